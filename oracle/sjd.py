@@ -1,0 +1,284 @@
+"""Speculative Jacobi Decoding state machine (test infrastructure; see
+oracle/__init__.py).  Follows Sec. 4.1 Steps 1-4 and Sec. 4.2 in the paper's
+order; plain auto-regressive sampling (Sec. 3.1) and greedy Jacobi decoding
+(Sec. 3.2) are included as the special cases the paper relates SJD to.
+
+Conventions fixed here (0-indexed)
+  * c[0..n) are fixed tokens (prompt of P tokens, then accepted tokens); the
+    window holds W_eff = min(W, P + N - n) drafts d_k for positions n + k.
+  * One step feeds [c[n-1], d_0 .. d_{W_eff-2}] at positions n-1 .. n+W_eff-2
+    (the KV cache therefore holds rows for c[0..n-1)); logits row k predicts
+    position n + k.  Rows are rounded to their storage dtype before use.
+  * The token drawn by Eq. 2 is fixed at once together with the accepted
+    prefix, so every step fixes at least one token.
+  * A freshly initialised slot carries the law it was drawn from: uniform
+    1/V for a random token, a point mass for a copied neighbour.
+  * Uniforms: Philox4x32-10 keyed by the seed, counter = (absolute position,
+    step index, sequence id, stream tag); see oracle/philox.py.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+from . import philox
+from .model import KVCache, OracleModel, round_to_storage
+from .sampling import (FLAG_DONE, Q_ONEHOT, Q_ROW, Q_UNIFORM, QDesc, VerifyResult, icdf,
+                       verify_window, warp)
+
+INIT_RANDOM = 0       # Sec. 4.2: uniform random candidate
+INIT_COPY_ABOVE = 1   # Sec. 4.2 (b): repeat the token one grid row above
+INIT_COPY_LEFT = 2    # Sec. 4.2 (a): repeat the left neighbour
+
+
+@dataclass
+class SampleCfg:
+    temperature: float = 1.0
+    top_k: int = 2000
+    seed: int = 0
+    window: int = 16
+    init: int = INIT_RANDOM
+    grid_stride: int = 0       # tokens per image row (incl. any row-end token)
+    n_generate: int = 0
+    logits_dtype: str = "f32"  # storage dtype of the logits: 'f32' or 'bf16'
+
+
+@dataclass
+class SJDState:
+    prompt_len: int
+    committed: list                    # c[0..n)
+    drafts: list = field(default_factory=list)
+    qdescs: list = field(default_factory=list)
+    step: int = 0
+    seq: int = 0
+    flags: int = 0
+
+    @property
+    def n(self) -> int:
+        return len(self.committed)
+
+
+@dataclass
+class StepRecord:
+    n_accepted: int
+    committed: list
+    drafts: list
+    kinds: list
+    flags: int
+    verify: VerifyResult | None
+    logits: np.ndarray | None          # stored logits rows of this step [W_eff][V]
+    q_draft: list = field(default_factory=list)   # q(d) of each new draft under its own descriptor
+
+
+# ----------------------------------------------------------------------------------------------
+# models: anything with  prefill(prompt)  and
+#                        step_logits(committed, drafts_in) -> [len(drafts_in)+1][V]
+# ----------------------------------------------------------------------------------------------
+class CachedModel:
+    """OracleModel driven with a KV cache: rows for c[0..n-1) stay cached, the
+    rejected tail is rolled back by truncation (stale rows are overwritten)."""
+
+    def __init__(self, model: OracleModel, capacity: int):
+        self.model = model
+        self.cache: KVCache = model.new_cache(capacity)
+
+    def prefill(self, prompt):
+        self.cache.truncate(0)
+        if len(prompt) > 1:
+            self.model.forward_window(self.cache, prompt[:-1], 0, want_logits=False)
+
+    def step_logits(self, committed, drafts_in):
+        n = len(committed)
+        self.cache.truncate(n - 1)
+        return self.model.forward_window(self.cache, [committed[-1]] + list(drafts_in), n - 1)
+
+
+class RecomputeModel:
+    """Same function without a cache: full causal forward of everything."""
+
+    def __init__(self, model: OracleModel):
+        self.model = model
+
+    def prefill(self, prompt):
+        pass
+
+    def step_logits(self, committed, drafts_in):
+        full = self.model.forward_full(list(committed) + list(drafts_in))
+        return full[len(committed) - 1:]
+
+
+class TableModel:
+    """Tiny context-dependent categorical model for brute-force pins:
+    logits(prefix) = table[index of the last `order` tokens]."""
+
+    def __init__(self, vocab: int, order: int, seed: int, scale: float = 1.5):
+        rng = np.random.default_rng(seed)
+        self.vocab, self.order = vocab, order
+        self.table = rng.normal(0.0, scale, size=(vocab ** order, vocab))
+
+    def logits_after(self, prefix):
+        ctx = [0] * self.order + [int(t) for t in prefix]
+        idx = 0
+        for t in ctx[-self.order:]:
+            idx = idx * self.vocab + t
+        return self.table[idx]
+
+    def prefill(self, prompt):
+        pass
+
+    def step_logits(self, committed, drafts_in):
+        seq = list(committed) + list(drafts_in)
+        n = len(committed)
+        return np.stack([self.logits_after(seq[:n + k]) for k in range(len(drafts_in) + 1)])
+
+
+# ----------------------------------------------------------------------------------------------
+# window construction (Step 4, Sec. 4.2)
+# ----------------------------------------------------------------------------------------------
+def _fresh_slot(state: SJDState, drafts, scfg: SampleCfg, vocab: int, t_pos: int, step_tag: int):
+    """Token and q descriptor for a newly initialised slot at absolute position t_pos.
+    `drafts` are the slots of the new window already filled (positions n .. t_pos-1)."""
+    stride = {INIT_COPY_ABOVE: scfg.grid_stride, INIT_COPY_LEFT: 1}.get(scfg.init, 0)
+    src = t_pos - stride
+    if scfg.init != INIT_RANDOM and stride > 0 and src >= state.prompt_len:
+        n = state.n
+        tok = state.committed[src] if src < n else drafts[src - n]
+        return int(tok), QDesc(Q_ONEHOT)
+    tok = philox.init_token(scfg.seed, t_pos, step_tag, state.seq, vocab)
+    return int(tok), QDesc(Q_UNIFORM)
+
+
+def _fill_window(state: SJDState, scfg: SampleCfg, vocab: int, step_tag: int):
+    w_eff = max(0, min(scfg.window, state.prompt_len + scfg.n_generate - state.n))
+    del state.drafts[w_eff:]
+    del state.qdescs[w_eff:]
+    while len(state.drafts) < w_eff:
+        t_pos = state.n + len(state.drafts)
+        tok, qd = _fresh_slot(state, state.drafts, scfg, vocab, t_pos, step_tag)
+        state.drafts.append(tok)
+        state.qdescs.append(qd)
+
+
+def sjd_begin(prompt, scfg: SampleCfg, vocab: int, seq: int = 0) -> SJDState:
+    """State after pre-filling the prompt: an all-fresh first window (Sec. 4.1:
+    the method starts with a window of initialised candidate tokens)."""
+    assert len(prompt) >= 1
+    st = SJDState(prompt_len=len(prompt), committed=[int(t) for t in prompt], seq=seq)
+    _fill_window(st, scfg, vocab, philox.STEP_INITIAL_WINDOW)
+    return st
+
+
+def q_of_draft(qd: QDesc, draft: int, vocab: int, scfg: SampleCfg) -> float:
+    return float(qd.dist(draft, vocab, scfg.temperature, scfg.top_k)[int(draft)])
+
+
+def sjd_step(state: SJDState, model, scfg: SampleCfg, vocab: int, logits_override=None) -> StepRecord:
+    """One SJD iteration (Steps 1-4).  `logits_override` replaces the forward
+    pass by externally supplied stored logits rows (lock-step comparisons)."""
+    n = state.n
+    w_eff = len(state.drafts)
+    if w_eff == 0:
+        state.flags |= FLAG_DONE
+        return StepRecord(0, [], [], [], FLAG_DONE, None, None)
+    j = state.step
+
+    # Step 2: one forward pass over the window
+    if logits_override is not None:
+        stored = np.asarray(logits_override, dtype=np.float64)[:w_eff]
+    else:
+        raw = model.step_logits(state.committed, state.drafts[:w_eff - 1])
+        stored = round_to_storage(raw, scfg.logits_dtype)
+
+    # Step 3: verification scan, calibrated resample, refinement
+    uniforms = [philox.verify_uniforms(scfg.seed, n + k, j, state.seq) for k in range(w_eff)]
+    vr = verify_window(stored, state.drafts, state.qdescs, uniforms, scfg.temperature, scfg.top_k)
+
+    # fixed tokens grow by the accepted prefix (+ the resampled token)
+    state.committed.extend(vr.committed)
+    # Step 4: unaccepted (re-drawn) tokens carry this iteration's rows as their q
+    state.drafts = list(vr.redraft)
+    state.qdescs = [QDesc(Q_ROW, row=stored[k].copy()) for k in vr.redraft_rows]
+    state.step = j + 1
+    _fill_window(state, scfg, vocab, j)
+    flags = vr.flags
+    if state.n >= state.prompt_len + scfg.n_generate:
+        flags |= FLAG_DONE
+    state.flags |= flags
+    return StepRecord(
+        n_accepted=vr.n_accepted, committed=list(vr.committed), drafts=list(state.drafts),
+        kinds=[qd.kind for qd in state.qdescs], flags=flags, verify=vr, logits=stored,
+        q_draft=[q_of_draft(qd, d, vocab, scfg) for qd, d in zip(state.qdescs, state.drafts)])
+
+
+def sjd_generate(prompt, model, scfg: SampleCfg, vocab: int, seq: int = 0, max_steps=None):
+    """Run SJD until N tokens are fixed.  Returns (generated tokens, number of
+    forward passes, per-step committed counts)."""
+    model.prefill(list(prompt))
+    st = sjd_begin(prompt, scfg, vocab, seq)
+    steps, accepted = 0, []
+    target = len(prompt) + scfg.n_generate
+    while st.n < target:
+        rec = sjd_step(st, model, scfg, vocab)
+        steps += 1
+        accepted.append(len(rec.committed))
+        if max_steps is not None and steps >= max_steps:
+            break
+    return st.committed[len(prompt):], steps, accepted
+
+
+def ar_generate(prompt, model, scfg: SampleCfg, vocab: int, seq: int = 0):
+    """Ordinary next-token sampling (Sec. 3.1): one forward pass per token.
+    Token at position t uses the re-draft uniform of (t, step = t - P)."""
+    model.prefill(list(prompt))
+    c = [int(t) for t in prompt]
+    p_len = len(prompt)
+    for i in range(scfg.n_generate):
+        row = round_to_storage(model.step_logits(c, []), scfg.logits_dtype)[0]
+        u = philox.verify_uniforms(scfg.seed, len(c), i, seq)[2]
+        tok, _ = icdf(warp(row, scfg.temperature, scfg.top_k), u)
+        c.append(tok)
+    return c[p_len:], scfg.n_generate
+
+
+def greedy_ar_generate(prompt, model, n_generate: int, logits_dtype: str = "f32"):
+    model.prefill(list(prompt))
+    c = [int(t) for t in prompt]
+    for _ in range(n_generate):
+        row = round_to_storage(model.step_logits(c, []), logits_dtype)[0]
+        c.append(int(np.argmax(row)))
+    return c[len(prompt):]
+
+
+def jacobi_generate(prompt, model, n_generate: int, window: int, vocab: int, seed: int = 0,
+                    logits_dtype: str = "f32", seq: int = 0):
+    """Greedy Jacobi decoding (Sec. 3.2): every window slot is replaced by the
+    argmax of its row each iteration; the prefix of slots that did not change
+    is fixed, and so is the first changed slot (its context is already fixed).
+    New slots are random tokens drawn exactly as SJD's random initialisation
+    draws them.  Returns (tokens, forward passes)."""
+    model.prefill(list(prompt))
+    c = [int(t) for t in prompt]
+    p_len = len(prompt)
+    total = p_len + n_generate
+
+    def refill(drafts, step_tag):
+        w_eff = min(window, total - len(c))
+        drafts = drafts[:w_eff]
+        while len(drafts) < w_eff:
+            drafts.append(philox.init_token(seed, len(c) + len(drafts), step_tag, seq, vocab))
+        return drafts
+
+    drafts = refill([], philox.STEP_INITIAL_WINDOW)
+    passes = 0
+    while len(c) < total:
+        rows = round_to_storage(model.step_logits(c, drafts[:-1]), logits_dtype)
+        new = [int(np.argmax(r)) for r in rows]
+        a = 0
+        while a < len(drafts) and drafts[a] == new[a]:
+            a += 1
+        fixed = new[:a + 1] if a < len(drafts) else new[:a]
+        c.extend(fixed)
+        drafts = refill(new[len(fixed):], passes)
+        passes += 1
+    return c[p_len:], passes
