@@ -1,0 +1,217 @@
+/*
+ * libsjd - one Speculative Jacobi Decoding (SJD) iteration on one GPU (sm_100a).
+ *
+ * The library runs the per-iteration hot path of SJD for a decoder-only
+ * image-token transformer (arXiv 2410.01699, Sec. 4.1 Steps 1-4, Eqs. 1-3,
+ * Sec. 4.2): a window of W draft tokens goes through the model in a single
+ * forward pass against a KV cache, each draft is accepted with probability
+ * min(1, p/q), the first rejected position is resampled from
+ * norm(max(0, p - q)), the rest of the window is re-drawn from the new
+ * distributions, and the window slides over the accepted tokens.
+ *
+ * Conventions
+ *   - Every function returns SJD_OK (0) or a negative sjd_status.  Nothing
+ *     throws, aborts or prints.
+ *   - "device" pointers are CUDA device pointers of the current device;
+ *     "host" pointers are ordinary host memory.  Pointers named in
+ *     sjd_step_out may be device memory or pinned (mapped) host memory.
+ *   - The caller owns all device memory: weights, the workspace and the
+ *     outputs.  The library owns only the small host-side context.  Weights
+ *     are borrowed for the lifetime of the context and never written.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default
+ *     stream).  Work is enqueued asynchronously; no call synchronises the
+ *     device except sjd_init (table upload) and sjd_last_device_status.
+ *   - Matrices are row-major [out_features][in_features] (y = x W^T).
+ *   - All sequences of a batch share prompt length, n_generate and the
+ *     sampling configuration; the Philox counter carries the sequence id.
+ *
+ * Random numbers: Philox4x32-10 (Salmon et al., SC'11), key = 64-bit seed,
+ * counter = (absolute position, step index, sequence id, stream tag).
+ * Stream tag 0: word 0 -> acceptance test (Eq. 1), word 1 -> residual
+ * resample (Eq. 2), word 2 -> re-draft (Eq. 3).  Stream tag 1: word 0 ->
+ * random token of a freshly initialised slot, floor(word * V / 2^32).  A
+ * uniform is (word >> 8) * 2^-24.  The first window uses step 0xFFFFFFFF.
+ */
+#ifndef SJD_H_
+#define SJD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sjd_ctx sjd_ctx; /* opaque; created by sjd_init, freed by sjd_destroy */
+
+typedef enum {
+  SJD_OK = 0,
+  SJD_ERR_BAD_ARG = -1,        /* null pointer, non-positive size, T <= 0, top_k < 1 ...      */
+  SJD_ERR_CAPACITY = -2,       /* batch/window/sequence/workspace/vocab beyond what was sized */
+  SJD_ERR_UNSUPPORTED = -3,    /* shape or dtype the kernels do not cover                     */
+  SJD_ERR_CUDA = -4,           /* a CUDA runtime call failed; see sjd_last_cuda_error         */
+  SJD_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait ran out                          */
+  SJD_ERR_STATE = -6           /* call out of order (step before prefill ...)                 */
+} sjd_status;
+
+typedef enum { SJD_F32 = 0, SJD_BF16 = 1 } sjd_dtype;
+
+/* How new window slots are initialised (Sec. 4.2). */
+typedef enum {
+  SJD_INIT_RANDOM = 0,     /* uniform random token; carries q = 1/V                         */
+  SJD_INIT_COPY_ABOVE = 1, /* token at position - grid_stride (strategy (b)); q = point mass */
+  SJD_INIT_COPY_LEFT = 2   /* token at position - 1 (strategy (a)); q = point mass           */
+} sjd_init_kind;
+
+/* The law a draft token was drawn from (Step 1: "the probability corresponding to the draft"). */
+typedef enum {
+  SJD_Q_ROW = 0,     /* top-k softmax of the logits row that produced it one iteration ago */
+  SJD_Q_UNIFORM = 1, /* 1/V                                                                */
+  SJD_Q_ONEHOT = 2   /* point mass on the draft itself                                     */
+} sjd_q_kind;
+
+/* bits of sjd_step_out.flags */
+#define SJD_FLAG_NEAR_TIE_ACCEPT 1u /* some scanned row had |u - min(1,p/q)| < 1e-4 with p/q < 1  */
+#define SJD_FLAG_RESIDUAL_EMPTY 4u  /* sum max(0,p-q) == 0 at the rejected row: sampled from p    */
+#define SJD_FLAG_NONFINITE 8u       /* a logits row held NaN or +inf (treated as -inf)            */
+#define SJD_FLAG_DONE 16u           /* all n_generate tokens of this sequence are fixed           */
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, ffn_hidden, vocab;
+  float rope_theta; /* rotary base; pairs (i, i + head_dim/2), angle pos * theta^(-2i/head_dim) */
+  float rms_eps;
+  int32_t dtype;    /* sjd_dtype of weights, activations, KV cache and stored logits */
+  int32_t max_batch, max_seq, max_window;
+} sjd_model_cfg;
+
+/* Device pointers, borrowed.  Per-layer entries are HOST arrays of n_layers device pointers. */
+typedef struct {
+  const void *tok_emb;    /* [vocab][d_model]                 */
+  const void *final_norm; /* [d_model]                        */
+  const void *lm_head;    /* [vocab][d_model]                 */
+  const void *const *attn_norm; /* [d_model]                  */
+  const void *const *wq;        /* [n_heads*head_dim][d_model]    */
+  const void *const *wk;        /* [n_kv_heads*head_dim][d_model] */
+  const void *const *wv;        /* [n_kv_heads*head_dim][d_model] */
+  const void *const *wo;        /* [d_model][n_heads*head_dim]    */
+  const void *const *ffn_norm;  /* [d_model]                  */
+  const void *const *w_gate;    /* [ffn_hidden][d_model]      */
+  const void *const *w_up;      /* [ffn_hidden][d_model]      */
+  const void *const *w_down;    /* [d_model][ffn_hidden]      */
+} sjd_weights;
+
+typedef struct {
+  float temperature;   /* > 0; logits are divided by it before top-k (the paper has none: 1.0) */
+  int32_t top_k;       /* >= 1; entries equal to the k-th largest are all kept; >= V: no filter */
+  uint64_t seed;       /* Philox key                                                            */
+  int32_t window;      /* W, Jacobi window size (Sec. 4.1)                                      */
+  int32_t init;        /* sjd_init_kind                                                         */
+  int32_t grid_stride; /* tokens per image row incl. any row-end token (COPY_ABOVE)             */
+  int32_t n_generate;  /* N, image tokens to generate per sequence                              */
+  int32_t seq_base;    /* global id of sequence 0 of this batch (Philox counter word 2): a batch    */
+                       /* sharded over several GPUs draws the same numbers wherever a sequence runs  */
+} sjd_sample_cfg;
+
+/* Results of one step.  Any pointer may be NULL (that output is skipped). */
+typedef struct {
+  int32_t *n_accepted;      /* [B]    drafts accepted by Eq. 1 this step (0..W)                    */
+  int32_t *n_committed;     /* [B]    tokens fixed this step: accepted (+1 resampled); 0 when done */
+  int32_t *committed;       /* [B][W] those tokens, left-aligned, rest -1                          */
+  int32_t *draft;           /* [B][W] the next window's draft tokens, rest -1                      */
+  int32_t *q_kind;          /* [B][W] sjd_q_kind of each new draft, rest -1                        */
+  float *q_draft;           /* [B][W] q(draft) of each new draft under its own law, rest 0         */
+  int32_t *total_committed; /* [B]    n after the step (prompt + fixed tokens)                     */
+  uint32_t *flags;          /* [B]    SJD_FLAG_* bits raised by this step                          */
+} sjd_step_out;
+
+/*
+ * Bytes of caller-provided device workspace a context needs: KV cache
+ * [layer][batch][k|v][kv_head][max_seq][head_dim], two logits buffers
+ * [max_batch][max_window][vocab] (this iteration's p rows are the next
+ * iteration's q rows: the buffers swap, nothing is copied), activations, GEMM
+ * split-K partials, per-row verification scratch and decoding state.
+ * Returns 0 for an invalid configuration.
+ */
+size_t sjd_workspace_bytes(const sjd_model_cfg *cfg);
+
+/*
+ * Create a context (Sec. 3.1: the auto-regressive transformer; Sec. 4.1: its
+ * use on a window).  `workspace` is device memory of at least
+ * sjd_workspace_bytes(cfg), 256-byte aligned, owned by the caller and must
+ * outlive the context.  Uploads the rotary table (synchronous).
+ * Errors: BAD_ARG (null / non-positive / odd head_dim / n_heads not a
+ * multiple of n_kv_heads), CAPACITY (workspace too small), UNSUPPORTED
+ * (head_dim > 256, window > 64, unknown dtype), CUDA.
+ */
+int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weights *weights, void *workspace,
+             size_t workspace_bytes);
+
+/*
+ * Pre-fill (Sec. 4.1, first sentence): run the model over prompt tokens
+ * c[0..P-1) so that their keys/values are cached (the last prompt token is
+ * the first input of step 0), then build the first window of W freshly
+ * initialised drafts (Sec. 4.2).  prompt: device int32 [batch][prompt_len],
+ * prompt_len >= 1.  Resets the step index to 0.
+ * Errors: BAD_ARG; CAPACITY (batch > max_batch, window > max_window,
+ * prompt_len + n_generate > max_seq); CUDA.
+ */
+int sjd_prefill(sjd_ctx *ctx, int batch, const int32_t *prompt, int prompt_len,
+                const sjd_sample_cfg *sample, void *cuda_stream);
+
+/*
+ * One SJD iteration for every sequence of the batch (Sec. 4.1 Steps 1-4):
+ *   inputs  [c[n-1], d_0 .. d_{W_eff-2}] at positions n-1 .. n+W_eff-2,
+ *           W_eff = min(W, P + N - n);
+ *   forward one pass; logits row k (stored in cfg.dtype) predicts position n+k;
+ *   verify  acc_k = u_k < min(1, p_k[d_k] / q_k[d_k]) scanned left to right (Eq. 1);
+ *           at the first rejected row a: t ~ max(0, p_a - q_a) / sum (Eq. 2),
+ *           fixed at once after d_0..d_{a-1}; rows k > a: d'_k ~ p_k (Eq. 3);
+ *   slide   the re-drawn tokens move left by the number of fixed tokens, new
+ *           slots are initialised (Sec. 4.2), rejected keys/values are
+ *           rolled back (overwritten by the next step).
+ * Sampling is by inverse CDF in token order.  Asynchronous on the stream.
+ * A finished sequence reports n_committed = 0 and SJD_FLAG_DONE.
+ * Errors: STATE (no prefill), BAD_ARG, CUDA.
+ */
+int sjd_step(sjd_ctx *ctx, const sjd_step_out *out, void *cuda_stream);
+
+/* Current window (drafts, their laws, n) without stepping; fields n_accepted,
+ * n_committed, committed and flags of `out` are not written. */
+int sjd_get_window(sjd_ctx *ctx, const sjd_step_out *out, void *cuda_stream);
+
+/* Copy the stored logits of the last step, [batch][window][vocab] in cfg.dtype,
+ * to dst (device or host); for parity checks.  Errors: STATE, CAPACITY (bytes too small). */
+int sjd_peek_logits(sjd_ctx *ctx, void *dst, size_t bytes, void *cuda_stream);
+
+/*
+ * The verification of Step 3 in isolation (Eqs. 1-3) on caller-supplied
+ * logits.  logits_cur / logits_prev: device [batch][window][vocab] of
+ * logits_dtype (this iteration's rows; the rows the drafts were drawn from);
+ * draft: device int32 [batch][window]; q_kind: device int32 [batch][window]
+ * or NULL (all SJD_Q_ROW); base_pos: device int32 [batch], absolute position
+ * of window slot 0 (Philox counter), or NULL (all 0).  Outputs as sjd_step:
+ * `draft` receives the re-drawn tokens of rows a+1.. left-aligned (no new
+ * slots are initialised), total_committed = base_pos + n_committed.
+ * ws: device scratch of sjd_verify_workspace_bytes(batch, window) bytes.
+ * Errors: BAD_ARG, CAPACITY (ws too small, window > 64, vocab too large), CUDA.
+ */
+size_t sjd_verify_workspace_bytes(int batch, int window);
+int sjd_verify(int batch, int window, int vocab, int logits_dtype, const void *logits_cur,
+               const void *logits_prev, const int32_t *draft, const int32_t *q_kind,
+               const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
+               const sjd_step_out *out, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Synchronises the context's last stream and returns SJD_OK, SJD_ERR_DEVICE_TIMEOUT
+ * or SJD_ERR_CUDA according to the device status word. */
+int sjd_last_device_status(sjd_ctx *ctx);
+
+/* cudaError_t of the last failed CUDA call made on behalf of this thread (0 if none). */
+int sjd_last_cuda_error(void);
+
+void sjd_destroy(sjd_ctx *ctx);
+const char *sjd_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SJD_H_ */

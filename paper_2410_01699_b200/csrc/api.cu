@@ -1,0 +1,86 @@
+// C-ABI entry points that need no context: isolated verification, error strings.
+#include <string.h>
+
+#include "common.cuh"
+
+namespace sjd {
+thread_local int g_last_cuda_error = 0;
+
+int check_sample_cfg(const sjd_sample_cfg *s, int vocab) {
+  if (!s) return SJD_ERR_BAD_ARG;
+  if (!(s->temperature > 0.0f) || s->top_k < 1 || s->window < 1) return SJD_ERR_BAD_ARG;
+  if (s->window > 64) return SJD_ERR_CAPACITY;
+  if (s->init < SJD_INIT_RANDOM || s->init > SJD_INIT_COPY_LEFT) return SJD_ERR_BAD_ARG;
+  if (s->init == SJD_INIT_COPY_ABOVE && s->grid_stride < 1) return SJD_ERR_BAD_ARG;
+  if (s->seq_base < 0) return SJD_ERR_BAD_ARG;
+  (void)vocab;
+  return SJD_OK;
+}
+}  // namespace sjd
+
+using namespace sjd;
+
+extern "C" size_t sjd_verify_workspace_bytes(int batch, int window) { return verify_scratch_bytes(batch, window); }
+
+extern "C" int sjd_verify(int batch, int window, int vocab, int logits_dtype, const void *logits_cur,
+                          const void *logits_prev, const int32_t *draft, const int32_t *q_kind,
+                          const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
+                          const sjd_step_out *out, void *ws, size_t ws_bytes, void *cuda_stream) {
+  if (batch < 1 || window < 1 || vocab < 1 || !logits_cur || !draft || !sample || !out || !ws)
+    return SJD_ERR_BAD_ARG;
+  if (!logits_prev && !q_kind) return SJD_ERR_BAD_ARG;  // rows of law SJD_Q_ROW need their logits
+  if (logits_dtype != SJD_F32 && logits_dtype != SJD_BF16) return SJD_ERR_UNSUPPORTED;
+  if (window > 64) return SJD_ERR_CAPACITY;
+  if (!(sample->temperature > 0.0f) || sample->top_k < 1) return SJD_ERR_BAD_ARG;
+  const size_t need = verify_scratch_bytes(batch, window);
+  if (ws_bytes < need) return SJD_ERR_CAPACITY;
+  if (((uintptr_t)ws & 15u) != 0) return SJD_ERR_BAD_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+  const size_t rows = (size_t)batch * window;
+  char *w = (char *)ws;
+  VerifyParams p;
+  memset(&p, 0, sizeof(p));
+  p.logits[0] = logits_cur;
+  p.logits[1] = logits_prev ? logits_prev : logits_cur;
+  p.stats[0] = (RowStats *)w;
+  p.stats[1] = (RowStats *)(w + rows * sizeof(RowStats));
+  p.row_out = (RowOut *)(w + 2 * rows * sizeof(RowStats));
+  p.seq_counter = (int32_t *)(w + 2 * rows * sizeof(RowStats) + rows * sizeof(RowOut));
+  p.done_counter = p.seq_counter + batch;
+  SJD_CUDA(cudaMemsetAsync(p.seq_counter, 0, ((size_t)batch + 1) * sizeof(int32_t), stream));
+  p.draft = draft;
+  p.q_kind = q_kind;
+  p.q_row = nullptr;
+  p.prev_stats_valid = 0;
+  p.w_eff = nullptr;
+  p.base_pos = base_pos;
+  p.step_ptr = nullptr;
+  p.step = step;
+  p.B = batch;
+  p.W = window;
+  p.V = vocab;
+  p.temperature = sample->temperature;
+  p.top_k = sample->top_k;
+  p.seed_lo = (uint32_t)(sample->seed & 0xFFFFFFFFull);
+  p.seed_hi = (uint32_t)(sample->seed >> 32);
+  p.seq_base = (uint32_t)sample->seq_base;
+  p.e2e = 0;
+  p.out = *out;
+  return launch_verify(p, logits_dtype, stream);
+}
+
+extern "C" int sjd_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" const char *sjd_strerror(int status) {
+  switch (status) {
+    case SJD_OK: return "ok";
+    case SJD_ERR_BAD_ARG: return "bad argument";
+    case SJD_ERR_CAPACITY: return "capacity exceeded (batch, window, sequence, vocabulary or workspace)";
+    case SJD_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case SJD_ERR_CUDA: return "CUDA runtime error (see sjd_last_cuda_error)";
+    case SJD_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case SJD_ERR_STATE: return "call out of order";
+    default: return "unknown status";
+  }
+}

@@ -1,0 +1,171 @@
+// Shared declarations of the SJD CUDA library: status helpers, Philox4x32-10,
+// small warp/block primitives, and the launch prototypes of every kernel file.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sjd.h"
+
+namespace sjd {
+
+extern thread_local int g_last_cuda_error;
+
+#define SJD_CUDA(expr)                          \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) {                   \
+      ::sjd::g_last_cuda_error = (int)e__;      \
+      return SJD_ERR_CUDA;                      \
+    }                                           \
+  } while (0)
+
+#define SJD_CHECK_LAUNCH() SJD_CUDA(cudaGetLastError())
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): 128-bit counter, 64-bit key, ten rounds of
+// two 32x32->64 multiplies with a Weyl key schedule.
+// ---------------------------------------------------------------------------------------------
+struct Philox4 {
+  uint32_t w[4];
+};
+
+__host__ __device__ inline Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)M0 * c0;
+    const uint64_t p1 = (uint64_t)M1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+    k0 += W0;
+    k1 += W1;
+  }
+  Philox4 out;
+  out.w[0] = c0; out.w[1] = c1; out.w[2] = c2; out.w[3] = c3;
+  return out;
+}
+
+constexpr uint32_t kStreamVerify = 0u;         // words 0,1,2: accept / residual / re-draft uniforms
+constexpr uint32_t kStreamInit = 1u;           // word 0: random token of a fresh slot
+constexpr uint32_t kStepInitialWindow = 0xFFFFFFFFu;
+
+__host__ __device__ inline float u24(uint32_t word) { return (float)(word >> 8) * (1.0f / 16777216.0f); }
+
+// ---------------------------------------------------------------------------------------------
+// warp helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Per-row verification records (device scratch)
+// ---------------------------------------------------------------------------------------------
+struct RowStats {      // what is needed to evaluate p(x) of a stored logits row at any x
+  uint32_t tau_key;    // order-preserving key of the top-k threshold (entries with key >= it are kept)
+  float xmax;          // largest logit of the row (-inf for a row with no finite entry)
+  float z;             // sum over kept entries of exp((x - xmax) / T)
+  uint32_t flags;      // SJD_FLAG_NONFINITE
+};
+
+struct RowOut {
+  float p_draft;       // p_k[d_k]
+  float q_draft;       // q_k[d_k]
+  float thr;           // min(1, p/q)
+  int32_t accept;      // u_acc < thr
+  int32_t redraft_tok; // d'_k ~ p_k (Eq. 3)
+  float redraft_p;     // p_k[d'_k]: the q the re-drawn token carries
+  int32_t resample_tok;// t_k ~ norm(max(0, p_k - q_k)) if this row rejected (Eq. 2), else -1
+  uint32_t flags;
+};
+
+// Decoding state of a context, all device-resident (see engine.cu)
+struct SeqState {
+  int32_t *committed;   // [B][max_seq]
+  int32_t *n;           // [B] committed count
+  int32_t *w_eff;       // [B] drafts in the current window
+  int32_t *draft;       // [B][W]
+  int32_t *q_kind;      // [B][W]
+  int32_t *q_row;       // [B][W] row of the previous logits buffer that produced the draft
+  float *q_draft;       // [B][W]
+  int32_t *in_tok;      // [B][W] model inputs of the next step
+  int32_t *in_pos;      // [B][W] their absolute positions, -1 = inactive row
+  int32_t max_seq;
+  int32_t prompt_len;
+  int32_t n_generate;
+  int32_t init;
+  int32_t grid_stride;
+};
+
+struct VerifyParams {
+  const void *logits[2];   // [B][W][V]; index (step & 1) is this iteration's buffer when use_step_ptr
+  RowStats *stats[2];      // [B][W] alongside
+  const int32_t *draft;    // [B][W]
+  const int32_t *q_kind;   // [B][W] or null (all ROW)
+  const int32_t *q_row;    // [B][W] or null (slot k was produced by row k)
+  int prev_stats_valid;    // stats of the previous buffer are already there (end-to-end mode)
+  RowOut *row_out;         // [B][W]
+  int32_t *seq_counter;    // [B] zero on entry, zero on exit
+  int32_t *done_counter;   // [1] zero on entry, zero on exit
+  const int32_t *w_eff;    // [B] or null (= W)
+  const int32_t *base_pos; // [B] absolute position of slot 0, or null (0)
+  uint32_t *step_ptr;      // device step index (end-to-end), bumped by the last block
+  uint32_t step;           // used when step_ptr == null
+  int B, W, V;
+  int staged;              // row fits the dynamic shared buffer
+  float temperature;
+  int top_k;
+  uint32_t seed_lo, seed_hi;
+  uint32_t seq_base;       // global id of sequence 0 (batch sharded across GPUs)
+  int e2e;                 // 1: update SeqState (window slide); 0: isolated verification
+  SeqState st;
+  sjd_step_out out;
+};
+
+// kernel launchers (each returns an sjd_status)
+int launch_verify(const VerifyParams &p, int dtype, cudaStream_t stream);
+size_t verify_scratch_bytes(int batch, int window);
+int check_sample_cfg(const sjd_sample_cfg *s, int vocab);
+
+// ---- model forward (model_kernels.cu, attention.cu); `dtype` selects float / bf16 storage
+enum GemmEpilogue { EPI_STORE_F32 = 0, EPI_STORE_T = 1, EPI_ADD_F32 = 2 };
+
+// C[M][N] (epilogue) = A[M][K] * Wt[N][K]^T, fp32 accumulation.  A and Wt are of `dtype`;
+// C is fp32 (EPI_STORE_F32, EPI_ADD_F32: C += product) or `dtype` (EPI_STORE_T).  lda/ldc in elements.
+int launch_gemm_simt(int dtype, const void *A, int lda, const void *Wt, void *C, int ldc, int M, int N, int K,
+                     int epilogue, cudaStream_t stream);
+// x[m][:] = tok_emb[tok[m]][:]  (fp32 residual stream)
+int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, int M, int d, int vocab,
+                 cudaStream_t stream);
+// h[m][:] = x[m][:] * gain[:] / sqrt(mean(x[m]^2) + eps), stored as `dtype`
+int launch_rmsnorm(int dtype, const float *x, const void *gain, void *h, int M, int d, float eps, cudaStream_t stream);
+// Rotate q and k by their absolute position (pairs i, i + hd/2), store q as `dtype` [M][H*hd],
+// append k and v to the cache row in_pos[m] of sequence m / rows_per_seq.  Rows with in_pos < 0 are skipped.
+struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
+  void *base;
+  int n_kv_heads, max_seq, head_dim;
+};
+int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, void *q,
+                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
+// act[m][f] = silu(gu[m][f]) * gu[m][F + f], stored as `dtype`
+int launch_swiglu(int dtype, const float *gu, void *act, int M, int F, cudaStream_t stream);
+// Window-causal attention: query row m (sequence m / rows_per_seq, position in_pos[m]) attends cache rows
+// 0 .. in_pos[m].  out [M][H*hd] of `dtype`.  partial: fp32 scratch [M][H][splits][hd + 2].
+int launch_attention(int dtype, const void *q, KvLayout kv, const int32_t *in_pos, void *out, float *partial,
+                     int M, int rows_per_seq, int n_heads, int splits, cudaStream_t stream);
+
+}  // namespace sjd

@@ -1,0 +1,398 @@
+// Context, workspace layout and the per-step launch sequence (Sec. 4.1: pre-fill, then one forward
+// pass + verification + window slide per iteration).  All decoding state (committed tokens, window,
+// counters, step index) lives in device memory, so consecutive steps are enqueued back to back with
+// no host round trip.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace sjd {
+namespace {
+
+inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+inline size_t esize(int dtype) { return dtype == SJD_F32 ? 4 : 2; }
+
+int attention_splits(int n_heads, int batch) {
+  int s = (2 * 148 + n_heads * batch - 1) / (n_heads * batch);
+  return s < 1 ? 1 : (s > 16 ? 16 : s);
+}
+
+struct Layout {
+  size_t kv, logits[2], stats[2], row_out, counters, step, status;
+  size_t x, h, qkv, q, attn, gu, act, partial, rope;
+  size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
+  size_t total;
+};
+
+bool cfg_valid(const sjd_model_cfg *c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->d_model < 1 || c->n_heads < 1 || c->n_kv_heads < 1 || c->head_dim < 2 ||
+      c->ffn_hidden < 1 || c->vocab < 1 || c->max_batch < 1 || c->max_seq < 2 || c->max_window < 1)
+    return false;
+  if (c->head_dim % 2 != 0 || c->n_heads % c->n_kv_heads != 0) return false;
+  if (!(c->rms_eps > 0.0f) || !(c->rope_theta > 0.0f)) return false;
+  return true;
+}
+
+Layout make_layout(const sjd_model_cfg &c) {
+  Layout L;
+  const size_t es = esize(c.dtype);
+  const size_t Mx = (size_t)c.max_batch * c.max_window;
+  const size_t nq = (size_t)c.n_heads * c.head_dim, nk = (size_t)c.n_kv_heads * c.head_dim;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align256(bytes);
+    return o;
+  };
+  L.kv = take((size_t)c.n_layers * c.max_batch * 2 * nk * c.max_seq * es);
+  L.logits[0] = take(Mx * c.vocab * es);
+  L.logits[1] = take(Mx * c.vocab * es);
+  L.stats[0] = take(Mx * sizeof(RowStats));
+  L.stats[1] = take(Mx * sizeof(RowStats));
+  L.row_out = take(Mx * sizeof(RowOut));
+  L.counters = take(((size_t)c.max_batch + 1) * 4);
+  L.step = take(4);
+  L.status = take(4);
+  L.x = take(Mx * c.d_model * 4);
+  L.h = take(Mx * c.d_model * es);
+  L.qkv = take(Mx * (nq + 2 * nk) * 4);
+  L.q = take(Mx * nq * es);
+  L.attn = take(Mx * nq * es);
+  L.gu = take(Mx * 2 * c.ffn_hidden * 4);
+  L.act = take(Mx * c.ffn_hidden * es);
+  size_t part = 0;
+  for (int b = 1; b <= c.max_batch; ++b) {
+    const size_t need = (size_t)b * c.max_window * c.n_heads * attention_splits(c.n_heads, b) * (c.head_dim + 2);
+    part = need > part ? need : part;
+  }
+  L.partial = take(part * 4);
+  L.rope = take((size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2));
+  L.committed = take((size_t)c.max_batch * c.max_seq * 4);
+  L.n = take((size_t)c.max_batch * 4);
+  L.w_eff = take((size_t)c.max_batch * 4);
+  L.draft = take(Mx * 4);
+  L.q_kind = take(Mx * 4);
+  L.q_row = take(Mx * 4);
+  L.q_draft = take(Mx * 4);
+  L.in_tok = take(Mx * 4);
+  L.in_pos = take(Mx * 4);
+  L.total = off;
+  return L;
+}
+
+__global__ void prefill_setup_kernel(const int32_t *prompt, int P, SeqState st, uint32_t *step, int32_t *counters,
+                                     int B) {
+  const int b = blockIdx.x;
+  for (int i = threadIdx.x; i < P; i += blockDim.x) st.committed[(size_t)b * st.max_seq + i] = prompt[(size_t)b * P + i];
+  if (threadIdx.x == 0) {
+    st.n[b] = P;
+    st.w_eff[b] = 0;
+    counters[b] = 0;
+    if (b == 0) {
+      counters[B] = 0;
+      *step = kStepInitialWindow;
+    }
+  }
+}
+
+__global__ void prefill_inputs_kernel(const int32_t *prompt, int P, int c0, int rows, int32_t *in_tok, int32_t *in_pos) {
+  const int b = blockIdx.x;
+  for (int k = threadIdx.x; k < rows; k += blockDim.x) {
+    const int pos = c0 + k;
+    const bool act = pos < P - 1;
+    in_tok[b * rows + k] = act ? prompt[(size_t)b * P + pos] : 0;
+    in_pos[b * rows + k] = act ? pos : -1;
+  }
+}
+
+__global__ void get_window_kernel(SeqState st, sjd_step_out o, int W) {
+  const int b = blockIdx.x;
+  for (int k = threadIdx.x; k < W; k += blockDim.x) {
+    const int i = b * W + k;
+    if (o.draft) o.draft[i] = st.draft[i];
+    if (o.q_kind) o.q_kind[i] = st.q_kind[i];
+    if (o.q_draft) o.q_draft[i] = st.q_draft[i];
+  }
+  if (threadIdx.x == 0 && o.total_committed) o.total_committed[b] = st.n[b];
+}
+
+}  // namespace
+}  // namespace sjd
+
+using namespace sjd;
+
+struct sjd_ctx {
+  sjd_model_cfg cfg;
+  Layout lay;
+  char *ws;
+  const void *tok_emb, *final_norm, *lm_head;
+  std::vector<const void *> attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down;
+  sjd_sample_cfg sample;
+  int batch, prompt_len, window;
+  bool prefilled;
+  uint32_t host_step;  // number of sjd_step calls since prefill == device step index
+  cudaStream_t last_stream;
+
+  template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
+  SeqState state() const {
+    SeqState st;
+    st.committed = at<int32_t>(lay.committed);
+    st.n = at<int32_t>(lay.n);
+    st.w_eff = at<int32_t>(lay.w_eff);
+    st.draft = at<int32_t>(lay.draft);
+    st.q_kind = at<int32_t>(lay.q_kind);
+    st.q_row = at<int32_t>(lay.q_row);
+    st.q_draft = at<float>(lay.q_draft);
+    st.in_tok = at<int32_t>(lay.in_tok);
+    st.in_pos = at<int32_t>(lay.in_pos);
+    st.max_seq = cfg.max_seq;
+    st.prompt_len = prompt_len;
+    st.n_generate = sample.n_generate;
+    st.init = sample.init;
+    st.grid_stride = sample.grid_stride;
+    return st;
+  }
+  KvLayout kv_layer(int l) const {
+    KvLayout kv;
+    const size_t per_layer = (size_t)cfg.max_batch * 2 * cfg.n_kv_heads * cfg.max_seq * cfg.head_dim * esize(cfg.dtype);
+    kv.base = ws + lay.kv + (size_t)l * per_layer;
+    kv.n_kv_heads = cfg.n_kv_heads;
+    kv.max_seq = cfg.max_seq;
+    kv.head_dim = cfg.head_dim;
+    return kv;
+  }
+};
+
+namespace sjd {
+namespace {
+
+// One forward pass of M = batch * rows_per_seq rows whose tokens / positions are in st.in_tok / in_pos.
+int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream) {
+  const sjd_model_cfg &g = c->cfg;
+  const int dt = g.dtype;
+  const int M = c->batch * rows_per_seq;
+  const int d = g.d_model, F = g.ffn_hidden;
+  const int nq = g.n_heads * g.head_dim, nk = g.n_kv_heads * g.head_dim, nqkv = nq + 2 * nk;
+  const SeqState st = c->state();
+  float *x = c->at<float>(c->lay.x);
+  void *h = c->ws + c->lay.h;
+  float *qkv = c->at<float>(c->lay.qkv);
+  void *q = c->ws + c->lay.q;
+  void *attn = c->ws + c->lay.attn;
+  float *gu = c->at<float>(c->lay.gu);
+  void *act = c->ws + c->lay.act;
+  float *partial = c->at<float>(c->lay.partial);
+  const float2 *rope = c->at<float2>(c->lay.rope);
+  const int splits = attention_splits(g.n_heads, c->batch);
+  int rc;
+#define SJD_TRY(call) do { rc = (call); if (rc != SJD_OK) return rc; } while (0)
+  SJD_TRY(launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
+  for (int l = 0; l < g.n_layers; ++l) {
+    SJD_TRY(launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream));
+    SJD_TRY(launch_gemm_simt(dt, h, d, c->wq[l], qkv, nqkv, M, nq, d, EPI_STORE_F32, stream));
+    SJD_TRY(launch_gemm_simt(dt, h, d, c->wk[l], qkv + nq, nqkv, M, nk, d, EPI_STORE_F32, stream));
+    SJD_TRY(launch_gemm_simt(dt, h, d, c->wv[l], qkv + nq + nk, nqkv, M, nk, d, EPI_STORE_F32, stream));
+    const KvLayout kv = c->kv_layer(l);
+    SJD_TRY(launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
+    SJD_TRY(launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream));
+    SJD_TRY(launch_gemm_simt(dt, attn, nq, c->wo[l], x, d, M, d, nq, EPI_ADD_F32, stream));
+    SJD_TRY(launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream));
+    SJD_TRY(launch_gemm_simt(dt, h, d, c->w_gate[l], gu, 2 * F, M, F, d, EPI_STORE_F32, stream));
+    SJD_TRY(launch_gemm_simt(dt, h, d, c->w_up[l], gu + F, 2 * F, M, F, d, EPI_STORE_F32, stream));
+    SJD_TRY(launch_swiglu(dt, gu, act, M, F, stream));
+    SJD_TRY(launch_gemm_simt(dt, act, F, c->w_down[l], x, d, M, d, F, EPI_ADD_F32, stream));
+  }
+  if (logits_out) {
+    SJD_TRY(launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream));
+    SJD_TRY(launch_gemm_simt(dt, h, d, c->lm_head, logits_out, g.vocab, M, g.vocab, d, EPI_STORE_T, stream));
+  }
+#undef SJD_TRY
+  return SJD_OK;
+}
+
+int run_verify(sjd_ctx *c, const sjd_step_out *out, cudaStream_t stream) {
+  VerifyParams p;
+  memset(&p, 0, sizeof(p));
+  const SeqState st = c->state();
+  p.logits[0] = c->ws + c->lay.logits[0];
+  p.logits[1] = c->ws + c->lay.logits[1];
+  p.stats[0] = c->at<RowStats>(c->lay.stats[0]);
+  p.stats[1] = c->at<RowStats>(c->lay.stats[1]);
+  p.draft = st.draft;
+  p.q_kind = st.q_kind;
+  p.q_row = st.q_row;
+  p.prev_stats_valid = 1;
+  p.row_out = c->at<RowOut>(c->lay.row_out);
+  p.seq_counter = c->at<int32_t>(c->lay.counters);
+  p.done_counter = p.seq_counter + c->batch;
+  p.w_eff = st.w_eff;
+  p.base_pos = nullptr;
+  p.step_ptr = c->at<uint32_t>(c->lay.step);
+  p.B = c->batch;
+  p.W = c->window;
+  p.V = c->cfg.vocab;
+  p.temperature = c->sample.temperature;
+  p.top_k = c->sample.top_k;
+  p.seed_lo = (uint32_t)(c->sample.seed & 0xFFFFFFFFull);
+  p.seed_hi = (uint32_t)(c->sample.seed >> 32);
+  p.seq_base = (uint32_t)c->sample.seq_base;
+  p.e2e = 1;
+  p.st = st;
+  if (out) p.out = *out;
+  return launch_verify(p, c->cfg.dtype, stream);
+}
+
+}  // namespace
+}  // namespace sjd
+
+extern "C" size_t sjd_workspace_bytes(const sjd_model_cfg *cfg) {
+  if (!cfg_valid(cfg) || (cfg->dtype != SJD_F32 && cfg->dtype != SJD_BF16)) return 0;
+  return make_layout(*cfg).total;
+}
+
+extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weights *w, void *workspace,
+                        size_t workspace_bytes) {
+  if (!out || !cfg || !w || !workspace) return SJD_ERR_BAD_ARG;
+  *out = nullptr;
+  if (!cfg_valid(cfg)) return SJD_ERR_BAD_ARG;
+  if (cfg->dtype != SJD_F32 && cfg->dtype != SJD_BF16) return SJD_ERR_UNSUPPORTED;
+  if (cfg->head_dim > 128 || cfg->max_window > 64) return SJD_ERR_UNSUPPORTED;
+  if (((uintptr_t)workspace & 255u) != 0) return SJD_ERR_BAD_ARG;
+  if (!w->tok_emb || !w->final_norm || !w->lm_head || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
+      !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down)
+    return SJD_ERR_BAD_ARG;
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (!w->attn_norm[l] || !w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->ffn_norm[l] || !w->w_gate[l] ||
+        !w->w_up[l] || !w->w_down[l])
+      return SJD_ERR_BAD_ARG;
+  const Layout lay = make_layout(*cfg);
+  if (workspace_bytes < lay.total) return SJD_ERR_CAPACITY;
+
+  sjd_ctx *c = new (std::nothrow) sjd_ctx();
+  if (!c) return SJD_ERR_BAD_ARG;
+  c->cfg = *cfg;
+  c->lay = lay;
+  c->ws = (char *)workspace;
+  c->tok_emb = w->tok_emb;
+  c->final_norm = w->final_norm;
+  c->lm_head = w->lm_head;
+  const int L = cfg->n_layers;
+  c->attn_norm.assign(w->attn_norm, w->attn_norm + L);
+  c->wq.assign(w->wq, w->wq + L);
+  c->wk.assign(w->wk, w->wk + L);
+  c->wv.assign(w->wv, w->wv + L);
+  c->wo.assign(w->wo, w->wo + L);
+  c->ffn_norm.assign(w->ffn_norm, w->ffn_norm + L);
+  c->w_gate.assign(w->w_gate, w->w_gate + L);
+  c->w_up.assign(w->w_up, w->w_up + L);
+  c->w_down.assign(w->w_down, w->w_down + L);
+  c->prefilled = false;
+  c->batch = c->prompt_len = c->window = 0;
+  c->host_step = 0;
+  c->last_stream = nullptr;
+  memset(&c->sample, 0, sizeof(c->sample));
+
+  // rotary table in double precision: (cos, sin)(pos * theta^(-2i/hd))
+  const int half = cfg->head_dim / 2;
+  std::vector<float2> table((size_t)cfg->max_seq * half);
+  for (int i = 0; i < half; ++i) {
+    const double inv_freq = pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
+    for (int pos = 0; pos < cfg->max_seq; ++pos) {
+      const double a = (double)pos * inv_freq;
+      table[(size_t)pos * half + i] = make_float2((float)cos(a), (float)sin(a));
+    }
+  }
+  cudaError_t e = cudaMemcpy(c->ws + lay.rope, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemset(c->ws + lay.counters, 0, ((size_t)cfg->max_batch + 1) * 4);
+  if (e == cudaSuccess) e = cudaMemset(c->ws + lay.status, 0, 4);
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    delete c;
+    return SJD_ERR_CUDA;
+  }
+  *out = c;
+  return SJD_OK;
+}
+
+extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int prompt_len, const sjd_sample_cfg *sample,
+                           void *cuda_stream) {
+  if (!c || !prompt || !sample || batch < 1 || prompt_len < 1) return SJD_ERR_BAD_ARG;
+  int rc = check_sample_cfg(sample, c->cfg.vocab);
+  if (rc != SJD_OK) return rc;
+  if (sample->n_generate < 0) return SJD_ERR_BAD_ARG;
+  if (batch > c->cfg.max_batch || sample->window > c->cfg.max_window) return SJD_ERR_CAPACITY;
+  if ((long)prompt_len + sample->n_generate > c->cfg.max_seq) return SJD_ERR_CAPACITY;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  c->sample = *sample;
+  c->batch = batch;
+  c->prompt_len = prompt_len;
+  c->window = sample->window;
+  c->host_step = 0;
+  c->last_stream = stream;
+  c->prefilled = false;
+  const SeqState st = c->state();
+  prefill_setup_kernel<<<batch, 128, 0, stream>>>(prompt, prompt_len, st, c->at<uint32_t>(c->lay.step),
+                                                  c->at<int32_t>(c->lay.counters), batch);
+  SJD_CHECK_LAUNCH();
+  // cache keys/values of c[0..P-1) in chunks of max_window rows per sequence
+  const int rows = c->cfg.max_window;
+  for (int c0 = 0; c0 < prompt_len - 1; c0 += rows) {
+    prefill_inputs_kernel<<<batch, 64, 0, stream>>>(prompt, prompt_len, c0, rows, st.in_tok, st.in_pos);
+    SJD_CHECK_LAUNCH();
+    rc = forward(c, rows, nullptr, stream);
+    if (rc != SJD_OK) return rc;
+  }
+  // first window: no rows to verify (w_eff = 0), the slide initialises every slot (Sec. 4.2) with the
+  // initial-window step tag and bumps the step index to 0
+  rc = run_verify(c, nullptr, stream);
+  if (rc != SJD_OK) return rc;
+  c->prefilled = true;
+  return SJD_OK;
+}
+
+extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) {
+  if (!c) return SJD_ERR_BAD_ARG;
+  if (!c->prefilled) return SJD_ERR_STATE;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  c->last_stream = stream;
+  const int cur = (int)(c->host_step & 1u);
+  int rc = forward(c, c->window, c->ws + c->lay.logits[cur], stream);
+  if (rc != SJD_OK) return rc;
+  rc = run_verify(c, out, stream);
+  if (rc != SJD_OK) return rc;
+  c->host_step += 1;
+  return SJD_OK;
+}
+
+extern "C" int sjd_get_window(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) {
+  if (!c || !out) return SJD_ERR_BAD_ARG;
+  if (!c->prefilled) return SJD_ERR_STATE;
+  get_window_kernel<<<c->batch, 64, 0, (cudaStream_t)cuda_stream>>>(c->state(), *out, c->window);
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
+
+extern "C" int sjd_peek_logits(sjd_ctx *c, void *dst, size_t bytes, void *cuda_stream) {
+  if (!c || !dst) return SJD_ERR_BAD_ARG;
+  if (!c->prefilled || c->host_step == 0) return SJD_ERR_STATE;
+  const size_t need = (size_t)c->batch * c->window * c->cfg.vocab * esize(c->cfg.dtype);
+  if (bytes < need) return SJD_ERR_CAPACITY;
+  const int last = (int)((c->host_step - 1) & 1u);
+  SJD_CUDA(cudaMemcpyAsync(dst, c->ws + c->lay.logits[last], need, cudaMemcpyDefault, (cudaStream_t)cuda_stream));
+  return SJD_OK;
+}
+
+extern "C" int sjd_last_device_status(sjd_ctx *c) {
+  if (!c) return SJD_ERR_BAD_ARG;
+  SJD_CUDA(cudaStreamSynchronize(c->last_stream));
+  int32_t status = 0;
+  SJD_CUDA(cudaMemcpy(&status, c->ws + c->lay.status, 4, cudaMemcpyDeviceToHost));
+  return status == 0 ? SJD_OK : SJD_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" void sjd_destroy(sjd_ctx *c) { delete c; }

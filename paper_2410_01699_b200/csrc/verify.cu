@@ -1,0 +1,722 @@
+// Fused verify-and-resample kernel (Sec. 4.1 Step 3, Eqs. 1-3) and the window slide of Step 4.
+//
+// One thread block per window row.  A block
+//   1. (only when the draft's law is a logits row whose statistics are not cached) stages the
+//      previous-iteration row in shared memory and computes its top-k threshold and softmax
+//      denominator;
+//   2. stages this iteration's row, finds the top-k threshold with an exact MSB-first radix select
+//      on order-preserving keys (ties at the threshold are all kept), computes the softmax
+//      denominator as per-chunk partial sums in token order;
+//   3. evaluates p(d)/q(d) against the Philox uniform (Eq. 1), draws the re-draft token from p by
+//      inverse CDF (Eq. 3) and, if the row rejected, the residual token from max(0, p - q) (Eq. 2);
+//   4. publishes a 32-byte record.  The last block of a sequence to finish (an atomic ticket, no
+//      waiting) scans the records left to right, fixes the accepted prefix and slides the window
+//      (Step 4, Sec. 4.2).
+// Logits are read once from HBM; later passes hit the shared-memory copy.  Rows too large for
+// shared memory are re-read through L2.  No floating-point atomics: every sum has a fixed order.
+#include <float.h>
+
+#include "common.cuh"
+
+namespace sjd {
+namespace {
+
+constexpr int kMaxChunks = 1024;   // 32 vectors of 16 bytes per chunk
+constexpr int kMaxThreads = 1024;
+
+// ------------------------------------------------------------------------------------ elements
+template <typename T>
+struct Elt;
+
+template <>
+struct Elt<float> {
+  static constexpr int VEC = 4;
+  static constexpr int KEYBITS = 32;
+  static constexpr uint32_t NEG_INF = 0xFF800000u;
+  __device__ static __forceinline__ uint32_t get(const uint4 &v, int t) {
+    return t == 0 ? v.x : t == 1 ? v.y : t == 2 ? v.z : v.w;
+  }
+  __device__ static __forceinline__ void set(uint4 &v, int t, uint32_t b) {
+    if (t == 0) v.x = b; else if (t == 1) v.y = b; else if (t == 2) v.z = b; else v.w = b;
+  }
+  __device__ static __forceinline__ uint32_t load_bits(const float *p) { return __float_as_uint(__ldg(p)); }
+  __device__ static __forceinline__ bool bad(uint32_t b) {
+    return (b & 0x7FFFFFFFu) > 0x7F800000u || b == 0x7F800000u;
+  }
+  __device__ static __forceinline__ uint32_t key(uint32_t b) { return (b & 0x80000000u) ? ~b : (b | 0x80000000u); }
+  __device__ static __forceinline__ uint32_t unkey(uint32_t k) { return (k & 0x80000000u) ? (k ^ 0x80000000u) : ~k; }
+  __device__ static __forceinline__ float val(uint32_t b) { return __uint_as_float(b); }
+};
+
+template <>
+struct Elt<__nv_bfloat16> {
+  static constexpr int VEC = 8;
+  static constexpr int KEYBITS = 16;
+  static constexpr uint32_t NEG_INF = 0xFF80u;
+  __device__ static __forceinline__ uint32_t word(const uint4 &v, int i) {
+    return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w;
+  }
+  __device__ static __forceinline__ uint32_t get(const uint4 &v, int t) {
+    return (word(v, t >> 1) >> ((t & 1) * 16)) & 0xFFFFu;
+  }
+  __device__ static __forceinline__ void set(uint4 &v, int t, uint32_t b) {
+    const uint32_t sh = (t & 1) * 16;
+    const uint32_t m = ~(0xFFFFu << sh);
+    const int i = t >> 1;
+    if (i == 0) v.x = (v.x & m) | (b << sh);
+    else if (i == 1) v.y = (v.y & m) | (b << sh);
+    else if (i == 2) v.z = (v.z & m) | (b << sh);
+    else v.w = (v.w & m) | (b << sh);
+  }
+  __device__ static __forceinline__ uint32_t load_bits(const __nv_bfloat16 *p) {
+    return (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(p));
+  }
+  __device__ static __forceinline__ bool bad(uint32_t b) { return (b & 0x7FFFu) > 0x7F80u || b == 0x7F80u; }
+  __device__ static __forceinline__ uint32_t key(uint32_t b) { return (b & 0x8000u) ? (~b & 0xFFFFu) : (b | 0x8000u); }
+  __device__ static __forceinline__ uint32_t unkey(uint32_t k) { return (k & 0x8000u) ? (k ^ 0x8000u) : (~k & 0xFFFFu); }
+  __device__ static __forceinline__ float val(uint32_t b) { return __uint_as_float(b << 16); }
+};
+
+// ------------------------------------------------------------------------------------ scratch
+struct Scratch {
+  double chunk_excl[kMaxChunks + 1];  // exclusive prefix of chunk sums; [NC] = total
+  float chunk_sum[kMaxChunks];
+  uint32_t hist[256];
+  uint32_t redu[32];
+  uint32_t sel_bin, count_above, bad;
+  int sel_chunk, last_chunk;
+  int tok;
+  float tok_w;
+  int is_last;
+};
+
+// A logits row seen as 16-byte vectors aligned in global memory: vector j holds elements
+// j*VEC - off .. j*VEC - off + VEC - 1; elements outside [0, V) read as -inf.
+template <typename T>
+struct Row {
+  const T *g;
+  int V, off, NV;
+  const uint4 *s;  // shared-memory copy (sanitised), or null
+
+  __device__ void init(const T *row, int v) {
+    g = row;
+    V = v;
+    off = (int)(((uintptr_t)row & 15u) / sizeof(T));
+    NV = (off + v + Elt<T>::VEC - 1) / Elt<T>::VEC;
+    s = nullptr;
+  }
+  // sanitised vector straight from global memory
+  __device__ __forceinline__ uint4 load_global(int j, uint32_t &bad) const {
+    using E = Elt<T>;
+    const int i0 = j * E::VEC - off;
+    uint4 v;
+    if (i0 >= 0 && i0 + E::VEC <= V) {
+      v = __ldg(reinterpret_cast<const uint4 *>(g + i0));
+    } else {
+      v = make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int t = 0; t < E::VEC; ++t) {
+        const int i = i0 + t;
+        E::set(v, t, (i >= 0 && i < V) ? E::load_bits(g + i) : E::NEG_INF);
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < E::VEC; ++t) {
+      if (E::bad(E::get(v, t))) {
+        E::set(v, t, E::NEG_INF);
+        bad = 1;
+      }
+    }
+    return v;
+  }
+  __device__ __forceinline__ uint4 vec(int j) const {
+    uint32_t ignore = 0;
+    return s ? s[j] : load_global(j, ignore);
+  }
+  // sanitised bits of element i (0 <= i < V)
+  __device__ __forceinline__ uint32_t element(int i) const {
+    uint32_t b = Elt<T>::load_bits(g + i);
+    return Elt<T>::bad(b) ? Elt<T>::NEG_INF : b;
+  }
+};
+
+// weight of one element under a row's statistics: exp((x - xmax)/T) inside the top-k set, else 0
+template <typename T>
+struct PWeight {
+  uint32_t tau_key;
+  float xmax, inv_t;
+  bool degenerate;  // no finite entry: all mass on token 0
+  __device__ void init(const RowStats &st, float inv_temperature) {
+    tau_key = st.tau_key;
+    xmax = st.xmax;
+    inv_t = inv_temperature;
+    degenerate = !(st.xmax > -FLT_MAX);
+  }
+  __device__ __forceinline__ float one(uint32_t bits, int idx) const {
+    if (degenerate) return idx == 0 ? 1.0f : 0.0f;
+    return Elt<T>::key(bits) >= tau_key ? expf((Elt<T>::val(bits) - xmax) * inv_t) : 0.0f;
+  }
+};
+
+template <typename T>
+struct PRowWeights {  // functor: weights of vector j of a row
+  Row<T> row;
+  PWeight<T> pw;
+  __device__ __forceinline__ void operator()(int j, float *w) const {
+    const uint4 v = row.vec(j);
+    const int i0 = j * Elt<T>::VEC - row.off;
+#pragma unroll
+    for (int t = 0; t < Elt<T>::VEC; ++t) w[t] = pw.one(Elt<T>::get(v, t), i0 + t);
+  }
+};
+
+template <typename T>
+struct ResidualWeights {  // functor: max(0, p - q) for vector j (in the p row's vector space)
+  Row<T> prow, qrow;
+  PWeight<T> pw, qw;
+  float inv_zp, inv_zq;
+  int kind, draft, V;
+  __device__ __forceinline__ void operator()(int j, float *w) const {
+    using E = Elt<T>;
+    const uint4 v = prow.vec(j);
+    const int i0 = j * E::VEC - prow.off;
+    uint4 qv = make_uint4(0, 0, 0, 0);
+    const bool qvec = (kind == SJD_Q_ROW) && (qrow.off == prow.off);
+    if (qvec) qv = qrow.vec(j);
+#pragma unroll
+    for (int t = 0; t < E::VEC; ++t) {
+      const int i = i0 + t;
+      const float p = pw.one(E::get(v, t), i) * inv_zp;
+      float q;
+      if (kind == SJD_Q_ROW) {
+        const bool in = (i >= 0 && i < V);
+        const uint32_t qb = qvec ? E::get(qv, t) : (in ? qrow.element(i) : E::NEG_INF);
+        q = qw.one(qb, i) * inv_zq;
+      } else if (kind == SJD_Q_UNIFORM) {
+        q = 1.0f / (float)V;
+      } else {
+        q = (i == draft) ? 1.0f : 0.0f;
+      }
+      w[t] = (i >= 0 && i < V) ? fmaxf(0.0f, p - q) : 0.0f;
+    }
+  }
+};
+
+// ------------------------------------------------------------------------------------ radix select
+// warp 0: locate, from the top, the histogram bin holding the `remaining`-th largest key
+__device__ void find_bin(Scratch &sc, uint32_t remaining) {
+  const int lane = threadIdx.x & 31;
+  uint32_t c[8], tot = 0;
+#pragma unroll
+  for (int b = 0; b < 8; ++b) {
+    c[b] = sc.hist[lane * 8 + b];
+    tot += c[b];
+  }
+  uint32_t incl = tot;  // sum over lanes >= lane
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_down_sync(0xffffffffu, incl, o);
+    if (lane + o < 32) incl += y;
+  }
+  const uint32_t above = incl - tot;
+  const bool hit = (above < remaining) && (remaining <= incl);
+  const uint32_t ballot = __ballot_sync(0xffffffffu, hit);
+  if (ballot == 0) {  // remaining exceeds the population: keep everything
+    if (lane == 0) {
+      sc.sel_bin = 0;
+      sc.count_above = incl - c[0];
+    }
+    return;
+  }
+  if (hit) {
+    uint32_t acc = above;
+#pragma unroll
+    for (int b = 7; b >= 0; --b) {
+      const uint32_t nxt = acc + c[b];
+      if (acc < remaining && remaining <= nxt) {
+        sc.sel_bin = lane * 8 + b;
+        sc.count_above = acc;
+      }
+      acc = nxt;
+    }
+  }
+}
+
+// Stage the row (optional), histogram the top digit, find the largest key.  Returns max key.
+template <typename T>
+__device__ uint32_t stage_first_pass(Row<T> &row, uint4 *stage, Scratch &sc, bool need_hist) {
+  using E = Elt<T>;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  for (int i = tid; i < 256; i += nt) sc.hist[i] = 0;
+  if (tid == 0) sc.bad = 0;
+  __syncthreads();
+  uint32_t kmax = 0, bad = 0;
+  for (int j0 = tid; j0 < row.NV; j0 += 4 * nt) {
+    uint4 v[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int j = j0 + r * nt;
+      if (j < row.NV) v[r] = row.load_global(j, bad);
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int j = j0 + r * nt;
+      if (j < row.NV) {
+        if (stage) stage[j] = v[r];
+#pragma unroll
+        for (int t = 0; t < E::VEC; ++t) {
+          const uint32_t k = E::key(E::get(v[r], t));
+          kmax = max(kmax, k);
+          if (need_hist) atomicAdd(&sc.hist[k >> (E::KEYBITS - 8)], 1u);
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+  if ((tid & 31) == 0) sc.redu[tid >> 5] = kmax;
+  if (bad) sc.bad = 1;
+  __syncthreads();
+  if (stage) row.s = stage;
+  kmax = 0;
+  for (int w = 0; w < (nt >> 5); ++w) kmax = max(kmax, sc.redu[w]);
+  return kmax;
+}
+
+// Exact key of the top_k-th largest element (histogram of digit 0 already in sc.hist).
+template <typename T>
+__device__ uint32_t select_threshold(const Row<T> &row, Scratch &sc, uint32_t top_k) {
+  using E = Elt<T>;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  uint32_t prefix = 0, remaining = top_k;
+  constexpr int PASSES = E::KEYBITS / 8;
+  for (int pass = 0; pass < PASSES; ++pass) {
+    const int shift = E::KEYBITS - 8 * (pass + 1);
+    if (pass > 0) {
+      for (int i = tid; i < 256; i += nt) sc.hist[i] = 0;
+      __syncthreads();
+      const uint32_t hi_mask_shift = shift + 8;
+      for (int j = tid; j < row.NV; j += nt) {
+        const uint4 v = row.vec(j);
+#pragma unroll
+        for (int t = 0; t < E::VEC; ++t) {
+          const uint32_t k = E::key(E::get(v, t));
+          if ((k >> hi_mask_shift) == (prefix >> hi_mask_shift)) atomicAdd(&sc.hist[(k >> shift) & 255u], 1u);
+        }
+      }
+      __syncthreads();
+    }
+    if (tid < 32) find_bin(sc, remaining);
+    __syncthreads();
+    prefix |= sc.sel_bin << shift;
+    remaining -= sc.count_above;
+    __syncthreads();
+  }
+  return prefix;
+}
+
+// ------------------------------------------------------------------------------------ sums & sampling
+// Per-chunk sums of the functor's weights in token order, then their exclusive prefix in fp64.
+template <int VEC, typename F>
+__device__ void chunk_sums(const F &f, int NV, Scratch &sc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+  const int NC = (NV + 31) >> 5;
+  for (int c = warp; c < NC; c += nw) {
+    const int j = c * 32 + lane;
+    float s = 0.0f;
+    if (j < NV) {
+      float w[VEC];
+      f(j, w);
+#pragma unroll
+      for (int t = 0; t < VEC; ++t) s += w[t];
+    }
+    float incl = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (lane == 31) sc.chunk_sum[c] = incl;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int per = (NC + 31) >> 5;
+    const int lo = min(NC, lane * per), hi = min(NC, lo + per);
+    double loc = 0.0;
+    for (int c = lo; c < hi; ++c) loc += (double)sc.chunk_sum[c];
+    double incl = loc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const double y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    double run = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (lane == 0) run = 0.0;
+    for (int c = lo; c < hi; ++c) {
+      sc.chunk_excl[c] = run;
+      run += (double)sc.chunk_sum[c];
+    }
+    if (lane == 31) sc.chunk_excl[NC] = incl;
+  }
+  __syncthreads();
+}
+
+// Inverse CDF in token order over the functor's weights (chunk_sums must have run with the same
+// functor): smallest index i with w_i > 0 and cumsum_i > u * total.  Result in sc.tok / sc.tok_w.
+template <int VEC, typename F>
+__device__ void sample_icdf(const F &f, int NV, int off, Scratch &sc, float u) {
+  const int tid = threadIdx.x, lane = tid & 31, nt = blockDim.x;
+  const int NC = (NV + 31) >> 5;
+  const double total = sc.chunk_excl[NC];
+  const double target = (double)u * total;
+  if (tid == 0) {
+    sc.sel_chunk = 0x7fffffff;
+    sc.last_chunk = -1;
+    sc.tok = 0;
+    sc.tok_w = 0.0f;
+  }
+  __syncthreads();
+  for (int c = tid; c < NC; c += nt) {
+    if (sc.chunk_sum[c] > 0.0f) {
+      atomicMax(&sc.last_chunk, c);
+      if (sc.chunk_excl[c] <= target && target < sc.chunk_excl[c + 1]) atomicMin(&sc.sel_chunk, c);
+    }
+  }
+  __syncthreads();
+  if (tid < 32) {
+    int c = sc.sel_chunk;
+    const bool fallback = (c == 0x7fffffff);
+    if (fallback) c = sc.last_chunk;
+    if (c >= 0) {
+      const int j = c * 32 + lane;
+      float w[VEC];
+      float s = 0.0f;
+#pragma unroll
+      for (int t = 0; t < VEC; ++t) w[t] = 0.0f;
+      if (j < NV) {
+        f(j, w);
+#pragma unroll
+        for (int t = 0; t < VEC; ++t) s += w[t];
+      }
+      float incl = s;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+      if (lane == 0) excl = 0.0f;
+      const double base = sc.chunk_excl[c];
+      const bool cond = !fallback && (base + (double)incl > target);
+      const uint32_t ballot = __ballot_sync(0xffffffffu, cond);
+      const uint32_t pos = __ballot_sync(0xffffffffu, s > 0.0f);
+      int sel_lane;
+      bool take_last = false;
+      if (ballot != 0) {
+        sel_lane = __ffs(ballot) - 1;
+      } else {
+        sel_lane = 31 - __clz(pos);  // pos != 0 because the chunk sum is positive
+        take_last = true;
+      }
+      if (lane == sel_lane) {
+        double acc = base + (double)excl;
+        int found = -1, last = -1;
+#pragma unroll
+        for (int t = 0; t < VEC; ++t) {
+          if (w[t] > 0.0f) {
+            acc += (double)w[t];
+            last = t;
+            if (found < 0 && !take_last && acc > target) found = t;
+          }
+        }
+        const int t_sel = found >= 0 ? found : last;
+        float wsel = 0.0f;
+#pragma unroll
+        for (int t = 0; t < VEC; ++t)
+          if (t == t_sel) wsel = w[t];
+        sc.tok = j * VEC + t_sel - off;
+        sc.tok_w = wsel;
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// Threshold + denominator of one row; leaves chunk sums of the row's weights in the scratch.
+template <typename T>
+__device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t,
+                                   PRowWeights<T> &f) {
+  using E = Elt<T>;
+  const bool need_select = top_k < row.V;
+  const uint32_t kmax = stage_first_pass<T>(row, stage, sc, need_select);
+  RowStats st;
+  st.flags = sc.bad ? SJD_FLAG_NONFINITE : 0u;
+  st.tau_key = need_select ? select_threshold<T>(row, sc, (uint32_t)top_k) : 0u;
+  st.xmax = E::val(E::unkey(kmax));
+  f.row = row;
+  f.pw.init(st, inv_t);
+  chunk_sums<E::VEC>(f, row.NV, sc);
+  st.z = (float)sc.chunk_excl[(row.NV + 31) >> 5];
+  return st;
+}
+
+// ------------------------------------------------------------------------------------ finalize
+__device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step) {
+  const int W = p.W;
+  const int w_eff = p.w_eff ? p.w_eff[b] : W;
+  const RowOut *ro = p.row_out + (size_t)b * W;
+  const int32_t *old_draft = p.draft + (size_t)b * W;
+  const sjd_step_out &o = p.out;
+  uint32_t flags = 0;
+  int a = w_eff;
+  for (int k = 0; k < w_eff; ++k) {
+    const uint32_t rf = __ldcg(&ro[k].flags);
+    flags |= rf & SJD_FLAG_NONFINITE;
+    if (a == w_eff) {
+      flags |= rf & SJD_FLAG_NEAR_TIE_ACCEPT;
+      if (!__ldcg(&ro[k].accept)) {
+        a = k;
+        flags |= rf & SJD_FLAG_RESIDUAL_EMPTY;
+      }
+    }
+  }
+  const int m = (a < w_eff) ? a + 1 : w_eff;
+  const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
+  const int n2 = base + m;
+
+  // fixed tokens: accepted drafts, then the resampled one
+  for (int i = 0; i < W; ++i) {
+    int tok = -1;
+    if (i < a) tok = old_draft[i];
+    else if (i == a && a < w_eff) tok = __ldcg(&ro[a].resample_tok);
+    if (o.committed) o.committed[(size_t)b * W + i] = tok;
+    if (p.e2e && i < m) p.st.committed[(size_t)b * p.st.max_seq + base + i] = tok;
+  }
+
+  int w2 = 0, kept = 0;
+  if (p.e2e) {
+    const int total = p.st.prompt_len + p.st.n_generate;
+    w2 = max(0, min(W, total - n2));
+    kept = (a < w_eff) ? min(w_eff - a - 1, w2) : 0;
+    if (n2 >= total) flags |= SJD_FLAG_DONE;
+  } else {
+    kept = (a < w_eff) ? (w_eff - a - 1) : 0;
+    w2 = kept;
+  }
+  int32_t *nd = p.e2e ? p.st.draft + (size_t)b * W : nullptr;
+  int32_t *nk = p.e2e ? p.st.q_kind + (size_t)b * W : nullptr;
+  int32_t *nr = p.e2e ? p.st.q_row + (size_t)b * W : nullptr;
+  float *nq = p.e2e ? p.st.q_draft + (size_t)b * W : nullptr;
+  for (int s = 0; s < W; ++s) {
+    int tok = -1, kind = -1, qrow = 0;
+    float q = 0.0f;
+    if (s < kept) {
+      const int k = a + 1 + s;
+      tok = __ldcg(&ro[k].redraft_tok);
+      q = __ldcg(&ro[k].redraft_p);
+      kind = SJD_Q_ROW;
+      qrow = k;
+    } else if (s < w2) {  // freshly initialised slot (end-to-end mode only), Sec. 4.2
+      const int t_pos = n2 + s;
+      const int stride = p.st.init == SJD_INIT_COPY_ABOVE ? p.st.grid_stride
+                         : p.st.init == SJD_INIT_COPY_LEFT ? 1 : 0;
+      const int src = t_pos - stride;
+      if (p.st.init != SJD_INIT_RANDOM && stride > 0 && src >= p.st.prompt_len) {
+        tok = src < n2 ? p.st.committed[(size_t)b * p.st.max_seq + src] : nd[src - n2];
+        kind = SJD_Q_ONEHOT;
+        q = 1.0f;
+      } else {
+        const Philox4 r = philox4x32_10((uint32_t)t_pos, step, p.seq_base + (uint32_t)b, kStreamInit,
+                                        p.seed_lo, p.seed_hi);
+        tok = (int)(((uint64_t)r.w[0] * (uint64_t)p.V) >> 32);
+        kind = SJD_Q_UNIFORM;
+        q = 1.0f / (float)p.V;
+      }
+    }
+    if (p.e2e) {
+      nd[s] = tok;
+      nk[s] = kind;
+      nr[s] = qrow;
+      nq[s] = q;
+    }
+    if (o.draft) o.draft[(size_t)b * W + s] = tok;
+    if (o.q_kind) o.q_kind[(size_t)b * W + s] = kind;
+    if (o.q_draft) o.q_draft[(size_t)b * W + s] = q;
+  }
+  if (p.e2e) {
+    p.st.n[b] = n2;
+    p.st.w_eff[b] = w2;
+    int32_t *it = p.st.in_tok + (size_t)b * W;
+    int32_t *ip = p.st.in_pos + (size_t)b * W;
+    for (int k = 0; k < W; ++k) {
+      const bool act = k < w2;
+      it[k] = act ? (k == 0 ? p.st.committed[(size_t)b * p.st.max_seq + n2 - 1] : nd[k - 1]) : 0;
+      ip[k] = act ? n2 - 1 + k : -1;
+    }
+  }
+  if (o.n_accepted) o.n_accepted[b] = a;
+  if (o.n_committed) o.n_committed[b] = m;
+  if (o.total_committed) o.total_committed[b] = n2;
+  if (o.flags) o.flags[b] = flags;
+}
+
+// ------------------------------------------------------------------------------------ kernel
+template <typename T>
+__global__ void __launch_bounds__(kMaxThreads) verify_rows_kernel(const VerifyParams p) {
+  using E = Elt<T>;
+  extern __shared__ uint4 dyn_smem[];
+  __shared__ Scratch sc;
+  uint4 *stage = p.staged ? dyn_smem : nullptr;
+
+  const int r = blockIdx.x;
+  const int b = r / p.W, k = r % p.W;
+  const int tid = threadIdx.x;
+  const int w_eff = p.w_eff ? p.w_eff[b] : p.W;
+  const uint32_t step = p.step_ptr ? *p.step_ptr : p.step;
+  const int cur = p.step_ptr ? (int)(step & 1u) : 0;
+  const float inv_t = 1.0f / p.temperature;
+
+  if (k < w_eff) {
+    const int kind = p.q_kind ? p.q_kind[r] : SJD_Q_ROW;
+    const int d = p.draft[r];
+    const bool d_ok = d >= 0 && d < p.V;
+    const int qr = p.q_row ? p.q_row[r] : k;
+    const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
+    const Philox4 rnd = philox4x32_10((uint32_t)(base + k), step, p.seq_base + (uint32_t)b, kStreamVerify,
+                                      p.seed_lo, p.seed_hi);
+    const float u_acc = u24(rnd.w[0]), u_res = u24(rnd.w[1]), u_draft = u24(rnd.w[2]);
+
+    const T *qbase = reinterpret_cast<const T *>(p.logits[cur ^ 1]) + ((size_t)b * p.W + qr) * p.V;
+    const T *pbase = reinterpret_cast<const T *>(p.logits[cur]) + (size_t)r * p.V;
+
+    // ---- the law of the draft
+    Row<T> qrow;
+    qrow.init(qbase, p.V);
+    RowStats qs;
+    qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
+    PRowWeights<T> qf;
+    float q_d;
+    if (kind == SJD_Q_ROW) {
+      if (p.prev_stats_valid) {
+        qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
+      } else {
+        qs = row_statistics<T>(qrow, stage, sc, p.top_k, inv_t, qf);
+        if (tid == 0) p.stats[cur ^ 1][r] = qs;
+        __syncthreads();
+        qrow.s = nullptr;  // the staging buffer is about to be reused
+      }
+      qf.row = qrow;
+      qf.pw.init(qs, inv_t);
+      q_d = d_ok ? qf.pw.one(qrow.element(d), d) / qs.z : 1.0f;
+    } else if (kind == SJD_Q_UNIFORM) {
+      q_d = 1.0f / (float)p.V;
+    } else {
+      q_d = 1.0f;
+    }
+
+    // ---- this iteration's distribution
+    Row<T> prow;
+    prow.init(pbase, p.V);
+    PRowWeights<T> pf;
+    const RowStats ps = row_statistics<T>(prow, stage, sc, p.top_k, inv_t, pf);
+    if (tid == 0) p.stats[cur][r] = ps;
+    const float p_d = d_ok ? pf.pw.one(prow.element(d), d) / ps.z : 0.0f;
+
+    // ---- Eq. 1
+    float ratio;
+    if (q_d > 0.0f) ratio = p_d / q_d;
+    else ratio = p_d > 0.0f ? INFINITY : 0.0f;
+    const float thr = fminf(1.0f, ratio);
+    const bool accept = u_acc < thr;
+    uint32_t flags = ps.flags | (kind == SJD_Q_ROW ? qs.flags : 0u);
+    if (thr < 1.0f && fabsf(u_acc - thr) < 1e-4f) flags |= SJD_FLAG_NEAR_TIE_ACCEPT;
+
+    // ---- Eq. 3: re-draft from p (used if an earlier row rejects)
+    sample_icdf<E::VEC>(pf, prow.NV, prow.off, sc, u_draft);
+    const int redraft_tok = sc.tok;
+    const float redraft_p = sc.tok_w / ps.z;
+    __syncthreads();
+
+    // ---- Eq. 2: residual resample (used if this is the first rejected row)
+    int resample_tok = -1;
+    if (!accept) {
+      ResidualWeights<T> rf;
+      rf.prow = prow; rf.qrow = qrow; rf.pw = pf.pw; rf.qw = qf.pw;
+      rf.inv_zp = 1.0f / ps.z; rf.inv_zq = 1.0f / qs.z;
+      rf.kind = kind; rf.draft = d; rf.V = p.V;
+      if (kind != SJD_Q_ROW) rf.qw = pf.pw;
+      chunk_sums<E::VEC>(rf, prow.NV, sc);
+      if (sc.chunk_excl[(prow.NV + 31) >> 5] > 0.0) {
+        sample_icdf<E::VEC>(rf, prow.NV, prow.off, sc, u_res);
+      } else {
+        flags |= SJD_FLAG_RESIDUAL_EMPTY;
+        __syncthreads();
+        chunk_sums<E::VEC>(pf, prow.NV, sc);
+        sample_icdf<E::VEC>(pf, prow.NV, prow.off, sc, u_res);
+      }
+      resample_tok = sc.tok;
+    }
+    if (tid == 0) {
+      RowOut ro;
+      ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
+      ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok; ro.flags = flags;
+      p.row_out[r] = ro;
+    }
+  }
+
+  // ---- ticket: the last block of the sequence slides the window
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    const int old = atomicAdd(&p.seq_counter[b], 1);
+    sc.is_last = (old == p.W - 1);
+    if (sc.is_last) {
+      __threadfence();
+      finalize_sequence(p, b, step);
+      p.seq_counter[b] = 0;
+      __threadfence();
+      const int done = atomicAdd(p.done_counter, 1);
+      if (done == p.B - 1) {  // every block has read the step index by now
+        *p.done_counter = 0;
+        if (p.step_ptr) *p.step_ptr = step + 1u;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+size_t verify_scratch_bytes(int batch, int window) {
+  if (batch <= 0 || window <= 0) return 0;
+  const size_t rows = (size_t)batch * window;
+  size_t b = 0;
+  b += 2 * rows * sizeof(RowStats);
+  b += rows * sizeof(RowOut);
+  b += ((size_t)batch + 1) * sizeof(int32_t);
+  return (b + 255) / 256 * 256;
+}
+
+template <typename T>
+static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
+  VerifyParams p = p_in;
+  constexpr int VEC = Elt<T>::VEC;
+  const long nv_max = ((long)p.V + 2 * VEC - 2) / VEC + 1;
+  if ((nv_max + 31) / 32 > kMaxChunks) return SJD_ERR_CAPACITY;
+  const size_t stage_bytes = (size_t)nv_max * 16;
+  p.staged = stage_bytes <= 160 * 1024 ? 1 : 0;
+  const size_t dyn = p.staged ? stage_bytes : 0;
+  int threads = nv_max <= 1024 ? 128 : nv_max <= 4096 ? 256 : nv_max <= 16384 ? 512 : 1024;
+  if (dyn > 48 * 1024)
+    SJD_CUDA(cudaFuncSetAttribute(verify_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+  verify_rows_kernel<T><<<p.B * p.W, threads, dyn, stream>>>(p);
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
+
+int launch_verify(const VerifyParams &p, int dtype, cudaStream_t stream) {
+  if (dtype == SJD_F32) return launch_verify_t<float>(p, stream);
+  if (dtype == SJD_BF16) return launch_verify_t<__nv_bfloat16>(p, stream);
+  return SJD_ERR_UNSUPPORTED;
+}
+
+}  // namespace sjd

@@ -1,0 +1,146 @@
+"""GPU parity of sjd_init / sjd_prefill / sjd_step (through the C-ABI) against the CPU checker in
+lock-step: before every step the checker holds the library's state; it recomputes the logits
+itself (compared within the storage-dtype tolerance) and re-takes every decision of the step from
+the library's stored logits (compared exactly, near-ties flagged)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.sjd import INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, SampleCfg
+from paper_2410_01699_b200 import binding as B
+from paper_2410_01699_b200.inputs import WORKLOADS, make_prompt, make_weights
+from tests.parity_util import LockStepSequence
+
+pytestmark = pytest.mark.gpu
+
+LOGIT_TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+def run_lockstep(wl, batch=1, max_steps=None, init=INIT_RANDOM, check_logits_every=1, gain_jitter=0.1, window=None,
+                 n_generate=None, seq_base=0, top_k=None):
+    window = window or wl.window
+    n_generate = wl.n_generate if n_generate is None else n_generate
+    top_k = top_k or wl.top_k
+    weights = make_weights(wl, gain_jitter=gain_jitter)
+    prompt = make_prompt(wl, batch)
+    cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=wl.prompt_len + n_generate + 8, max_window=window)
+    ctx = B.Context(cfg, B.weights_to_device(weights))
+    sample = B.make_sample_cfg(temperature=wl.temperature, top_k=top_k, seed=wl.philox_seed, window=window,
+                               init=init, grid_stride=wl.grid_stride, n_generate=n_generate, seq_base=seq_base)
+    scfg = SampleCfg(temperature=wl.temperature, top_k=top_k, seed=wl.philox_seed, window=window, init=init,
+                     grid_stride=wl.grid_stride, n_generate=n_generate, logits_dtype=wl.dtype)
+    ctx.prefill(torch.from_numpy(prompt).cuda(), sample)
+    out = B.StepOut(batch, window)
+    ctx.get_window(out)
+    h = out.host()
+    seqs = [LockStepSequence(wl, weights, prompt[b], scfg, seq_base + b, LOGIT_TOL[wl.dtype]) for b in range(batch)]
+    for b, s in enumerate(seqs):
+        s.check_window(h["draft"][b], h["q_kind"][b], h["q_draft"][b], h["total_committed"][b])
+    steps = 0
+    total = wl.prompt_len + n_generate
+    committed = [list(prompt[b]) for b in range(batch)]
+    while any(s.st.n < total for s in seqs):
+        ctx.step(out)
+        logits = ctx.peek_logits().to(torch.float64).cpu().numpy()
+        h = out.host()
+        for b, s in enumerate(seqs):
+            ob = {k: v[b] for k, v in h.items()}
+            s.step(logits[b], ob, check_logits=(steps % check_logits_every == 0))
+            committed[b] += [int(t) for t in ob["committed"][:int(ob["n_committed"])]]
+            assert committed[b] == s.st.committed
+        steps += 1
+        assert steps <= n_generate, "more forward passes than tokens"
+        if max_steps and steps >= max_steps:
+            break
+    assert ctx.device_status() == B.SJD_OK
+    return ctx, seqs, steps, out
+
+
+def test_tiny_fp32_full_generation():
+    """The tiny fp32 configuration end to end: 256 tokens, W = 16, top-k 64, random initialisation."""
+    wl = WORKLOADS["tiny"]
+    ctx, seqs, steps, out = run_lockstep(wl)
+    s = seqs[0]
+    assert s.st.n == wl.prompt_len + wl.n_generate
+    assert steps <= wl.n_generate
+    assert s.max_logit_err <= 1e-4
+    assert s.stats.flagged <= max(3, 0.02 * s.stats.decisions), s.stats
+    # a finished sequence: further steps fix nothing and say so
+    ctx.step(out)
+    h = out.host()
+    assert h["n_committed"][0] == 0 and h["flags"][0] & B.SJD_FLAG_DONE
+    assert h["total_committed"][0] == wl.prompt_len + wl.n_generate
+
+
+@pytest.mark.parametrize("init", [INIT_COPY_ABOVE, INIT_COPY_LEFT])
+def test_tiny_spatial_initialisation(init):
+    wl = WORKLOADS["tiny"]
+    run_lockstep(wl, init=init, n_generate=100)
+
+
+def test_tiny_batch_of_three_and_ragged_window():
+    """Independent sequences in one batch; window 11 does not divide anything; sequence ids offset."""
+    wl = WORKLOADS["tiny"]
+    ctx, seqs, steps, _ = run_lockstep(wl, batch=3, window=11, n_generate=61, seq_base=5)
+    assert all(s.st.n == wl.prompt_len + 61 for s in seqs)
+
+
+def test_tiny_window_of_one_is_ordinary_sampling():
+    wl = WORKLOADS["tiny"]
+    ctx, seqs, steps, _ = run_lockstep(wl, window=1, n_generate=24)
+    assert steps == 24
+
+
+def test_tiny_top1_is_greedy_decoding():
+    from oracle.model import OracleModel
+    from oracle.sjd import CachedModel, greedy_ar_generate
+    from tests.parity_util import oracle_model_cfg
+    wl = WORKLOADS["tiny"]
+    ctx, seqs, steps, _ = run_lockstep(wl, n_generate=48, top_k=1, gain_jitter=0.0)
+    weights = make_weights(wl)
+    greedy = greedy_ar_generate(list(make_prompt(wl)[0]),
+                                CachedModel(OracleModel(oracle_model_cfg(wl), weights), 80), 48)
+    assert seqs[0].st.committed[wl.prompt_len:] == greedy
+    assert steps <= 48
+
+
+def test_small_bf16_gqa_generation():
+    """bf16 storage, grouped-query attention, sizes that are not multiples of the tile sizes."""
+    wl = WORKLOADS["small-bf16"]
+    ctx, seqs, steps, _ = run_lockstep(wl, batch=2)
+    for s in seqs:
+        assert s.max_logit_err <= 2e-2
+        assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
+
+
+@pytest.mark.parametrize("name,steps", [("7b-2l", 4), ("8b-gqa-2l", 3)])
+def test_large_shapes_two_layers(name, steps):
+    """The 7B / 8B-GQA layer shapes (d 4096, SwiGLU 11008 / 14336, vocab 65536 / 184320, W 32 / 64,
+    top-k 2000 / 2048) at two layers, a few lock-step steps."""
+    wl = WORKLOADS[name]
+    ctx, seqs, n, _ = run_lockstep(wl, max_steps=steps, gain_jitter=0.0)
+    assert seqs[0].max_logit_err <= 2e-2
+
+
+def test_api_errors_and_state():
+    wl = WORKLOADS["tiny"]
+    weights = B.weights_to_device(make_weights(wl))
+    cfg = B.make_model_cfg(wl, max_batch=2, max_seq=64, max_window=8)
+    ctx = B.Context(cfg, weights)
+    with pytest.raises(B.SJDError) as e:
+        ctx.step(None)
+    assert e.value.status == B.SJD_ERR_STATE
+    prompt = torch.from_numpy(make_prompt(wl, 2)).cuda()
+    for kw, status in [(dict(window=9), B.SJD_ERR_CAPACITY), (dict(n_generate=60), B.SJD_ERR_CAPACITY),
+                       (dict(temperature=0.0), B.SJD_ERR_BAD_ARG), (dict(top_k=0), B.SJD_ERR_BAD_ARG),
+                       (dict(init=1, grid_stride=0), B.SJD_ERR_BAD_ARG)]:
+        args = dict(top_k=10, window=8, n_generate=20)
+        args.update(kw)
+        with pytest.raises(B.SJDError) as e:
+            ctx.prefill(prompt, B.make_sample_cfg(**args))
+        assert e.value.status == status, kw
+    bad = B.make_model_cfg(wl, max_batch=0, max_seq=64, max_window=8)
+    assert B.sjd_workspace_bytes(bad) == 0
+    with pytest.raises(B.SJDError):
+        B.Context(B.make_model_cfg(wl.with_(head_dim=63), 1, 64, 8), weights)
+    torch.cuda.synchronize()

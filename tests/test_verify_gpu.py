@@ -1,0 +1,152 @@
+"""GPU parity of the fused verify-and-resample kernel (sjd_verify through the C-ABI) against the
+CPU checker, element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2410_01699_b200 import binding as B
+from paper_2410_01699_b200.inputs import make_verify_case, round_bf16
+from tests.parity_util import ParityStats, compare_window, oracle_verify_case
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_gpu(case, logits_prev=True):
+    dt = torch.bfloat16 if case.dtype == "bf16" else torch.float32
+    cur = torch.from_numpy(case.logits_cur).to("cuda").to(dt)
+    prev = torch.from_numpy(case.logits_prev).to("cuda").to(dt) if logits_prev else None
+    draft = torch.from_numpy(case.draft).cuda()
+    kind = torch.from_numpy(case.q_kind.astype(np.int32)).cuda()
+    base = torch.from_numpy(case.base_pos).cuda()
+    out = B.StepOut(case.batch, case.window)
+    sample = B.make_sample_cfg(temperature=case.temperature, top_k=case.top_k, seed=case.seed, window=case.window)
+    B.sjd_verify(cur, prev, draft, kind, base, sample, case.step, out)
+    return out.host()
+
+
+def _check_case(case, prob_tol=1e-5, max_flag_frac=0.03):
+    got = _run_gpu(case)
+    stats = ParityStats()
+    for b in range(case.batch):
+        vr, qdescs = oracle_verify_case(case, b)
+        gpu = dict(n_accepted=got["n_accepted"][b], committed=got["committed"][b], draft=got["draft"][b],
+                   q_draft=got["q_draft"][b])
+        st = compare_window(vr, gpu, case.logits_cur[b].astype(np.float64), case.draft[b], qdescs, case.temperature,
+                            case.top_k, prob_tol, where=f"seq {b}")
+        stats.merge(st)
+        if st.skipped_sequences == 0:
+            assert got["n_committed"][b] == len(vr.committed)
+            assert got["total_committed"][b] == case.base_pos[b] + len(vr.committed)
+            kept = len(vr.redraft)
+            assert list(got["q_kind"][b][:kept]) == [B.SJD_Q_ROW] * kept
+            assert all(x == -1 for x in got["draft"][b][kept:]) and all(x == -1 for x in got["q_kind"][b][kept:])
+    assert stats.flagged <= max(2, max_flag_frac * stats.decisions), f"too many near-ties: {stats}"
+    return stats
+
+
+@pytest.mark.parametrize("batch", [1, 4])
+def test_verify_workload_shape(batch):
+    """The isolated-verification workload: W = 32 rows over a 16384 vocabulary, bf16, top-k 2000."""
+    _check_case(make_verify_case(batch))
+
+
+def test_verify_full_batch_sampled():
+    """Largest batch of the workload in the launch configuration the benchmark times; the checker
+    re-computes a sample of the sequences one by one."""
+    case = make_verify_case(32)
+    got = _run_gpu(case)
+    stats = ParityStats()
+    for b in (0, 7, 19, 31):
+        vr, qdescs = oracle_verify_case(case, b)
+        gpu = dict(n_accepted=got["n_accepted"][b], committed=got["committed"][b], draft=got["draft"][b],
+                   q_draft=got["q_draft"][b])
+        stats.merge(compare_window(vr, gpu, case.logits_cur[b].astype(np.float64), case.draft[b], qdescs,
+                                   case.temperature, case.top_k, 1e-5, where=f"seq {b}"))
+    # properties that hold for every sequence
+    assert np.all(got["n_committed"] >= 1) and np.all(got["n_committed"] <= 32)
+    assert np.all((got["n_committed"] == got["n_accepted"] + 1) | (got["n_accepted"] == 32))
+    for b in range(32):
+        a = got["n_accepted"][b]
+        assert list(got["committed"][b][:a]) == list(case.draft[b][:a])
+    assert stats.flagged <= 3
+
+
+@pytest.mark.parametrize("dtype,vocab,window,top_k", [
+    ("bf16", 16001, 29, 2000),   # ragged: rows not 16-byte aligned, odd window
+    ("f32", 1024, 16, 64),       # the tiny end-to-end model's head
+    ("f32", 1000, 7, 1000),      # top_k == V: no filtering
+    ("bf16", 4099, 5, 1),        # top-1
+    ("bf16", 65536, 4, 2000),    # 128 KB rows (the 7B head)
+    ("bf16", 184320, 2, 2048),   # rows larger than shared memory
+    ("f32", 50000, 3, 500),      # fp32 rows beyond the staging buffer
+])
+def test_verify_shapes(dtype, vocab, window, top_k):
+    case = make_verify_case(2, window=window, vocab=vocab, dtype=dtype, top_k=top_k, seed=7 + vocab)
+    _check_case(case, max_flag_frac=0.06)
+
+
+def test_verify_mixed_laws():
+    """Slots whose draft came from a uniform initialisation (q = 1/V) or a copy (point mass)."""
+    case = make_verify_case(6, window=16, vocab=4096, top_k=300, seed=11, mixed_kinds=True)
+    _check_case(case)
+
+
+def test_verify_temperature_and_ties():
+    case = make_verify_case(3, window=8, vocab=8192, top_k=500, temperature=0.7, seed=5)
+    _check_case(case)
+    # coarse logits: many exact ties at the top-k threshold (all must be kept)
+    case = make_verify_case(3, window=8, vocab=8192, top_k=500, seed=6)
+    case.logits_cur = round_bf16(np.round(case.logits_cur * 2) / 2)
+    case.logits_prev = round_bf16(np.round(case.logits_prev * 2) / 2)
+    _check_case(case)
+
+
+def test_verify_identical_rows_accept_everything():
+    """p == q bit for bit: every ratio is 1 and every draft is accepted for any uniform."""
+    case = make_verify_case(2, window=12, vocab=4096, top_k=100, seed=3)
+    case.logits_prev = case.logits_cur.copy()
+    got = _run_gpu(case)
+    assert list(got["n_accepted"]) == [12, 12] and list(got["n_committed"]) == [12, 12]
+    assert np.array_equal(got["committed"], case.draft)
+    assert np.all(got["draft"] == -1)
+
+
+def test_verify_nonfinite_rows_are_flagged():
+    case = make_verify_case(2, window=4, vocab=2048, top_k=50, seed=9)
+    case.logits_cur[0, 1, 5] = np.nan
+    case.logits_cur[0, 1, 9] = np.inf
+    got = _check_and_flags(case)
+    assert got["flags"][0] & B.SJD_FLAG_NONFINITE
+    assert not (got["flags"][1] & B.SJD_FLAG_NONFINITE)
+
+
+def _check_and_flags(case):
+    _check_case(case)
+    return _run_gpu(case)
+
+
+def test_verify_is_deterministic():
+    case = make_verify_case(4, window=16, vocab=16384, seed=21)
+    a, b = _run_gpu(case), _run_gpu(case)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+
+
+def test_verify_argument_errors():
+    out = B.StepOut(1, 4)
+    s = B.make_sample_cfg(top_k=10, window=4)
+    cur = torch.zeros(1, 4, 128, device="cuda")
+    d = torch.zeros(1, 4, dtype=torch.int32, device="cuda")
+    ws = torch.empty(B.sjd_verify_workspace_bytes(1, 4), dtype=torch.uint8, device="cuda")
+    L = B.lib()
+    import ctypes as C
+    args = lambda **kw: [kw.get("b", 1), kw.get("w", 4), 128, kw.get("dt", 0), C.c_void_p(cur.data_ptr()),
+                         C.c_void_p(cur.data_ptr()), C.c_void_p(d.data_ptr()), None, None, C.byref(kw.get("s", s)), 0,
+                         C.byref(out.c), C.c_void_p(ws.data_ptr()), kw.get("n", ws.numel()), None]
+    assert L.sjd_verify(*args()) == B.SJD_OK
+    assert L.sjd_verify(*args(b=0)) == B.SJD_ERR_BAD_ARG
+    assert L.sjd_verify(*args(dt=5)) == B.SJD_ERR_UNSUPPORTED
+    assert L.sjd_verify(*args(n=16)) == B.SJD_ERR_CAPACITY
+    assert L.sjd_verify(*args(s=B.make_sample_cfg(temperature=0.0, top_k=10))) == B.SJD_ERR_BAD_ARG
+    assert L.sjd_verify(*args(s=B.make_sample_cfg(top_k=0))) == B.SJD_ERR_BAD_ARG
+    torch.cuda.synchronize()
