@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the SJD hot path: committed image tokens per second.
+
+One "step" = one SJD iteration (window forward pass against the KV cache, fused verify-and-resample,
+window slide) of the 7B-shaped decoder (32 layers, d 4096, 32 heads, SwiGLU 11008, vocab 65536, bf16,
+random init), batch 1, W = 32, top-k 2000, prompt 64.  Inputs are synthetic and seeded.
+
+  python bench.py --gpus N --steps K --warmup W            # this library (N > 1: under torchrun)
+  python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
+
+Prints ONE JSON line.  `value` is device-timed with everything resident in HBM; `e2e` goes through the
+C-ABI with pinned host buffers for the prompt (copied in) and the step results (written out) and a
+host read of the results every step; `roofline` is the weight-streaming GEMM (the dominant kernel)
+against the measured HBM copy bandwidth; `cpu_baseline` is the oracle timed on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "committed_image_tokens_per_sec"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["source"] = "measured"
+        return d
+    return dict(FALLBACK_PEAKS)
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            parts = [p.strip() for p in s.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle on the host cores (reference arm and cpu_baseline leg)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(wl, steps: int, warmup: int, tokens_per_step: float | None):
+    """Times oracle SJD iterations on a bounded sample of the workload: the same window (W rows
+    against the pre-filled prompt) through ONE of the n_layers decoder layers plus the lm_head and
+    the full verification, then scales the time by streamed-parameter count to the full depth."""
+    import numpy as np
+    import torch
+
+    from oracle.model import OracleModel
+    from oracle.sjd import CachedModel, SampleCfg, sjd_begin, sjd_step
+    from paper_2410_01699_b200.inputs import make_prompt, make_weights
+    from tests.parity_util import oracle_model_cfg
+
+    cores = len(os.sched_getaffinity(0))
+    torch.set_num_threads(cores)
+    sample_wl = wl.with_(n_layers=1)
+    weights = make_weights(sample_wl)
+    model = CachedModel(OracleModel(oracle_model_cfg(sample_wl), weights), wl.prompt_len + wl.n_generate + 1,
+                        kv_storage=wl.dtype)
+    scfg = SampleCfg(wl.temperature, wl.top_k, wl.philox_seed, wl.window, 0, wl.grid_stride, wl.n_generate, wl.dtype)
+    prompt = [int(t) for t in make_prompt(wl, 1)[0]]
+    model.prefill(prompt)
+    st = sjd_begin(prompt, scfg, wl.vocab)
+    times, committed = [], 0
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        rec = sjd_step(st, model, scfg, wl.vocab)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+            committed += len(rec.committed)
+    t_sample = float(np.mean(times))
+    # the part that does not scale with depth (embedding, lm_head, verification): the same
+    # iteration on a zero-layer model
+    head_wl = wl.with_(n_layers=0)
+    head = CachedModel(OracleModel(oracle_model_cfg(head_wl), dict(weights, layers=[])), wl.prompt_len + wl.n_generate + 1,
+                       kv_storage=wl.dtype)
+    head.prefill(prompt)
+    st0 = sjd_begin(prompt, scfg, wl.vocab)
+    t0 = time.perf_counter()
+    sjd_step(st0, head, scfg, wl.vocab)
+    t_head = time.perf_counter() - t0
+    t_layer = max(t_sample - t_head, 0.0)
+    t_full = t_layer * wl.n_layers + t_head
+    tps = tokens_per_step if tokens_per_step else committed / max(1, len(times))
+    return {"value": tps / t_full, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": ("%d oracle SJD iterations (W=%d rows, prompt %d) of 1 of %d layers + lm_head + verification: "
+                       "%.2f s each; layer part scaled x%d to full depth => %.1f s per iteration (extrapolated); "
+                       "%.3f committed tokens per iteration" %
+                       (len(times), wl.window, wl.prompt_len, wl.n_layers, t_sample, wl.n_layers, t_full, tps)),
+            "seconds_per_step_full_depth": t_full}
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 8))
+    warm = max(0, min(args.warmup, 1))
+    t0 = time.perf_counter()
+    res = oracle_sample(wl, steps, warm, None)
+    line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["seconds_per_step_full_depth"] * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(wl, 1), "gpu_launches": 0,
+            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "note": "CPU oracle (fp64, numpy); timed steps capped at %d; wall %.0f s" % (steps, time.perf_counter() - t0)}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl, batch_per_gpu):
+    return {"workload": "7B-shaped decoder, one SJD iteration per step (BASELINE configs[2])", "name": wl.name,
+            "n_layers": wl.n_layers, "d_model": wl.d_model, "n_heads": wl.n_heads, "n_kv_heads": wl.n_kv_heads,
+            "ffn_hidden": wl.ffn_hidden, "vocab": wl.vocab, "prompt_len": wl.prompt_len, "n_generate": wl.n_generate,
+            "window": wl.window, "top_k": wl.top_k, "temperature": wl.temperature, "init": "random",
+            "batch_per_gpu": batch_per_gpu, "parallelism": "independent sequences per GPU, no collective",
+            "l2": "inputs (13.5 GB of weights per step) exceed L2; no flush needed"}
+
+
+# ------------------------------------------------------------------------------------------------
+# this library
+# ------------------------------------------------------------------------------------------------
+def run_library(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2410_01699_b200 import binding as B
+    from paper_2410_01699_b200.inputs import make_prompt, make_weights
+    from paper_2410_01699_b200.sharding import shard_sequences
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    batch = args.batch
+    seq_base, _ = shard_sequences(batch * world, world, rank)
+
+    weights = make_weights(wl, device=dev)
+    max_seq = wl.prompt_len + wl.n_generate + 8
+    ctx = B.Context(B.make_model_cfg(wl, batch, max_seq, wl.window), weights, device=dev)
+    sample = B.make_sample_cfg(wl.temperature, wl.top_k, wl.philox_seed, wl.window, B.SJD_INIT_RANDOM,
+                               wl.grid_stride, wl.n_generate, seq_base=seq_base)
+    prompt_host = torch.from_numpy(make_prompt(wl, batch * world)[seq_base:seq_base + batch].copy()).pin_memory()
+    prompt_dev = prompt_host.to(dev)
+    out_dev = B.StepOut(batch, wl.window, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K steps enqueued back to back, no host round trip
+    ctx.prefill(prompt_dev, sample)
+    committed_acc = torch.zeros(batch, dtype=torch.int64, device=dev)
+    for _ in range(args.warmup):
+        ctx.step(out_dev)
+    barrier()
+    clocks = ClockSampler(local)
+    clocks.start()
+    launches0 = B.sjd_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        ctx.step(out_dev)
+        committed_acc += out_dev.n_committed  # device-side add of the step's result, no sync
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = B.sjd_launch_count() - launches0
+    clk = clocks.stop()
+    tokens = int(committed_acc.sum().item())
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+        tk = torch.tensor([tokens], dtype=torch.int64, device=dev)
+        dist.all_reduce(tk)
+        tokens = int(tk.item())
+    assert ctx.device_status() == B.SJD_OK
+    value = tokens / (ms * 1e-3)
+    tokens_per_step = tokens / (args.steps * batch * world)
+
+    # ---- per-kernel-class device time (separate traced steps, CUDA events on the launching stream)
+    trace_steps = max(3, min(10, args.steps))
+    ctx.trace(True)
+    for _ in range(trace_steps):
+        ctx.step(out_dev)
+    tr = ctx.trace_read()
+    ctx.trace(False)
+    peaks = measured_peaks()
+    gemm_ms_per_launch = tr["ms"]["gemm"] / max(1, tr["launches"]["gemm"])
+    achieved = tr["gemm_weight_bytes"] / (tr["ms"]["gemm"] * 1e-3) / 1e9 if tr["ms"]["gemm"] > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "projection GEMMs (weight streaming, M = %d rows)" % (batch * wl.window),
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                "peak_source": "of " + peaks["source"], "traffic": None,
+                "algorithmic_bytes_per_step": tr["gemm_weight_bytes"] / trace_steps,
+                "launches_per_step": tr["launches"]["gemm"] / trace_steps, "avg_launch_ms": gemm_ms_per_launch,
+                "step_ms_by_class": {k: v / trace_steps for k, v in tr["ms"].items()}}
+
+    # ---- end to end through the C-ABI with host buffers: prompt copied in from pinned memory, results
+    # written to pinned host memory and read by the host after every step
+    out_host = B.StepOut(batch, wl.window, pinned=True)
+    e2e_steps = args.steps
+    barrier()
+    t0 = time.perf_counter()
+    prompt_dev.copy_(prompt_host, non_blocking=True)
+    ctx.prefill(prompt_dev, sample)
+    e2e_tokens = 0
+    for _ in range(e2e_steps):
+        ctx.step(out_host)
+        stream.synchronize()
+        e2e_tokens += int(out_host.n_committed.sum())
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+        tk = torch.tensor([e2e_tokens], dtype=torch.int64, device=dev)
+        dist.all_reduce(tk)
+        e2e_tokens = int(tk.item())
+    out_bytes = sum(getattr(out_host, n).numel() * 4 for n in ("n_accepted", "n_committed", "committed", "draft",
+                                                                "q_kind", "q_draft", "total_committed", "flags"))
+    e2e = {"value": e2e_tokens / e2e_s, "unit": UNIT,
+           "h2d_bytes_per_step": prompt_host.numel() * 4 / e2e_steps, "d2h_bytes_per_step": out_bytes,
+           "note": "includes pre-fill of the %d-token prompt; host waits for and reads every step's results" % wl.prompt_len}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = oracle_sample(wl, 2, 1, tokens_per_step)
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(wl, batch),
+                "clocks": clk, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+                "sjd": {"committed_tokens_per_step": tokens_per_step,
+                        "steps_per_image_est": wl.n_generate / tokens_per_step if tokens_per_step else None,
+                        "step_floor_ms_at_measured_hbm": wl.step_weight_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e3}}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="7b")
+    ap.add_argument("--batch", type=int, default=1, help="sequences per GPU")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2410_01699_b200.inputs import WORKLOADS
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_library(args, wl)
+
+
+if __name__ == "__main__":
+    main()

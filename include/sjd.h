@@ -208,6 +208,21 @@ int sjd_last_device_status(sjd_ctx *ctx);
 /* cudaError_t of the last failed CUDA call made on behalf of this thread (0 if none). */
 int sjd_last_cuda_error(void);
 
+/* Number of kernels this library has launched in this process (all contexts, all calls). */
+int64_t sjd_launch_count(void);
+
+/*
+ * Diagnostics: where the time of Step 2 / Step 3 goes.  sjd_trace(ctx, 1) zeroes the totals and
+ * makes every following sjd_step bracket each kernel launch with CUDA events on the caller's
+ * stream and end with a stream synchronisation (so traced steps are slower and must not be the
+ * ones a throughput figure is taken from); sjd_trace(ctx, 0) switches it off.  sjd_trace_read
+ * returns, per class {0: projection GEMMs, 1: attention, 2: verify + window slide, 3: the rest},
+ * the summed device milliseconds and launch counts (host arrays of 4), and the weight bytes the
+ * traced GEMM launches had to stream (out_features * in_features * element size, summed).
+ */
+int sjd_trace(sjd_ctx *ctx, int enable);
+int sjd_trace_read(sjd_ctx *ctx, double *ms, int64_t *launches, double *gemm_weight_bytes);
+
 void sjd_destroy(sjd_ctx *ctx);
 const char *sjd_strerror(int status);
 

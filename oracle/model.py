@@ -21,6 +21,15 @@ Sec. 3.2, Sec. 4.1 Step 2); its models are 7B Llama/Chameleon-style decoders
 
 Weights are taken exactly as given (bf16-rounded values are exact inputs) and
 every intermediate stays fp64; nothing is blocked, fused or reordered.
+
+Stored tensors.  The paper never states a precision.  The workloads fix a
+storage dtype (fp32 or bf16) for the two tensors that persist across
+iterations: the logits handed to the verification (rounded by
+round_to_storage before use) and the KV cache.  A KVCache created with
+storage 'f32' / 'bf16' therefore rounds keys (after RoPE) and values to that
+dtype as they are written, exactly like the stored logits; storage 'f64'
+(default) is the plain definition and makes the cached forward identical to
+the full causal forward.
 """
 from __future__ import annotations
 
@@ -83,7 +92,9 @@ def softmax_rows(s):
 class KVCache:
     """Keys (after RoPE) and values of the positions already run, per layer."""
 
-    def __init__(self, cfg: ModelCfg, capacity: int):
+    def __init__(self, cfg: ModelCfg, capacity: int, storage: str = "f64"):
+        assert storage in ("f64", "f32", "bf16")
+        self.storage = storage
         shape = (cfg.n_layers, capacity, cfg.n_kv_heads, cfg.head_dim)
         self.k = np.zeros(shape, dtype=np.float64)
         self.v = np.zeros(shape, dtype=np.float64)
@@ -104,8 +115,8 @@ class OracleModel:
         assert cfg.n_heads % cfg.n_kv_heads == 0
         assert cfg.head_dim % 2 == 0
 
-    def new_cache(self, capacity: int) -> KVCache:
-        return KVCache(self.cfg, capacity)
+    def new_cache(self, capacity: int, storage: str = "f64") -> KVCache:
+        return KVCache(self.cfg, capacity, storage)
 
     def _attention(self, q, k_all, v_all, q_pos):
         """q: [T][H][hd]; k_all, v_all: [S][KVh][hd] for positions 0..S-1;
@@ -137,6 +148,9 @@ class OracleModel:
         if cache is not None:
             p0 = int(positions[0])
             assert p0 == cache.length, "window must start right after the cached prefix"
+            if cache.storage != "f64":
+                k = round_to_storage(k, cache.storage)
+                v = round_to_storage(v, cache.storage)
             cache.k[li, p0:p0 + t_len] = k
             cache.v[li, p0:p0 + t_len] = v
             k_all = cache.k[li, :p0 + t_len]

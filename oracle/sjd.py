@@ -79,9 +79,9 @@ class CachedModel:
     """OracleModel driven with a KV cache: rows for c[0..n-1) stay cached, the
     rejected tail is rolled back by truncation (stale rows are overwritten)."""
 
-    def __init__(self, model: OracleModel, capacity: int):
+    def __init__(self, model: OracleModel, capacity: int, kv_storage: str = "f64"):
         self.model = model
-        self.cache: KVCache = model.new_cache(capacity)
+        self.cache: KVCache = model.new_cache(capacity, kv_storage)
 
     def prefill(self, prompt):
         self.cache.truncate(0)

@@ -27,7 +27,7 @@ TORCH_DTYPES = {SJD_F32: torch.float32, SJD_BF16: torch.bfloat16}
 
 EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_get_window", "sjd_peek_logits",
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
-           "sjd_destroy", "sjd_strerror"]
+           "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read"]
 
 
 class SJDError(RuntimeError):
@@ -101,6 +101,11 @@ def lib():
     L.sjd_last_device_status.restype = C.c_int
     L.sjd_last_device_status.argtypes = [C.c_void_p]
     L.sjd_last_cuda_error.restype = C.c_int
+    L.sjd_launch_count.restype = C.c_int64
+    L.sjd_trace.restype = C.c_int
+    L.sjd_trace.argtypes = [C.c_void_p, C.c_int]
+    L.sjd_trace_read.restype = C.c_int
+    L.sjd_trace_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_double)]
     L.sjd_destroy.restype = None
     L.sjd_destroy.argtypes = [C.c_void_p]
     L.sjd_strerror.restype = C.c_char_p
@@ -219,6 +224,17 @@ class Context:
         _check(lib().sjd_peek_logits(self._ctx, _ptr(t), t.numel() * t.element_size(), _stream()), "sjd_peek_logits")
         return t
 
+    def trace(self, enable: bool):
+        _check(lib().sjd_trace(self._ctx, 1 if enable else 0), "sjd_trace")
+
+    def trace_read(self):
+        """{'ms': {class: ms}, 'launches': {class: n}, 'gemm_weight_bytes': float}"""
+        ms, n, wb = (C.c_double * 4)(), (C.c_int64 * 4)(), C.c_double()
+        _check(lib().sjd_trace_read(self._ctx, ms, n, C.byref(wb)), "sjd_trace_read")
+        names = ("gemm", "attention", "verify", "other")
+        return {"ms": dict(zip(names, list(ms))), "launches": dict(zip(names, list(n))),
+                "gemm_weight_bytes": float(wb.value)}
+
     def device_status(self) -> int:
         return int(lib().sjd_last_device_status(self._ctx))
 
@@ -232,6 +248,10 @@ class Context:
             self.close()
         except Exception:
             pass
+
+
+def sjd_launch_count() -> int:
+    return int(lib().sjd_launch_count())
 
 
 def weights_to_device(weights: dict, device="cuda") -> dict:

@@ -5,6 +5,7 @@
 
 namespace sjd {
 thread_local int g_last_cuda_error = 0;
+std::atomic<long long> g_launch_count{0};
 
 int check_sample_cfg(const sjd_sample_cfg *s, int vocab) {
   if (!s) return SJD_ERR_BAD_ARG;
@@ -71,6 +72,8 @@ extern "C" int sjd_verify(int batch, int window, int vocab, int logits_dtype, co
 }
 
 extern "C" int sjd_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" int64_t sjd_launch_count(void) { return (int64_t)g_launch_count.load(); }
 
 extern "C" const char *sjd_strerror(int status) {
   switch (status) {

@@ -13,9 +13,6 @@ namespace {
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-template <typename T> __device__ __forceinline__ T from_f(float v);
-template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
-template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 constexpr int TK = 32;        // keys per tile (one per lane)
 constexpr int NWARPS = 8;
@@ -24,7 +21,7 @@ constexpr int MAXD = 4;       // head dims per lane: head_dim <= 128
 
 template <typename T>
 __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
-    const T *__restrict__ q, KvLayout kv, const int32_t *__restrict__ in_pos, float *__restrict__ partial,
+    const float *__restrict__ q, KvLayout kv, const int32_t *__restrict__ in_pos, float *__restrict__ partial,
     int rows_per_seq, int n_heads, int splits) {
   extern __shared__ float smem[];
   const int hd = kv.head_dim;
@@ -50,7 +47,7 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
   }
   for (int i = tid; i < W * hd; i += blockDim.x) {
     const int qi = i / hd, d = i % hd;
-    Qs[i] = to_f<T>(q[((size_t)(m0 + qi) * n_heads + h) * hd + d]);
+    Qs[i] = q[((size_t)(m0 + qi) * n_heads + h) * hd + d];
   }
   __syncthreads();
   const int len = s_len;
@@ -156,14 +153,13 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
   }
 }
 
-template <typename T>
 __global__ void attention_combine_kernel(const float *__restrict__ partial, const int32_t *__restrict__ in_pos,
-                                         T *__restrict__ out, int n_heads, int hd, int splits) {
+                                         float *__restrict__ out, int n_heads, int hd, int splits) {
   const int m = blockIdx.x, h = blockIdx.y;
   const float *src = partial + ((size_t)m * n_heads + h) * splits * (hd + 2);
-  T *dst = out + ((size_t)m * n_heads + h) * hd;
+  float *dst = out + ((size_t)m * n_heads + h) * hd;
   if (in_pos[m] < 0) {
-    for (int d = threadIdx.x; d < hd; d += blockDim.x) dst[d] = from_f<T>(0.0f);
+    for (int d = threadIdx.x; d < hd; d += blockDim.x) dst[d] = 0.0f;
     return;
   }
   float gmax = -INFINITY;
@@ -179,12 +175,12 @@ __global__ void attention_combine_kernel(const float *__restrict__ partial, cons
       const float ms = src[(size_t)s * (hd + 2)];
       if (ms > -INFINITY) acc += src[(size_t)s * (hd + 2) + 2 + d] * expf(ms - gmax);
     }
-    dst[d] = from_f<T>(denom > 0.0f ? acc / denom : 0.0f);
+    dst[d] = denom > 0.0f ? acc / denom : 0.0f;
   }
 }
 
 template <typename T>
-int attention_t(const void *q, KvLayout kv, const int32_t *in_pos, void *out, float *partial, int M, int rows_per_seq,
+int attention_t(const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial, int M, int rows_per_seq,
                 int n_heads, int splits, cudaStream_t stream) {
   const int hd = kv.head_dim, W = rows_per_seq;
   if (W > NWARPS * MAXQ || hd > 32 * MAXD || M % W != 0) return SJD_ERR_UNSUPPORTED;
@@ -192,18 +188,17 @@ int attention_t(const void *q, KvLayout kv, const int32_t *in_pos, void *out, fl
   if (smem > 48 * 1024)
     SJD_CUDA(cudaFuncSetAttribute(attention_partial_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(n_heads, M / W, splits);
-  attention_partial_kernel<T><<<grid, NWARPS * 32, smem, stream>>>(reinterpret_cast<const T *>(q), kv, in_pos, partial,
+  attention_partial_kernel<T><<<grid, NWARPS * 32, smem, stream>>>(q, kv, in_pos, partial,
                                                                   W, n_heads, splits);
   SJD_CHECK_LAUNCH();
-  attention_combine_kernel<T><<<dim3(M, n_heads), 128, 0, stream>>>(partial, in_pos, reinterpret_cast<T *>(out),
-                                                                   n_heads, hd, splits);
+  attention_combine_kernel<<<dim3(M, n_heads), 128, 0, stream>>>(partial, in_pos, out, n_heads, hd, splits);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
 
 }  // namespace
 
-int launch_attention(int dtype, const void *q, KvLayout kv, const int32_t *in_pos, void *out, float *partial, int M,
+int launch_attention(int dtype, const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial, int M,
                      int rows_per_seq, int n_heads, int splits, cudaStream_t stream) {
   if (dtype == SJD_F32) return attention_t<float>(q, kv, in_pos, out, partial, M, rows_per_seq, n_heads, splits, stream);
   if (dtype == SJD_BF16)

@@ -6,11 +6,14 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "sjd.h"
 
 namespace sjd {
 
 extern thread_local int g_last_cuda_error;
+extern std::atomic<long long> g_launch_count;  // kernels launched by this library in this process
 
 #define SJD_CUDA(expr)                          \
   do {                                          \
@@ -21,7 +24,11 @@ extern thread_local int g_last_cuda_error;
     }                                           \
   } while (0)
 
-#define SJD_CHECK_LAUNCH() SJD_CUDA(cudaGetLastError())
+#define SJD_CHECK_LAUNCH()                                              \
+  do {                                                                  \
+    ::sjd::g_launch_count.fetch_add(1, std::memory_order_relaxed);      \
+    SJD_CUDA(cudaGetLastError());                                       \
+  } while (0)
 
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): 128-bit counter, 64-bit key, ten rounds of
@@ -144,28 +151,28 @@ int check_sample_cfg(const sjd_sample_cfg *s, int vocab);
 // ---- model forward (model_kernels.cu, attention.cu); `dtype` selects float / bf16 storage
 enum GemmEpilogue { EPI_STORE_F32 = 0, EPI_STORE_T = 1, EPI_ADD_F32 = 2 };
 
-// C[M][N] (epilogue) = A[M][K] * Wt[N][K]^T, fp32 accumulation.  A and Wt are of `dtype`;
+// C[M][N] (epilogue) = A[M][K] * Wt[N][K]^T, fp32 accumulation.  A is fp32, Wt is of `dtype`;
 // C is fp32 (EPI_STORE_F32, EPI_ADD_F32: C += product) or `dtype` (EPI_STORE_T).  lda/ldc in elements.
 int launch_gemm_simt(int dtype, const void *A, int lda, const void *Wt, void *C, int ldc, int M, int N, int K,
                      int epilogue, cudaStream_t stream);
 // x[m][:] = tok_emb[tok[m]][:]  (fp32 residual stream)
 int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, int M, int d, int vocab,
                  cudaStream_t stream);
-// h[m][:] = x[m][:] * gain[:] / sqrt(mean(x[m]^2) + eps), stored as `dtype`
-int launch_rmsnorm(int dtype, const float *x, const void *gain, void *h, int M, int d, float eps, cudaStream_t stream);
-// Rotate q and k by their absolute position (pairs i, i + hd/2), store q as `dtype` [M][H*hd],
+// h[m][:] = x[m][:] * gain[:] / sqrt(mean(x[m]^2) + eps)  (gain of `dtype`)
+int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M, int d, float eps, cudaStream_t stream);
+// Rotate q and k by their absolute position (pairs i, i + hd/2), store q as fp32 [M][H*hd],
 // append k and v to the cache row in_pos[m] of sequence m / rows_per_seq.  Rows with in_pos < 0 are skipped.
 struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
   void *base;
   int n_kv_heads, max_seq, head_dim;
 };
-int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, void *q,
+int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
                        KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
-// act[m][f] = silu(gu[m][f]) * gu[m][F + f], stored as `dtype`
-int launch_swiglu(int dtype, const float *gu, void *act, int M, int F, cudaStream_t stream);
+// act[m][f] = silu(gu[m][f]) * gu[m][F + f]
+int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream);
 // Window-causal attention: query row m (sequence m / rows_per_seq, position in_pos[m]) attends cache rows
-// 0 .. in_pos[m].  out [M][H*hd] of `dtype`.  partial: fp32 scratch [M][H][splits][hd + 2].
-int launch_attention(int dtype, const void *q, KvLayout kv, const int32_t *in_pos, void *out, float *partial,
+// 0 .. in_pos[m].  q, out: fp32 [M][H*hd]; cache of `dtype`.  partial: fp32 scratch [M][H][splits][hd + 2].
+int launch_attention(int dtype, const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial,
                      int M, int rows_per_seq, int n_heads, int splits, cudaStream_t stream);
 
 }  // namespace sjd

@@ -59,12 +59,12 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.step = take(4);
   L.status = take(4);
   L.x = take(Mx * c.d_model * 4);
-  L.h = take(Mx * c.d_model * es);
+  L.h = take(Mx * c.d_model * 4);
   L.qkv = take(Mx * (nq + 2 * nk) * 4);
-  L.q = take(Mx * nq * es);
-  L.attn = take(Mx * nq * es);
+  L.q = take(Mx * nq * 4);
+  L.attn = take(Mx * nq * 4);
   L.gu = take(Mx * 2 * c.ffn_hidden * 4);
-  L.act = take(Mx * c.ffn_hidden * es);
+  L.act = take(Mx * c.ffn_hidden * 4);
   size_t part = 0;
   for (int b = 1; b <= c.max_batch; ++b) {
     const size_t need = (size_t)b * c.max_window * c.n_heads * attention_splits(c.n_heads, b) * (c.head_dim + 2);
@@ -84,6 +84,53 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.total = off;
   return L;
 }
+
+// Optional per-class timing of the launches of a step with CUDA events on the launching stream
+// (diagnostics: which kernels the step time goes to).  Off by default; when on, every launch is
+// bracketed by two events and each step ends with a stream synchronisation.
+enum TraceClass { TC_GEMM = 0, TC_ATTENTION = 1, TC_VERIFY = 2, TC_OTHER = 3, TC_COUNT = 4 };
+struct Tracer {
+  bool on = false;
+  std::vector<cudaEvent_t> ev;
+  std::vector<int> cls;
+  size_t used = 0;
+  double ms[TC_COUNT] = {0, 0, 0, 0};
+  long long launches[TC_COUNT] = {0, 0, 0, 0};
+  double gemm_weight_bytes = 0;
+  void begin(int c, cudaStream_t s) {
+    if (!on) return;
+    if (used + 2 > ev.size()) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      cudaEventCreate(&a);
+      cudaEventCreate(&b);
+      ev.push_back(a);
+      ev.push_back(b);
+    }
+    cls.push_back(c);
+    cudaEventRecord(ev[used], s);
+  }
+  void end(cudaStream_t s) {
+    if (!on) return;
+    cudaEventRecord(ev[used + 1], s);
+    used += 2;
+  }
+  int flush(cudaStream_t s) {
+    if (!on || used == 0) return SJD_OK;
+    SJD_CUDA(cudaStreamSynchronize(s));
+    for (size_t i = 0; i < used; i += 2) {
+      float t = 0.0f;
+      SJD_CUDA(cudaEventElapsedTime(&t, ev[i], ev[i + 1]));
+      ms[cls[i / 2]] += t;
+      launches[cls[i / 2]] += 1;
+    }
+    used = 0;
+    cls.clear();
+    return SJD_OK;
+  }
+  ~Tracer() {
+    for (cudaEvent_t e : ev) cudaEventDestroy(e);
+  }
+};
 
 __global__ void prefill_setup_kernel(const int32_t *prompt, int P, SeqState st, uint32_t *step, int32_t *counters,
                                      int B) {
@@ -137,6 +184,7 @@ struct sjd_ctx {
   bool prefilled;
   uint32_t host_step;  // number of sjd_step calls since prefill == device step index
   cudaStream_t last_stream;
+  Tracer tracer;
 
   template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
   SeqState state() const {
@@ -180,37 +228,43 @@ int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream)
   const int nq = g.n_heads * g.head_dim, nk = g.n_kv_heads * g.head_dim, nqkv = nq + 2 * nk;
   const SeqState st = c->state();
   float *x = c->at<float>(c->lay.x);
-  void *h = c->ws + c->lay.h;
+  float *h = c->at<float>(c->lay.h);
   float *qkv = c->at<float>(c->lay.qkv);
-  void *q = c->ws + c->lay.q;
-  void *attn = c->ws + c->lay.attn;
+  float *q = c->at<float>(c->lay.q);
+  float *attn = c->at<float>(c->lay.attn);
   float *gu = c->at<float>(c->lay.gu);
-  void *act = c->ws + c->lay.act;
+  float *act = c->at<float>(c->lay.act);
   float *partial = c->at<float>(c->lay.partial);
   const float2 *rope = c->at<float2>(c->lay.rope);
   const int splits = attention_splits(g.n_heads, c->batch);
   int rc;
+  Tracer &tr = c->tracer;
+  const double es = (double)esize(dt);
 #define SJD_TRY(call) do { rc = (call); if (rc != SJD_OK) return rc; } while (0)
-  SJD_TRY(launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
+#define SJD_TR(klass, call) do { tr.begin(klass, stream); rc = (call); tr.end(stream); if (rc != SJD_OK) return rc; } while (0)
+#define SJD_GEMM(n_out, k_in, call) do { if (tr.on) tr.gemm_weight_bytes += (double)(n_out) * (double)(k_in) * es; SJD_TR(TC_GEMM, call); } while (0)
+  SJD_TR(TC_OTHER, launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
   for (int l = 0; l < g.n_layers; ++l) {
-    SJD_TRY(launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream));
-    SJD_TRY(launch_gemm_simt(dt, h, d, c->wq[l], qkv, nqkv, M, nq, d, EPI_STORE_F32, stream));
-    SJD_TRY(launch_gemm_simt(dt, h, d, c->wk[l], qkv + nq, nqkv, M, nk, d, EPI_STORE_F32, stream));
-    SJD_TRY(launch_gemm_simt(dt, h, d, c->wv[l], qkv + nq + nk, nqkv, M, nk, d, EPI_STORE_F32, stream));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream));
+    SJD_GEMM(nq, d, launch_gemm_simt(dt, h, d, c->wq[l], qkv, nqkv, M, nq, d, EPI_STORE_F32, stream));
+    SJD_GEMM(nk, d, launch_gemm_simt(dt, h, d, c->wk[l], qkv + nq, nqkv, M, nk, d, EPI_STORE_F32, stream));
+    SJD_GEMM(nk, d, launch_gemm_simt(dt, h, d, c->wv[l], qkv + nq + nk, nqkv, M, nk, d, EPI_STORE_F32, stream));
     const KvLayout kv = c->kv_layer(l);
-    SJD_TRY(launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
-    SJD_TRY(launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream));
-    SJD_TRY(launch_gemm_simt(dt, attn, nq, c->wo[l], x, d, M, d, nq, EPI_ADD_F32, stream));
-    SJD_TRY(launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream));
-    SJD_TRY(launch_gemm_simt(dt, h, d, c->w_gate[l], gu, 2 * F, M, F, d, EPI_STORE_F32, stream));
-    SJD_TRY(launch_gemm_simt(dt, h, d, c->w_up[l], gu + F, 2 * F, M, F, d, EPI_STORE_F32, stream));
-    SJD_TRY(launch_swiglu(dt, gu, act, M, F, stream));
-    SJD_TRY(launch_gemm_simt(dt, act, F, c->w_down[l], x, d, M, d, F, EPI_ADD_F32, stream));
+    SJD_TR(TC_OTHER, launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
+    SJD_TR(TC_ATTENTION, launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream));
+    SJD_GEMM(d, nq, launch_gemm_simt(dt, attn, nq, c->wo[l], x, d, M, d, nq, EPI_ADD_F32, stream));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream));
+    SJD_GEMM(F, d, launch_gemm_simt(dt, h, d, c->w_gate[l], gu, 2 * F, M, F, d, EPI_STORE_F32, stream));
+    SJD_GEMM(F, d, launch_gemm_simt(dt, h, d, c->w_up[l], gu + F, 2 * F, M, F, d, EPI_STORE_F32, stream));
+    SJD_TR(TC_OTHER, launch_swiglu(gu, act, M, F, stream));
+    SJD_GEMM(d, F, launch_gemm_simt(dt, act, F, c->w_down[l], x, d, M, d, F, EPI_ADD_F32, stream));
   }
   if (logits_out) {
-    SJD_TRY(launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream));
-    SJD_TRY(launch_gemm_simt(dt, h, d, c->lm_head, logits_out, g.vocab, M, g.vocab, d, EPI_STORE_T, stream));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream));
+    SJD_GEMM(g.vocab, d, launch_gemm_simt(dt, h, d, c->lm_head, logits_out, g.vocab, M, g.vocab, d, EPI_STORE_T, stream));
   }
+#undef SJD_GEMM
+#undef SJD_TR
 #undef SJD_TRY
   return SJD_OK;
 }
@@ -363,10 +417,12 @@ extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) 
   const int cur = (int)(c->host_step & 1u);
   int rc = forward(c, c->window, c->ws + c->lay.logits[cur], stream);
   if (rc != SJD_OK) return rc;
+  c->tracer.begin(TC_VERIFY, stream);
   rc = run_verify(c, out, stream);
+  c->tracer.end(stream);
   if (rc != SJD_OK) return rc;
   c->host_step += 1;
-  return SJD_OK;
+  return c->tracer.flush(stream);
 }
 
 extern "C" int sjd_get_window(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) {
@@ -393,6 +449,31 @@ extern "C" int sjd_last_device_status(sjd_ctx *c) {
   int32_t status = 0;
   SJD_CUDA(cudaMemcpy(&status, c->ws + c->lay.status, 4, cudaMemcpyDeviceToHost));
   return status == 0 ? SJD_OK : SJD_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" int sjd_trace(sjd_ctx *c, int enable) {
+  if (!c) return SJD_ERR_BAD_ARG;
+  c->tracer.on = enable != 0;
+  c->tracer.used = 0;
+  c->tracer.cls.clear();
+  if (enable) {
+    for (int i = 0; i < TC_COUNT; ++i) {
+      c->tracer.ms[i] = 0;
+      c->tracer.launches[i] = 0;
+    }
+    c->tracer.gemm_weight_bytes = 0;
+  }
+  return SJD_OK;
+}
+
+extern "C" int sjd_trace_read(sjd_ctx *c, double *ms, int64_t *launches, double *gemm_weight_bytes) {
+  if (!c || !ms || !launches || !gemm_weight_bytes) return SJD_ERR_BAD_ARG;
+  for (int i = 0; i < TC_COUNT; ++i) {
+    ms[i] = c->tracer.ms[i];
+    launches[i] = c->tracer.launches[i];
+  }
+  *gemm_weight_bytes = c->tracer.gemm_weight_bytes;
+  return SJD_OK;
 }
 
 extern "C" void sjd_destroy(sjd_ctx *c) { delete c; }

@@ -1,7 +1,7 @@
 // Generic kernels of the decoder forward pass (Sec. 3.1: the auto-regressive transformer; Sec. 4.1
 // Step 2: one pass over the window).  These cover every shape and both dtypes with plain FMA
-// arithmetic and fp32 accumulation; the bf16 weight-streaming tensor-core GEMM lives in gemm_tc.cu
-// and takes over for the shapes it supports.
+// arithmetic and fp32 accumulation.  Activations between kernels are fp32 (they are a few hundred KB);
+// only weights, the KV cache and the stored logits are in the model dtype.
 #include "common.cuh"
 
 namespace sjd {
@@ -20,7 +20,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float
 constexpr int GM = 32, GN = 64, GK = 32;
 
 template <typename T, int EPI>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const T *__restrict__ A, int lda, const T *__restrict__ Wt,
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const float *__restrict__ A, int lda, const T *__restrict__ Wt,
                                                         void *__restrict__ Cv, int ldc, int M, int N, int K) {
   __shared__ float As[GM][GK + 1];
   __shared__ float Ws[GN][GK + 1];
@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T *__restrict__ A,
     for (int i = tid; i < GM * GK; i += 256) {
       const int r = i / GK, c = i % GK;
       const int m = m0 + r, k = k0 + c;
-      As[r][c] = (m < M && k < K) ? to_f<T>(A[(size_t)m * lda + k]) : 0.0f;
+      As[r][c] = (m < M && k < K) ? A[(size_t)m * lda + k] : 0.0f;
     }
     for (int i = tid; i < GN * GK; i += 256) {
       const int r = i / GK, c = i % GK;
@@ -72,7 +72,7 @@ template <typename T>
 int gemm_simt_t(const void *A, int lda, const void *Wt, void *C, int ldc, int M, int N, int K, int epi,
                 cudaStream_t stream) {
   dim3 grid((N + GN - 1) / GN, (M + GM - 1) / GM);
-  const T *a = reinterpret_cast<const T *>(A);
+  const float *a = reinterpret_cast<const float *>(A);
   const T *w = reinterpret_cast<const T *>(Wt);
   if (epi == EPI_STORE_F32) gemm_simt_kernel<T, EPI_STORE_F32><<<grid, 256, 0, stream>>>(a, lda, w, C, ldc, M, N, K);
   else if (epi == EPI_STORE_T) gemm_simt_kernel<T, EPI_STORE_T><<<grid, 256, 0, stream>>>(a, lda, w, C, ldc, M, N, K);
@@ -96,7 +96,7 @@ __global__ void embed_kernel(const T *__restrict__ emb, const int32_t *__restric
 // ------------------------------------------------------------------------------------ RMSNorm
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ gain,
-                                                      T *__restrict__ h, int d, float eps) {
+                                                      float *__restrict__ h, int d, float eps) {
   __shared__ float red[8];
   const int m = blockIdx.x, tid = threadIdx.x;
   const float *row = x + (size_t)m * d;
@@ -109,13 +109,13 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
 #pragma unroll
   for (int w = 0; w < 8; ++w) tot += red[w];
   const float scale = rsqrtf(tot / (float)d + eps);
-  for (int i = tid; i < d; i += 256) h[(size_t)m * d + i] = from_f<T>(row[i] * scale * to_f<T>(gain[i]));
+  for (int i = tid; i < d; i += 256) h[(size_t)m * d + i] = row[i] * scale * to_f<T>(gain[i]);
 }
 
 // ------------------------------------------------------------------------------------ RoPE + KV append
 template <typename T>
 __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t *__restrict__ in_pos,
-                                   const float2 *__restrict__ rope, T *__restrict__ q, KvLayout kv, int rows_per_seq,
+                                   const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
                                    int n_heads) {
   const int m = blockIdx.x;
   const int pos = in_pos[m];
@@ -133,8 +133,8 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t 
     const float2 c = cs[j];
     if (head < n_heads) {
       const float x1 = row[head * hd + j], x2 = row[head * hd + j + half];
-      q[(size_t)m * nq + head * hd + j] = from_f<T>(x1 * c.x - x2 * c.y);
-      q[(size_t)m * nq + head * hd + j + half] = from_f<T>(x2 * c.x + x1 * c.y);
+      q[(size_t)m * nq + head * hd + j] = x1 * c.x - x2 * c.y;
+      q[(size_t)m * nq + head * hd + j + half] = x2 * c.x + x1 * c.y;
     } else {
       const int kh = head - n_heads;
       const float x1 = row[nq + kh * hd + j], x2 = row[nq + kh * hd + j + half];
@@ -150,13 +150,12 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t 
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU
-template <typename T>
-__global__ void swiglu_kernel(const float *__restrict__ gu, T *__restrict__ act, int M, int F) {
+__global__ void swiglu_kernel(const float *__restrict__ gu, float *__restrict__ act, int M, int F) {
   const size_t total = (size_t)M * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t m = i / F, f = i % F;
     const float g = gu[m * 2 * F + f], u = gu[m * 2 * F + F + f];
-    act[i] = from_f<T>(g / (1.0f + expf(-g)) * u);
+    act[i] = g / (1.0f + expf(-g)) * u;
   }
 }
 
@@ -182,25 +181,24 @@ int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, i
   return SJD_OK;
 }
 
-int launch_rmsnorm(int dtype, const float *x, const void *gain, void *h, int M, int d, float eps, cudaStream_t stream) {
-  SJD_DISPATCH(dtype, (rmsnorm_kernel<T><<<M, 256, 0, stream>>>(x, reinterpret_cast<const T *>(gain),
-                                                               reinterpret_cast<T *>(h), d, eps)));
+int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M, int d, float eps, cudaStream_t stream) {
+  SJD_DISPATCH(dtype, (rmsnorm_kernel<T><<<M, 256, 0, stream>>>(x, reinterpret_cast<const T *>(gain), h, d, eps)));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
 
-int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, void *q,
+int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
                        KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
-  SJD_DISPATCH(dtype, (rope_append_kernel<T><<<M, 256, 0, stream>>>(qkv, in_pos, rope_table, reinterpret_cast<T *>(q),
-                                                                   kv, rows_per_seq, n_heads)));
+  SJD_DISPATCH(dtype, (rope_append_kernel<T><<<M, 256, 0, stream>>>(qkv, in_pos, rope_table, q, kv, rows_per_seq,
+                                                                   n_heads)));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
 
-int launch_swiglu(int dtype, const float *gu, void *act, int M, int F, cudaStream_t stream) {
+int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream) {
   const size_t total = (size_t)M * F;
   const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
-  SJD_DISPATCH(dtype, (swiglu_kernel<T><<<blocks, 256, 0, stream>>>(gu, reinterpret_cast<T *>(act), M, F)));
+  swiglu_kernel<<<blocks, 256, 0, stream>>>(gu, act, M, F);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

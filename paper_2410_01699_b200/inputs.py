@@ -84,21 +84,22 @@ def torch_dtype(name: str):
 
 
 def _randn(shape, std, gen, dtype):
-    return (torch.randn(shape, generator=gen, dtype=torch.float32) * std).to(dtype)
+    return (torch.randn(shape, generator=gen, dtype=torch.float32, device=gen.device) * std).to(dtype)
 
 
-def make_weights(wl: Workload, gain_jitter: float = 0.0, std: float = 0.02):
-    """Random-init weights N(0, std^2) rounded to the workload dtype (CPU tensors).
-    Matrices are [out_features][in_features].  Norm gains are 1 (+ optional jitter so
-    tests exercise the gain path)."""
+def make_weights(wl: Workload, gain_jitter: float = 0.0, std: float = 0.02, device="cpu"):
+    """Random-init weights N(0, std^2) rounded to the workload dtype.  Matrices are
+    [out_features][in_features].  Norm gains are 1 (+ optional jitter so tests exercise the
+    gain path).  Generated on `device` with that device's generator: CPU tensors are what
+    parity tests feed to both sides; the benchmark generates its 7B weights on the GPU."""
     dt = torch_dtype(wl.dtype)
-    gen = torch.Generator().manual_seed(wl.weight_seed)
+    gen = torch.Generator(device=device).manual_seed(wl.weight_seed)
     d, hd = wl.d_model, wl.head_dim
 
     def gain():
-        g = torch.ones(d, dtype=torch.float32)
+        g = torch.ones(d, dtype=torch.float32, device=gen.device)
         if gain_jitter:
-            g = g + gain_jitter * torch.randn(d, generator=gen)
+            g = g + gain_jitter * torch.randn(d, generator=gen, device=gen.device)
         return g.to(dt)
 
     w = {"tok_emb": _randn((wl.vocab, d), std, gen, dt), "layers": []}

@@ -65,9 +65,9 @@ def test_rope_properties():
     assert np.count_nonzero(np.abs(r) > 1e-15) == 2
 
 
-def _torch_forward(cfg: ModelCfg, w, tokens):
+def _torch_forward(cfg: ModelCfg, w, tokens, kv_cast=None):
     """Independent fp64 forward built from torch library ops (sdpa, rms_norm, silu, complex
-    multiplication for the rotary step)."""
+    multiplication for the rotary step).  kv_cast: torch dtype keys/values are cast through."""
     t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
     tok = torch.as_tensor(tokens)
     x = t(w["tok_emb"])[tok]
@@ -86,6 +86,8 @@ def _torch_forward(cfg: ModelCfg, w, tokens):
         q = rot((h @ t(lw["wq"]).T).view(T, cfg.n_heads, hd))
         k = rot((h @ t(lw["wk"]).T).view(T, cfg.n_kv_heads, hd))
         v = (h @ t(lw["wv"]).T).view(T, cfg.n_kv_heads, hd)
+        if kv_cast is not None:
+            k, v = k.to(kv_cast).to(torch.float64), v.to(kv_cast).to(torch.float64)
         rep = cfg.n_heads // cfg.n_kv_heads
         k = k.repeat_interleave(rep, dim=1)
         v = v.repeat_interleave(rep, dim=1)
@@ -121,6 +123,25 @@ def test_window_forward_with_cache_equals_full_forward():
     cache.truncate(12)
     again = m.forward_window(cache, tokens[12:23], 12)
     np.testing.assert_allclose(again, full[12:23], rtol=1e-10, atol=1e-12)
+
+
+@pytest.mark.parametrize("storage,cast", [("bf16", torch.bfloat16), ("f32", torch.float32)])
+def test_cache_storage_rounding_equals_casting_keys_and_values(storage, cast):
+    """A cache of storage dtype s holds keys/values rounded to s: same logits as a library forward
+    whose keys and values are cast through that dtype; and it does change the result for bf16."""
+    w = _weights(CFG, seed=11)
+    m = OracleModel(CFG, w)
+    tokens = np.random.default_rng(12).integers(0, CFG.vocab, size=21)
+    cache = m.new_cache(32, storage)
+    m.forward_window(cache, tokens[:8], 0, want_logits=False)
+    got = np.concatenate([m.forward_window(cache, tokens[8:15], 8), m.forward_window(cache, tokens[15:21], 15)])
+    ref = _torch_forward(CFG, w, tokens, kv_cast=cast)[8:21]
+    np.testing.assert_allclose(got, ref, rtol=1e-9, atol=1e-11)
+    plain = m.forward_full(tokens)[8:21]
+    if storage == "bf16":
+        assert 1e-5 < np.abs(got - plain).max() < 0.05
+    else:
+        assert np.abs(got - plain).max() < 1e-6
 
 
 def test_causality():
