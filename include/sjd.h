@@ -201,6 +201,32 @@ int sjd_verify(int batch, int window, int vocab, int logits_dtype, const void *l
                const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
                const sjd_step_out *out, void *ws, size_t ws_bytes, void *cuda_stream);
 
+/*
+ * sjd_verify without a scratch argument, for callers that cannot allocate device memory: code that
+ * runs where cudaMalloc is forbidden or would stall the device (inside a serving loop with a latency
+ * budget, in a host thread that owns no allocator, in a plug-in that is handed only its input and
+ * output buffers).  (The paper has no counterpart; this is a packaging variant of the same kernel.)
+ *
+ * Same arguments, outputs and results as sjd_verify, minus ws / ws_bytes.  The per-row scratch lives
+ * in a fixed array inside the library image, SJD_VERIFY_STATIC_MAX_ROWS rows (about 130 KB); every
+ * GPU that loads the library holds that array until the process exits.  The call performs no
+ * cudaMalloc / cudaFree and calls no allocating routine; inputs and outputs stay the caller's.
+ *   - Limits: batch * window <= SJD_VERIFY_STATIC_MAX_ROWS and batch <= SJD_VERIFY_STATIC_MAX_BATCH,
+ *     else SJD_ERR_CAPACITY (nothing is launched).
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents; the call
+ *     clears the counters that must start at zero.  Two calls that overlap on the GPU (different
+ *     streams, or different threads or contexts of the same process on one device) race on it:
+ *     serialise them.  sjd_verify with separate workspaces has no such restriction.
+ */
+#define SJD_VERIFY_STATIC_MAX_ROWS 2048
+#define SJD_VERIFY_STATIC_MAX_BATCH 256
+int sjd_verify_static(int batch, int window, int vocab, int logits_dtype, const void *logits_cur,
+                      const void *logits_prev, const int32_t *draft, const int32_t *q_kind,
+                      const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
+                      const sjd_step_out *out, void *cuda_stream);
+
 /* Synchronises the context's last stream and returns SJD_OK, SJD_ERR_DEVICE_TIMEOUT
  * or SJD_ERR_CUDA according to the device status word. */
 int sjd_last_device_status(sjd_ctx *ctx);

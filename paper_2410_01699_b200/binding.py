@@ -27,7 +27,7 @@ TORCH_DTYPES = {SJD_F32: torch.float32, SJD_BF16: torch.bfloat16}
 
 EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_get_window", "sjd_peek_logits",
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
-           "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read"]
+           "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static"]
 
 
 class SJDError(RuntimeError):
@@ -98,6 +98,10 @@ def lib():
     L.sjd_verify.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.POINTER(sjd_sample_cfg), C.c_uint32, C.POINTER(sjd_step_out), C.c_void_p,
                              C.c_size_t, C.c_void_p]
+    L.sjd_verify_static.restype = C.c_int
+    L.sjd_verify_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_void_p, C.POINTER(sjd_sample_cfg), C.c_uint32, C.POINTER(sjd_step_out),
+                                    C.c_void_p]
     L.sjd_last_device_status.restype = C.c_int
     L.sjd_last_device_status.argtypes = [C.c_void_p]
     L.sjd_last_cuda_error.restype = C.c_int
@@ -179,6 +183,21 @@ def sjd_verify(logits_cur, logits_prev, draft, q_kind, base_pos, sample: sjd_sam
                           C.byref(sample), C.c_uint32(step), C.byref(out.c), _ptr(ws), ws.numel(), _stream())
     _check(st, "sjd_verify")
     return ws
+
+
+SJD_VERIFY_STATIC_MAX_ROWS, SJD_VERIFY_STATIC_MAX_BATCH = 2048, 256
+
+
+def sjd_verify_static(logits_cur, logits_prev, draft, q_kind, base_pos, sample: sjd_sample_cfg, step: int,
+                      out: StepOut):
+    """sjd_verify for callers that cannot allocate: no scratch argument, the library's built-in
+    scratch array is used (batch * window <= SJD_VERIFY_STATIC_MAX_ROWS).  Calls on one device must
+    not overlap; make the first call on a device outside any stream capture."""
+    b, w, v = logits_cur.shape
+    dt = {torch.float32: SJD_F32, torch.bfloat16: SJD_BF16}[logits_cur.dtype]
+    st = lib().sjd_verify_static(b, w, v, dt, _ptr(logits_cur), _ptr(logits_prev), _ptr(draft), _ptr(q_kind),
+                                 _ptr(base_pos), C.byref(sample), C.c_uint32(step), C.byref(out.c), _stream())
+    _check(st, "sjd_verify_static")
 
 
 class Context:
