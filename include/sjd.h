@@ -227,6 +227,22 @@ int sjd_verify_static(int batch, int window, int vocab, int logits_dtype, const 
                       const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
                       const sjd_step_out *out, void *cuda_stream);
 
+/*
+ * One projection of the forward pass (Sec. 4.1 Step 2) in isolation, on the tensor-core
+ * weight-streaming kernel sjd_step uses for bf16 models:
+ *     out[m][n] (+)= sum_k x[m][k] * w[n][k]      (fp32 accumulation)
+ * x: device fp32 [M][K] (split internally into bf16 hi + lo parts, so activations keep ~16 bits of
+ * mantissa); w: device bf16 [N][K]; out: device fp32 [M][N], overwritten (accumulate = 0) or added
+ * to (accumulate != 0).  Covered shapes: 1 <= M <= 128, N a multiple of 128, K a multiple of 64,
+ * compute capability 10.x; anything else returns SJD_ERR_UNSUPPORTED (sjd_step then uses its generic
+ * kernel).  ws: device scratch of sjd_gemm_workspace_bytes(M, K), 256-byte aligned; after the stream
+ * has drained its first int32 is 0, or non-zero if a bounded device-side wait ran out.
+ * Errors: BAD_ARG, UNSUPPORTED, CAPACITY (ws too small), CUDA.
+ */
+size_t sjd_gemm_workspace_bytes(int M, int K);
+int sjd_gemm(int M, int N, int K, const float *x, const void *w, float *out, int accumulate, void *ws,
+             size_t ws_bytes, void *cuda_stream);
+
 /* Synchronises the context's last stream and returns SJD_OK, SJD_ERR_DEVICE_TIMEOUT
  * or SJD_ERR_CUDA according to the device status word. */
 int sjd_last_device_status(sjd_ctx *ctx);

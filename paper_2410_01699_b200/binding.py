@@ -27,7 +27,8 @@ TORCH_DTYPES = {SJD_F32: torch.float32, SJD_BF16: torch.bfloat16}
 
 EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_get_window", "sjd_peek_logits",
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
-           "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static"]
+           "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static",
+           "sjd_gemm_workspace_bytes", "sjd_gemm"]
 
 
 class SJDError(RuntimeError):
@@ -102,6 +103,11 @@ def lib():
     L.sjd_verify_static.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.POINTER(sjd_sample_cfg), C.c_uint32, C.POINTER(sjd_step_out),
                                     C.c_void_p]
+    L.sjd_gemm_workspace_bytes.restype = C.c_size_t
+    L.sjd_gemm_workspace_bytes.argtypes = [C.c_int, C.c_int]
+    L.sjd_gemm.restype = C.c_int
+    L.sjd_gemm.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                           C.c_size_t, C.c_void_p]
     L.sjd_last_device_status.restype = C.c_int
     L.sjd_last_device_status.argtypes = [C.c_void_p]
     L.sjd_last_cuda_error.restype = C.c_int
@@ -198,6 +204,22 @@ def sjd_verify_static(logits_cur, logits_prev, draft, q_kind, base_pos, sample: 
     st = lib().sjd_verify_static(b, w, v, dt, _ptr(logits_cur), _ptr(logits_prev), _ptr(draft), _ptr(q_kind),
                                  _ptr(base_pos), C.byref(sample), C.c_uint32(step), C.byref(out.c), _stream())
     _check(st, "sjd_verify_static")
+
+
+def sjd_gemm(x, w, out=None, accumulate=False):
+    """out[M][N] (+)= x[M][K] @ w[N][K]^T on the tensor-core weight-streaming kernel.
+    x: float32 cuda, w: bfloat16 cuda.  Returns (out, status word tensor)."""
+    m, k = x.shape
+    n = w.shape[0]
+    if out is None:
+        out = torch.zeros(m, n, dtype=torch.float32, device=x.device)
+    nbytes = int(lib().sjd_gemm_workspace_bytes(m, k))
+    if nbytes == 0:
+        raise SJDError(SJD_ERR_UNSUPPORTED, "sjd_gemm_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=x.device)
+    _check(lib().sjd_gemm(m, n, k, _ptr(x), _ptr(w), _ptr(out), 1 if accumulate else 0, _ptr(ws), nbytes, _stream()),
+           "sjd_gemm")
+    return out, ws[:4].view(torch.int32)
 
 
 class Context:

@@ -154,12 +154,19 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
 }
 
 __global__ void attention_combine_kernel(const float *__restrict__ partial, const int32_t *__restrict__ in_pos,
-                                         float *__restrict__ out, int n_heads, int hd, int splits) {
+                                         float *__restrict__ out, int n_heads, int hd, int splits, HiLoOut hilo) {
   const int m = blockIdx.x, h = blockIdx.y;
   const float *src = partial + ((size_t)m * n_heads + h) * splits * (hd + 2);
-  float *dst = out + ((size_t)m * n_heads + h) * hd;
+  const size_t base = ((size_t)m * n_heads + h) * hd;
+  float *dst = out + base;
   if (in_pos[m] < 0) {
-    for (int d = threadIdx.x; d < hd; d += blockDim.x) dst[d] = 0.0f;
+    for (int d = threadIdx.x; d < hd; d += blockDim.x) {
+      dst[d] = 0.0f;
+      if (hilo.base) {
+        hilo.base[base + d] = __float2bfloat16_rn(0.0f);
+        hilo.base[hilo.lo_offset + base + d] = __float2bfloat16_rn(0.0f);
+      }
+    }
     return;
   }
   float gmax = -INFINITY;
@@ -175,13 +182,19 @@ __global__ void attention_combine_kernel(const float *__restrict__ partial, cons
       const float ms = src[(size_t)s * (hd + 2)];
       if (ms > -INFINITY) acc += src[(size_t)s * (hd + 2) + 2 + d] * expf(ms - gmax);
     }
-    dst[d] = denom > 0.0f ? acc / denom : 0.0f;
+    const float v = denom > 0.0f ? acc / denom : 0.0f;
+    dst[d] = v;
+    if (hilo.base) {
+      const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+      hilo.base[base + d] = hi;
+      hilo.base[hilo.lo_offset + base + d] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
   }
 }
 
 template <typename T>
 int attention_t(const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial, int M, int rows_per_seq,
-                int n_heads, int splits, cudaStream_t stream) {
+                int n_heads, int splits, cudaStream_t stream, HiLoOut hilo) {
   const int hd = kv.head_dim, W = rows_per_seq;
   if (W > NWARPS * MAXQ || hd > 32 * MAXD || M % W != 0) return SJD_ERR_UNSUPPORTED;
   const size_t smem = sizeof(float) * ((size_t)W * hd + TK * (hd + 1) + TK * hd + (size_t)W * TK);
@@ -191,7 +204,7 @@ int attention_t(const float *q, KvLayout kv, const int32_t *in_pos, float *out, 
   attention_partial_kernel<T><<<grid, NWARPS * 32, smem, stream>>>(q, kv, in_pos, partial,
                                                                   W, n_heads, splits);
   SJD_CHECK_LAUNCH();
-  attention_combine_kernel<<<dim3(M, n_heads), 128, 0, stream>>>(partial, in_pos, out, n_heads, hd, splits);
+  attention_combine_kernel<<<dim3(M, n_heads), 128, 0, stream>>>(partial, in_pos, out, n_heads, hd, splits, hilo);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
@@ -199,10 +212,11 @@ int attention_t(const float *q, KvLayout kv, const int32_t *in_pos, float *out, 
 }  // namespace
 
 int launch_attention(int dtype, const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial, int M,
-                     int rows_per_seq, int n_heads, int splits, cudaStream_t stream) {
-  if (dtype == SJD_F32) return attention_t<float>(q, kv, in_pos, out, partial, M, rows_per_seq, n_heads, splits, stream);
+                     int rows_per_seq, int n_heads, int splits, cudaStream_t stream, HiLoOut hilo) {
+  if (dtype == SJD_F32)
+    return attention_t<float>(q, kv, in_pos, out, partial, M, rows_per_seq, n_heads, splits, stream, hilo);
   if (dtype == SJD_BF16)
-    return attention_t<__nv_bfloat16>(q, kv, in_pos, out, partial, M, rows_per_seq, n_heads, splits, stream);
+    return attention_t<__nv_bfloat16>(q, kv, in_pos, out, partial, M, rows_per_seq, n_heads, splits, stream, hilo);
   return SJD_ERR_UNSUPPORTED;
 }
 

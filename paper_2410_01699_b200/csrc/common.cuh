@@ -155,11 +155,33 @@ enum GemmEpilogue { EPI_STORE_F32 = 0, EPI_STORE_T = 1, EPI_ADD_F32 = 2 };
 // C is fp32 (EPI_STORE_F32, EPI_ADD_F32: C += product) or `dtype` (EPI_STORE_T).  lda/ldc in elements.
 int launch_gemm_simt(int dtype, const void *A, int lda, const void *Wt, void *C, int ldc, int M, int N, int K,
                      int epilogue, cudaStream_t stream);
+// ---- tensor-core weight-streaming GEMM (gemm_tc.cu), bf16 weights
+struct alignas(64) TensorMap {   // an encoded TMA descriptor (same size and alignment as the driver's)
+  unsigned char bytes[128];
+};
+// bf16 row-major [rows][cols] matrix cut into boxes of box_rows x 64 columns, 128-byte swizzle
+int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols, int box_rows);
+bool gemm_tc_supported(int M, int N, int K);
+size_t gemm_tc_partial_floats(int n_ctas, int max_rows);
+// out[M][N] (epilogue) = X * W^T with X given as two bf16 planes (hi at row 0, lo at row x_lo_row of
+// x_map, each [rows][K]); partials / tickets / status: device scratch (tickets zero on entry and exit)
+int launch_gemm_tc(const TensorMap &w_map, const TensorMap &x_map, int x_lo_row, void *out, int ldc, int M, int N, int K,
+                   int epilogue, float *partials, int *tickets, int *status, int n_ctas, cudaStream_t stream);
+// Optional second output of the activation-producing kernels: the value split as bf16 hi + bf16 lo
+// (hi = bf16(v), lo = bf16(v - hi)), planes `lo_offset` elements apart, row stride = row length.
+struct HiLoOut {
+  __nv_bfloat16 *base;   // null: not wanted
+  size_t lo_offset;
+};
+
+int launch_split_hilo(const float *x, HiLoOut o, size_t total, cudaStream_t stream);
+
 // x[m][:] = tok_emb[tok[m]][:]  (fp32 residual stream)
 int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, int M, int d, int vocab,
                  cudaStream_t stream);
 // h[m][:] = x[m][:] * gain[:] / sqrt(mean(x[m]^2) + eps)  (gain of `dtype`)
-int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M, int d, float eps, cudaStream_t stream);
+int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M, int d, float eps, cudaStream_t stream,
+                   HiLoOut hilo = HiLoOut{nullptr, 0});
 // Rotate q and k by their absolute position (pairs i, i + hd/2), store q as fp32 [M][H*hd],
 // append k and v to the cache row in_pos[m] of sequence m / rows_per_seq.  Rows with in_pos < 0 are skipped.
 struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
@@ -169,10 +191,11 @@ struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
 int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
                        KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
 // act[m][f] = silu(gu[m][f]) * gu[m][F + f]
-int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream);
+int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream, HiLoOut hilo = HiLoOut{nullptr, 0});
 // Window-causal attention: query row m (sequence m / rows_per_seq, position in_pos[m]) attends cache rows
 // 0 .. in_pos[m].  q, out: fp32 [M][H*hd]; cache of `dtype`.  partial: fp32 scratch [M][H][splits][hd + 2].
 int launch_attention(int dtype, const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial,
-                     int M, int rows_per_seq, int n_heads, int splits, cudaStream_t stream);
+                     int M, int rows_per_seq, int n_heads, int splits, cudaStream_t stream,
+                     HiLoOut hilo = HiLoOut{nullptr, 0});
 
 }  // namespace sjd

@@ -5,6 +5,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <map>
 #include <new>
 #include <vector>
 
@@ -21,9 +22,24 @@ int attention_splits(int n_heads, int batch) {
   return s < 1 ? 1 : (s > 16 ? 16 : s);
 }
 
+constexpr int kMaxGemmCtas = 160;    // persistent CTAs of the tensor-core GEMM (one per SM)
+constexpr int kMaxGemmTiles = 4096;  // 128-row weight tiles per matrix (vocabulary up to 524288)
+
+struct WMap {
+  TensorMap map;
+  bool valid = false;
+};
+struct LayerMaps {
+  WMap wq, wk, wv, wo, w_gate, w_up, w_down;
+};
+struct XMaps {
+  TensorMap h, attn, act;
+};
+
 struct Layout {
   size_t kv, logits[2], stats[2], row_out, counters, step, status;
   size_t x, h, qkv, q, attn, gu, act, partial, rope;
+  size_t xs_h, xs_attn, xs_act, gemm_partials, gemm_tickets;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t total;
 };
@@ -71,6 +87,13 @@ Layout make_layout(const sjd_model_cfg &c) {
     part = need > part ? need : part;
   }
   L.partial = take(part * 4);
+  // bf16 hi/lo planes of the GEMM inputs, stream-K partials and tickets (tensor-core path)
+  const size_t Ma = (Mx + 15) / 16 * 16;
+  L.xs_h = take(2 * Ma * c.d_model * 2);
+  L.xs_attn = take(2 * Ma * nq * 2);
+  L.xs_act = take(2 * Ma * c.ffn_hidden * 2);
+  L.gemm_partials = take(gemm_tc_partial_floats(kMaxGemmCtas, (int)(Ma < 128 ? Ma : 128)) * 4);
+  L.gemm_tickets = take(kMaxGemmTiles * 4);
   L.rope = take((size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2));
   L.committed = take((size_t)c.max_batch * c.max_seq * 4);
   L.n = take((size_t)c.max_batch * 4);
@@ -185,6 +208,12 @@ struct sjd_ctx {
   uint32_t host_step;  // number of sjd_step calls since prefill == device step index
   cudaStream_t last_stream;
   Tracer tracer;
+  bool use_tc = false;   // bf16 model on a device with tensor memory: tensor-core GEMM path
+  int n_ctas = 0;
+  std::vector<LayerMaps> wmaps;
+  WMap wmap_head;
+  std::map<int, XMaps> xmaps;   // keyed by padded row count
+  int rows_alloc() const { return ((cfg.max_batch * cfg.max_window) + 15) / 16 * 16; }
 
   template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
   SeqState state() const {
@@ -242,28 +271,56 @@ int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream)
   const double es = (double)esize(dt);
 #define SJD_TRY(call) do { rc = (call); if (rc != SJD_OK) return rc; } while (0)
 #define SJD_TR(klass, call) do { tr.begin(klass, stream); rc = (call); tr.end(stream); if (rc != SJD_OK) return rc; } while (0)
-#define SJD_GEMM(n_out, k_in, call) do { if (tr.on) tr.gemm_weight_bytes += (double)(n_out) * (double)(k_in) * es; SJD_TR(TC_GEMM, call); } while (0)
+  // activations as bf16 hi/lo planes for the tensor-core GEMM (only when that path is live)
+  const bool tc = c->use_tc && M <= 128;
+  const int Ma = c->rows_alloc();
+  const HiLoOut hl_h{tc ? c->at<__nv_bfloat16>(c->lay.xs_h) : nullptr, (size_t)Ma * d};
+  const HiLoOut hl_attn{tc ? c->at<__nv_bfloat16>(c->lay.xs_attn) : nullptr, (size_t)Ma * nq};
+  const HiLoOut hl_act{tc ? c->at<__nv_bfloat16>(c->lay.xs_act) : nullptr, (size_t)Ma * F};
+  const int Mp = (M + 15) / 16 * 16;
+  const XMaps *xm = nullptr;
+  if (tc) {
+    auto it = c->xmaps.find(Mp);
+    if (it != c->xmaps.end()) xm = &it->second;
+  }
+  // xsel: 0 = normalised hidden state, 1 = attention output, 2 = SwiGLU output
+  auto gemm = [&](int xsel, const WMap &wm, const void *w, const float *a, int lda, void *out, int ldc, int n_out,
+                  int k_in, int epi) -> int {
+    if (tr.on) tr.gemm_weight_bytes += (double)n_out * (double)k_in * es;
+    tr.begin(TC_GEMM, stream);
+    int r;
+    if (xm && wm.valid && gemm_tc_supported(M, n_out, k_in)) {
+      const TensorMap &x_map = xsel == 0 ? xm->h : xsel == 1 ? xm->attn : xm->act;
+      r = launch_gemm_tc(wm.map, x_map, Ma, out, ldc, M, n_out, k_in, epi, c->at<float>(c->lay.gemm_partials),
+                         c->at<int>(c->lay.gemm_tickets), c->at<int>(c->lay.status), c->n_ctas, stream);
+    } else {
+      r = launch_gemm_simt(dt, a, lda, w, out, ldc, M, n_out, k_in, epi, stream);
+    }
+    tr.end(stream);
+    return r;
+  };
   SJD_TR(TC_OTHER, launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
   for (int l = 0; l < g.n_layers; ++l) {
-    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream));
-    SJD_GEMM(nq, d, launch_gemm_simt(dt, h, d, c->wq[l], qkv, nqkv, M, nq, d, EPI_STORE_F32, stream));
-    SJD_GEMM(nk, d, launch_gemm_simt(dt, h, d, c->wk[l], qkv + nq, nqkv, M, nk, d, EPI_STORE_F32, stream));
-    SJD_GEMM(nk, d, launch_gemm_simt(dt, h, d, c->wv[l], qkv + nq + nk, nqkv, M, nk, d, EPI_STORE_F32, stream));
+    const LayerMaps &lm = c->wmaps[l];
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream, hl_h));
+    SJD_TRY(gemm(0, lm.wq, c->wq[l], h, d, qkv, nqkv, nq, d, EPI_STORE_F32));
+    SJD_TRY(gemm(0, lm.wk, c->wk[l], h, d, qkv + nq, nqkv, nk, d, EPI_STORE_F32));
+    SJD_TRY(gemm(0, lm.wv, c->wv[l], h, d, qkv + nq + nk, nqkv, nk, d, EPI_STORE_F32));
     const KvLayout kv = c->kv_layer(l);
     SJD_TR(TC_OTHER, launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
-    SJD_TR(TC_ATTENTION, launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream));
-    SJD_GEMM(d, nq, launch_gemm_simt(dt, attn, nq, c->wo[l], x, d, M, d, nq, EPI_ADD_F32, stream));
-    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream));
-    SJD_GEMM(F, d, launch_gemm_simt(dt, h, d, c->w_gate[l], gu, 2 * F, M, F, d, EPI_STORE_F32, stream));
-    SJD_GEMM(F, d, launch_gemm_simt(dt, h, d, c->w_up[l], gu + F, 2 * F, M, F, d, EPI_STORE_F32, stream));
-    SJD_TR(TC_OTHER, launch_swiglu(gu, act, M, F, stream));
-    SJD_GEMM(d, F, launch_gemm_simt(dt, act, F, c->w_down[l], x, d, M, d, F, EPI_ADD_F32, stream));
+    SJD_TR(TC_ATTENTION,
+           launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream, hl_attn));
+    SJD_TRY(gemm(1, lm.wo, c->wo[l], attn, nq, x, d, d, nq, EPI_ADD_F32));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream, hl_h));
+    SJD_TRY(gemm(0, lm.w_gate, c->w_gate[l], h, d, gu, 2 * F, F, d, EPI_STORE_F32));
+    SJD_TRY(gemm(0, lm.w_up, c->w_up[l], h, d, gu + F, 2 * F, F, d, EPI_STORE_F32));
+    SJD_TR(TC_OTHER, launch_swiglu(gu, act, M, F, stream, hl_act));
+    SJD_TRY(gemm(2, lm.w_down, c->w_down[l], act, F, x, d, d, F, EPI_ADD_F32));
   }
   if (logits_out) {
-    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream));
-    SJD_GEMM(g.vocab, d, launch_gemm_simt(dt, h, d, c->lm_head, logits_out, g.vocab, M, g.vocab, d, EPI_STORE_T, stream));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream, hl_h));
+    SJD_TRY(gemm(0, c->wmap_head, c->lm_head, h, d, logits_out, g.vocab, g.vocab, d, EPI_STORE_T));
   }
-#undef SJD_GEMM
 #undef SJD_TR
 #undef SJD_TRY
   return SJD_OK;
@@ -369,6 +426,33 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
     delete c;
     return SJD_ERR_CUDA;
   }
+  // tensor-core path: bf16 weights on a device of compute capability 10.x; one TMA descriptor per
+  // weight matrix whose shape the kernel covers (the others use the generic kernel)
+  c->wmaps.resize(L);
+  int dev = 0, cc_major = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && cfg->dtype == SJD_BF16 &&
+      cc_major == 10 && sms > 0) {
+    c->use_tc = true;
+    c->n_ctas = sms < kMaxGemmCtas ? sms : kMaxGemmCtas;
+    const int d = cfg->d_model, F = cfg->ffn_hidden;
+    const int nq = cfg->n_heads * cfg->head_dim, nk = cfg->n_kv_heads * cfg->head_dim;
+    auto mk = [&](WMap &m, const void *w, int n_out, int k_in) {
+      m.valid = n_out % 128 == 0 && k_in % 64 == 0 && n_out / 128 <= kMaxGemmTiles &&
+                make_tensor_map_bf16(&m.map, w, n_out, k_in, 128) == SJD_OK;
+    };
+    for (int l = 0; l < L; ++l) {
+      LayerMaps &lm = c->wmaps[l];
+      mk(lm.wq, c->wq[l], nq, d);
+      mk(lm.wk, c->wk[l], nk, d);
+      mk(lm.wv, c->wv[l], nk, d);
+      mk(lm.wo, c->wo[l], d, nq);
+      mk(lm.w_gate, c->w_gate[l], F, d);
+      mk(lm.w_up, c->w_up[l], F, d);
+      mk(lm.w_down, c->w_down[l], d, F);
+    }
+    mk(c->wmap_head, c->lm_head, cfg->vocab, d);
+  }
   *out = c;
   return SJD_OK;
 }
@@ -389,6 +473,21 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
   c->host_step = 0;
   c->last_stream = stream;
   c->prefilled = false;
+  if (c->use_tc) {
+    // activation descriptors for the two row counts used: the step's window and the pre-fill chunk
+    const int Ma = c->rows_alloc();
+    const int nq = c->cfg.n_heads * c->cfg.head_dim;
+    const int row_counts[2] = {batch * sample->window, batch * c->cfg.max_window};
+    for (int i = 0; i < 2; ++i) {
+      const int Mp = (row_counts[i] + 15) / 16 * 16;
+      if (row_counts[i] > 128 || c->xmaps.count(Mp)) continue;
+      XMaps xm;
+      const bool ok = make_tensor_map_bf16(&xm.h, c->ws + c->lay.xs_h, 2L * Ma, c->cfg.d_model, Mp) == SJD_OK &&
+                      make_tensor_map_bf16(&xm.attn, c->ws + c->lay.xs_attn, 2L * Ma, nq, Mp) == SJD_OK &&
+                      make_tensor_map_bf16(&xm.act, c->ws + c->lay.xs_act, 2L * Ma, c->cfg.ffn_hidden, Mp) == SJD_OK;
+      if (ok) c->xmaps[Mp] = xm;
+    }
+  }
   const SeqState st = c->state();
   prefill_setup_kernel<<<batch, 128, 0, stream>>>(prompt, prompt_len, st, c->at<uint32_t>(c->lay.step),
                                                   c->at<int32_t>(c->lay.counters), batch);

@@ -14,6 +14,13 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+__device__ __forceinline__ void store_hilo(const HiLoOut &o, size_t idx, float v) {
+  if (!o.base) return;
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  o.base[idx] = hi;
+  o.base[o.lo_offset + idx] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
 // ------------------------------------------------------------------------------------ GEMM (FMA)
 // 32 x 64 output tile per block of 256 threads, K in slices of 32; every access is bounds-checked so
 // any M, N, K (683, 1408, ...) works.  Sums run over k in increasing order: deterministic.
@@ -96,7 +103,7 @@ __global__ void embed_kernel(const T *__restrict__ emb, const int32_t *__restric
 // ------------------------------------------------------------------------------------ RMSNorm
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ gain,
-                                                      float *__restrict__ h, int d, float eps) {
+                                                      float *__restrict__ h, int d, float eps, HiLoOut hilo) {
   __shared__ float red[8];
   const int m = blockIdx.x, tid = threadIdx.x;
   const float *row = x + (size_t)m * d;
@@ -109,7 +116,11 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
 #pragma unroll
   for (int w = 0; w < 8; ++w) tot += red[w];
   const float scale = rsqrtf(tot / (float)d + eps);
-  for (int i = tid; i < d; i += 256) h[(size_t)m * d + i] = row[i] * scale * to_f<T>(gain[i]);
+  for (int i = tid; i < d; i += 256) {
+    const float v = row[i] * scale * to_f<T>(gain[i]);
+    h[(size_t)m * d + i] = v;
+    store_hilo(hilo, (size_t)m * d + i, v);
+  }
 }
 
 // ------------------------------------------------------------------------------------ RoPE + KV append
@@ -150,12 +161,14 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t 
 }
 
 // ------------------------------------------------------------------------------------ SwiGLU
-__global__ void swiglu_kernel(const float *__restrict__ gu, float *__restrict__ act, int M, int F) {
+__global__ void swiglu_kernel(const float *__restrict__ gu, float *__restrict__ act, int M, int F, HiLoOut hilo) {
   const size_t total = (size_t)M * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t m = i / F, f = i % F;
     const float g = gu[m * 2 * F + f], u = gu[m * 2 * F + F + f];
-    act[i] = g / (1.0f + expf(-g)) * u;
+    const float v = g / (1.0f + expf(-g)) * u;
+    act[i] = v;
+    store_hilo(hilo, i, v);
   }
 }
 
@@ -181,8 +194,9 @@ int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, i
   return SJD_OK;
 }
 
-int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M, int d, float eps, cudaStream_t stream) {
-  SJD_DISPATCH(dtype, (rmsnorm_kernel<T><<<M, 256, 0, stream>>>(x, reinterpret_cast<const T *>(gain), h, d, eps)));
+int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M, int d, float eps, cudaStream_t stream,
+                   HiLoOut hilo) {
+  SJD_DISPATCH(dtype, (rmsnorm_kernel<T><<<M, 256, 0, stream>>>(x, reinterpret_cast<const T *>(gain), h, d, eps, hilo)));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
@@ -195,12 +209,29 @@ int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const
   return SJD_OK;
 }
 
-int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream) {
+int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream, HiLoOut hilo) {
   const size_t total = (size_t)M * F;
   const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
-  swiglu_kernel<<<blocks, 256, 0, stream>>>(gu, act, M, F);
+  swiglu_kernel<<<blocks, 256, 0, stream>>>(gu, act, M, F, hilo);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
 
+}  // namespace sjd
+
+namespace sjd {
+namespace {
+__global__ void split_hilo_kernel(const float *__restrict__ x, HiLoOut o, size_t total) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+    store_hilo(o, i, x[i]);
+}
+}  // namespace
+
+// hi/lo bf16 planes of an fp32 matrix (same row stride), for the tensor-core GEMM
+int launch_split_hilo(const float *x, HiLoOut o, size_t total, cudaStream_t stream) {
+  const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
+  split_hilo_kernel<<<blocks, 256, 0, stream>>>(x, o, total);
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
 }  // namespace sjd
