@@ -421,6 +421,7 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
   cudaError_t e = cudaMemcpy(c->ws + lay.rope, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.counters, 0, ((size_t)cfg->max_batch + 1) * 4);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.status, 0, 4);
+  if (e == cudaSuccess) e = cudaMemset(c->ws + lay.gemm_tickets, 0, (size_t)kMaxGemmTiles * 4);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     delete c;
