@@ -235,11 +235,11 @@ int sjd_verify_static(int batch, int window, int vocab, int logits_dtype, const 
  * mantissa); w: device bf16 [N][K]; out: device fp32 [M][N], overwritten (accumulate = 0) or added
  * to (accumulate != 0).  Covered shapes: 1 <= M <= 128, N a multiple of 128, K a multiple of 64,
  * compute capability 10.x; anything else returns SJD_ERR_UNSUPPORTED (sjd_step then uses its generic
- * kernel).  ws: device scratch of sjd_gemm_workspace_bytes(M, K), 256-byte aligned; after the stream
+ * kernel).  ws: device scratch of sjd_gemm_workspace_bytes(M, N, K), 256-byte aligned; after the stream
  * has drained its first int32 is 0, or non-zero if a bounded device-side wait ran out.
  * Errors: BAD_ARG, UNSUPPORTED, CAPACITY (ws too small), CUDA.
  */
-size_t sjd_gemm_workspace_bytes(int M, int K);
+size_t sjd_gemm_workspace_bytes(int M, int N, int K);
 int sjd_gemm(int M, int N, int K, const float *x, const void *w, float *out, int accumulate, void *ws,
              size_t ws_bytes, void *cuda_stream);
 

@@ -104,7 +104,7 @@ def lib():
                                     C.c_void_p, C.POINTER(sjd_sample_cfg), C.c_uint32, C.POINTER(sjd_step_out),
                                     C.c_void_p]
     L.sjd_gemm_workspace_bytes.restype = C.c_size_t
-    L.sjd_gemm_workspace_bytes.argtypes = [C.c_int, C.c_int]
+    L.sjd_gemm_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
     L.sjd_gemm.restype = C.c_int
     L.sjd_gemm.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                            C.c_size_t, C.c_void_p]
@@ -213,7 +213,7 @@ def sjd_gemm(x, w, out=None, accumulate=False):
     n = w.shape[0]
     if out is None:
         out = torch.zeros(m, n, dtype=torch.float32, device=x.device)
-    nbytes = int(lib().sjd_gemm_workspace_bytes(m, k))
+    nbytes = int(lib().sjd_gemm_workspace_bytes(m, n, k))
     if nbytes == 0:
         raise SJDError(SJD_ERR_UNSUPPORTED, "sjd_gemm_workspace_bytes")
     ws = torch.empty(nbytes, dtype=torch.uint8, device=x.device)

@@ -91,35 +91,37 @@ extern "C" const char *sjd_strerror(int status) {
 // ---- the projection of Step 2 in isolation (tensor-core weight-streaming GEMM)
 namespace {
 inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
-constexpr int kGemmCtasMax = 160, kGemmTilesMax = 4096;
+constexpr int kGemmSmsMax = 160;
 }  // namespace
 
-extern "C" size_t sjd_gemm_workspace_bytes(int M, int K) {
-  if (M < 1 || M > 128 || K < 1) return 0;
+extern "C" size_t sjd_gemm_workspace_bytes(int M, int N, int K) {
+  if (!gemm_tc_supported(M, N, K)) return 0;
   const int mp = (M + 15) / 16 * 16;
-  return 256 + up256((size_t)kGemmTilesMax * 4) + up256(gemm_tc_partial_floats(kGemmCtasMax, mp) * 4) +
-         up256((size_t)2 * mp * K * 2);
+  const int splits = gemm_tc_splits(N / 128, K / 64, kGemmSmsMax);
+  return 256 + up256((size_t)splits * M * N * 4) + up256((size_t)2 * mp * K * 2);
 }
 
 extern "C" int sjd_gemm(int M, int N, int K, const float *x, const void *w, float *out, int accumulate, void *ws,
                         size_t ws_bytes, void *cuda_stream) {
   if (M < 1 || N < 1 || K < 1 || !x || !w || !out || !ws) return SJD_ERR_BAD_ARG;
-  if (!gemm_tc_supported(M, N, K) || N / 128 > kGemmTilesMax) return SJD_ERR_UNSUPPORTED;
+  if (!gemm_tc_supported(M, N, K)) return SJD_ERR_UNSUPPORTED;
   if (((uintptr_t)ws & 255u) != 0) return SJD_ERR_BAD_ARG;
-  if (ws_bytes < sjd_gemm_workspace_bytes(M, K)) return SJD_ERR_CAPACITY;
+  if (ws_bytes < sjd_gemm_workspace_bytes(M, N, K)) return SJD_ERR_CAPACITY;
   int dev = 0, cc_major = 0, sms = 0;
   SJD_CUDA(cudaGetDevice(&dev));
   SJD_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
   SJD_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   if (cc_major != 10) return SJD_ERR_UNSUPPORTED;
+  sms = sms < kGemmSmsMax ? sms : kGemmSmsMax;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   const int mp = (M + 15) / 16 * 16;
+  const int splits = gemm_tc_splits(N / 128, K / 64, sms);
+  const int splits_max = gemm_tc_splits(N / 128, K / 64, kGemmSmsMax);
   char *p = (char *)ws;
   int *status = (int *)p;
-  int *tickets = (int *)(p + 256);
-  float *partials = (float *)(p + 256 + up256((size_t)kGemmTilesMax * 4));
-  __nv_bfloat16 *xs = (__nv_bfloat16 *)((char *)partials + up256(gemm_tc_partial_floats(kGemmCtasMax, mp) * 4));
-  SJD_CUDA(cudaMemsetAsync(p, 0, 256 + up256((size_t)kGemmTilesMax * 4), stream));
+  float *planes = (float *)(p + 256);
+  __nv_bfloat16 *xs = (__nv_bfloat16 *)(p + 256 + up256((size_t)splits_max * M * N * 4));
+  SJD_CUDA(cudaMemsetAsync(p, 0, 256, stream));
   SJD_CUDA(cudaMemsetAsync(xs, 0, (size_t)2 * mp * K * 2, stream));
   int rc = launch_split_hilo(x, HiLoOut{xs, (size_t)mp * K}, (size_t)M * K, stream);
   if (rc != SJD_OK) return rc;
@@ -128,6 +130,22 @@ extern "C" int sjd_gemm(int M, int N, int K, const float *x, const void *w, floa
   if (rc != SJD_OK) return rc;
   rc = make_tensor_map_bf16(&xm, xs, 2L * mp, K, mp);
   if (rc != SJD_OK) return rc;
-  return launch_gemm_tc(wm, xm, mp, out, N, M, N, K, accumulate ? EPI_ADD_F32 : EPI_STORE_F32, partials, tickets, status,
-                        sms < kGemmCtasMax ? sms : kGemmCtasMax, stream);
+  GemmTcCall g;
+  memset(&g, 0, sizeof(g));
+  g.w_map[0] = g.w_map[1] = g.w_map[2] = &wm;
+  g.n_mats = 1;
+  g.n_out[0] = N;
+  g.x_map = &xm;
+  g.x_lo_row = mp;
+  g.M = M;
+  g.K = K;
+  g.splits = splits;
+  g.out = planes;
+  g.plane_stride = (size_t)M * N;
+  g.ldc = N;
+  g.store_bf16 = 0;
+  g.status = status;
+  rc = launch_gemm_tc(g, stream);
+  if (rc != SJD_OK) return rc;
+  return launch_sum_planes(planes, (size_t)M * N, splits, out, (size_t)M * N, accumulate, stream);
 }

@@ -162,11 +162,35 @@ struct alignas(64) TensorMap {   // an encoded TMA descriptor (same size and ali
 // bf16 row-major [rows][cols] matrix cut into boxes of box_rows x 64 columns, 128-byte swizzle
 int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols, int box_rows);
 bool gemm_tc_supported(int M, int N, int K);
-size_t gemm_tc_partial_floats(int n_ctas, int max_rows);
-// out[M][N] (epilogue) = X * W^T with X given as two bf16 planes (hi at row 0, lo at row x_lo_row of
-// x_map, each [rows][K]); partials / tickets / status: device scratch (tickets zero on entry and exit)
-int launch_gemm_tc(const TensorMap &w_map, const TensorMap &x_map, int x_lo_row, void *out, int ldc, int M, int N, int K,
-                   int epilogue, float *partials, int *tickets, int *status, int n_ctas, cudaStream_t stream);
+int gemm_tc_splits(int tiles, int k_blocks, int n_sms);
+// One launch over up to three weight matrices that share the activation operand X (two bf16 planes:
+// hi at row 0, lo at row x_lo_row of x_map, each [rows][K]).  Matrix j has n_out[j] rows and writes
+// output columns [col_off[j], col_off[j] + n_out[j]).  splits > 1 (or store_bf16 == 0): fp32 planes
+// out[s][m][ldc], plane_stride elements apart, one per K split; store_bf16 (splits == 1): bf16 out[m][ldc].
+struct GemmTcCall {
+  const TensorMap *w_map[3];
+  int n_mats;
+  int n_out[3], col_off[3];
+  const TensorMap *x_map;
+  int x_lo_row;
+  int M, K;
+  int splits;
+  void *out;
+  size_t plane_stride;
+  int ldc;
+  int store_bf16;
+  int *status;
+};
+int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream);
+int launch_sum_planes(const float *planes, size_t plane_stride, int splits, float *out, size_t total, int accumulate,
+                      cudaStream_t stream);
+// The fp32 partial planes a GEMM launch left: value(m, col) = sum_s base[s * plane_stride + m * ld + col]
+struct PlaneSet {
+  const float *base;
+  size_t plane_stride;
+  int ld;
+  int splits;     // 0: no planes (nothing to add)
+};
 // Optional second output of the activation-producing kernels: the value split as bf16 hi + bf16 lo
 // (hi = bf16(v), lo = bf16(v - hi)), planes `lo_offset` elements apart, row stride = row length.
 struct HiLoOut {
@@ -175,6 +199,11 @@ struct HiLoOut {
 };
 
 int launch_split_hilo(const float *x, HiLoOut o, size_t total, cudaStream_t stream);
+// consumer kernels of the tensor-core path (fused_kernels.cu)
+struct KvLayout;
+int launch_resid_norm(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOut h, int M, int d, float eps,
+                      cudaStream_t stream);
+int launch_swiglu_finish(PlaneSet ps, HiLoOut act, int M, int F, cudaStream_t stream);
 
 // x[m][:] = tok_emb[tok[m]][:]  (fp32 residual stream)
 int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, int M, int d, int vocab,
@@ -190,6 +219,8 @@ struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
 };
 int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
                        KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
+int launch_qkv_finish(int dtype, PlaneSet ps, const int32_t *in_pos, const float2 *rope_table, float *q, KvLayout kv, int M,
+                      int rows_per_seq, int n_heads, cudaStream_t stream);
 // act[m][f] = silu(gu[m][f]) * gu[m][F + f]
 int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream, HiLoOut hilo = HiLoOut{nullptr, 0});
 // Window-causal attention: query row m (sequence m / rows_per_seq, position in_pos[m]) attends cache rows

@@ -22,8 +22,7 @@ int attention_splits(int n_heads, int batch) {
   return s < 1 ? 1 : (s > 16 ? 16 : s);
 }
 
-constexpr int kMaxGemmCtas = 160;    // persistent CTAs of the tensor-core GEMM (one per SM)
-constexpr int kMaxGemmTiles = 4096;  // 128-row weight tiles per matrix (vocabulary up to 524288)
+constexpr int kMaxGemmCtas = 160;    // upper bound on the SM count used to size split-K scratch
 
 struct WMap {
   TensorMap map;
@@ -39,7 +38,7 @@ struct XMaps {
 struct Layout {
   size_t kv, logits[2], stats[2], row_out, counters, step, status;
   size_t x, h, qkv, q, attn, gu, act, partial, rope;
-  size_t xs_h, xs_attn, xs_act, gemm_partials, gemm_tickets;
+  size_t xs_h, xs_attn, xs_act, gemm_planes;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t total;
 };
@@ -92,8 +91,19 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.xs_h = take(2 * Ma * c.d_model * 2);
   L.xs_attn = take(2 * Ma * nq * 2);
   L.xs_act = take(2 * Ma * c.ffn_hidden * 2);
-  L.gemm_partials = take(gemm_tc_partial_floats(kMaxGemmCtas, (int)(Ma < 128 ? Ma : 128)) * 4);
-  L.gemm_tickets = take(kMaxGemmTiles * 4);
+  {
+    // fp32 partial planes of one GEMM launch: the largest splits * rows * columns over the launches
+    const int rows = (int)(Mx < 128 ? Mx : 128);
+    const int tiles[4] = {(int)((nq + 2 * nk) / 128), c.d_model / 128, 2 * c.ffn_hidden / 128, c.d_model / 128};
+    const int kbs[4] = {c.d_model / 64, (int)(nq / 64), c.d_model / 64, c.ffn_hidden / 64};
+    const size_t cols[4] = {nq + 2 * nk, (size_t)c.d_model, (size_t)2 * c.ffn_hidden, (size_t)c.d_model};
+    size_t need = 0;
+    for (int i = 0; i < 4; ++i) {
+      const size_t n = (size_t)gemm_tc_splits(tiles[i] > 0 ? tiles[i] : 1, kbs[i], kMaxGemmCtas) * rows * cols[i];
+      need = n > need ? n : need;
+    }
+    L.gemm_planes = take(need * 4);
+  }
   L.rope = take((size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2));
   L.committed = take((size_t)c.max_batch * c.max_seq * 4);
   L.n = take((size_t)c.max_batch * 4);
@@ -209,6 +219,7 @@ struct sjd_ctx {
   cudaStream_t last_stream;
   Tracer tracer;
   bool use_tc = false;   // bf16 model on a device with tensor memory: tensor-core GEMM path
+  bool all_tc = false;   // every projection of the model is covered by it
   int n_ctas = 0;
   std::vector<LayerMaps> wmaps;
   WMap wmap_head;
@@ -249,7 +260,12 @@ namespace sjd {
 namespace {
 
 // One forward pass of M = batch * rows_per_seq rows whose tokens / positions are in st.in_tok / in_pos.
-int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream) {
+// Two pipelines: the tensor-core one (bf16 model, every projection covered by the weight-streaming
+// GEMM: partial planes + fused consumer kernels) and the generic one (any dtype and shape).
+#define SJD_TRY(call) do { rc = (call); if (rc != SJD_OK) return rc; } while (0)
+#define SJD_TR(klass, call) do { tr.begin(klass, stream); rc = (call); tr.end(stream); if (rc != SJD_OK) return rc; } while (0)
+
+int forward_generic(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream) {
   const sjd_model_cfg &g = c->cfg;
   const int dt = g.dtype;
   const int M = c->batch * rows_per_seq;
@@ -269,61 +285,142 @@ int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream)
   int rc;
   Tracer &tr = c->tracer;
   const double es = (double)esize(dt);
-#define SJD_TRY(call) do { rc = (call); if (rc != SJD_OK) return rc; } while (0)
-#define SJD_TR(klass, call) do { tr.begin(klass, stream); rc = (call); tr.end(stream); if (rc != SJD_OK) return rc; } while (0)
-  // activations as bf16 hi/lo planes for the tensor-core GEMM (only when that path is live)
-  const bool tc = c->use_tc && M <= 128;
-  const int Ma = c->rows_alloc();
-  const HiLoOut hl_h{tc ? c->at<__nv_bfloat16>(c->lay.xs_h) : nullptr, (size_t)Ma * d};
-  const HiLoOut hl_attn{tc ? c->at<__nv_bfloat16>(c->lay.xs_attn) : nullptr, (size_t)Ma * nq};
-  const HiLoOut hl_act{tc ? c->at<__nv_bfloat16>(c->lay.xs_act) : nullptr, (size_t)Ma * F};
-  const int Mp = (M + 15) / 16 * 16;
-  const XMaps *xm = nullptr;
-  if (tc) {
-    auto it = c->xmaps.find(Mp);
-    if (it != c->xmaps.end()) xm = &it->second;
-  }
-  // xsel: 0 = normalised hidden state, 1 = attention output, 2 = SwiGLU output
-  auto gemm = [&](int xsel, const WMap &wm, const void *w, const float *a, int lda, void *out, int ldc, int n_out,
-                  int k_in, int epi) -> int {
+  auto gemm = [&](const void *w, const float *a, int lda, void *out, int ldc, int n_out, int k_in, int epi) -> int {
     if (tr.on) tr.gemm_weight_bytes += (double)n_out * (double)k_in * es;
     tr.begin(TC_GEMM, stream);
-    int r;
-    if (xm && wm.valid && gemm_tc_supported(M, n_out, k_in)) {
-      const TensorMap &x_map = xsel == 0 ? xm->h : xsel == 1 ? xm->attn : xm->act;
-      r = launch_gemm_tc(wm.map, x_map, Ma, out, ldc, M, n_out, k_in, epi, c->at<float>(c->lay.gemm_partials),
-                         c->at<int>(c->lay.gemm_tickets), c->at<int>(c->lay.status), c->n_ctas, stream);
-    } else {
-      r = launch_gemm_simt(dt, a, lda, w, out, ldc, M, n_out, k_in, epi, stream);
-    }
+    const int r = launch_gemm_simt(dt, a, lda, w, out, ldc, M, n_out, k_in, epi, stream);
     tr.end(stream);
     return r;
   };
   SJD_TR(TC_OTHER, launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
   for (int l = 0; l < g.n_layers; ++l) {
-    const LayerMaps &lm = c->wmaps[l];
-    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream, hl_h));
-    SJD_TRY(gemm(0, lm.wq, c->wq[l], h, d, qkv, nqkv, nq, d, EPI_STORE_F32));
-    SJD_TRY(gemm(0, lm.wk, c->wk[l], h, d, qkv + nq, nqkv, nk, d, EPI_STORE_F32));
-    SJD_TRY(gemm(0, lm.wv, c->wv[l], h, d, qkv + nq + nk, nqkv, nk, d, EPI_STORE_F32));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->attn_norm[l], h, M, d, g.rms_eps, stream));
+    SJD_TRY(gemm(c->wq[l], h, d, qkv, nqkv, nq, d, EPI_STORE_F32));
+    SJD_TRY(gemm(c->wk[l], h, d, qkv + nq, nqkv, nk, d, EPI_STORE_F32));
+    SJD_TRY(gemm(c->wv[l], h, d, qkv + nq + nk, nqkv, nk, d, EPI_STORE_F32));
     const KvLayout kv = c->kv_layer(l);
     SJD_TR(TC_OTHER, launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
-    SJD_TR(TC_ATTENTION,
-           launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream, hl_attn));
-    SJD_TRY(gemm(1, lm.wo, c->wo[l], attn, nq, x, d, d, nq, EPI_ADD_F32));
-    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream, hl_h));
-    SJD_TRY(gemm(0, lm.w_gate, c->w_gate[l], h, d, gu, 2 * F, F, d, EPI_STORE_F32));
-    SJD_TRY(gemm(0, lm.w_up, c->w_up[l], h, d, gu + F, 2 * F, F, d, EPI_STORE_F32));
-    SJD_TR(TC_OTHER, launch_swiglu(gu, act, M, F, stream, hl_act));
-    SJD_TRY(gemm(2, lm.w_down, c->w_down[l], act, F, x, d, d, F, EPI_ADD_F32));
+    SJD_TR(TC_ATTENTION, launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream));
+    SJD_TRY(gemm(c->wo[l], attn, nq, x, d, d, nq, EPI_ADD_F32));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream));
+    SJD_TRY(gemm(c->w_gate[l], h, d, gu, 2 * F, F, d, EPI_STORE_F32));
+    SJD_TRY(gemm(c->w_up[l], h, d, gu + F, 2 * F, F, d, EPI_STORE_F32));
+    SJD_TR(TC_OTHER, launch_swiglu(gu, act, M, F, stream));
+    SJD_TRY(gemm(c->w_down[l], act, F, x, d, d, F, EPI_ADD_F32));
   }
   if (logits_out) {
-    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream, hl_h));
-    SJD_TRY(gemm(0, c->wmap_head, c->lm_head, h, d, logits_out, g.vocab, g.vocab, d, EPI_STORE_T));
+    SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->final_norm, h, M, d, g.rms_eps, stream));
+    SJD_TRY(gemm(c->lm_head, h, d, logits_out, g.vocab, g.vocab, d, EPI_STORE_T));
   }
+  return SJD_OK;
+}
+
+int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, cudaStream_t stream) {
+  const sjd_model_cfg &g = c->cfg;
+  const int dt = g.dtype;
+  const int M = c->batch * rows_per_seq;
+  const int d = g.d_model, F = g.ffn_hidden;
+  const int nq = g.n_heads * g.head_dim, nk = g.n_kv_heads * g.head_dim, nqkv = nq + 2 * nk;
+  const SeqState st = c->state();
+  float *x = c->at<float>(c->lay.x);
+  float *q = c->at<float>(c->lay.q);
+  float *attn = c->at<float>(c->lay.attn);
+  float *partial = c->at<float>(c->lay.partial);
+  float *planes = c->at<float>(c->lay.gemm_planes);
+  int *status = c->at<int>(c->lay.status);
+  const float2 *rope = c->at<float2>(c->lay.rope);
+  const int att_splits = attention_splits(g.n_heads, c->batch);
+  const int Ma = c->rows_alloc();
+  const HiLoOut hl_h{c->at<__nv_bfloat16>(c->lay.xs_h), (size_t)Ma * d};
+  const HiLoOut hl_attn{c->at<__nv_bfloat16>(c->lay.xs_attn), (size_t)Ma * nq};
+  const HiLoOut hl_act{c->at<__nv_bfloat16>(c->lay.xs_act), (size_t)Ma * F};
+  int rc;
+  Tracer &tr = c->tracer;
+
+  // one GEMM launch over n_mats matrices sharing the activation operand; returns the planes it wrote
+  auto gemm = [&](const WMap *const *wm, int n_mats, const int *n_out, const TensorMap &x_map, int k_in, int ldc, void *out,
+                  bool bf16_out, PlaneSet *ps) -> int {
+    GemmTcCall call;
+    memset(&call, 0, sizeof(call));
+    int tiles = 0, col = 0;
+    for (int j = 0; j < n_mats; ++j) {
+      call.w_map[j] = &wm[j]->map;
+      call.n_out[j] = n_out[j];
+      call.col_off[j] = col;
+      col += n_out[j];
+      tiles += n_out[j] / 128;
+      if (tr.on) tr.gemm_weight_bytes += (double)n_out[j] * (double)k_in * 2.0;
+    }
+    for (int j = n_mats; j < 3; ++j) call.w_map[j] = call.w_map[0];
+    call.n_mats = n_mats;
+    call.x_map = &x_map;
+    call.x_lo_row = Ma;
+    call.M = M;
+    call.K = k_in;
+    call.splits = bf16_out ? 1 : gemm_tc_splits(tiles, k_in / 64, c->n_ctas);
+    call.out = out;
+    call.plane_stride = (size_t)M * ldc;
+    call.ldc = ldc;
+    call.store_bf16 = bf16_out ? 1 : 0;
+    call.status = status;
+    if (ps) *ps = PlaneSet{reinterpret_cast<const float *>(out), call.plane_stride, ldc, call.splits};
+    tr.begin(TC_GEMM, stream);
+    const int r = launch_gemm_tc(call, stream);
+    tr.end(stream);
+    return r;
+  };
+
+  SJD_TR(TC_OTHER, launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
+  PlaneSet pending{nullptr, 0, 0, 0};   // planes still to be added into the residual stream
+  for (int l = 0; l < g.n_layers; ++l) {
+    const LayerMaps &lm = c->wmaps[l];
+    PlaneSet ps;
+    SJD_TR(TC_OTHER, launch_resid_norm(dt, x, pending, c->attn_norm[l], hl_h, M, d, g.rms_eps, stream));
+    {
+      const WMap *wm[3] = {&lm.wq, &lm.wk, &lm.wv};
+      const int n_out[3] = {nq, nk, nk};
+      SJD_TRY(gemm(wm, 3, n_out, xm.h, d, nqkv, planes, false, &ps));
+    }
+    const KvLayout kv = c->kv_layer(l);
+    SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
+    SJD_TR(TC_ATTENTION,
+           launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, att_splits, stream, hl_attn));
+    {
+      const WMap *wm[1] = {&lm.wo};
+      const int n_out[1] = {d};
+      SJD_TRY(gemm(wm, 1, n_out, xm.attn, nq, d, planes, false, &ps));
+    }
+    SJD_TR(TC_OTHER, launch_resid_norm(dt, x, ps, c->ffn_norm[l], hl_h, M, d, g.rms_eps, stream));
+    {
+      const WMap *wm[2] = {&lm.w_gate, &lm.w_up};
+      const int n_out[2] = {F, F};
+      SJD_TRY(gemm(wm, 2, n_out, xm.h, d, 2 * F, planes, false, &ps));
+    }
+    SJD_TR(TC_OTHER, launch_swiglu_finish(ps, hl_act, M, F, stream));
+    {
+      const WMap *wm[1] = {&lm.w_down};
+      const int n_out[1] = {d};
+      SJD_TRY(gemm(wm, 1, n_out, xm.act, F, d, planes, false, &pending));
+    }
+  }
+  if (logits_out) {
+    SJD_TR(TC_OTHER, launch_resid_norm(dt, x, pending, c->final_norm, hl_h, M, d, g.rms_eps, stream));
+    const WMap *wm[1] = {&c->wmap_head};
+    const int n_out[1] = {g.vocab};
+    SJD_TRY(gemm(wm, 1, n_out, xm.h, d, g.vocab, logits_out, true, nullptr));
+  }
+  return SJD_OK;
+}
 #undef SJD_TR
 #undef SJD_TRY
-  return SJD_OK;
+
+int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream) {
+  const int M = c->batch * rows_per_seq;
+  if (c->use_tc && c->all_tc && M <= 128) {
+    auto it = c->xmaps.find((M + 15) / 16 * 16);
+    if (it != c->xmaps.end()) return forward_tc(c, it->second, rows_per_seq, logits_out, stream);
+  }
+  return forward_generic(c, rows_per_seq, logits_out, stream);
 }
 
 int run_verify(sjd_ctx *c, const sjd_step_out *out, cudaStream_t stream) {
@@ -421,7 +518,6 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
   cudaError_t e = cudaMemcpy(c->ws + lay.rope, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.counters, 0, ((size_t)cfg->max_batch + 1) * 4);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.status, 0, 4);
-  if (e == cudaSuccess) e = cudaMemset(c->ws + lay.gemm_tickets, 0, (size_t)kMaxGemmTiles * 4);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     delete c;
@@ -439,8 +535,7 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
     const int d = cfg->d_model, F = cfg->ffn_hidden;
     const int nq = cfg->n_heads * cfg->head_dim, nk = cfg->n_kv_heads * cfg->head_dim;
     auto mk = [&](WMap &m, const void *w, int n_out, int k_in) {
-      m.valid = n_out % 128 == 0 && k_in % 64 == 0 && n_out / 128 <= kMaxGemmTiles &&
-                make_tensor_map_bf16(&m.map, w, n_out, k_in, 128) == SJD_OK;
+      m.valid = n_out % 128 == 0 && k_in % 64 == 0 && make_tensor_map_bf16(&m.map, w, n_out, k_in, 128) == SJD_OK;
     };
     for (int l = 0; l < L; ++l) {
       LayerMaps &lm = c->wmaps[l];
@@ -453,6 +548,12 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
       mk(lm.w_down, c->w_down[l], d, F);
     }
     mk(c->wmap_head, c->lm_head, cfg->vocab, d);
+    c->all_tc = c->wmap_head.valid && d <= 8192;
+    for (int l = 0; l < L; ++l) {
+      const LayerMaps &lm = c->wmaps[l];
+      c->all_tc = c->all_tc && lm.wq.valid && lm.wk.valid && lm.wv.valid && lm.wo.valid && lm.w_gate.valid &&
+                  lm.w_up.valid && lm.w_down.valid;
+    }
   }
   *out = c;
   return SJD_OK;

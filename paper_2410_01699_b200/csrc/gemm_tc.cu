@@ -1,21 +1,22 @@
-// Weight-streaming projection GEMM for sm_100a:  out[m][n] (epilogue)= sum_k X[m][k] * W[n][k]
+// Weight-streaming projection GEMM for sm_100a:  P[s][m][n] = sum_{k in split s} X[m][k] * W[n][k]
 // (Sec. 4.1 Step 2: the one forward pass over the window; every projection of the decoder).
 //
-// Shape of the problem: M = batch * window is 8..128 rows, the weight matrix W [N][K] (bf16) is tens
-// to hundreds of MB and is read exactly once per step, so the kernel is bound by HBM bandwidth and its
+// Shape of the problem: M = batch * window is 8..128 rows, the weight matrices (bf16) are tens to
+// hundreds of MB and are read exactly once per step, so the kernel is bound by HBM bandwidth and its
 // job is to keep every SM's TMA queue full.
 //   * W is the 128-row operand of tcgen05.mma (M = 128), the tokens are the N dimension.  The fp32
 //     activations arrive split into two bf16 planes, hi = bf16(x) and lo = bf16(x - hi); both planes
 //     are columns of the same MMA (N = 2 * Mp), and the epilogue adds the two halves: activations keep
-//     ~16 bits of mantissa at no cost in bytes.
-//   * One persistent CTA per SM.  The (tile, k-block) units are split evenly over the CTAs (stream-K);
-//     a CTA whose range covers only part of a tile's K range writes an fp32 partial and takes a
-//     ticket; the last CTA of a tile adds the partials in CTA order (fixed order: deterministic) and
-//     runs the epilogue.  No floating-point atomics.
+//     ~16 bits of mantissa at no cost in weight bytes.
+//   * One CTA per (128-row weight tile, K split); two CTAs are resident per SM.  A launch covers up to
+//     three weight matrices that share the activation operand (Q|K|V, gate|up), so their tiles form
+//     one grid.  With more than one K split every CTA writes an fp32 partial plane; the consumer
+//     kernel (residual + RMSNorm, RoPE + cache append, SwiGLU, or a plain sum) adds the planes in
+//     split order: deterministic, no atomics, no serial reduction tail inside the GEMM.
 //   * Warp 0 issues TMA loads (128B-swizzled 128x64 W tiles with an evict-first L2 policy, plus the
 //     activation tiles) into a ring of shared-memory stages guarded by mbarriers; warp 1 issues the
-//     MMAs into one of two TMEM accumulators and commits to the stage's "empty" barrier; warps 2-5
-//     drain the accumulator with tcgen05.ld while the next segment's MMAs run.
+//     MMAs into a TMEM accumulator and commits to the stage's "empty" barrier; warps 2-5 drain the
+//     accumulator with tcgen05.ld and store.
 //   * Every wait is bounded: after ~2 s a role records an error in the status word and leaves; the
 //     CTA still frees its TMEM.
 #include <cuda.h>
@@ -31,19 +32,21 @@ constexpr int UMMA_K = 16;
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 100 * 1024;   // per CTA, so that two CTAs fit one SM
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
 struct GemmParams {
-  void *out;              // fp32 or bf16 [M][ldc]
+  void *out;              // fp32 planes [splits][M][ldc], or bf16 [M][ldc] when store_bf16
+  size_t plane_stride;    // elements between planes
   int ldc;
   int M;                  // valid token rows
   int Mp;                 // token rows padded to a multiple of 16 (MMA N = 2 * Mp)
   int x_lo_row;           // row of the lo plane inside the activation tensor map
-  int n_tiles, k_blocks;  // N / 128, K / 64
+  int k_blocks, splits;   // K / 64, K splits (gridDim.y)
+  int tile_end[3];        // matrix j owns tiles [tile_end[j-1], tile_end[j])
+  int col_off[3];         // first output column of matrix j
   int stages;
-  int epilogue;
-  float *partials;        // [gridDim.x][2][2 * Mp][128]
-  int *tickets;           // [n_tiles], zero on entry and on exit
+  int store_bf16;
   int *status;            // device status word (non-zero = a bounded wait ran out)
 };
 
@@ -55,9 +58,6 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
   uint32_t ok;
@@ -102,6 +102,9 @@ __device__ __forceinline__ void tma_load_2d_nohint(void *dst, const CUtensorMap 
       ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
       : "memory");
 }
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 
 // shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
@@ -132,17 +135,14 @@ __device__ __forceinline__ void umma_commit(uint64_t *bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
-  uint32_t r[16];
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t *r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // AND of a predicate over the 128 epilogue threads (named barrier 1): keeps their control flow uniform
 __device__ __forceinline__ bool epilogue_all(bool pred) {
@@ -158,63 +158,41 @@ __device__ __forceinline__ bool epilogue_all(bool pred) {
   return r != 0;
 }
 
-// ---------------------------------------------------------------------------------- work split
-struct Split {
-  long total, q, r;   // units, units per CTA (floor), CTAs with one extra
-  __device__ void init(long units, int ctas) {
-    total = units;
-    q = units / ctas;
-    r = units % ctas;
-  }
-  __device__ long begin(int c) const { return (long)c * q + (c < r ? c : r); }
-  __device__ int owner(long u) const {
-    const long b = r * (q + 1);
-    if (u < b) return (int)(u / (q + 1));
-    return (int)(r + (u - b) / (q > 0 ? q : 1));
-  }
-};
-
-template <int EPI>
-__device__ __forceinline__ void store_out(const GemmParams &p, int m, int n, float v) {
-  if (m >= p.M) return;
-  const size_t idx = (size_t)m * p.ldc + n;
-  if (EPI == EPI_STORE_F32) reinterpret_cast<float *>(p.out)[idx] = v;
-  else if (EPI == EPI_ADD_F32) reinterpret_cast<float *>(p.out)[idx] += v;
-  else reinterpret_cast<__nv_bfloat16 *>(p.out)[idx] = __float2bfloat16_rn(v);
-}
-
 // ---------------------------------------------------------------------------------- kernel
-template <int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
+__global__ void __launch_bounds__(kThreads, 2)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant__ CUtensorMap w_map1,
+               const __grid_constant__ CUtensorMap w_map2, const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full[2], bar_acc_empty[2];
+  __shared__ uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full;
   __shared__ uint32_t s_tmem_base;
-  __shared__ int s_last;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int cta = blockIdx.x, n_cta = gridDim.x;
+  const int tile = blockIdx.x, split = blockIdx.y;
   const int NN = 2 * p.Mp;                                   // MMA N
   const int x_tile_bytes = NN * TILE_K * 2;
   const int stage_bytes = W_TILE_BYTES + x_tile_bytes;
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
-  Split sp;
-  sp.init((long)p.n_tiles * p.k_blocks, n_cta);
-  const long u_begin = sp.begin(cta), u_end = sp.begin(cta + 1);
+  // which weight matrix this tile belongs to
+  const int mat = tile < p.tile_end[0] ? 0 : (tile < p.tile_end[1] ? 1 : 2);
+  const CUtensorMap *w_map = mat == 0 ? &w_map0 : (mat == 1 ? &w_map1 : &w_map2);
+  const int tile_in_mat = tile - (mat == 0 ? 0 : p.tile_end[mat - 1]);
+  // this CTA's k-blocks
+  const int kb_begin = (int)(((long)split * p.k_blocks) / p.splits);
+  const int kb_end = (int)(((long)(split + 1) * p.k_blocks) / p.splits);
+  const int n_kb = kb_end - kb_begin;
 
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < 2 * NN) tmem_cols <<= 1;
+  while ((int)tmem_cols < NN) tmem_cols <<= 1;
 
   if (tid == 0) {
+    tma_prefetch_desc(w_map);
+    tma_prefetch_desc(&x_map);
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(&bar_full[s], 1);
       mbar_init(&bar_empty[s], 1);
     }
-    mbar_init(&bar_acc_full[0], 1);
-    mbar_init(&bar_acc_full[1], 1);
-    mbar_init(&bar_acc_empty[0], 4);
-    mbar_init(&bar_acc_empty[1], 4);
+    mbar_init(&bar_acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -231,137 +209,82 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0 && u_begin < u_end) {
+    if (lane == 0) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-      long it = 0;
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
-      for (long u = u_begin; u < u_end && ok; ++u, ++it) {
-        const int tile = (int)(u / p.k_blocks), kb = (int)(u % p.k_blocks);
-        const int s = (int)(it % p.stages);
-        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
+      int it = 0;
+      for (; it < n_kb; ++it) {
         if (!mbar_wait(&bar_empty[s], ph ^ 1u)) { ok = false; break; }
-        uint8_t *dst = smem + (size_t)s * stage_bytes;
+        uint8_t *dst = smem + s * stage_bytes;
+        const int kcol = (kb_begin + it) * TILE_K;
         mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
-        tma_load_2d(dst, &w_map, kb * TILE_K, tile * TILE_N, &bar_full[s], policy);
-        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kb * TILE_K, 0, &bar_full[s]);
-        tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kb * TILE_K, p.x_lo_row, &bar_full[s]);
+        tma_load_2d(dst, w_map, kcol, tile_in_mat * TILE_N, &bar_full[s], policy);
+        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, 0, &bar_full[s]);
+        tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row, &bar_full[s]);
+        if (++s == p.stages) { s = 0; ph ^= 1u; }
       }
       if (!ok) {
         atomicExch(p.status, 1);
         // leave no copy in flight: wait (bounded) for the stages armed most recently
-        const long armed = it < p.stages ? it : p.stages;
-        for (long j = it - armed; j < it; ++j) mbar_wait(&bar_full[j % p.stages], (uint32_t)((j / p.stages) & 1));
+        const int armed = it < p.stages ? it : p.stages;
+        for (int j = it - armed; j < it; ++j) mbar_wait(&bar_full[j % p.stages], (uint32_t)((j / p.stages) & 1));
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && u_begin < u_end) {
+    if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(NN);
-      long it = 0;
-      int seg = 0;
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
-      for (long u = u_begin; u < u_end && ok; ++seg) {
-        const int kb0 = (int)(u % p.k_blocks);
-        const long seg_end = min(u_end, u - kb0 + p.k_blocks);
-        const int buf = seg & 1;
-        if (!mbar_wait(&bar_acc_empty[buf], (uint32_t)(((seg >> 1) & 1) ^ 1))) { ok = false; break; }
+      for (int it = 0; it < n_kb; ++it) {
+        if (!mbar_wait(&bar_full[s], ph)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_addr = tmem_base + (uint32_t)(buf * NN);
-        bool first = true;
-        for (; u < seg_end; ++u, ++it) {
-          const int s = (int)(it % p.stages);
-          const uint32_t ph = (uint32_t)((it / p.stages) & 1);
-          if (!mbar_wait(&bar_full[s], ph)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-          const uint32_t b_addr = a_addr + W_TILE_BYTES;
+        const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
+        const uint32_t b_addr = a_addr + W_TILE_BYTES;
 #pragma unroll
-          for (int k = 0; k < TILE_K / UMMA_K; ++k) {
-            umma_bf16(d_addr, umma_desc_sw128(a_addr + k * UMMA_K * 2), umma_desc_sw128(b_addr + k * UMMA_K * 2), idesc,
-                      !(first && k == 0));
-          }
-          first = false;
-          umma_commit(&bar_empty[s]);   // frees the stage once these MMAs have read it
+        for (int k = 0; k < TILE_K / UMMA_K; ++k) {
+          umma_bf16(tmem_base, umma_desc_sw128(a_addr + k * UMMA_K * 2), umma_desc_sw128(b_addr + k * UMMA_K * 2), idesc,
+                    !(it == 0 && k == 0));
         }
-        if (ok) umma_commit(&bar_acc_full[buf]);
+        umma_commit(&bar_empty[s]);   // frees the stage once these MMAs have read it
+        if (++s == p.stages) { s = 0; ph ^= 1u; }
       }
-      if (!ok) atomicExch(p.status, 2);
+      if (ok) umma_commit(&bar_acc_full);
+      else atomicExch(p.status, 2);
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps (2..5)
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const int row = quarter * 32 + lane;          // weight row inside the tile
-    int seg = 0;
-    bool ok = true;
-    for (long u = u_begin; u < u_end && ok; ++seg) {
-      const int tile = (int)(u / p.k_blocks), kb0 = (int)(u % p.k_blocks);
-      const long seg_end = min(u_end, u - kb0 + p.k_blocks);
-      const int kb1 = kb0 + (int)(seg_end - u);
-      const bool full_tile = (kb0 == 0 && kb1 == p.k_blocks);
-      const int buf = seg & 1;
-      if (!epilogue_all(mbar_wait(&bar_acc_full[buf], (uint32_t)((seg >> 1) & 1)))) { ok = false; break; }
+    const bool ok = epilogue_all(mbar_wait(&bar_acc_full, 0));
+    if (ok) {
       tc_fence_after();
-      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NN);
-      const int n = tile * TILE_N + row;
-      if (full_tile) {
-        for (int m0 = 0; m0 < p.Mp; m0 += 16) {
-          float hi[16], lo[16];
-          tmem_ld16(t_addr + m0, hi);
-          tmem_ld16(t_addr + p.Mp + m0, lo);
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      const int n = p.col_off[mat] + tile_in_mat * TILE_N + row;
+      float *plane = reinterpret_cast<float *>(p.out) + (size_t)split * p.plane_stride;
+      __nv_bfloat16 *out_bf16 = reinterpret_cast<__nv_bfloat16 *>(p.out);
+      for (int m0 = 0; m0 < p.Mp; m0 += 16) {
+        uint32_t hi[16], lo[16];
+        tmem_ld16_issue(t_addr + m0, hi);
+        tmem_ld16_issue(t_addr + p.Mp + m0, lo);
+        tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 16; ++i) store_out<EPI>(p, m0 + i, n, hi[i] + lo[i]);
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-      } else {
-        // partial K range: park the fp32 partial, take a ticket; the last arrival reduces the tile
-        const int which = kb0 > 0 ? 0 : 1;
-        float *slot = p.partials + ((size_t)(cta * 2 + which) * NN) * TILE_N;
-        for (int c0 = 0; c0 < NN; c0 += 16) {
-          float v[16];
-          tmem_ld16(t_addr + c0, v);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) __stcg(&slot[(size_t)(c0 + i) * TILE_N + row], v[i]);
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
-        __threadfence();
-        // all four epilogue warps must have stored before the ticket is taken
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        const int c_lo = sp.owner((long)tile * p.k_blocks), c_hi = sp.owner((long)(tile + 1) * p.k_blocks - 1);
-        if (tid == 64) {
-          __threadfence();
-          const int old = atomicAdd(&p.tickets[tile], 1);
-          s_last = (old == c_hi - c_lo);
-          if (s_last) p.tickets[tile] = 0;
-          __threadfence();
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (s_last) {
-          for (int m0 = 0; m0 < p.Mp; m0 += 16) {
-            float acc[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
-            for (int half = 0; half < 2; ++half) {
-              for (int c = c_lo; c <= c_hi; ++c) {
-                const int wch = sp.begin(c) > (long)tile * p.k_blocks ? 0 : 1;
-                const float *src = p.partials + ((size_t)(c * 2 + wch) * NN) * TILE_N;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) acc[i] += __ldcg(&src[(size_t)(half * p.Mp + m0 + i) * TILE_N + row]);
-              }
-            }
-#pragma unroll
-            for (int i = 0; i < 16; ++i) store_out<EPI>(p, m0 + i, n, acc[i]);
+        for (int i = 0; i < 16; ++i) {
+          const int m = m0 + i;
+          if (m < p.M) {
+            const float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+            if (p.store_bf16) out_bf16[(size_t)m * p.ldc + n] = __float2bfloat16_rn(v);
+            else plane[(size_t)m * p.ldc + n] = v;
           }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // s_last is reused by the next segment
       }
-      u = seg_end;
+    } else if (tid == 64) {
+      atomicExch(p.status, 3);
     }
-    if (!ok) atomicExch(p.status, 3);
   }
 
   tc_fence_before();
@@ -388,6 +311,16 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// plain sum of split planes (sjd_gemm): out[m][n] (+)= sum_s P[s][m][n]
+__global__ void sum_planes_kernel(const float *__restrict__ planes, size_t plane_stride, int splits, float *__restrict__ out,
+                                  size_t total, int accumulate) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    float acc = 0.0f;
+    for (int s = 0; s < splits; ++s) acc += planes[(size_t)s * plane_stride + i];
+    out[i] = accumulate ? out[i] + acc : acc;
+  }
+}
+
 }  // namespace
 
 // bf16 row-major [rows][cols] matrix viewed as boxes of box_rows x 64 columns with 128-byte swizzle
@@ -408,44 +341,66 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
 
 bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 128 && N % TILE_N == 0 && K % TILE_K == 0; }
 
-size_t gemm_tc_partial_floats(int n_ctas, int max_rows) {
-  const int mp = (max_rows + 15) / 16 * 16;
-  return (size_t)n_ctas * 2 * (2 * mp) * TILE_N;
+// K splits for a launch of `tiles` weight tiles: about two CTAs per SM, at least 8 k-blocks per CTA
+int gemm_tc_splits(int tiles, int k_blocks, int n_sms) {
+  int s = (2 * n_sms + tiles - 1) / tiles;
+  const int cap = k_blocks / 8 > 1 ? k_blocks / 8 : 1;
+  s = s > cap ? cap : s;
+  s = s > 16 ? 16 : s;
+  return s < 1 ? 1 : s;
 }
 
-int launch_gemm_tc(const TensorMap &w_map, const TensorMap &x_map, int x_lo_row, void *out, int ldc, int M, int N, int K,
-                   int epilogue, float *partials, int *tickets, int *status, int n_ctas, cudaStream_t stream) {
-  if (!gemm_tc_supported(M, N, K)) return SJD_ERR_UNSUPPORTED;
+int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
+  if (g.n_mats < 1 || g.n_mats > 3 || g.splits < 1) return SJD_ERR_BAD_ARG;
   GemmParams p;
-  p.out = out;
-  p.ldc = ldc;
-  p.M = M;
-  p.Mp = (M + 15) / 16 * 16;
-  p.x_lo_row = x_lo_row;
-  p.n_tiles = N / TILE_N;
-  p.k_blocks = K / TILE_K;
-  p.epilogue = epilogue;
-  p.partials = partials;
-  p.tickets = tickets;
-  p.status = status;
+  int tiles = 0;
+  for (int j = 0; j < 3; ++j) {
+    if (j < g.n_mats) {
+      if (!gemm_tc_supported(g.M, g.n_out[j], g.K)) return SJD_ERR_UNSUPPORTED;
+      tiles += g.n_out[j] / TILE_N;
+    }
+    p.tile_end[j] = tiles;
+    p.col_off[j] = j < g.n_mats ? g.col_off[j] : 0;
+  }
+  if (g.store_bf16 && g.splits != 1) return SJD_ERR_BAD_ARG;
+  p.out = g.out;
+  p.plane_stride = g.plane_stride;
+  p.ldc = g.ldc;
+  p.M = g.M;
+  p.Mp = (g.M + 15) / 16 * 16;
+  p.x_lo_row = g.x_lo_row;
+  p.k_blocks = g.K / TILE_K;
+  p.splits = g.splits;
+  p.store_bf16 = g.store_bf16;
+  p.status = g.status;
   const int stage_bytes = W_TILE_BYTES + 2 * p.Mp * TILE_K * 2;
-  int stages = (200 * 1024) / stage_bytes;
+  int stages = kSmemBudget / stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : stages;
   if (stages < 2) return SJD_ERR_UNSUPPORTED;
   p.stages = stages;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  const CUtensorMap &wm = reinterpret_cast<const CUtensorMap &>(w_map);
-  const CUtensorMap &xm = reinterpret_cast<const CUtensorMap &>(x_map);
-#define SJD_LAUNCH_TC(E)                                                                                         \
-  do {                                                                                                           \
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
-    gemm_tc_kernel<E><<<n_ctas, kThreads, smem, stream>>>(wm, xm, p);                                            \
-  } while (0)
-  if (epilogue == EPI_STORE_F32) SJD_LAUNCH_TC(EPI_STORE_F32);
-  else if (epilogue == EPI_ADD_F32) SJD_LAUNCH_TC(EPI_ADD_F32);
-  else if (epilogue == EPI_STORE_T) SJD_LAUNCH_TC(EPI_STORE_T);
-  else return SJD_ERR_BAD_ARG;
-#undef SJD_LAUNCH_TC
+  const CUtensorMap &w0 = reinterpret_cast<const CUtensorMap &>(*g.w_map[0]);
+  const CUtensorMap &w1 = reinterpret_cast<const CUtensorMap &>(*g.w_map[g.n_mats > 1 ? 1 : 0]);
+  const CUtensorMap &w2 = reinterpret_cast<const CUtensorMap &>(*g.w_map[g.n_mats > 2 ? 2 : 0]);
+  const CUtensorMap &xm = reinterpret_cast<const CUtensorMap &>(*g.x_map);
+  // opt in to > 48 KB of dynamic shared memory, once per device
+  static bool configured[64] = {};
+  int dev = 0;
+  SJD_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
+  if (!configured[dev]) {
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
+    configured[dev] = true;
+  }
+  gemm_tc_kernel<<<dim3(tiles, g.splits), kThreads, smem, stream>>>(w0, w1, w2, xm, p);
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
+
+int launch_sum_planes(const float *planes, size_t plane_stride, int splits, float *out, size_t total, int accumulate,
+                      cudaStream_t stream) {
+  const int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
+  sum_planes_kernel<<<blocks, 256, 0, stream>>>(planes, plane_stride, splits, out, total, accumulate);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -61,4 +61,4 @@ def test_gemm_rejects_uncovered_shapes():
     with pytest.raises(B.SJDError) as e:
         B.sjd_gemm(x, w)                      # K not a multiple of 64
     assert e.value.status == B.SJD_ERR_UNSUPPORTED
-    assert B.lib().sjd_gemm_workspace_bytes(129, 64) == 0
+    assert B.lib().sjd_gemm_workspace_bytes(129, 128, 64) == 0
