@@ -145,6 +145,7 @@ extern "C" int sjd_gemm(int M, int N, int K, const float *x, const void *w, floa
   g.ldc = N;
   g.store_bf16 = 0;
   g.status = status;
+  g.n_sms = sms;
   rc = launch_gemm_tc(g, stream);
   if (rc != SJD_OK) return rc;
   return launch_sum_planes(planes, (size_t)M * N, splits, out, (size_t)M * N, accumulate, stream);

@@ -180,6 +180,10 @@ struct GemmTcCall {
   int ldc;
   int store_bf16;
   int *status;
+  const float *ss_part;   // optional per-row RMS scale applied in the epilogue (see RowScale); null: none
+  int n_part;
+  float inv_d, eps;
+  int n_sms;
 };
 int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream);
 int launch_sum_planes(const float *planes, size_t plane_stride, int splits, float *out, size_t total, int accumulate,
@@ -201,9 +205,16 @@ struct HiLoOut {
 int launch_split_hilo(const float *x, HiLoOut o, size_t total, cudaStream_t stream);
 // consumer kernels of the tensor-core path (fused_kernels.cu)
 struct KvLayout;
-int launch_resid_norm(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOut h, int M, int d, float eps,
+// partial sums of squares of the residual rows: scale(m) = 1/sqrt(sum_j ss_part[m][j] * inv_d + eps)
+struct RowScale {
+  const float *ss_part;   // [M][n_part]; null: scale 1
+  int n_part;
+  float inv_d, eps;
+};
+int resid_gain_parts(int d);
+int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOut h, float *ss_part, int M, int d,
                       cudaStream_t stream);
-int launch_swiglu_finish(PlaneSet ps, HiLoOut act, int M, int F, cudaStream_t stream);
+int launch_swiglu_finish(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, cudaStream_t stream);
 
 // x[m][:] = tok_emb[tok[m]][:]  (fp32 residual stream)
 int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, int M, int d, int vocab,
@@ -219,8 +230,8 @@ struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
 };
 int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
                        KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
-int launch_qkv_finish(int dtype, PlaneSet ps, const int32_t *in_pos, const float2 *rope_table, float *q, KvLayout kv, int M,
-                      int rows_per_seq, int n_heads, cudaStream_t stream);
+int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
+                      KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
 // act[m][f] = silu(gu[m][f]) * gu[m][F + f]
 int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream, HiLoOut hilo = HiLoOut{nullptr, 0});
 // Window-causal attention: query row m (sequence m / rows_per_seq, position in_pos[m]) attends cache rows

@@ -38,7 +38,7 @@ struct XMaps {
 struct Layout {
   size_t kv, logits[2], stats[2], row_out, counters, step, status;
   size_t x, h, qkv, q, attn, gu, act, partial, rope;
-  size_t xs_h, xs_attn, xs_act, gemm_planes;
+  size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t total;
 };
@@ -104,6 +104,7 @@ Layout make_layout(const sjd_model_cfg &c) {
     }
     L.gemm_planes = take(need * 4);
   }
+  L.ss_part = take(Mx * (size_t)resid_gain_parts(c.d_model) * 4);
   L.rope = take((size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2));
   L.committed = take((size_t)c.max_batch * c.max_seq * 4);
   L.n = take((size_t)c.max_batch * 4);
@@ -334,6 +335,8 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
   const HiLoOut hl_h{c->at<__nv_bfloat16>(c->lay.xs_h), (size_t)Ma * d};
   const HiLoOut hl_attn{c->at<__nv_bfloat16>(c->lay.xs_attn), (size_t)Ma * nq};
   const HiLoOut hl_act{c->at<__nv_bfloat16>(c->lay.xs_act), (size_t)Ma * F};
+  float *ss_part = c->at<float>(c->lay.ss_part);
+  const RowScale rs{ss_part, resid_gain_parts(d), 1.0f / (float)d, g.rms_eps};
   int rc;
   Tracer &tr = c->tracer;
 
@@ -363,6 +366,13 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     call.ldc = ldc;
     call.store_bf16 = bf16_out ? 1 : 0;
     call.status = status;
+    call.n_sms = c->n_ctas;
+    if (bf16_out) {   // the logits projection applies the final norm's row scale itself
+      call.ss_part = rs.ss_part;
+      call.n_part = rs.n_part;
+      call.inv_d = rs.inv_d;
+      call.eps = rs.eps;
+    }
     if (ps) *ps = PlaneSet{reinterpret_cast<const float *>(out), call.plane_stride, ldc, call.splits};
     tr.begin(TC_GEMM, stream);
     const int r = launch_gemm_tc(call, stream);
@@ -375,14 +385,14 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
   for (int l = 0; l < g.n_layers; ++l) {
     const LayerMaps &lm = c->wmaps[l];
     PlaneSet ps;
-    SJD_TR(TC_OTHER, launch_resid_norm(dt, x, pending, c->attn_norm[l], hl_h, M, d, g.rms_eps, stream));
+    SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->attn_norm[l], hl_h, ss_part, M, d, stream));
     {
       const WMap *wm[3] = {&lm.wq, &lm.wk, &lm.wv};
       const int n_out[3] = {nq, nk, nk};
       SJD_TRY(gemm(wm, 3, n_out, xm.h, d, nqkv, planes, false, &ps));
     }
     const KvLayout kv = c->kv_layer(l);
-    SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
+    SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
     SJD_TR(TC_ATTENTION,
            launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, att_splits, stream, hl_attn));
     {
@@ -390,13 +400,13 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       const int n_out[1] = {d};
       SJD_TRY(gemm(wm, 1, n_out, xm.attn, nq, d, planes, false, &ps));
     }
-    SJD_TR(TC_OTHER, launch_resid_norm(dt, x, ps, c->ffn_norm[l], hl_h, M, d, g.rms_eps, stream));
+    SJD_TR(TC_OTHER, launch_resid_gain(dt, x, ps, c->ffn_norm[l], hl_h, ss_part, M, d, stream));
     {
       const WMap *wm[2] = {&lm.w_gate, &lm.w_up};
       const int n_out[2] = {F, F};
       SJD_TRY(gemm(wm, 2, n_out, xm.h, d, 2 * F, planes, false, &ps));
     }
-    SJD_TR(TC_OTHER, launch_swiglu_finish(ps, hl_act, M, F, stream));
+    SJD_TR(TC_OTHER, launch_swiglu_finish(ps, rs, hl_act, M, F, stream));
     {
       const WMap *wm[1] = {&lm.w_down};
       const int n_out[1] = {d};
@@ -404,7 +414,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     }
   }
   if (logits_out) {
-    SJD_TR(TC_OTHER, launch_resid_norm(dt, x, pending, c->final_norm, hl_h, M, d, g.rms_eps, stream));
+    SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->final_norm, hl_h, ss_part, M, d, stream));
     const WMap *wm[1] = {&c->wmap_head};
     const int n_out[1] = {g.vocab};
     SJD_TRY(gemm(wm, 1, n_out, xm.h, d, g.vocab, logits_out, true, nullptr));
@@ -548,7 +558,7 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
       mk(lm.w_down, c->w_down[l], d, F);
     }
     mk(c->wmap_head, c->lm_head, cfg->vocab, d);
-    c->all_tc = c->wmap_head.valid && d <= 8192;
+    c->all_tc = c->wmap_head.valid;
     for (int l = 0; l < L; ++l) {
       const LayerMaps &lm = c->wmaps[l];
       c->all_tc = c->all_tc && lm.wq.valid && lm.wk.valid && lm.wv.valid && lm.wo.valid && lm.w_gate.valid &&

@@ -26,55 +26,61 @@ __device__ __forceinline__ float sum_planes(const PlaneSet &ps, size_t idx) {
   return acc;
 }
 
-// x[m][:] += sum_s P[s][m][:]  (residual connection), then h = rmsnorm(x; gain) as bf16 hi/lo planes.
-// One block per row; the sum of squares is reduced in a fixed tree.
-constexpr int RN_THREADS = 512;
-constexpr int RN_MAX_PER_THREAD = 16;   // d_model <= 8192
+// Per-row RMS scale from the partial sums of squares a resid_gain launch left:
+// scale(m) = 1 / sqrt(mean(x[m]^2) + eps).  The scale is a per-row scalar, so it commutes with the
+// projection that follows the normalisation and is applied by that projection's consumer.
+__device__ __forceinline__ float row_scale(const RowScale &rs, int m) {
+  if (!rs.ss_part) return 1.0f;
+  float tot = 0.0f;
+  for (int j = 0; j < rs.n_part; ++j) tot += __ldg(rs.ss_part + (size_t)m * rs.n_part + j);
+  return rsqrtf(tot * rs.inv_d + rs.eps);
+}
+
+// x[m][:] += sum_s P[s][m][:]  (residual connection); emits x * gain as bf16 hi/lo planes (the RMS
+// scale is applied downstream) and this block's share of sum(x^2).  Grid (rows, column chunks of 1024).
+constexpr int RG_THREADS = 256;
+constexpr int RG_COLS = RG_THREADS * 4;
 
 template <typename T>
-__global__ void __launch_bounds__(RN_THREADS) resid_norm_kernel(float *__restrict__ x, PlaneSet ps, const T *__restrict__ gain,
-                                                               HiLoOut h, int d, float eps) {
-  __shared__ float red[RN_THREADS / 32];
-  const int m = blockIdx.x, tid = threadIdx.x;
-  float *row = x + (size_t)m * d;
-  float v[RN_MAX_PER_THREAD];
-  float ss = 0.0f;
-#pragma unroll
-  for (int j = 0; j < RN_MAX_PER_THREAD; ++j) {
-    const int i = tid + j * RN_THREADS;
-    v[j] = 0.0f;
-    if (i < d) {
-      float t = row[i];
-      if (ps.splits > 0) t += sum_planes(ps, (size_t)m * ps.ld + i);
-      v[j] = t;
-      ss = fmaf(t, t, ss);
+__global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restrict__ x, PlaneSet ps, const T *__restrict__ gain,
+                                                               HiLoOut h, float *__restrict__ ss_part, int d) {
+  __shared__ float red[RG_THREADS / 32];
+  const int m = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;
+  const int c0 = chunk * RG_COLS + tid * 4;
+  float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  if (c0 < d) {   // d is a multiple of 4
+    const float4 t = *reinterpret_cast<const float4 *>(x + (size_t)m * d + c0);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    for (int s = 0; s < ps.splits; ++s) {
+      const float4 pv = __ldg(reinterpret_cast<const float4 *>(ps.base + (size_t)s * ps.plane_stride + (size_t)m * ps.ld + c0));
+      v[0] += pv.x; v[1] += pv.y; v[2] += pv.z; v[3] += pv.w;
     }
+    if (ps.splits > 0) *reinterpret_cast<float4 *>(x + (size_t)m * d + c0) = make_float4(v[0], v[1], v[2], v[3]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) put_hilo(h, (size_t)m * d + c0 + i, v[i] * to_f<T>(gain[c0 + i]));
   }
+  float ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
   ss = warp_sum(ss);
   if ((tid & 31) == 0) red[tid >> 5] = ss;
   __syncthreads();
-  float tot = 0.0f;
+  if (tid == 0) {
+    float tot = 0.0f;
 #pragma unroll
-  for (int w = 0; w < RN_THREADS / 32; ++w) tot += red[w];
-  const float scale = rsqrtf(tot / (float)d + eps);
-#pragma unroll
-  for (int j = 0; j < RN_MAX_PER_THREAD; ++j) {
-    const int i = tid + j * RN_THREADS;
-    if (i < d) {
-      if (ps.splits > 0) row[i] = v[j];
-      put_hilo(h, (size_t)m * d + i, v[j] * scale * to_f<T>(gain[i]));
-    }
+    for (int w = 0; w < RG_THREADS / 32; ++w) tot += red[w];
+    ss_part[(size_t)m * gridDim.y + chunk] = tot;
   }
 }
 
-// q,k,v = sum of the QKV planes; rotate q and k (pairs i, i + hd/2) by the row's absolute position;
-// q -> fp32 [M][H*hd]; k, v -> cache row in_pos[m].  One block per (row, head slot).
+// q,k,v = scale * sum of the QKV planes; rotate q and k (pairs i, i + hd/2) by the row's absolute
+// position; q -> fp32 [M][H*hd]; k, v -> cache row in_pos[m].  One block per (row, head slot).
 template <typename T>
-__global__ void qkv_finish_kernel(PlaneSet ps, const int32_t *__restrict__ in_pos, const float2 *__restrict__ rope,
-                                  float *__restrict__ q, KvLayout kv, int rows_per_seq, int n_heads) {
+__global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__restrict__ in_pos,
+                                  const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
+                                  int n_heads) {
   const int m = blockIdx.x, slot = blockIdx.y;
   const int pos = in_pos[m];
   if (pos < 0) return;
+  const float sc = row_scale(rs, m);
   const int b = m / rows_per_seq;
   const int hd = kv.head_dim, half = hd >> 1, nkv = kv.n_kv_heads;
   const int nq = n_heads * hd, nk = nkv * hd;
@@ -86,7 +92,7 @@ __global__ void qkv_finish_kernel(PlaneSet ps, const int32_t *__restrict__ in_po
     const int col0 = is_q ? slot * hd : nq + (slot - n_heads) * hd;
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
       const float2 c = rope[(size_t)pos * half + j];
-      const float x1 = sum_planes(ps, rbase + col0 + j), x2 = sum_planes(ps, rbase + col0 + j + half);
+      const float x1 = sc * sum_planes(ps, rbase + col0 + j), x2 = sc * sum_planes(ps, rbase + col0 + j + half);
       const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
       if (is_q) {
         q[(size_t)m * nq + slot * hd + j] = r1;
@@ -100,52 +106,58 @@ __global__ void qkv_finish_kernel(PlaneSet ps, const int32_t *__restrict__ in_po
   } else {
     const int kh = slot - n_heads - nkv;
     T *dst = vbase + ((size_t)kh * kv.max_seq + pos) * hd;
-    for (int j = threadIdx.x; j < hd; j += blockDim.x) dst[j] = from_f<T>(sum_planes(ps, rbase + nq + nk + kh * hd + j));
+    for (int j = threadIdx.x; j < hd; j += blockDim.x)
+      dst[j] = from_f<T>(sc * sum_planes(ps, rbase + nq + nk + kh * hd + j));
   }
 }
 
-// act = silu(sum gate planes) * (sum up planes) as bf16 hi/lo planes; planes are [S][M][2F] (gate | up)
-__global__ void swiglu_finish_kernel(PlaneSet ps, HiLoOut act, int M, int F) {
+// act = silu(scale * sum gate planes) * (scale * sum up planes) as bf16 hi/lo planes; planes [S][M][2F]
+__global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F) {
   const size_t total = (size_t)M * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t m = i / F, f = i % F;
-    const float g = sum_planes(ps, m * ps.ld + f), u = sum_planes(ps, m * ps.ld + F + f);
+    const float sc = row_scale(rs, (int)m);
+    const float g = sc * sum_planes(ps, m * ps.ld + f), u = sc * sum_planes(ps, m * ps.ld + F + f);
     put_hilo(act, i, g / (1.0f + expf(-g)) * u);
   }
 }
 
 }  // namespace
 
-int launch_resid_norm(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOut h, int M, int d, float eps,
+int resid_gain_parts(int d) { return (d + RG_COLS - 1) / RG_COLS; }
+
+int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOut h, float *ss_part, int M, int d,
                       cudaStream_t stream) {
-  if (d > RN_THREADS * RN_MAX_PER_THREAD) return SJD_ERR_UNSUPPORTED;
+  if (d % 4 != 0) return SJD_ERR_UNSUPPORTED;
+  const dim3 grid(M, resid_gain_parts(d));
   if (dtype == SJD_F32)
-    resid_norm_kernel<float><<<M, RN_THREADS, 0, stream>>>(x, ps, reinterpret_cast<const float *>(gain), h, d, eps);
+    resid_gain_kernel<float><<<grid, RG_THREADS, 0, stream>>>(x, ps, reinterpret_cast<const float *>(gain), h, ss_part, d);
   else if (dtype == SJD_BF16)
-    resid_norm_kernel<__nv_bfloat16><<<M, RN_THREADS, 0, stream>>>(x, ps, reinterpret_cast<const __nv_bfloat16 *>(gain), h, d, eps);
+    resid_gain_kernel<__nv_bfloat16><<<grid, RG_THREADS, 0, stream>>>(x, ps, reinterpret_cast<const __nv_bfloat16 *>(gain), h,
+                                                                     ss_part, d);
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
 
-int launch_qkv_finish(int dtype, PlaneSet ps, const int32_t *in_pos, const float2 *rope_table, float *q, KvLayout kv, int M,
-                      int rows_per_seq, int n_heads, cudaStream_t stream) {
+int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
+                      KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
   const dim3 grid(M, n_heads + 2 * kv.n_kv_heads);
   if (dtype == SJD_F32)
-    qkv_finish_kernel<float><<<grid, 64, 0, stream>>>(ps, in_pos, rope_table, q, kv, rows_per_seq, n_heads);
+    qkv_finish_kernel<float><<<grid, 64, 0, stream>>>(ps, rs, in_pos, rope_table, q, kv, rows_per_seq, n_heads);
   else if (dtype == SJD_BF16)
-    qkv_finish_kernel<__nv_bfloat16><<<grid, 64, 0, stream>>>(ps, in_pos, rope_table, q, kv, rows_per_seq, n_heads);
+    qkv_finish_kernel<__nv_bfloat16><<<grid, 64, 0, stream>>>(ps, rs, in_pos, rope_table, q, kv, rows_per_seq, n_heads);
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
 
-int launch_swiglu_finish(PlaneSet ps, HiLoOut act, int M, int F, cudaStream_t stream) {
+int launch_swiglu_finish(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, cudaStream_t stream) {
   const size_t total = (size_t)M * F;
   const int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
-  swiglu_finish_kernel<<<blocks, 256, 0, stream>>>(ps, act, M, F);
+  swiglu_finish_kernel<<<blocks, 256, 0, stream>>>(ps, rs, act, M, F);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

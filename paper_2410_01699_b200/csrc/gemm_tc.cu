@@ -48,6 +48,9 @@ struct GemmParams {
   int stages;
   int store_bf16;
   int *status;            // device status word (non-zero = a bounded wait ran out)
+  const float *ss_part;   // optional [M][n_part] partial sums of squares: rows are scaled by
+  int n_part;             //   1 / sqrt(sum_j ss_part[m][j] * inv_d + eps) before they are stored
+  float inv_d, eps;
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -276,7 +279,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         for (int i = 0; i < 16; ++i) {
           const int m = m0 + i;
           if (m < p.M) {
-            const float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+            float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
+            if (p.ss_part) {
+              float tot = 0.0f;
+              for (int j = 0; j < p.n_part; ++j) tot += __ldg(p.ss_part + (size_t)m * p.n_part + j);
+              v *= rsqrtf(tot * p.inv_d + p.eps);
+            }
             if (p.store_bf16) out_bf16[(size_t)m * p.ldc + n] = __float2bfloat16_rn(v);
             else plane[(size_t)m * p.ldc + n] = v;
           }
@@ -341,10 +349,11 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
 
 bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 128 && N % TILE_N == 0 && K % TILE_K == 0; }
 
-// K splits for a launch of `tiles` weight tiles: about two CTAs per SM, at least 8 k-blocks per CTA
+// K splits for a launch of `tiles` weight tiles: at most two CTAs per SM in a single wave, at least
+// 16 k-blocks (256 KB of weights) per CTA so that set-up and drain stay small next to the streaming
 int gemm_tc_splits(int tiles, int k_blocks, int n_sms) {
-  int s = (2 * n_sms + tiles - 1) / tiles;
-  const int cap = k_blocks / 8 > 1 ? k_blocks / 8 : 1;
+  int s = (2 * n_sms) / tiles;
+  const int cap = k_blocks / 16 > 1 ? k_blocks / 16 : 1;
   s = s > cap ? cap : s;
   s = s > 16 ? 16 : s;
   return s < 1 ? 1 : s;
@@ -373,8 +382,14 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.splits = g.splits;
   p.store_bf16 = g.store_bf16;
   p.status = g.status;
+  p.ss_part = g.ss_part;
+  p.n_part = g.n_part;
+  p.inv_d = g.inv_d;
+  p.eps = g.eps;
   const int stage_bytes = W_TILE_BYTES + 2 * p.Mp * TILE_K * 2;
-  int stages = kSmemBudget / stage_bytes;
+  // one CTA per SM or fewer: give each the deeper ring
+  const int budget = (g.n_sms > 0 && tiles * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
+  int stages = budget / stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : stages;
   if (stages < 2) return SJD_ERR_UNSUPPORTED;
   p.stages = stages;
@@ -389,7 +404,7 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   SJD_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
   if (!configured[dev]) {
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
     configured[dev] = true;
   }
   gemm_tc_kernel<<<dim3(tiles, g.splits), kThreads, smem, stream>>>(w0, w1, w2, xm, p);
