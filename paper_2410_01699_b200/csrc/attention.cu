@@ -211,6 +211,13 @@ int attention_t(const float *q, KvLayout kv, const int32_t *in_pos, float *out, 
 
 }  // namespace
 
+int launch_attention_combine(const float *partial, const int32_t *in_pos, float *out, int M, int n_heads, int head_dim,
+                             int splits, cudaStream_t stream, HiLoOut hilo) {
+  attention_combine_kernel<<<dim3(M, n_heads), 128, 0, stream>>>(partial, in_pos, out, n_heads, head_dim, splits, hilo);
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
+
 int launch_attention(int dtype, const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial, int M,
                      int rows_per_seq, int n_heads, int splits, cudaStream_t stream, HiLoOut hilo) {
   if (dtype == SJD_F32)

@@ -1,0 +1,357 @@
+// Window-causal split-KV attention on tensor cores for bf16 caches (Sec. 3.2 / Sec. 4.1 Step 2: the W
+// window queries attend the cached prefix plus the in-window causal block).
+//
+// One CTA per (query head, sequence, key range).  K and V tiles of 64 keys are staged in shared memory
+// by TMA (128-byte swizzle, two 64-dim boxes per 128-dim head) through a ring of mbarrier-guarded
+// stages; each warp owns 16 query rows, keeps Q (pre-scaled, split into bf16 hi + lo), the running
+// max / sum and the fp32 output accumulators in registers and runs QK^T and PV as m16n8k16 bf16
+// mma.sync with ldmatrix-fed operands.  The probabilities are split hi + lo as well, so neither
+// operand loses more than ~2^-17 relative.  The kernel is bound by streaming K/V once from HBM (GQA
+// heads of a group share their tiles through L2).  Partials (max, sum, unnormalised output) go to the
+// merge kernel of attention.cu.  Every barrier wait is bounded.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace sjd {
+namespace {
+
+constexpr int KT = 64;                 // keys per tile
+constexpr int kStagesAttn = 3;
+constexpr unsigned long long kWaitNsAttn = 2000000000ull;
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool bar_try(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool bar_wait(uint64_t *bar, uint32_t parity) {
+  if (bar_try(bar, parity)) return true;
+  unsigned long long t0, t1;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (bar_try(bar, parity)) return true;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+    if (t1 - t0 > kWaitNsAttn) return false;
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_addr(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_addr(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// two floats -> packed bf16 hi pair and bf16 lo pair (lo = value - hi, rounded)
+__device__ __forceinline__ void split_pair(float x, float y, uint32_t &hi, uint32_t &lo) {
+  const __nv_bfloat16 hx = __float2bfloat16_rn(x), hy = __float2bfloat16_rn(y);
+  const __nv_bfloat16 lx = __float2bfloat16_rn(x - __bfloat162float(hx)), ly = __float2bfloat16_rn(y - __bfloat162float(hy));
+  hi = (uint32_t)__bfloat16_as_ushort(hx) | ((uint32_t)__bfloat16_as_ushort(hy) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(lx) | ((uint32_t)__bfloat16_as_ushort(ly) << 16);
+}
+
+struct AttnParams {
+  const float *q;        // [M][H*HD]
+  const int32_t *in_pos; // [M]
+  float *partial;        // [M][H][splits][HD + 2]
+  int *status;
+  int rows_per_seq, n_heads, n_kv_heads, splits;
+  int plane0;            // first cache plane of this layer: planes are [b][k|v][kv_head]
+};
+
+template <int HD>
+__global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
+  constexpr int HALVES = HD / 64;                // 64-dim (128-byte) boxes per row
+  constexpr int TILE_BYTES = KT * HD * 2;        // one of K or V
+  constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ uint64_t bar_full[kStagesAttn];
+  __shared__ int s_pos[64];
+  uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+
+  const int h = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int W = p.rows_per_seq;
+  const int kvh = h / (p.n_heads / p.n_kv_heads);
+  const int m0 = b * W;
+  const int g = lane >> 2, tq = lane & 3;
+
+  if (tid < 64) s_pos[tid] = tid < W ? p.in_pos[m0 + tid] : -1;
+  if (tid == 0) {
+    for (int s = 0; s < kStagesAttn; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bar_full[s])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  int len = 0;
+  for (int i = 0; i < W; ++i) len = max(len, s_pos[i] + 1);
+  int chunk = (len + p.splits - 1) / p.splits;
+  chunk = (chunk + KT - 1) / KT * KT;
+  const int k_begin = split * chunk;
+  const int k_end = min(len, k_begin + chunk);
+  const int n_tiles = k_end > k_begin ? (k_end - k_begin + KT - 1) / KT : 0;
+  const int plane_k = p.plane0 + (b * 2 + 0) * p.n_kv_heads + kvh;
+  const int plane_v = p.plane0 + (b * 2 + 1) * p.n_kv_heads + kvh;
+
+  auto issue = [&](int t) {   // thread 0: load tile t into its stage
+    const int s = t % kStagesAttn;
+    uint8_t *dst = smem + s * STAGE_BYTES;
+    const int key0 = k_begin + t * KT;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&bar_full[s])), "r"(STAGE_BYTES)
+                 : "memory");
+#pragma unroll
+    for (int hf = 0; hf < HALVES; ++hf) {
+      tma_load_3d(dst + hf * (KT * 128), &kv_map, hf * 64, key0, plane_k, &bar_full[s]);
+      tma_load_3d(dst + TILE_BYTES + hf * (KT * 128), &kv_map, hf * 64, key0, plane_v, &bar_full[s]);
+    }
+  };
+  if (tid == 0)
+    for (int t = 0; t < n_tiles && t < kStagesAttn; ++t) issue(t);
+
+  // this thread's two query rows
+  const int r0 = warp * 16 + g, r1 = r0 + 8;
+  const int pos0 = r0 < W ? s_pos[r0] : -1, pos1 = r1 < W ? s_pos[r1] : -1;
+  // Q fragments, pre-scaled by log2(e) / sqrt(HD), split hi / lo
+  uint32_t qh[HD / 16][4], ql[HD / 16][4];
+  {
+    const float sc = 1.4426950408889634f * rsqrtf((float)HD);
+    const float *q0 = p.q + ((size_t)(m0 + r0) * p.n_heads + h) * HD;
+    const float *q1 = p.q + ((size_t)(m0 + r1) * p.n_heads + h) * HD;
+#pragma unroll
+    for (int ks = 0; ks < HD / 16; ++ks) {
+      const int c = ks * 16 + tq * 2;
+      float2 a = make_float2(0.f, 0.f), bq = a, cq = a, dq = a;
+      if (pos0 >= 0) {
+        a = *reinterpret_cast<const float2 *>(q0 + c);
+        cq = *reinterpret_cast<const float2 *>(q0 + c + 8);
+      }
+      if (pos1 >= 0) {
+        bq = *reinterpret_cast<const float2 *>(q1 + c);
+        dq = *reinterpret_cast<const float2 *>(q1 + c + 8);
+      }
+      split_pair(a.x * sc, a.y * sc, qh[ks][0], ql[ks][0]);
+      split_pair(bq.x * sc, bq.y * sc, qh[ks][1], ql[ks][1]);
+      split_pair(cq.x * sc, cq.y * sc, qh[ks][2], ql[ks][2]);
+      split_pair(dq.x * sc, dq.y * sc, qh[ks][3], ql[ks][3]);
+    }
+  }
+
+  float o[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
+
+  bool ok = true;
+  for (int t = 0; t < n_tiles; ++t) {
+    const int s = t % kStagesAttn;
+    const bool got = bar_wait(&bar_full[s], (uint32_t)((t / kStagesAttn) & 1));
+    if (!__syncthreads_and(got)) { ok = false; break; }
+    const uint32_t kbase = smem_addr(smem + s * STAGE_BYTES), vbase = kbase + TILE_BYTES;
+    const int key0 = k_begin + t * KT;
+
+    // ---- S = Q K^T  (16 rows x 64 keys per warp)
+    float sacc[KT / 8][4];
+#pragma unroll
+    for (int i = 0; i < KT / 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.0f;
+#pragma unroll
+    for (int ks = 0; ks < HD / 16; ++ks) {
+      const int half = ks >> 2, c0 = (ks & 3) * 2;
+#pragma unroll
+      for (int nb = 0; nb < KT / 8; nb += 2) {
+        const int row = nb * 8 + (lane & 7) + ((lane >> 4) & 1) * 8;
+        const int chunkc = c0 + ((lane >> 3) & 1);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(kbase + half * (KT * 128) + row * 128 + ((chunkc ^ (row & 7)) << 4), b0, b1, b2, b3);
+        mma_bf16(sacc[nb], qh[ks], b0, b1);
+        mma_bf16(sacc[nb], ql[ks], b0, b1);
+        mma_bf16(sacc[nb + 1], qh[ks], b2, b3);
+        mma_bf16(sacc[nb + 1], ql[ks], b2, b3);
+      }
+    }
+    // ---- mask, online softmax (base 2)
+    float tmax0 = -INFINITY, tmax1 = -INFINITY;
+#pragma unroll
+    for (int nb = 0; nb < KT / 8; ++nb) {
+      const int j = key0 + nb * 8 + tq * 2;
+      if (!(j <= pos0 && j < k_end)) sacc[nb][0] = -INFINITY;
+      if (!(j + 1 <= pos0 && j + 1 < k_end)) sacc[nb][1] = -INFINITY;
+      if (!(j <= pos1 && j < k_end)) sacc[nb][2] = -INFINITY;
+      if (!(j + 1 <= pos1 && j + 1 < k_end)) sacc[nb][3] = -INFINITY;
+      tmax0 = fmaxf(tmax0, fmaxf(sacc[nb][0], sacc[nb][1]));
+      tmax1 = fmaxf(tmax1, fmaxf(sacc[nb][2], sacc[nb][3]));
+    }
+    tmax0 = fmaxf(tmax0, __shfl_xor_sync(0xffffffffu, tmax0, 1));
+    tmax0 = fmaxf(tmax0, __shfl_xor_sync(0xffffffffu, tmax0, 2));
+    tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, 1));
+    tmax1 = fmaxf(tmax1, __shfl_xor_sync(0xffffffffu, tmax1, 2));
+    const float mn0 = fmaxf(m_run[0], tmax0), mn1 = fmaxf(m_run[1], tmax1);
+    const float al0 = mn0 > -INFINITY ? exp2f(m_run[0] - mn0) : 1.0f;   // exp2f(-inf) = 0 for a fresh row
+    const float al1 = mn1 > -INFINITY ? exp2f(m_run[1] - mn1) : 1.0f;
+    const float sub0 = mn0 > -INFINITY ? mn0 : 0.0f, sub1 = mn1 > -INFINITY ? mn1 : 0.0f;
+    m_run[0] = mn0;
+    m_run[1] = mn1;
+    float ls0 = 0.0f, ls1 = 0.0f;
+    uint32_t ph[KT / 16][4], pl[KT / 16][4];
+#pragma unroll
+    for (int nb = 0; nb < KT / 8; ++nb) {
+      const float p0 = exp2f(sacc[nb][0] - sub0), p1 = exp2f(sacc[nb][1] - sub0);
+      const float p2 = exp2f(sacc[nb][2] - sub1), p3 = exp2f(sacc[nb][3] - sub1);
+      ls0 += p0 + p1;
+      ls1 += p2 + p3;
+      const int kk = nb >> 1, hi8 = (nb & 1) * 2;   // A fragment regs: {row g, row g+8} x {keys 0-7, keys 8-15}
+      split_pair(p0, p1, ph[kk][hi8], pl[kk][hi8]);
+      split_pair(p2, p3, ph[kk][hi8 + 1], pl[kk][hi8 + 1]);
+    }
+    l_run[0] = l_run[0] * al0 + ls0;
+    l_run[1] = l_run[1] * al1 + ls1;
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) {
+      o[i][0] *= al0; o[i][1] *= al0;
+      o[i][2] *= al1; o[i][3] *= al1;
+    }
+    // ---- O += P V
+#pragma unroll
+    for (int kk = 0; kk < KT / 16; ++kk) {
+#pragma unroll
+      for (int cd = 0; cd < HD / 8; cd += 2) {
+        const int row = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int chunkc = cd + ((lane >> 4) & 1);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(vbase + (chunkc >> 3) * (KT * 128) + row * 128 + (((chunkc & 7) ^ (row & 7)) << 4), b0, b1, b2, b3);
+        mma_bf16(o[cd], ph[kk], b0, b1);
+        mma_bf16(o[cd], pl[kk], b0, b1);
+        mma_bf16(o[cd + 1], ph[kk], b2, b3);
+        mma_bf16(o[cd + 1], pl[kk], b2, b3);
+      }
+    }
+    __syncthreads();   // every warp is done with this stage
+    if (tid == 0 && t + kStagesAttn < n_tiles) issue(t + kStagesAttn);
+  }
+  if (!ok) {
+    if (tid == 0) atomicExch(p.status, 4);
+    // leave no copy in flight: wait (bounded) for the stages that were armed
+    if (tid == 0)
+      for (int t = 0; t < n_tiles && t < kStagesAttn; ++t) bar_wait(&bar_full[t % kStagesAttn], 0);
+    return;
+  }
+
+  // ---- partial record per (row, head, split): [max (natural log units), sum, o[HD]]
+  l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
+  l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
+  l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
+  l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+#pragma unroll
+  for (int rr = 0; rr < 2; ++rr) {
+    const int r = rr == 0 ? r0 : r1;
+    if (r >= W) continue;
+    float *dst = p.partial + (((size_t)(m0 + r) * p.n_heads + h) * p.splits + split) * (HD + 2);
+    if (tq == 0) {
+      dst[0] = m_run[rr] > -INFINITY ? m_run[rr] * 0.6931471805599453f : -INFINITY;
+      dst[1] = l_run[rr];
+    }
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i)
+      *reinterpret_cast<float2 *>(dst + 2 + i * 8 + tq * 2) = make_float2(o[i][rr * 2], o[i][rr * 2 + 1]);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn3)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+// bf16 cache [planes][max_seq][head_dim] as boxes of 64 keys x 64 dims, 128-byte swizzle
+int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_seq, int head_dim) {
+  static EncodeTiledFn3 fn = nullptr;
+  if (!fn) {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn3>(sym);
+  }
+  if (!fn) return SJD_ERR_UNSUPPORTED;
+  if (((uintptr_t)base & 15u) != 0 || (head_dim != 64 && head_dim != 128)) return SJD_ERR_UNSUPPORTED;
+  cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)max_seq, (cuuint64_t)planes};
+  cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)max_seq * head_dim * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)KT, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(reinterpret_cast<CUtensorMap *>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base),
+                        dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SJD_OK : SJD_ERR_CUDA;
+}
+
+bool attention_mma_supported(int head_dim, int rows_per_seq) { return (head_dim == 64 || head_dim == 128) && rows_per_seq <= 64; }
+
+// partial kernel only; the caller merges with the combine kernel of attention.cu
+int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
+                         int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads, int head_dim, int splits,
+                         cudaStream_t stream) {
+  if (!attention_mma_supported(head_dim, rows_per_seq) || M % rows_per_seq != 0) return SJD_ERR_UNSUPPORTED;
+  AttnParams p;
+  p.q = q;
+  p.in_pos = in_pos;
+  p.partial = partial;
+  p.status = status;
+  p.rows_per_seq = rows_per_seq;
+  p.n_heads = n_heads;
+  p.n_kv_heads = n_kv_heads;
+  p.splits = splits;
+  p.plane0 = plane0;
+  const int threads = 32 * ((rows_per_seq + 15) / 16);
+  const dim3 grid(n_heads, M / rows_per_seq, splits);
+  const CUtensorMap &km = reinterpret_cast<const CUtensorMap &>(kv_map);
+  const size_t smem = (size_t)kStagesAttn * 2 * KT * head_dim * 2 + 1024;
+  static bool configured[64][2] = {};
+  int dev = 0;
+  SJD_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
+  if (head_dim == 128) {
+    if (!configured[dev][1]) {
+      SJD_CUDA(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      configured[dev][1] = true;
+    }
+    attention_mma_kernel<128><<<grid, threads, smem, stream>>>(km, p);
+  } else {
+    if (!configured[dev][0]) {
+      SJD_CUDA(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      configured[dev][0] = true;
+    }
+    attention_mma_kernel<64><<<grid, threads, smem, stream>>>(km, p);
+  }
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
+
+}  // namespace sjd

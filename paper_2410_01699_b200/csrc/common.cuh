@@ -239,5 +239,14 @@ int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream
 int launch_attention(int dtype, const float *q, KvLayout kv, const int32_t *in_pos, float *out, float *partial,
                      int M, int rows_per_seq, int n_heads, int splits, cudaStream_t stream,
                      HiLoOut hilo = HiLoOut{nullptr, 0});
+// merge of the split-KV partials only (used after launch_attention_mma)
+int launch_attention_combine(const float *partial, const int32_t *in_pos, float *out, int M, int n_heads, int head_dim,
+                             int splits, cudaStream_t stream, HiLoOut hilo);
+// tensor-core split-KV attention for bf16 caches (attention_mma.cu)
+int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_seq, int head_dim);
+bool attention_mma_supported(int head_dim, int rows_per_seq);
+int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
+                         int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads, int head_dim, int splits,
+                         cudaStream_t stream);
 
 }  // namespace sjd

@@ -225,6 +225,8 @@ struct sjd_ctx {
   std::vector<LayerMaps> wmaps;
   WMap wmap_head;
   std::map<int, XMaps> xmaps;   // keyed by padded row count
+  TensorMap kv_map;             // whole KV cache as [planes][max_seq][head_dim]
+  bool kv_map_valid = false;
   int rows_alloc() const { return ((cfg.max_batch * cfg.max_window) + 15) / 16 * 16; }
 
   template <typename T> T *at(size_t off) const { return reinterpret_cast<T *>(ws + off); }
@@ -393,8 +395,15 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     }
     const KvLayout kv = c->kv_layer(l);
     SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
-    SJD_TR(TC_ATTENTION,
-           launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, att_splits, stream, hl_attn));
+    if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
+      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, status, M,
+                                                rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim, att_splits, stream));
+      SJD_TR(TC_ATTENTION,
+             launch_attention_combine(partial, st.in_pos, attn, M, g.n_heads, g.head_dim, att_splits, stream, hl_attn));
+    } else {
+      SJD_TR(TC_ATTENTION,
+             launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, att_splits, stream, hl_attn));
+    }
     {
       const WMap *wm[1] = {&lm.wo};
       const int n_out[1] = {d};
@@ -559,6 +568,13 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
     }
     mk(c->wmap_head, c->lm_head, cfg->vocab, d);
     c->all_tc = c->wmap_head.valid;
+    // the cache as one 3-D tensor map for the tensor-core attention; unwritten rows must read as finite
+    // numbers (a masked probability of 0 times NaN would poison the output), so the cache starts at zero
+    const long planes = (long)L * cfg->max_batch * 2 * cfg->n_kv_heads;
+    if (attention_mma_supported(cfg->head_dim, cfg->max_window) &&
+        make_kv_tensor_map(&c->kv_map, c->ws + lay.kv, planes, cfg->max_seq, cfg->head_dim) == SJD_OK &&
+        cudaMemset(c->ws + lay.kv, 0, (size_t)planes * cfg->max_seq * cfg->head_dim * 2) == cudaSuccess)
+      c->kv_map_valid = true;
     for (int l = 0; l < L; ++l) {
       const LayerMaps &lm = c->wmaps[l];
       c->all_tc = c->all_tc && lm.wq.valid && lm.wk.valid && lm.wv.valid && lm.wo.valid && lm.w_gate.valid &&
