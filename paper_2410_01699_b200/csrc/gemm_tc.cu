@@ -32,7 +32,23 @@ constexpr int UMMA_K = 16;
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
-constexpr int kSmemBudget = 100 * 1024;   // per CTA, so that two CTAs fit one SM
+// tunables (defaults chosen by measurement on B200; see profiles/)
+#ifndef SJD_GEMM_SMEM_BUDGET
+#define SJD_GEMM_SMEM_BUDGET (100 * 1024)   // ring bytes per CTA when two CTAs share an SM
+#endif
+#ifndef SJD_GEMM_DEEP_RING
+#define SJD_GEMM_DEEP_RING 1                // double the ring when the grid has at most one CTA per SM
+#endif
+#ifndef SJD_GEMM_L2_PROMO
+#define SJD_GEMM_L2_PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
+#ifndef SJD_GEMM_MIN_KB
+#define SJD_GEMM_MIN_KB 16                  // fewest k-blocks (of 16 KB of weights) a CTA should stream
+#endif
+#ifndef SJD_GEMM_CTAS_PER_SM
+#define SJD_GEMM_CTAS_PER_SM 2
+#endif
+constexpr int kSmemBudget = SJD_GEMM_SMEM_BUDGET;
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
 struct GemmParams {
@@ -343,7 +359,7 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
   cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(reinterpret_cast<CUtensorMap *>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base),
                         dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        SJD_GEMM_L2_PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SJD_OK : SJD_ERR_CUDA;
 }
 
@@ -352,8 +368,8 @@ bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 128 && N % T
 // K splits for a launch of `tiles` weight tiles: at most two CTAs per SM in a single wave, at least
 // 16 k-blocks (256 KB of weights) per CTA so that set-up and drain stay small next to the streaming
 int gemm_tc_splits(int tiles, int k_blocks, int n_sms) {
-  int s = (2 * n_sms) / tiles;
-  const int cap = k_blocks / 16 > 1 ? k_blocks / 16 : 1;
+  int s = (SJD_GEMM_CTAS_PER_SM * n_sms) / tiles;
+  const int cap = k_blocks / SJD_GEMM_MIN_KB > 1 ? k_blocks / SJD_GEMM_MIN_KB : 1;
   s = s > cap ? cap : s;
   s = s > 16 ? 16 : s;
   return s < 1 ? 1 : s;
@@ -388,7 +404,7 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.eps = g.eps;
   const int stage_bytes = W_TILE_BYTES + 2 * p.Mp * TILE_K * 2;
   // one CTA per SM or fewer: give each the deeper ring
-  const int budget = (g.n_sms > 0 && tiles * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
+  const int budget = (SJD_GEMM_DEEP_RING && g.n_sms > 0 && tiles * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
   int stages = budget / stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : stages;
   if (stages < 2) return SJD_ERR_UNSUPPORTED;
