@@ -155,6 +155,8 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
 
 __global__ void attention_combine_kernel(const float *__restrict__ partial, const int32_t *__restrict__ in_pos,
                                          float *__restrict__ out, int n_heads, int hd, int splits, HiLoOut hilo) {
+  pdl_trigger();
+  pdl_wait();
   const int m = blockIdx.x, h = blockIdx.y;
   const float *src = partial + ((size_t)m * n_heads + h) * splits * (hd + 2);
   const size_t base = ((size_t)m * n_heads + h) * hd;
@@ -213,7 +215,8 @@ int attention_t(const float *q, KvLayout kv, const int32_t *in_pos, float *out, 
 
 int launch_attention_combine(const float *partial, const int32_t *in_pos, float *out, int M, int n_heads, int head_dim,
                              int splits, cudaStream_t stream, HiLoOut hilo) {
-  attention_combine_kernel<<<dim3(M, n_heads), 128, 0, stream>>>(partial, in_pos, out, n_heads, head_dim, splits, hilo);
+  SJD_CUDA(launch_kernel(attention_combine_kernel, dim3(M, n_heads), dim3(128), 0, stream, partial, in_pos, out, n_heads,
+                         head_dim, splits, hilo));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

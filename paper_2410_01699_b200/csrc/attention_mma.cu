@@ -97,6 +97,8 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   __shared__ int s_pos[64];
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
+  pdl_trigger();
+  pdl_wait();   // keys/values of this step were written by the preceding kernel
   const int h = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int W = p.rows_per_seq;
@@ -342,13 +344,13 @@ int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, co
       SJD_CUDA(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       configured[dev][1] = true;
     }
-    attention_mma_kernel<128><<<grid, threads, smem, stream>>>(km, p);
+    SJD_CUDA(launch_kernel(attention_mma_kernel<128>, grid, dim3(threads), smem, stream, km, p));
   } else {
     if (!configured[dev][0]) {
       SJD_CUDA(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       configured[dev][0] = true;
     }
-    attention_mma_kernel<64><<<grid, threads, smem, stream>>>(km, p);
+    SJD_CUDA(launch_kernel(attention_mma_kernel<64>, grid, dim3(threads), smem, stream, km, p));
   }
   SJD_CHECK_LAUNCH();
   return SJD_OK;

@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include <atomic>
 
@@ -29,6 +30,36 @@ extern std::atomic<long long> g_launch_count;  // kernels launched by this libra
     ::sjd::g_launch_count.fetch_add(1, std::memory_order_relaxed);      \
     SJD_CUDA(cudaGetLastError());                                       \
   } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  While g_pdl is set, kernels are launched with the
+// programmatic-stream-serialization attribute: a kernel may start (set up, prefetch data that does
+// not depend on its predecessor) before the previous kernel in the stream has finished.  Every such
+// kernel calls pdl_trigger() early and pdl_wait() before it touches anything an earlier kernel writes
+// or still reads; outside such launches both are no-ops.
+// ---------------------------------------------------------------------------------------------
+extern thread_local bool g_pdl;
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args &&...args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): 128-bit counter, 64-bit key, ten rounds of

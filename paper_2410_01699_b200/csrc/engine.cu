@@ -437,7 +437,13 @@ int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream)
   const int M = c->batch * rows_per_seq;
   if (c->use_tc && c->all_tc && M <= 128) {
     auto it = c->xmaps.find((M + 15) / 16 * 16);
-    if (it != c->xmaps.end()) return forward_tc(c, it->second, rows_per_seq, logits_out, stream);
+    if (it != c->xmaps.end()) {
+      // every kernel of this pipeline waits for its predecessor itself: launch them overlapped
+      g_pdl = !c->tracer.on;
+      const int rc = forward_tc(c, it->second, rows_per_seq, logits_out, stream);
+      g_pdl = false;
+      return rc;
+    }
   }
   return forward_generic(c, rows_per_seq, logits_out, stream);
 }
@@ -645,7 +651,9 @@ extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) 
   int rc = forward(c, c->window, c->ws + c->lay.logits[cur], stream);
   if (rc != SJD_OK) return rc;
   c->tracer.begin(TC_VERIFY, stream);
+  g_pdl = !c->tracer.on;
   rc = run_verify(c, out, stream);
+  g_pdl = false;
   c->tracer.end(stream);
   if (rc != SJD_OK) return rc;
   c->host_step += 1;

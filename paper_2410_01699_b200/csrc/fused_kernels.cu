@@ -45,6 +45,8 @@ template <typename T>
 __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restrict__ x, PlaneSet ps, const T *__restrict__ gain,
                                                                HiLoOut h, float *__restrict__ ss_part, int d) {
   __shared__ float red[RG_THREADS / 32];
+  pdl_trigger();
+  pdl_wait();
   const int m = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;
   const int c0 = chunk * RG_COLS + tid * 4;
   float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -77,6 +79,8 @@ template <typename T>
 __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__restrict__ in_pos,
                                   const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
                                   int n_heads) {
+  pdl_trigger();
+  pdl_wait();
   const int m = blockIdx.x, slot = blockIdx.y;
   const int pos = in_pos[m];
   if (pos < 0) return;
@@ -113,6 +117,8 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
 
 // act = silu(scale * sum gate planes) * (scale * sum up planes) as bf16 hi/lo planes; planes [S][M][2F]
 __global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F) {
+  pdl_trigger();
+  pdl_wait();
   const size_t total = (size_t)M * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t m = i / F, f = i % F;
@@ -131,10 +137,11 @@ int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOu
   if (d % 4 != 0) return SJD_ERR_UNSUPPORTED;
   const dim3 grid(M, resid_gain_parts(d));
   if (dtype == SJD_F32)
-    resid_gain_kernel<float><<<grid, RG_THREADS, 0, stream>>>(x, ps, reinterpret_cast<const float *>(gain), h, ss_part, d);
+    SJD_CUDA(launch_kernel(resid_gain_kernel<float>, grid, dim3(RG_THREADS), 0, stream, x, ps,
+                           reinterpret_cast<const float *>(gain), h, ss_part, d));
   else if (dtype == SJD_BF16)
-    resid_gain_kernel<__nv_bfloat16><<<grid, RG_THREADS, 0, stream>>>(x, ps, reinterpret_cast<const __nv_bfloat16 *>(gain), h,
-                                                                     ss_part, d);
+    SJD_CUDA(launch_kernel(resid_gain_kernel<__nv_bfloat16>, grid, dim3(RG_THREADS), 0, stream, x, ps,
+                           reinterpret_cast<const __nv_bfloat16 *>(gain), h, ss_part, d));
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();
@@ -145,9 +152,11 @@ int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos
                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
   const dim3 grid(M, n_heads + 2 * kv.n_kv_heads);
   if (dtype == SJD_F32)
-    qkv_finish_kernel<float><<<grid, 64, 0, stream>>>(ps, rs, in_pos, rope_table, q, kv, rows_per_seq, n_heads);
+    SJD_CUDA(launch_kernel(qkv_finish_kernel<float>, grid, dim3(64), 0, stream, ps, rs, in_pos, rope_table, q, kv,
+                           rows_per_seq, n_heads));
   else if (dtype == SJD_BF16)
-    qkv_finish_kernel<__nv_bfloat16><<<grid, 64, 0, stream>>>(ps, rs, in_pos, rope_table, q, kv, rows_per_seq, n_heads);
+    SJD_CUDA(launch_kernel(qkv_finish_kernel<__nv_bfloat16>, grid, dim3(64), 0, stream, ps, rs, in_pos, rope_table, q, kv,
+                           rows_per_seq, n_heads));
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();
@@ -157,7 +166,7 @@ int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos
 int launch_swiglu_finish(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, cudaStream_t stream) {
   const size_t total = (size_t)M * F;
   const int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
-  swiglu_finish_kernel<<<blocks, 256, 0, stream>>>(ps, rs, act, M, F);
+  SJD_CUDA(launch_kernel(swiglu_finish_kernel, dim3(blocks), dim3(256), 0, stream, ps, rs, act, M, F));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

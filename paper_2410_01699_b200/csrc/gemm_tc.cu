@@ -185,6 +185,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   __shared__ uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full;
   __shared__ uint32_t s_tmem_base;
 
+  pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int NN = 2 * p.Mp;                                   // MMA N
@@ -231,10 +232,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
     if (lane == 0) {
       uint64_t policy;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-      int s = 0;
-      uint32_t ph = 0;
+      // The weights do not depend on the preceding kernel: fill the ring with W tiles right away,
+      // then wait for the predecessor before fetching the activation tiles it produced.
+      const int pre = n_kb < p.stages ? n_kb : p.stages;
+      for (int i = 0; i < pre; ++i) {
+        mbar_expect_tx(&bar_full[i], (uint32_t)stage_bytes);
+        tma_load_2d(smem + i * stage_bytes, w_map, (kb_begin + i) * TILE_K, tile_in_mat * TILE_N, &bar_full[i], policy);
+      }
+      pdl_wait();
+      for (int i = 0; i < pre; ++i) {
+        uint8_t *dst = smem + i * stage_bytes;
+        const int kcol = (kb_begin + i) * TILE_K;
+        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, 0, &bar_full[i]);
+        tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row, &bar_full[i]);
+      }
+      int s = pre == p.stages ? 0 : pre;
+      uint32_t ph = pre == p.stages ? 1u : 0u;
       bool ok = true;
-      int it = 0;
+      int it = pre;
       for (; it < n_kb; ++it) {
         if (!mbar_wait(&bar_empty[s], ph ^ 1u)) { ok = false; break; }
         uint8_t *dst = smem + s * stage_bytes;
@@ -282,6 +297,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
     const bool ok = epilogue_all(mbar_wait(&bar_acc_full, 0));
     if (ok) {
       tc_fence_after();
+      pdl_wait();   // the planes may still be read, and the row scales written, by the preceding kernel
       const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
       const int n = p.col_off[mat] + tile_in_mat * TILE_N + row;
       float *plane = reinterpret_cast<float *>(p.out) + (size_t)split * p.plane_stride;
@@ -423,7 +439,7 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
     SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
     configured[dev] = true;
   }
-  gemm_tc_kernel<<<dim3(tiles, g.splits), kThreads, smem, stream>>>(w0, w1, w2, xm, p);
+  SJD_CUDA(launch_kernel(gemm_tc_kernel, dim3(tiles, g.splits), dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

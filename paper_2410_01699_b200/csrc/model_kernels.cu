@@ -93,6 +93,8 @@ int gemm_simt_t(const void *A, int lda, const void *Wt, void *C, int ldc, int M,
 template <typename T>
 __global__ void embed_kernel(const T *__restrict__ emb, const int32_t *__restrict__ tok, float *__restrict__ x, int d,
                              int vocab) {
+  pdl_trigger();
+  pdl_wait();
   const int m = blockIdx.x;
   int t = tok[m];
   t = min(max(t, 0), vocab - 1);
@@ -189,7 +191,8 @@ int launch_gemm_simt(int dtype, const void *A, int lda, const void *Wt, void *C,
 
 int launch_embed(int dtype, const void *tok_emb, const int32_t *tok, float *x, int M, int d, int vocab,
                  cudaStream_t stream) {
-  SJD_DISPATCH(dtype, (embed_kernel<T><<<M, 256, 0, stream>>>(reinterpret_cast<const T *>(tok_emb), tok, x, d, vocab)));
+  SJD_DISPATCH(dtype, SJD_CUDA(launch_kernel(embed_kernel<T>, dim3(M), dim3(256), 0, stream, reinterpret_cast<const T *>(tok_emb),
+                                             tok, x, d, vocab)));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -567,6 +567,8 @@ __global__ void __launch_bounds__(kMaxThreads) verify_rows_kernel(const VerifyPa
   extern __shared__ uint4 dyn_smem[];
   __shared__ Scratch sc;
   uint4 *stage = p.staged ? dyn_smem : nullptr;
+  pdl_trigger();
+  pdl_wait();   // the logits come from the preceding kernel
 
   const int r = blockIdx.x;
   const int b = r / p.W, k = r % p.W;
@@ -708,7 +710,7 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
   int threads = nv_max <= 1024 ? 128 : nv_max <= 4096 ? 256 : nv_max <= 16384 ? 512 : 1024;
   if (dyn > 48 * 1024)
     SJD_CUDA(cudaFuncSetAttribute(verify_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-  verify_rows_kernel<T><<<p.B * p.W, threads, dyn, stream>>>(p);
+  SJD_CUDA(launch_kernel(verify_rows_kernel<T>, dim3(p.B * p.W), dim3(threads), dyn, stream, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
