@@ -165,7 +165,9 @@ int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos
 
 int launch_swiglu_finish(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, cudaStream_t stream) {
   const size_t total = (size_t)M * F;
-  const int blocks = (int)((total + 255) / 256 < 2368 ? (total + 255) / 256 : 2368);
+  // at most two blocks per SM: the whole grid must be resident at once for the next kernel to be
+  // scheduled early, and it must leave thread slots for that kernel's CTAs while it waits
+  const int blocks = (int)((total + 255) / 256 < 296 ? (total + 255) / 256 : 296);
   SJD_CUDA(launch_kernel(swiglu_finish_kernel, dim3(blocks), dim3(256), 0, stream, ps, rs, act, M, F));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
