@@ -218,6 +218,26 @@ struct sjd_ctx {
   bool prefilled;
   uint32_t host_step;  // number of sjd_step calls since prefill == device step index
   cudaStream_t last_stream;
+  // One captured CUDA graph per logits-buffer parity: a step is ~330 launches, and replaying a graph
+  // takes the host out of the critical path.  Keyed by the caller's output pointers.
+  struct StepGraph {
+    cudaGraphExec_t exec = nullptr;
+    sjd_step_out out;
+    bool has_out = false;
+    long long launches = 0;
+  } graphs[2];
+  cudaStream_t capture_stream = nullptr;
+  bool graphs_enabled = true;
+  void drop_graphs() {
+    for (int i = 0; i < 2; ++i) {
+      if (graphs[i].exec) cudaGraphExecDestroy(graphs[i].exec);
+      graphs[i].exec = nullptr;
+    }
+  }
+  ~sjd_ctx() {
+    drop_graphs();
+    if (capture_stream) cudaStreamDestroy(capture_stream);
+  }
   Tracer tracer;
   bool use_tc = false;   // bf16 model on a device with tensor memory: tensor-core GEMM path
   bool all_tc = false;   // every projection of the model is covered by it
@@ -607,6 +627,7 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
   c->host_step = 0;
   c->last_stream = stream;
   c->prefilled = false;
+  c->drop_graphs();
   if (c->use_tc) {
     // activation descriptors for the two row counts used: the step's window and the pre-fill chunk
     const int Ma = c->rows_alloc();
@@ -642,12 +663,9 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
   return SJD_OK;
 }
 
-extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) {
-  if (!c) return SJD_ERR_BAD_ARG;
-  if (!c->prefilled) return SJD_ERR_STATE;
-  cudaStream_t stream = (cudaStream_t)cuda_stream;
-  c->last_stream = stream;
-  const int cur = (int)(c->host_step & 1u);
+namespace {
+// forward pass + verification of one step, enqueued on `stream`
+int enqueue_step(sjd_ctx *c, const sjd_step_out *out, int cur, cudaStream_t stream) {
   int rc = forward(c, c->window, c->ws + c->lay.logits[cur], stream);
   if (rc != SJD_OK) return rc;
   c->tracer.begin(TC_VERIFY, stream);
@@ -655,6 +673,65 @@ extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) 
   rc = run_verify(c, out, stream);
   g_pdl = false;
   c->tracer.end(stream);
+  return rc;
+}
+
+bool same_out(const sjd_step_out &a, const sjd_step_out *b) {
+  sjd_step_out z;
+  memset(&z, 0, sizeof(z));
+  return memcmp(&a, b ? b : &z, sizeof(sjd_step_out)) == 0;
+}
+}  // namespace
+
+extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) {
+  if (!c) return SJD_ERR_BAD_ARG;
+  if (!c->prefilled) return SJD_ERR_STATE;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  c->last_stream = stream;
+  const int cur = (int)(c->host_step & 1u);
+  if (c->graphs_enabled && c->use_tc && !c->tracer.on) {
+    sjd_ctx::StepGraph &g = c->graphs[cur];
+    if (g.exec && !(g.has_out && same_out(g.out, out))) {
+      cudaGraphExecDestroy(g.exec);
+      g.exec = nullptr;
+    }
+    if (!g.exec) {
+      // capture on a private stream (the caller's may be the legacy default stream), replay on the caller's
+      if (!c->capture_stream && cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking) != cudaSuccess)
+        c->graphs_enabled = false;
+      if (c->graphs_enabled) {
+        const long long before = g_launch_count.load();
+        cudaGraph_t graph = nullptr;
+        bool ok = cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+        if (ok) {
+          const int rc = enqueue_step(c, out, cur, c->capture_stream);
+          const cudaError_t e = cudaStreamEndCapture(c->capture_stream, &graph);
+          ok = rc == SJD_OK && e == cudaSuccess && graph != nullptr;
+        }
+        const long long captured = g_launch_count.load() - before;   // kernels recorded, not run
+        g_launch_count.store(before);
+        if (ok) ok = cudaGraphInstantiate(&g.exec, graph, 0) == cudaSuccess;
+        if (graph) cudaGraphDestroy(graph);
+        if (ok) {
+          memset(&g.out, 0, sizeof(g.out));
+          if (out) g.out = *out;
+          g.has_out = true;
+          g.launches = captured;
+        } else {
+          g.exec = nullptr;
+          c->graphs_enabled = false;   // fall back to direct launches for good
+          cudaGetLastError();
+        }
+      }
+    }
+    if (g.exec) {
+      SJD_CUDA(cudaGraphLaunch(g.exec, stream));
+      g_launch_count.fetch_add(g.launches, std::memory_order_relaxed);
+      c->host_step += 1;
+      return SJD_OK;
+    }
+  }
+  const int rc = enqueue_step(c, out, cur, stream);
   if (rc != SJD_OK) return rc;
   c->host_step += 1;
   return c->tracer.flush(stream);
