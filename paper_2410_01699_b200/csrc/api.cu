@@ -151,3 +151,24 @@ extern "C" int sjd_gemm(int M, int N, int K, const float *x, const void *w, floa
   if (rc != SJD_OK) return rc;
   return launch_sum_planes(planes, (size_t)M * N, splits, out, (size_t)M * N, accumulate, stream);
 }
+
+#ifdef SJD_TIMELINE
+// timeline builds only: allocate / read the device timeline (see common.cuh)
+namespace sjd {
+void timeline_set_fused(TimelineBuf *);
+void timeline_set_gemm(TimelineBuf *);
+void timeline_set_attn(TimelineBuf *);
+void timeline_set_combine(TimelineBuf *);
+void timeline_set_verify(TimelineBuf *);
+}  // namespace sjd
+extern "C" int sjd_timeline_attach(void *device_buf) {
+  TimelineBuf *b = (TimelineBuf *)device_buf;
+  timeline_set_fused(b);
+  timeline_set_gemm(b);
+  timeline_set_attn(b);
+  timeline_set_combine(b);
+  timeline_set_verify(b);
+  return SJD_OK;
+}
+extern "C" size_t sjd_timeline_bytes(void) { return sizeof(TimelineBuf); }
+#endif

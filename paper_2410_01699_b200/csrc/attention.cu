@@ -8,6 +8,7 @@
 #include "common.cuh"
 
 namespace sjd {
+SJD_TIMELINE_TU(combine)
 namespace {
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
@@ -156,7 +157,9 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
 __global__ void attention_combine_kernel(const float *__restrict__ partial, const int32_t *__restrict__ in_pos,
                                          float *__restrict__ out, int n_heads, int hd, int splits, HiLoOut hilo) {
   pdl_trigger();
+  SJD_TL(TL_COMBINE, 0, threadIdx.x == 0);
   pdl_wait();
+  SJD_TL(TL_COMBINE, 1, threadIdx.x == 0);
   const int m = blockIdx.x, h = blockIdx.y;
   const float *src = partial + ((size_t)m * n_heads + h) * splits * (hd + 2);
   const size_t base = ((size_t)m * n_heads + h) * hd;

@@ -14,6 +14,7 @@
 #include "common.cuh"
 
 namespace sjd {
+SJD_TIMELINE_TU(attn)
 namespace {
 
 constexpr int KT = 64;                 // keys per tile
@@ -98,7 +99,9 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   pdl_trigger();
+  SJD_TL(TL_ATTN, 0, threadIdx.x == 0);
   pdl_wait();   // keys/values of this step were written by the preceding kernel
+  SJD_TL(TL_ATTN, 1, threadIdx.x == 0);
   const int h = blockIdx.x, b = blockIdx.y, split = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int W = p.rows_per_seq;
@@ -266,6 +269,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     return;
   }
 
+  SJD_TL(TL_ATTN, 2, threadIdx.x == 0);
   // ---- partial record per (row, head, split): [max (natural log units), sum, o[HD]]
   l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
   l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);

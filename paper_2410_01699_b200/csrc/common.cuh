@@ -62,6 +62,39 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 #endif
 
 // ---------------------------------------------------------------------------------------------
+// Optional device timeline (build with -DSJD_TIMELINE): block 0 of every kernel of the tensor-core
+// pipeline stamps %globaltimer at entry, after its grid-dependency wait and at its end into one
+// buffer, which shows how the overlapped launches really interleave.  Off in normal builds.
+// ---------------------------------------------------------------------------------------------
+#ifdef SJD_TIMELINE
+struct TimelineBuf {
+  unsigned int n;
+  unsigned int pad;
+  struct Rec { unsigned long long t; int tag; int phase; } rec[1 << 16];
+};
+#define SJD_TIMELINE_TU(name)                                                                       \
+  static __device__ TimelineBuf *g_tl_buf;                                                         \
+  void timeline_set_##name(TimelineBuf *p) { cudaMemcpyToSymbol(g_tl_buf, &p, sizeof(p)); }        \
+  __device__ __forceinline__ void tl_mark(int tag, int phase) {                                    \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && g_tl_buf) {                      \
+      unsigned long long t;                                                                        \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));                                         \
+      const unsigned int i = atomicAdd(&g_tl_buf->n, 1u);                                          \
+      if (i < (1u << 16)) {                                                                        \
+        g_tl_buf->rec[i].t = t;                                                                    \
+        g_tl_buf->rec[i].tag = tag;                                                                \
+        g_tl_buf->rec[i].phase = phase;                                                            \
+      }                                                                                            \
+    }                                                                                              \
+  }
+#define SJD_TL(tag, phase, cond) do { if (cond) tl_mark(tag, phase); } while (0)
+#else
+#define SJD_TIMELINE_TU(name)
+#define SJD_TL(tag, phase, cond) do { } while (0)
+#endif
+enum TimelineTag { TL_EMBED = 0, TL_RESID = 1, TL_GEMM = 2, TL_QKV = 3, TL_ATTN = 4, TL_COMBINE = 5, TL_SWIGLU = 6, TL_VERIFY = 7 };
+
+// ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): 128-bit counter, 64-bit key, ten rounds of
 // two 32x32->64 multiplies with a Weyl key schedule.
 // ---------------------------------------------------------------------------------------------

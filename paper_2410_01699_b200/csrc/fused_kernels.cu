@@ -5,6 +5,7 @@
 #include "common.cuh"
 
 namespace sjd {
+SJD_TIMELINE_TU(fused)
 namespace {
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
@@ -46,7 +47,9 @@ __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restric
                                                                HiLoOut h, float *__restrict__ ss_part, int d) {
   __shared__ float red[RG_THREADS / 32];
   pdl_trigger();
+  SJD_TL(TL_RESID, 0, threadIdx.x == 0);
   pdl_wait();
+  SJD_TL(TL_RESID, 1, threadIdx.x == 0);
   const int m = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x;
   const int c0 = chunk * RG_COLS + tid * 4;
   float v[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -71,6 +74,7 @@ __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restric
     for (int w = 0; w < RG_THREADS / 32; ++w) tot += red[w];
     ss_part[(size_t)m * gridDim.y + chunk] = tot;
   }
+  SJD_TL(TL_RESID, 2, threadIdx.x == 0);
 }
 
 // q,k,v = scale * sum of the QKV planes; rotate q and k (pairs i, i + hd/2) by the row's absolute
@@ -80,7 +84,9 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
                                   const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
                                   int n_heads) {
   pdl_trigger();
+  SJD_TL(TL_QKV, 0, threadIdx.x == 0);
   pdl_wait();
+  SJD_TL(TL_QKV, 1, threadIdx.x == 0);
   const int m = blockIdx.x, slot = blockIdx.y;
   const int pos = in_pos[m];
   if (pos < 0) return;
@@ -118,7 +124,9 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
 // act = silu(scale * sum gate planes) * (scale * sum up planes) as bf16 hi/lo planes; planes [S][M][2F]
 __global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F) {
   pdl_trigger();
+  SJD_TL(TL_SWIGLU, 0, threadIdx.x == 0);
   pdl_wait();
+  SJD_TL(TL_SWIGLU, 1, threadIdx.x == 0);
   const size_t total = (size_t)M * F;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t m = i / F, f = i % F;
@@ -126,6 +134,7 @@ __global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int 
     const float g = sc * sum_planes(ps, m * ps.ld + f), u = sc * sum_planes(ps, m * ps.ld + F + f);
     put_hilo(act, i, g / (1.0f + expf(-g)) * u);
   }
+  SJD_TL(TL_SWIGLU, 2, threadIdx.x == 0);
 }
 
 }  // namespace

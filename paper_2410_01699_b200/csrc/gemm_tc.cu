@@ -24,6 +24,7 @@
 #include "common.cuh"
 
 namespace sjd {
+SJD_TIMELINE_TU(gemm)
 namespace {
 
 constexpr int TILE_N = 128;   // weight rows per tile (MMA M)
@@ -186,6 +187,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   __shared__ uint32_t s_tmem_base;
 
   pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
+  SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
   const int NN = 2 * p.Mp;                                   // MMA N
@@ -239,7 +241,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         mbar_expect_tx(&bar_full[i], (uint32_t)stage_bytes);
         tma_load_2d(smem + i * stage_bytes, w_map, (kb_begin + i) * TILE_K, tile_in_mat * TILE_N, &bar_full[i], policy);
       }
+      SJD_TL(TL_GEMM, 3, true);
       pdl_wait();
+      SJD_TL(TL_GEMM, 1, true);
       for (int i = 0; i < pre; ++i) {
         uint8_t *dst = smem + i * stage_bytes;
         const int kcol = (kb_begin + i) * TILE_K;
@@ -325,6 +329,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
     } else if (tid == 64) {
       atomicExch(p.status, 3);
     }
+    SJD_TL(TL_GEMM, 2, tid == 64);
   }
 
   tc_fence_before();

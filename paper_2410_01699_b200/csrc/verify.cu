@@ -19,6 +19,7 @@
 #include "common.cuh"
 
 namespace sjd {
+SJD_TIMELINE_TU(verify)
 namespace {
 
 constexpr int kMaxChunks = 1024;   // 32 vectors of 16 bytes per chunk
@@ -568,7 +569,9 @@ __global__ void __launch_bounds__(kMaxThreads) verify_rows_kernel(const VerifyPa
   __shared__ Scratch sc;
   uint4 *stage = p.staged ? dyn_smem : nullptr;
   pdl_trigger();
+  SJD_TL(TL_VERIFY, 0, threadIdx.x == 0);
   pdl_wait();   // the logits come from the preceding kernel
+  SJD_TL(TL_VERIFY, 1, threadIdx.x == 0);
 
   const int r = blockIdx.x;
   const int b = r / p.W, k = r % p.W;
