@@ -315,10 +315,13 @@ def main():
     ap.add_argument("--workload", default="7b")
     ap.add_argument("--batch", type=int, default=1, help="sequences per GPU")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (longer KV prefix)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2410_01699_b200.inputs import WORKLOADS
     wl = WORKLOADS[args.workload]
+    if args.prompt_len:
+        wl = wl.with_(prompt_len=args.prompt_len)
     if args.impl == "reference":
         run_reference(args, wl)
     else:
