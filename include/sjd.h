@@ -243,6 +243,24 @@ size_t sjd_gemm_workspace_bytes(int M, int N, int K);
 int sjd_gemm(int M, int N, int K, const float *x, const void *w, float *out, int accumulate, void *ws,
              size_t ws_bytes, void *cuda_stream);
 
+/*
+ * The window-causal attention of the forward pass (Sec. 3.2 / Sec. 4.1 Step 2) in isolation, on the
+ * tensor-core split-KV kernel sjd_step uses for bf16 caches: query row m = b * window + k, at absolute
+ * position in_pos[m] (-1: inactive row, output zeros), attends cache rows 0 .. in_pos[m] of sequence b:
+ *     out[m][h] = softmax(q[m][h] . K[b][h / (H/KVh)][0..pos]^T / sqrt(head_dim)) V[b][...][0..pos]
+ * q, out: device fp32 [batch*window][n_heads*head_dim]; kv_cache: device bf16
+ * [batch][K|V][n_kv_heads][max_seq][head_dim], finite everywhere (rows beyond the positions are read
+ * and masked); in_pos: device int32 [batch*window].  Covered: head_dim 64 or 128, window <= 64,
+ * compute capability >= 9; anything else returns SJD_ERR_UNSUPPORTED.  ws: device scratch of
+ * sjd_attention_workspace_bytes(...), 256-byte aligned; its first int32 is non-zero after the stream
+ * has drained if a bounded device-side wait ran out.
+ * Errors: BAD_ARG, UNSUPPORTED, CAPACITY, CUDA.
+ */
+size_t sjd_attention_workspace_bytes(int batch, int window, int n_heads, int head_dim);
+int sjd_attention(int batch, int window, int n_heads, int n_kv_heads, int head_dim, int max_seq, const float *q,
+                  const void *kv_cache, const int32_t *in_pos, float *out, void *ws, size_t ws_bytes,
+                  void *cuda_stream);
+
 /* Synchronises the context's last stream and returns SJD_OK, SJD_ERR_DEVICE_TIMEOUT
  * or SJD_ERR_CUDA according to the device status word. */
 int sjd_last_device_status(sjd_ctx *ctx);

@@ -28,7 +28,7 @@ TORCH_DTYPES = {SJD_F32: torch.float32, SJD_BF16: torch.bfloat16}
 EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_get_window", "sjd_peek_logits",
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
            "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static",
-           "sjd_gemm_workspace_bytes", "sjd_gemm"]
+           "sjd_gemm_workspace_bytes", "sjd_gemm", "sjd_attention_workspace_bytes", "sjd_attention"]
 
 
 class SJDError(RuntimeError):
@@ -108,6 +108,10 @@ def lib():
     L.sjd_gemm.restype = C.c_int
     L.sjd_gemm.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                            C.c_size_t, C.c_void_p]
+    L.sjd_attention_workspace_bytes.restype = C.c_size_t
+    L.sjd_attention_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
+    L.sjd_attention.restype = C.c_int
+    L.sjd_attention.argtypes = [C.c_int] * 6 + [C.c_void_p] * 5 + [C.c_size_t, C.c_void_p]
     L.sjd_last_device_status.restype = C.c_int
     L.sjd_last_device_status.argtypes = [C.c_void_p]
     L.sjd_last_cuda_error.restype = C.c_int
@@ -219,6 +223,23 @@ def sjd_gemm(x, w, out=None, accumulate=False):
     ws = torch.empty(nbytes, dtype=torch.uint8, device=x.device)
     _check(lib().sjd_gemm(m, n, k, _ptr(x), _ptr(w), _ptr(out), 1 if accumulate else 0, _ptr(ws), nbytes, _stream()),
            "sjd_gemm")
+    return out, ws[:4].view(torch.int32)
+
+
+def sjd_attention(q, kv_cache, in_pos, window, n_kv_heads, out=None, ws=None):
+    """Window-causal attention on the tensor-core kernel.  q: float32 cuda [B*W][H][hd]; kv_cache:
+    bfloat16 cuda [B][2][KVh][max_seq][hd]; in_pos: int32 cuda [B*W].  Returns (out, status word)."""
+    m, h, hd = q.shape
+    b, max_seq = kv_cache.shape[0], kv_cache.shape[3]
+    if out is None:
+        out = torch.empty_like(q)
+    nbytes = int(lib().sjd_attention_workspace_bytes(b, window, h, hd))
+    if nbytes == 0:
+        raise SJDError(SJD_ERR_UNSUPPORTED, "sjd_attention_workspace_bytes")
+    if ws is None:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    _check(lib().sjd_attention(b, window, h, n_kv_heads, hd, max_seq, _ptr(q), _ptr(kv_cache), _ptr(in_pos), _ptr(out),
+                               _ptr(ws), nbytes, _stream()), "sjd_attention")
     return out, ws[:4].view(torch.int32)
 
 

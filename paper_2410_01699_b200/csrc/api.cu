@@ -172,3 +172,43 @@ extern "C" int sjd_timeline_attach(void *device_buf) {
 }
 extern "C" size_t sjd_timeline_bytes(void) { return sizeof(TimelineBuf); }
 #endif
+
+// ---- the window attention of Step 2 in isolation (tensor-core split-KV kernel, bf16 cache)
+namespace {
+int attn_splits(int n_heads, int batch) {
+  int s = (2 * 148) / (n_heads * batch);
+  return s < 1 ? 1 : (s > 16 ? 16 : s);
+}
+}  // namespace
+
+extern "C" size_t sjd_attention_workspace_bytes(int batch, int window, int n_heads, int head_dim) {
+  if (batch < 1 || window < 1 || n_heads < 1 || !attention_mma_supported(head_dim, window)) return 0;
+  return 256 + (size_t)batch * window * n_heads * attn_splits(n_heads, batch) * (head_dim + 2) * 4;
+}
+
+extern "C" int sjd_attention(int batch, int window, int n_heads, int n_kv_heads, int head_dim, int max_seq, const float *q,
+                             const void *kv_cache, const int32_t *in_pos, float *out, void *ws, size_t ws_bytes,
+                             void *cuda_stream) {
+  if (batch < 1 || window < 1 || n_heads < 1 || n_kv_heads < 1 || max_seq < 1 || !q || !kv_cache || !in_pos || !out || !ws)
+    return SJD_ERR_BAD_ARG;
+  if (n_heads % n_kv_heads != 0) return SJD_ERR_BAD_ARG;
+  if (!attention_mma_supported(head_dim, window)) return SJD_ERR_UNSUPPORTED;
+  if (((uintptr_t)ws & 255u) != 0) return SJD_ERR_BAD_ARG;
+  if (ws_bytes < sjd_attention_workspace_bytes(batch, window, n_heads, head_dim)) return SJD_ERR_CAPACITY;
+  int dev = 0, cc_major = 0;
+  SJD_CUDA(cudaGetDevice(&dev));
+  SJD_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (cc_major < 9) return SJD_ERR_UNSUPPORTED;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  int *status = (int *)ws;
+  float *partial = (float *)((char *)ws + 256);
+  SJD_CUDA(cudaMemsetAsync(status, 0, 256, stream));
+  TensorMap kv_map;
+  int rc = make_kv_tensor_map(&kv_map, kv_cache, (long)batch * 2 * n_kv_heads, max_seq, head_dim);
+  if (rc != SJD_OK) return rc;
+  const int splits = attn_splits(n_heads, batch);
+  const int M = batch * window;
+  rc = launch_attention_mma(kv_map, 0, q, in_pos, partial, status, M, window, n_heads, n_kv_heads, head_dim, splits, stream);
+  if (rc != SJD_OK) return rc;
+  return launch_attention_combine(partial, in_pos, out, M, n_heads, head_dim, splits, stream, HiLoOut{nullptr, 0});
+}

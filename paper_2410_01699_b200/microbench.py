@@ -6,6 +6,8 @@
 gemm    the weight-streaming projection (sjd_gemm): fp32 x[M][K], bf16 w[N][K]; reports the achieved
         weight-streaming rate N*K*2 bytes / time.  The weights rotate through enough copies to exceed
         the L2 cache, so every launch streams from HBM.
+attention BATCH PREFIX [--window W --heads H --kv-heads KVH --head-dim D]: the window attention
+        (sjd_attention) of W queries over PREFIX + W cached positions; reports K/V bytes / time.
 verify  the isolated verify-and-resample kernel (sjd_verify) on the synthetic verification workload;
         reports 2*B*W*V*2 bytes / time (current and previous logits read once each).
 
@@ -85,6 +87,32 @@ def bench_verify(batch, window, vocab, top_k, iters):
             "rows_per_s": batch * window / sec, "mean_accepted": float(out.host()["n_accepted"].mean())}
 
 
+def bench_attention(batch, window, prefix, n_heads, n_kv_heads, head_dim, iters):
+    g = torch.Generator(device="cuda").manual_seed(0)
+    max_seq = prefix + window
+    q = torch.randn(batch * window, n_heads, head_dim, generator=g, device="cuda")
+    kv_bytes = batch * 2 * n_kv_heads * max_seq * head_dim * 2
+    copies = max(1, min(8, (192 << 20) // kv_bytes + 1))
+    kvs = [torch.randn(batch, 2, n_kv_heads, max_seq, head_dim, generator=g, device="cuda").to(torch.bfloat16)
+           for _ in range(copies)]
+    pos = (prefix - 1 + torch.arange(window, dtype=torch.int32, device="cuda")).repeat(batch).contiguous()
+    out = torch.empty_like(q)
+    ws = torch.empty(int(B.lib().sjd_attention_workspace_bytes(batch, window, n_heads, head_dim)), dtype=torch.uint8,
+                     device="cuda")
+    status = [None]
+
+    def run(i):
+        _, status[0] = B.sjd_attention(q, kvs[i % copies], pos, window, n_kv_heads, out=out, ws=ws)
+
+    sec = _time(run, iters)
+    assert int(status[0].item()) == 0
+    peak, src = _peak()
+    gbs = kv_bytes / sec / 1e9
+    return {"kernel": "sjd_attention", "batch": batch, "window": window, "prefix": prefix, "n_heads": n_heads,
+            "n_kv_heads": n_kv_heads, "head_dim": head_dim, "us": sec * 1e6, "kv_GBps": gbs, "frac_of_hbm": gbs / peak,
+            "peak_GBps": peak, "peak_source": src, "note": "time includes the merge of the split-KV partials"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -99,8 +127,18 @@ def main():
     v.add_argument("--vocab", type=int, default=16384)
     v.add_argument("--top-k", type=int, default=2000)
     v.add_argument("--iters", type=int, default=50)
+    t = sub.add_parser("attention")
+    t.add_argument("batch", type=int)
+    t.add_argument("prefix", type=int)
+    t.add_argument("--window", type=int, default=32)
+    t.add_argument("--heads", type=int, default=32)
+    t.add_argument("--kv-heads", type=int, default=32)
+    t.add_argument("--head-dim", type=int, default=128)
+    t.add_argument("--iters", type=int, default=50)
     a = ap.parse_args()
-    if a.cmd == "gemm":
+    if a.cmd == "attention":
+        print(json.dumps(bench_attention(a.batch, a.window, a.prefix, a.heads, a.kv_heads, a.head_dim, a.iters)))
+    elif a.cmd == "gemm":
         print(json.dumps(bench_gemm(a.M, a.N, a.K, a.iters)))
     else:
         print(json.dumps(bench_verify(a.batch, a.window, a.vocab, a.top_k, a.iters)))
