@@ -32,11 +32,26 @@ def _peak():
     return 6650.0, "fallback"
 
 
-def _time(fn, iters, warmup=5):
+def _time(fn, iters, warmup=5, graph=False):
+    """Seconds per call.  graph=True records the `iters` calls into one CUDA graph and times replays of
+    it, so that a kernel of a few microseconds is not timed by the speed of the Python loop."""
     for _ in range(warmup):
         fn(0)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(iters):
+                fn(i)
+        g.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(5):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (5 * iters) * 1e-3
     e0.record()
     for i in range(iters):
         fn(i)
@@ -87,7 +102,7 @@ def bench_verify(batch, window, vocab, top_k, iters):
             "rows_per_s": batch * window / sec, "mean_accepted": float(out.host()["n_accepted"].mean())}
 
 
-def bench_attention(batch, window, prefix, n_heads, n_kv_heads, head_dim, iters):
+def bench_attention(batch, window, prefix, n_heads, n_kv_heads, head_dim, iters, graph=True):
     g = torch.Generator(device="cuda").manual_seed(0)
     max_seq = prefix + window
     q = torch.randn(batch * window, n_heads, head_dim, generator=g, device="cuda")
@@ -104,7 +119,7 @@ def bench_attention(batch, window, prefix, n_heads, n_kv_heads, head_dim, iters)
     def run(i):
         _, status[0] = B.sjd_attention(q, kvs[i % copies], pos, window, n_kv_heads, out=out, ws=ws)
 
-    sec = _time(run, iters)
+    sec = _time(run, iters, graph=graph)
     assert int(status[0].item()) == 0
     peak, src = _peak()
     gbs = kv_bytes / sec / 1e9
@@ -135,9 +150,10 @@ def main():
     t.add_argument("--kv-heads", type=int, default=32)
     t.add_argument("--head-dim", type=int, default=128)
     t.add_argument("--iters", type=int, default=50)
+    t.add_argument("--no-graph", action="store_true", help="time a plain Python loop of calls (for captures under ncu)")
     a = ap.parse_args()
     if a.cmd == "attention":
-        print(json.dumps(bench_attention(a.batch, a.window, a.prefix, a.heads, a.kv_heads, a.head_dim, a.iters)))
+        print(json.dumps(bench_attention(a.batch, a.window, a.prefix, a.heads, a.kv_heads, a.head_dim, a.iters, not a.no_graph)))
     elif a.cmd == "gemm":
         print(json.dumps(bench_gemm(a.M, a.N, a.K, a.iters)))
     else:
