@@ -95,14 +95,17 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.xs_act = take(2 * Ma * c.ffn_hidden * 2);
   {
     // fp32 partial planes of one GEMM launch: the largest splits * rows * columns over the launches
-    const int rows = (int)(Mx < 128 ? Mx : 128);
     const int tiles[4] = {(int)((nq + 2 * nk) / 128), c.d_model / 128, 2 * c.ffn_hidden / 128, c.d_model / 128};
     const int kbs[4] = {c.d_model / 64, (int)(nq / 64), c.d_model / 64, c.ffn_hidden / 64};
     const size_t cols[4] = {nq + 2 * nk, (size_t)c.d_model, (size_t)2 * c.ffn_hidden, (size_t)c.d_model};
     size_t need = 0;
     for (int i = 0; i < 4; ++i) {
-      const size_t n = (size_t)gemm_tc_splits(tiles[i] > 0 ? tiles[i] : 1, kbs[i], kMaxGemmCtas) * rows * cols[i];
-      need = n > need ? n : need;
+      for (size_t rows = 16; rows < Mx + 16 && rows <= 1024; rows += 16) {   // splits shrink as the token slabs grow
+        const size_t m = rows < Mx ? rows : Mx;
+        const int ctas = (tiles[i] > 0 ? tiles[i] : 1) * gemm_tc_plan((int)m).n_slabs;
+        const size_t n = (size_t)gemm_tc_splits(ctas, kbs[i], kMaxGemmCtas) * m * cols[i];
+        need = n > need ? n : need;
+      }
     }
     L.gemm_planes = take(need * 4);
   }
@@ -384,7 +387,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     call.x_lo_row = Ma;
     call.M = M;
     call.K = k_in;
-    call.splits = bf16_out ? 1 : gemm_tc_splits(tiles, k_in / 64, c->n_ctas);
+    call.splits = bf16_out ? 1 : gemm_tc_splits(tiles * gemm_tc_plan(M).n_slabs, k_in / 64, c->n_ctas);
     call.out = out;
     call.plane_stride = (size_t)M * ldc;
     call.ldc = ldc;
@@ -457,7 +460,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
 
 int forward(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t stream) {
   const int M = c->batch * rows_per_seq;
-  if (c->use_tc && c->all_tc && M <= 128) {
+  if (c->use_tc && c->all_tc && M <= 1024) {
     auto it = c->xmaps.find((M + 15) / 16 * 16);
     if (it != c->xmaps.end()) {
       // every kernel of this pipeline waits for its predecessor itself: launch them overlapped
@@ -637,11 +640,12 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
     const int row_counts[2] = {batch * sample->window, batch * c->cfg.max_window};
     for (int i = 0; i < 2; ++i) {
       const int Mp = (row_counts[i] + 15) / 16 * 16;
-      if (row_counts[i] > 128 || c->xmaps.count(Mp)) continue;
+      if (row_counts[i] > 1024 || c->xmaps.count(Mp)) continue;
       XMaps xm;
-      const bool ok = make_tensor_map_bf16(&xm.h, c->ws + c->lay.xs_h, 2L * Ma, c->cfg.d_model, Mp) == SJD_OK &&
-                      make_tensor_map_bf16(&xm.attn, c->ws + c->lay.xs_attn, 2L * Ma, nq, Mp) == SJD_OK &&
-                      make_tensor_map_bf16(&xm.act, c->ws + c->lay.xs_act, 2L * Ma, c->cfg.ffn_hidden, Mp) == SJD_OK;
+      const int box = gemm_tc_plan(row_counts[i]).slab_rows;
+      const bool ok = make_tensor_map_bf16(&xm.h, c->ws + c->lay.xs_h, 2L * Ma, c->cfg.d_model, box) == SJD_OK &&
+                      make_tensor_map_bf16(&xm.attn, c->ws + c->lay.xs_attn, 2L * Ma, nq, box) == SJD_OK &&
+                      make_tensor_map_bf16(&xm.act, c->ws + c->lay.xs_act, 2L * Ma, c->cfg.ffn_hidden, box) == SJD_OK;
       if (ok) c->xmaps[Mp] = xm;
     }
   }

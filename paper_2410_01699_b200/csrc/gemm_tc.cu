@@ -3,11 +3,14 @@
 //
 // Shape of the problem: M = batch * window is 8..128 rows, the weight matrices (bf16) are tens to
 // hundreds of MB and are read exactly once per step, so the kernel is bound by HBM bandwidth and its
-// job is to keep every SM's TMA queue full.
+// job is to keep every SM's TMA queue full.  Larger M (batches of images with wide windows, up to
+// 1024 rows) is cut into token slabs of at most 256 rows; the CTAs of the slabs of one weight tile
+// are neighbours in the grid, so the tile comes from HBM once and from L2 for the other slabs.
 //   * W is the 128-row operand of tcgen05.mma (M = 128), the tokens are the N dimension.  The fp32
 //     activations arrive split into two bf16 planes, hi = bf16(x) and lo = bf16(x - hi); both planes
 //     are columns of the same MMA (N = 2 * Mp), and the epilogue adds the two halves: activations keep
-//     ~16 bits of mantissa at no cost in weight bytes.
+//     ~16 bits of mantissa at no cost in weight bytes.  Above 128 rows the step is bound by the
+//     tensor pipe, not by bytes, and only the hi plane is multiplied (plain bf16 activations).
 //   * One CTA per (128-row weight tile, K split); two CTAs are resident per SM.  A launch covers up to
 //     three weight matrices that share the activation operand (Q|K|V, gate|up), so their tiles form
 //     one grid.  With more than one K split every CTA writes an fp32 partial plane; the consumer
@@ -49,6 +52,9 @@ constexpr int kMaxStages = 8;
 #ifndef SJD_GEMM_CTAS_PER_SM
 #define SJD_GEMM_CTAS_PER_SM 2
 #endif
+#ifndef SJD_GEMM_SPLIT_MAX_M
+#define SJD_GEMM_SPLIT_MAX_M 128            // most rows for which both the hi and the lo plane are multiplied
+#endif
 constexpr int kSmemBudget = SJD_GEMM_SMEM_BUDGET;
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
@@ -57,7 +63,9 @@ struct GemmParams {
   size_t plane_stride;    // elements between planes
   int ldc;
   int M;                  // valid token rows
-  int Mp;                 // token rows padded to a multiple of 16 (MMA N = 2 * Mp)
+  int Mp;                 // token rows of one slab, a multiple of 16 (MMA N = x_planes * Mp)
+  int n_slabs;            // token slabs; CTA blockIdx.x = weight tile * n_slabs + slab
+  int x_planes;           // 2: hi and lo planes of the activations, 1: hi only
   int x_lo_row;           // row of the lo plane inside the activation tensor map
   int k_blocks, splits;   // K / 64, K splits (gridDim.y)
   int tile_end[3];        // matrix j owns tiles [tile_end[j-1], tile_end[j])
@@ -189,8 +197,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
   SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tile = blockIdx.x, split = blockIdx.y;
-  const int NN = 2 * p.Mp;                                   // MMA N
+  const int tile = (int)blockIdx.x / p.n_slabs, split = blockIdx.y;
+  const int m_base = ((int)blockIdx.x - tile * p.n_slabs) * p.Mp;   // first token row of this CTA's slab
+  const int NN = p.x_planes * p.Mp;                          // MMA N
   const int x_tile_bytes = NN * TILE_K * 2;
   const int stage_bytes = W_TILE_BYTES + x_tile_bytes;
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -247,8 +256,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       for (int i = 0; i < pre; ++i) {
         uint8_t *dst = smem + i * stage_bytes;
         const int kcol = (kb_begin + i) * TILE_K;
-        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, 0, &bar_full[i]);
-        tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row, &bar_full[i]);
+        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, m_base, &bar_full[i]);
+        if (p.x_planes == 2)
+          tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[i]);
       }
       int s = pre == p.stages ? 0 : pre;
       uint32_t ph = pre == p.stages ? 1u : 0u;
@@ -260,8 +270,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         const int kcol = (kb_begin + it) * TILE_K;
         mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
         tma_load_2d(dst, w_map, kcol, tile_in_mat * TILE_N, &bar_full[s], policy);
-        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, 0, &bar_full[s]);
-        tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row, &bar_full[s]);
+        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, m_base, &bar_full[s]);
+        if (p.x_planes == 2)
+          tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[s]);
         if (++s == p.stages) { s = 0; ph ^= 1u; }
       }
       if (!ok) {
@@ -309,11 +320,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       for (int m0 = 0; m0 < p.Mp; m0 += 16) {
         uint32_t hi[16], lo[16];
         tmem_ld16_issue(t_addr + m0, hi);
-        tmem_ld16_issue(t_addr + p.Mp + m0, lo);
+        if (p.x_planes == 2) {
+          tmem_ld16_issue(t_addr + p.Mp + m0, lo);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) lo[i] = 0u;
+        }
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const int m = m0 + i;
+          const int m = m_base + m0 + i;
           if (m < p.M) {
             float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
             if (p.ss_part) {
@@ -384,7 +400,19 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
   return r == CUDA_SUCCESS ? SJD_OK : SJD_ERR_CUDA;
 }
 
-bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 128 && N % TILE_N == 0 && K % TILE_K == 0; }
+bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 1024 && N % TILE_N == 0 && K % TILE_K == 0; }
+
+// How M token rows are laid over the MMA N dimension (at most 256 columns per CTA): both activation
+// planes for M <= 128, the hi plane alone in slabs of at most 256 rows above that.
+GemmTcPlan gemm_tc_plan(int M) {
+  GemmTcPlan pl;
+  pl.x_planes = M <= SJD_GEMM_SPLIT_MAX_M ? 2 : 1;
+  const int cap = 256 / pl.x_planes;
+  pl.n_slabs = (M + cap - 1) / cap;
+  const int per = (M + pl.n_slabs - 1) / pl.n_slabs;
+  pl.slab_rows = (per + 15) / 16 * 16;
+  return pl;
+}
 
 // K splits for a launch of `tiles` weight tiles: at most two CTAs per SM in a single wave, at least
 // 16 k-blocks (256 KB of weights) per CTA so that set-up and drain stay small next to the streaming
@@ -412,8 +440,11 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.out = g.out;
   p.plane_stride = g.plane_stride;
   p.ldc = g.ldc;
+  const GemmTcPlan pl = gemm_tc_plan(g.M);
   p.M = g.M;
-  p.Mp = (g.M + 15) / 16 * 16;
+  p.Mp = pl.slab_rows;
+  p.n_slabs = pl.n_slabs;
+  p.x_planes = pl.x_planes;
   p.x_lo_row = g.x_lo_row;
   p.k_blocks = g.K / TILE_K;
   p.splits = g.splits;
@@ -423,9 +454,10 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.n_part = g.n_part;
   p.inv_d = g.inv_d;
   p.eps = g.eps;
-  const int stage_bytes = W_TILE_BYTES + 2 * p.Mp * TILE_K * 2;
+  const int stage_bytes = W_TILE_BYTES + p.x_planes * p.Mp * TILE_K * 2;
   // one CTA per SM or fewer: give each the deeper ring
-  const int budget = (SJD_GEMM_DEEP_RING && g.n_sms > 0 && tiles * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
+  const int budget =
+      (SJD_GEMM_DEEP_RING && g.n_sms > 0 && tiles * p.n_slabs * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
   int stages = budget / stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : stages;
   if (stages < 2) return SJD_ERR_UNSUPPORTED;
@@ -444,7 +476,7 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
     SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
     configured[dev] = true;
   }
-  SJD_CUDA(launch_kernel(gemm_tc_kernel, dim3(tiles, g.splits), dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  SJD_CUDA(launch_kernel(gemm_tc_kernel, dim3(tiles * p.n_slabs, g.splits), dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

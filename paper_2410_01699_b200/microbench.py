@@ -77,7 +77,8 @@ def bench_gemm(m, n, k, iters):
     peak, src = _peak()
     gbs = wbytes / sec / 1e9
     return {"kernel": "sjd_gemm", "M": m, "N": n, "K": k, "us": sec * 1e6, "weight_GBps": gbs, "frac_of_hbm": gbs / peak,
-            "peak_GBps": peak, "peak_source": src, "note": "time includes the hi/lo split and plane-sum launches of sjd_gemm"}
+            "peak_GBps": peak, "peak_source": src, "TFLOPs": 2.0 * m * n * k / sec / 1e12,
+            "note": "time includes the hi/lo split and plane-sum launches of sjd_gemm"}
 
 
 def bench_verify(batch, window, vocab, top_k, iters):

@@ -128,6 +128,7 @@ class LockStepSequence:
         self.st = sjd_begin(self.prompt, scfg, wl.vocab, seq=seq_id)
         self.stats = ParityStats(sequences=1)
         self.max_logit_err = 0.0
+        self.max_logit_excess = 0.0      # largest |diff| beyond half a storage ulp
         self.steps = 0
 
     def check_window(self, draft_row, kind_row, q_row, total):
@@ -161,7 +162,9 @@ class LockStepSequence:
             diff = np.abs(own - gpu_logits_rows[:w_eff])
             err = float(diff.max())
             self.max_logit_err = max(self.max_logit_err, err)
-            bad = diff > self.tol + storage_half_ulp(own, scfg.logits_dtype)
+            half_ulp = storage_half_ulp(own, scfg.logits_dtype)
+            self.max_logit_excess = max(self.max_logit_excess, float((diff - half_ulp).max()))
+            bad = diff > self.tol + half_ulp
             assert not bad.any(), (f"step {self.steps}: {int(bad.sum())} logits off by more than {self.tol} "
                                    f"+ half a storage ulp; max |diff| {err:.3e}")
         n_before = st.n

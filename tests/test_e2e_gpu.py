@@ -113,6 +113,16 @@ def test_small_bf16_gqa_generation():
         assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
 
 
+def test_small_bf16_many_rows():
+    """20 images x W = 16 = 320 rows per pass: the token-slab form of the projections (two slabs, hi
+    plane only) through pre-fill and three steps."""
+    wl = WORKLOADS["small-bf16"]
+    ctx, seqs, steps, _ = run_lockstep(wl, batch=20, max_steps=3)
+    for s in seqs:
+        assert s.max_logit_err <= 2e-2
+        assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
+
+
 @pytest.mark.parametrize("name,steps", [("7b-2l", 4), ("8b-gqa-2l", 3)])
 def test_large_shapes_two_layers(name, steps):
     """The 7B / 8B-GQA layer shapes (d 4096, SwiGLU 11008 / 14336, vocab 65536 / 184320, W 32 / 64,
