@@ -4,13 +4,14 @@
 // Shape of the problem: M = batch * window is 8..128 rows, the weight matrices (bf16) are tens to
 // hundreds of MB and are read exactly once per step, so the kernel is bound by HBM bandwidth and its
 // job is to keep every SM's TMA queue full.  Larger M (batches of images with wide windows, up to
-// 1024 rows) is cut into token slabs of at most 256 rows; the CTAs of the slabs of one weight tile
+// 1024 rows) is cut into token slabs of at most 128 rows; the CTAs of the slabs of one weight tile
 // are neighbours in the grid, so the tile comes from HBM once and from L2 for the other slabs.
 //   * W is the 128-row operand of tcgen05.mma (M = 128), the tokens are the N dimension.  The fp32
 //     activations arrive split into two bf16 planes, hi = bf16(x) and lo = bf16(x - hi); both planes
 //     are columns of the same MMA (N = 2 * Mp), and the epilogue adds the two halves: activations keep
-//     ~16 bits of mantissa at no cost in weight bytes.  Above 128 rows the step is bound by the
-//     tensor pipe, not by bytes, and only the hi plane is multiplied (plain bf16 activations).
+//     ~16 bits of mantissa at no cost in weight bytes.  (Multiplying the hi plane alone, i.e. plain
+//     bf16 activations, halves the tensor work of the many-row case but misses the 2e-2 logits
+//     tolerance at d_model 4096 already after two layers; it stays a compile-time option.)
 //   * One CTA per (128-row weight tile, K split); two CTAs are resident per SM.  A launch covers up to
 //     three weight matrices that share the activation operand (Q|K|V, gate|up), so their tiles form
 //     one grid.  With more than one K split every CTA writes an fp32 partial plane; the consumer
@@ -53,7 +54,7 @@ constexpr int kMaxStages = 8;
 #define SJD_GEMM_CTAS_PER_SM 2
 #endif
 #ifndef SJD_GEMM_SPLIT_MAX_M
-#define SJD_GEMM_SPLIT_MAX_M 128            // most rows for which both the hi and the lo plane are multiplied
+#define SJD_GEMM_SPLIT_MAX_M 1024           // most rows for which both the hi and the lo plane are multiplied
 #endif
 constexpr int kSmemBudget = SJD_GEMM_SMEM_BUDGET;
 constexpr unsigned long long kWaitNs = 2000000000ull;
@@ -402,8 +403,8 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
 
 bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 1024 && N % TILE_N == 0 && K % TILE_K == 0; }
 
-// How M token rows are laid over the MMA N dimension (at most 256 columns per CTA): both activation
-// planes for M <= 128, the hi plane alone in slabs of at most 256 rows above that.
+// How M token rows are laid over the MMA N dimension (at most 256 columns per CTA): slabs of at most
+// 128 rows with both activation planes (256 rows where only the hi plane is multiplied).
 GemmTcPlan gemm_tc_plan(int M) {
   GemmTcPlan pl;
   pl.x_planes = M <= SJD_GEMM_SPLIT_MAX_M ? 2 : 1;

@@ -114,8 +114,8 @@ def test_small_bf16_gqa_generation():
 
 
 def test_small_bf16_many_rows():
-    """20 images x W = 16 = 320 rows per pass: the token-slab form of the projections (two slabs, hi
-    plane only) through pre-fill and three steps."""
+    """20 images x W = 16 = 320 rows per pass: the token-slab form of the projections (three slabs of
+    112 rows) through pre-fill and three steps."""
     wl = WORKLOADS["small-bf16"]
     ctx, seqs, steps, _ = run_lockstep(wl, batch=20, max_steps=3)
     for s in seqs:
