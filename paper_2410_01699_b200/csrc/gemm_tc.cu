@@ -5,7 +5,10 @@
 // hundreds of MB and are read exactly once per step, so the kernel is bound by HBM bandwidth and its
 // job is to keep every SM's TMA queue full.  Larger M (batches of images with wide windows, up to
 // 1024 rows) is cut into token slabs of at most 128 rows; the CTAs of the slabs of one weight tile
-// are neighbours in the grid, so the tile comes from HBM once and from L2 for the other slabs.
+// are neighbours in the grid, so the tile comes from HBM once and from L2 for the other slabs.  With
+// several slabs the kernel is bound by the tensor pipe and by the L2-to-shared-memory traffic of its
+// operands, so each CTA then takes two adjacent weight tiles against one activation tile (two
+// accumulators, all 512 TMEM columns, one CTA per SM): 64 instead of 96 operand bytes per MMA clock.
 //   * W is the 128-row operand of tcgen05.mma (M = 128), the tokens are the N dimension.  The fp32
 //     activations arrive split into two bf16 planes, hi = bf16(x) and lo = bf16(x - hi); both planes
 //     are columns of the same MMA (N = 2 * Mp), and the epilogue adds the two halves: activations keep
@@ -65,7 +68,8 @@ struct GemmParams {
   int ldc;
   int M;                  // valid token rows
   int Mp;                 // token rows of one slab, a multiple of 16 (MMA N = x_planes * Mp)
-  int n_slabs;            // token slabs; CTA blockIdx.x = weight tile * n_slabs + slab
+  int n_slabs;            // token slabs; CTA blockIdx.x = (weight tile / w_tiles) * n_slabs + slab
+  int w_tiles;            // adjacent weight tiles per CTA (1 or 2), each with its own accumulator
   int x_planes;           // 2: hi and lo planes of the activations, 1: hi only
   int x_lo_row;           // row of the lo plane inside the activation tensor map
   int k_blocks, splits;   // K / 64, K splits (gridDim.y)
@@ -198,11 +202,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
   SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tile = (int)blockIdx.x / p.n_slabs, split = blockIdx.y;
-  const int m_base = ((int)blockIdx.x - tile * p.n_slabs) * p.Mp;   // first token row of this CTA's slab
+  const int unit = (int)blockIdx.x / p.n_slabs, split = blockIdx.y;
+  const int tile = unit * p.w_tiles;                         // first weight tile of this CTA
+  const int m_base = ((int)blockIdx.x - unit * p.n_slabs) * p.Mp;   // first token row of this CTA's slab
   const int NN = p.x_planes * p.Mp;                          // MMA N
   const int x_tile_bytes = NN * TILE_K * 2;
-  const int stage_bytes = W_TILE_BYTES + x_tile_bytes;
+  const int w_bytes = p.w_tiles * W_TILE_BYTES;
+  const int stage_bytes = w_bytes + x_tile_bytes;
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   // which weight matrix this tile belongs to
@@ -215,7 +221,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   const int n_kb = kb_end - kb_begin;
 
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < NN) tmem_cols <<= 1;
+  while ((int)tmem_cols < p.w_tiles * NN) tmem_cols <<= 1;
 
   if (tid == 0) {
     tma_prefetch_desc(w_map);
@@ -249,7 +255,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       const int pre = n_kb < p.stages ? n_kb : p.stages;
       for (int i = 0; i < pre; ++i) {
         mbar_expect_tx(&bar_full[i], (uint32_t)stage_bytes);
-        tma_load_2d(smem + i * stage_bytes, w_map, (kb_begin + i) * TILE_K, tile_in_mat * TILE_N, &bar_full[i], policy);
+        for (int j = 0; j < p.w_tiles; ++j)
+          tma_load_2d(smem + i * stage_bytes + j * W_TILE_BYTES, w_map, (kb_begin + i) * TILE_K, (tile_in_mat + j) * TILE_N,
+                      &bar_full[i], policy);
       }
       SJD_TL(TL_GEMM, 3, true);
       pdl_wait();
@@ -257,9 +265,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       for (int i = 0; i < pre; ++i) {
         uint8_t *dst = smem + i * stage_bytes;
         const int kcol = (kb_begin + i) * TILE_K;
-        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, m_base, &bar_full[i]);
+        tma_load_2d_nohint(dst + w_bytes, &x_map, kcol, m_base, &bar_full[i]);
         if (p.x_planes == 2)
-          tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[i]);
+          tma_load_2d_nohint(dst + w_bytes + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[i]);
       }
       int s = pre == p.stages ? 0 : pre;
       uint32_t ph = pre == p.stages ? 1u : 0u;
@@ -270,10 +278,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         uint8_t *dst = smem + s * stage_bytes;
         const int kcol = (kb_begin + it) * TILE_K;
         mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
-        tma_load_2d(dst, w_map, kcol, tile_in_mat * TILE_N, &bar_full[s], policy);
-        tma_load_2d_nohint(dst + W_TILE_BYTES, &x_map, kcol, m_base, &bar_full[s]);
+        for (int j = 0; j < p.w_tiles; ++j)
+          tma_load_2d(dst + j * W_TILE_BYTES, w_map, kcol, (tile_in_mat + j) * TILE_N, &bar_full[s], policy);
+        tma_load_2d_nohint(dst + w_bytes, &x_map, kcol, m_base, &bar_full[s]);
         if (p.x_planes == 2)
-          tma_load_2d_nohint(dst + W_TILE_BYTES + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[s]);
+          tma_load_2d_nohint(dst + w_bytes + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[s]);
         if (++s == p.stages) { s = 0; ph ^= 1u; }
       }
       if (!ok) {
@@ -294,11 +303,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         if (!mbar_wait(&bar_full[s], ph)) { ok = false; break; }
         tc_fence_after();
         const uint32_t a_addr = smem_u32(smem + s * stage_bytes);
-        const uint32_t b_addr = a_addr + W_TILE_BYTES;
+        const uint32_t b_addr = a_addr + w_bytes;
 #pragma unroll
         for (int k = 0; k < TILE_K / UMMA_K; ++k) {
-          umma_bf16(tmem_base, umma_desc_sw128(a_addr + k * UMMA_K * 2), umma_desc_sw128(b_addr + k * UMMA_K * 2), idesc,
-                    !(it == 0 && k == 0));
+          const uint64_t bdesc = umma_desc_sw128(b_addr + k * UMMA_K * 2);
+          for (int j = 0; j < p.w_tiles; ++j)
+            umma_bf16(tmem_base + j * NN, umma_desc_sw128(a_addr + j * W_TILE_BYTES + k * UMMA_K * 2), bdesc, idesc,
+                      !(it == 0 && k == 0));
         }
         umma_commit(&bar_empty[s]);   // frees the stage once these MMAs have read it
         if (++s == p.stages) { s = 0; ph ^= 1u; }
@@ -314,11 +325,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
     if (ok) {
       tc_fence_after();
       pdl_wait();   // the planes may still be read, and the row scales written, by the preceding kernel
-      const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      const int n = p.col_off[mat] + tile_in_mat * TILE_N + row;
       float *plane = reinterpret_cast<float *>(p.out) + (size_t)split * p.plane_stride;
       __nv_bfloat16 *out_bf16 = reinterpret_cast<__nv_bfloat16 *>(p.out);
-      for (int m0 = 0; m0 < p.Mp; m0 += 16) {
+      for (int jm = 0; jm < p.w_tiles * p.Mp; jm += 16) {
+        const int j = jm / p.Mp, m0 = jm - j * p.Mp;            // accumulator, first token row of the chunk
+        const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + j * NN;
+        const int n = p.col_off[mat] + (tile_in_mat + j) * TILE_N + row;
         uint32_t hi[16], lo[16];
         tmem_ld16_issue(t_addr + m0, hi);
         if (p.x_planes == 2) {
@@ -335,7 +347,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
             float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
             if (p.ss_part) {
               float tot = 0.0f;
-              for (int j = 0; j < p.n_part; ++j) tot += __ldg(p.ss_part + (size_t)m * p.n_part + j);
+              for (int jj = 0; jj < p.n_part; ++jj) tot += __ldg(p.ss_part + (size_t)m * p.n_part + jj);
               v *= rsqrtf(tot * p.inv_d + p.eps);
             }
             if (p.store_bf16) out_bf16[(size_t)m * p.ldc + n] = __float2bfloat16_rn(v);
@@ -403,22 +415,26 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
 
 bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 1024 && N % TILE_N == 0 && K % TILE_K == 0; }
 
-// How M token rows are laid over the MMA N dimension (at most 256 columns per CTA): slabs of at most
-// 128 rows with both activation planes (256 rows where only the hi plane is multiplied).
-GemmTcPlan gemm_tc_plan(int M) {
+// How M token rows are laid over the MMA N dimension (at most 256 columns per accumulator): slabs of
+// at most 128 rows with both activation planes (256 rows where only the hi plane is multiplied).
+// `tiles_even`: every weight matrix of the launch has an even number of 128-row tiles.
+GemmTcPlan gemm_tc_plan(int M, bool tiles_even) {
   GemmTcPlan pl;
   pl.x_planes = M <= SJD_GEMM_SPLIT_MAX_M ? 2 : 1;
   const int cap = 256 / pl.x_planes;
   pl.n_slabs = (M + cap - 1) / cap;
   const int per = (M + pl.n_slabs - 1) / pl.n_slabs;
   pl.slab_rows = (per + 15) / 16 * 16;
+  pl.w_tiles = (pl.n_slabs >= 2 && tiles_even) ? 2 : 1;
   return pl;
 }
 
-// K splits for a launch of `tiles` weight tiles: at most two CTAs per SM in a single wave, at least
-// 16 k-blocks (256 KB of weights) per CTA so that set-up and drain stay small next to the streaming
-int gemm_tc_splits(int tiles, int k_blocks, int n_sms) {
-  int s = (SJD_GEMM_CTAS_PER_SM * n_sms) / tiles;
+// K splits for a launch of `tiles` weight tiles: a single wave of the resident CTAs (two per SM, one
+// when a CTA holds two accumulators), at least 16 k-blocks (256 KB of weights) per CTA so that
+// set-up and drain stay small next to the streaming
+int gemm_tc_splits(const GemmTcPlan &pl, int tiles, int k_blocks, int n_sms) {
+  const int ctas = tiles / pl.w_tiles * pl.n_slabs;
+  int s = ((pl.w_tiles == 2 ? 1 : SJD_GEMM_CTAS_PER_SM) * n_sms) / (ctas > 0 ? ctas : 1);
   const int cap = k_blocks / SJD_GEMM_MIN_KB > 1 ? k_blocks / SJD_GEMM_MIN_KB : 1;
   s = s > cap ? cap : s;
   s = s > 16 ? 16 : s;
@@ -429,10 +445,12 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   if (g.n_mats < 1 || g.n_mats > 3 || g.splits < 1) return SJD_ERR_BAD_ARG;
   GemmParams p;
   int tiles = 0;
+  bool tiles_even = true;
   for (int j = 0; j < 3; ++j) {
     if (j < g.n_mats) {
       if (!gemm_tc_supported(g.M, g.n_out[j], g.K)) return SJD_ERR_UNSUPPORTED;
       tiles += g.n_out[j] / TILE_N;
+      tiles_even = tiles_even && (g.n_out[j] / TILE_N) % 2 == 0;
     }
     p.tile_end[j] = tiles;
     p.col_off[j] = j < g.n_mats ? g.col_off[j] : 0;
@@ -441,10 +459,11 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.out = g.out;
   p.plane_stride = g.plane_stride;
   p.ldc = g.ldc;
-  const GemmTcPlan pl = gemm_tc_plan(g.M);
+  const GemmTcPlan pl = gemm_tc_plan(g.M, tiles_even);
   p.M = g.M;
   p.Mp = pl.slab_rows;
   p.n_slabs = pl.n_slabs;
+  p.w_tiles = pl.w_tiles;
   p.x_planes = pl.x_planes;
   p.x_lo_row = g.x_lo_row;
   p.k_blocks = g.K / TILE_K;
@@ -455,10 +474,11 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.n_part = g.n_part;
   p.inv_d = g.inv_d;
   p.eps = g.eps;
-  const int stage_bytes = W_TILE_BYTES + p.x_planes * p.Mp * TILE_K * 2;
+  const int stage_bytes = p.w_tiles * W_TILE_BYTES + p.x_planes * p.Mp * TILE_K * 2;
+  const int ctas = tiles / p.w_tiles * p.n_slabs;
   // one CTA per SM or fewer: give each the deeper ring
   const int budget =
-      (SJD_GEMM_DEEP_RING && g.n_sms > 0 && tiles * p.n_slabs * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
+      (p.w_tiles == 2 || (SJD_GEMM_DEEP_RING && g.n_sms > 0 && ctas * g.splits <= g.n_sms)) ? 2 * kSmemBudget : kSmemBudget;
   int stages = budget / stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : stages;
   if (stages < 2) return SJD_ERR_UNSUPPORTED;
@@ -477,7 +497,7 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
     SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
     configured[dev] = true;
   }
-  SJD_CUDA(launch_kernel(gemm_tc_kernel, dim3(tiles * p.n_slabs, g.splits), dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  SJD_CUDA(launch_kernel(gemm_tc_kernel, dim3(ctas, g.splits), dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
