@@ -6,9 +6,10 @@
 // job is to keep every SM's TMA queue full.  Larger M (batches of images with wide windows, up to
 // 1024 rows) is cut into token slabs of at most 128 rows; the CTAs of the slabs of one weight tile
 // are neighbours in the grid, so the tile comes from HBM once and from L2 for the other slabs.  With
-// several slabs the kernel is bound by the tensor pipe and by the L2-to-shared-memory traffic of its
-// operands, so each CTA then takes two adjacent weight tiles against one activation tile (two
-// accumulators, all 512 TMEM columns, one CTA per SM): 64 instead of 96 operand bytes per MMA clock.
+// several slabs the kernel is bound by the tensor pipe (both activation planes are multiplied).
+// Optionally (SJD_GEMM_WIDE_W_TILES = 2) a CTA of a multi-slab launch takes two adjacent weight tiles
+// against one activation tile (two accumulators, all 512 TMEM columns, one CTA per SM: 64 instead of
+// 96 operand bytes per MMA clock); measured 10-15 % slower than two independent CTAs per SM.
 //   * W is the 128-row operand of tcgen05.mma (M = 128), the tokens are the N dimension.  The fp32
 //     activations arrive split into two bf16 planes, hi = bf16(x) and lo = bf16(x - hi); both planes
 //     are columns of the same MMA (N = 2 * Mp), and the epilogue adds the two halves: activations keep
@@ -55,6 +56,9 @@ constexpr int kMaxStages = 8;
 #endif
 #ifndef SJD_GEMM_CTAS_PER_SM
 #define SJD_GEMM_CTAS_PER_SM 2
+#endif
+#ifndef SJD_GEMM_WIDE_W_TILES
+#define SJD_GEMM_WIDE_W_TILES 1             // weight tiles per CTA in launches with several token slabs (1 or 2)
 #endif
 #ifndef SJD_GEMM_SPLIT_MAX_M
 #define SJD_GEMM_SPLIT_MAX_M 1024           // most rows for which both the hi and the lo plane are multiplied
@@ -425,7 +429,7 @@ GemmTcPlan gemm_tc_plan(int M, bool tiles_even) {
   pl.n_slabs = (M + cap - 1) / cap;
   const int per = (M + pl.n_slabs - 1) / pl.n_slabs;
   pl.slab_rows = (per + 15) / 16 * 16;
-  pl.w_tiles = (pl.n_slabs >= 2 && tiles_even) ? 2 : 1;
+  pl.w_tiles = (SJD_GEMM_WIDE_W_TILES == 2 && pl.n_slabs >= 2 && tiles_even) ? 2 : 1;
   return pl;
 }
 
