@@ -14,7 +14,16 @@
 //      (Step 4, Sec. 4.2).
 // Logits are read once from HBM; later passes hit the shared-memory copy.  Rows too large for
 // shared memory are re-read through L2.  No floating-point atomics: every sum has a fixed order.
+//
+// bf16 rows of at most 65536 entries take a leaner route through step 2: the block holds the row
+// in registers (eight 16-byte vectors per thread), finds the maximum with packed bf16 instructions,
+// histograms the top 12 key bits once, resolves the last 4 bits on the few entries of the selected
+// bin, and forms the chunk sums from registers.  Rows with NaN/+inf, without a finite entry, or
+// whose threshold lies next to +-0 (where bf16 comparison and key order differ) use the general
+// route above; both routes produce the same threshold and the same weights.
 #include <float.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -82,6 +91,8 @@ struct Elt<__nv_bfloat16> {
 struct Scratch {
   double chunk_excl[kMaxChunks + 1];  // exclusive prefix of chunk sums; [NC] = total
   float chunk_sum[kMaxChunks];
+  uint32_t hist12[4096];              // register-resident route: histogram of the top 12 key bits
+  uint32_t hist16[16];                //   and of the last 4 bits inside the selected bin
   uint32_t hist[256];
   uint32_t redu[32];
   uint32_t sel_bin, count_above, bad;
@@ -142,20 +153,27 @@ struct Row {
 };
 
 // weight of one element under a row's statistics: exp((x - xmax)/T) inside the top-k set, else 0
+// 2^x for x <= 0 (hardware approximation, 2 ulp; results below the normal range flush to 0)
+__device__ __forceinline__ float exp2_neg(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 template <typename T>
 struct PWeight {
   uint32_t tau_key;
-  float xmax, inv_t;
+  float xmax, scale;   // scale = log2(e) / T
   bool degenerate;  // no finite entry: all mass on token 0
   __device__ void init(const RowStats &st, float inv_temperature) {
     tau_key = st.tau_key;
     xmax = st.xmax;
-    inv_t = inv_temperature;
+    scale = inv_temperature * 1.4426950408889634f;
     degenerate = !(st.xmax > -FLT_MAX);
   }
   __device__ __forceinline__ float one(uint32_t bits, int idx) const {
     if (degenerate) return idx == 0 ? 1.0f : 0.0f;
-    return Elt<T>::key(bits) >= tau_key ? expf((Elt<T>::val(bits) - xmax) * inv_t) : 0.0f;
+    return Elt<T>::key(bits) >= tau_key ? exp2_neg((Elt<T>::val(bits) - xmax) * scale) : 0.0f;
   }
 };
 
@@ -317,6 +335,8 @@ __device__ uint32_t select_threshold(const Row<T> &row, Scratch &sc, uint32_t to
 }
 
 // ------------------------------------------------------------------------------------ sums & sampling
+__device__ void chunk_prefix(int NC, Scratch &sc);
+
 // Per-chunk sums of the functor's weights in token order, then their exclusive prefix in fp64.
 template <int VEC, typename F>
 __device__ void chunk_sums(const F &f, int NV, Scratch &sc) {
@@ -340,6 +360,12 @@ __device__ void chunk_sums(const F &f, int NV, Scratch &sc) {
     if (lane == 31) sc.chunk_sum[c] = incl;
   }
   __syncthreads();
+  chunk_prefix(NC, sc);
+}
+
+// Exclusive prefix of sc.chunk_sum[0..NC) in fp64 (warp 0), total in sc.chunk_excl[NC].
+__device__ void chunk_prefix(int NC, Scratch &sc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (warp == 0) {
     const int per = (NC + 31) >> 5;
     const int lo = min(NC, lane * per), hi = min(NC, lo + per);
@@ -443,6 +469,181 @@ __device__ void sample_icdf(const F &f, int NV, int off, Scratch &sc, float u) {
   __syncthreads();
 }
 
+// ------------------------------------------------------------------------------------ register-resident route
+__device__ __forceinline__ __nv_bfloat162 as_bf2(uint32_t w) { return *reinterpret_cast<__nv_bfloat162 *>(&w); }
+// order-preserving keys of both halves of a packed bf16 pair (same map as Elt<bf16>::key per half)
+__device__ __forceinline__ uint32_t key_pair(uint32_t w) {
+  const uint32_t neg = ((w >> 15) & 0x00010001u) * 0xFFFFu;   // 0xFFFF in the halves whose sign bit is set
+  return w ^ (neg | 0x80008000u);
+}
+__device__ __forceinline__ uint32_t word_of(const uint4 &v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+
+// Threshold, maximum and denominator of a 16-byte aligned bf16 row of NV <= 8 * blockDim.x vectors
+// held in registers: warp w owns chunks 8w .. 8w+7 (32 vectors each, the chunks of chunk_sums), lane
+// l holds vector l of each.  Leaves the staged copy, the chunk sums and their prefix exactly as
+// row_statistics does.  Returns false (block-uniform, nothing published) for rows it does not cover.
+__device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t,
+                                    PRowWeights<__nv_bfloat16> &f, RowStats &st) {
+  using E = Elt<__nv_bfloat16>;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
+  const int NV = row.NV, NC = (NV + 31) >> 5;
+  const bool need_select = top_k < row.V;
+  if (need_select)
+    for (int i = tid; i < 4096; i += nt) sc.hist12[i] = 0;
+  if (tid < 16) sc.hist16[tid] = 0;
+
+  // ---- load, stage, maximum
+  uint4 v[8];
+  const uint4 *g = reinterpret_cast<const uint4 *>(row.g);
+  const int j0 = warp * 256 + lane;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    v[i] = j < NV ? __ldg(g + j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+  }
+  __nv_bfloat162 m2 = as_bf2(v[0].x);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    if (j < NV) stage[j] = v[i];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(v[i], w)));
+  }
+  const __nv_bfloat16 m1 = __hmax_nan(__low2bfloat16(m2), __high2bfloat16(m2));
+  const uint32_t mbits = (uint32_t)__bfloat16_as_ushort(m1);
+  uint32_t kmax = (mbits & 0x7FFFu) > 0x7F80u ? 0xFFFFu : E::key(mbits);   // NaN sorts above everything
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) sc.redu[warp] = kmax;
+  __syncthreads();
+  kmax = 0;
+  for (int w = 0; w < nw; ++w) kmax = max(kmax, sc.redu[w]);
+  // NaN or +inf somewhere, or no finite entry at all: the general route sanitises and flags
+  if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
+  row.s = stage;
+
+  // ---- threshold
+  uint32_t tau_key = 0;
+  if (need_select) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (j0 + i * 32 < NV) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const uint32_t kk = key_pair(word_of(v[i], w));
+          atomicAdd(&sc.hist12[(kk >> 4) & 0xFFFu], 1u);
+          atomicAdd(&sc.hist12[kk >> 20], 1u);
+        }
+      }
+    }
+    __syncthreads();
+    for (int c = tid; c < 256; c += nt) {
+      uint32_t t = 0;
+#pragma unroll
+      for (int b = 0; b < 16; ++b) t += sc.hist12[c * 16 + b];
+      sc.hist[c] = t;
+    }
+    __syncthreads();
+    if (tid < 32) find_bin(sc, (uint32_t)top_k);
+    __syncthreads();
+    if (tid == 0) {   // the 16 fine bins of the selected coarse bin, from the top
+      const uint32_t cb = sc.sel_bin, k = (uint32_t)top_k;
+      uint32_t acc = sc.count_above, sel = cb * 16, above = acc;
+      for (int b = 15; b >= 0; --b) {
+        const uint32_t nxt = acc + sc.hist12[cb * 16 + b];
+        if (acc < k && k <= nxt) {
+          sel = cb * 16 + b;
+          above = acc;
+          break;
+        }
+        acc = nxt;
+      }
+      sc.sel_bin = sel;
+      sc.count_above = above;
+    }
+    __syncthreads();
+    const uint32_t sel12 = sc.sel_bin, above = sc.count_above;
+    if (sel12 == 0x7FFu || sel12 == 0x800u) {   // the bins of -0 and +0: bf16 comparison cannot tell them apart
+      __syncthreads();
+      return false;
+    }
+    // entries inside the selected bin: found with two packed comparisons per word, then counted by
+    // their last 4 key bits
+    const uint32_t kb_lo = sel12 << 4;
+    const uint32_t v_lo = E::unkey(kb_lo), v_hi = E::unkey(kb_lo | 15u);
+    const __nv_bfloat162 lo2 = as_bf2(v_lo | (v_lo << 16)), hi2 = as_bf2(v_hi | (v_hi << 16));
+    uint32_t cand = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (j0 + i * 32 < NV) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const __nv_bfloat162 x = as_bf2(word_of(v[i], w));
+          if (__hge2_mask(x, lo2) & __hle2_mask(x, hi2)) cand |= 1u << (i * 4 + w);
+        }
+      }
+    }
+    const uint32_t *stage_w = reinterpret_cast<const uint32_t *>(stage);
+    while (cand) {
+      const int idx = __ffs(cand) - 1;
+      cand &= cand - 1;
+      const uint32_t kk = key_pair(stage_w[(size_t)(j0 + (idx >> 2) * 32) * 4 + (idx & 3)]);
+      if (((kk >> 4) & 0xFFFu) == sel12) atomicAdd(&sc.hist16[kk & 15u], 1u);
+      if ((kk >> 20) == sel12) atomicAdd(&sc.hist16[(kk >> 16) & 15u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      const uint32_t need = (uint32_t)top_k - above;   // rank inside the bin, from the top
+      uint32_t acc = 0, t = kb_lo;
+      for (int b = 15; b >= 0; --b) {
+        acc += sc.hist16[b];
+        if (acc >= need) {
+          t = kb_lo | (uint32_t)b;
+          break;
+        }
+      }
+      sc.sel_bin = t;
+    }
+    __syncthreads();
+    tau_key = sc.sel_bin;
+  }
+
+  // ---- weights and chunk sums from registers
+  st.tau_key = tau_key;
+  st.xmax = E::val(E::unkey(kmax));
+  st.flags = 0;
+  f.row = row;
+  f.pw.init(st, inv_t);
+  const float tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
+  const float xmax = st.xmax, scale = f.pw.scale;
+  float s[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const uint32_t x = word_of(v[i], w);
+      const float a = __uint_as_float(x << 16), b = __uint_as_float(x & 0xFFFF0000u);
+      acc += a >= tau_f ? exp2_neg((a - xmax) * scale) : 0.0f;
+      acc += b >= tau_f ? exp2_neg((b - xmax) * scale) : 0.0f;
+    }
+    s[i] = acc;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
+  }
+  __syncthreads();
+  chunk_prefix(NC, sc);
+  st.z = (float)sc.chunk_excl[NC];
+  return true;
+}
+
 // Threshold + denominator of one row; leaves chunk sums of the row's weights in the scratch.
 template <typename T>
 __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t,
@@ -459,6 +660,21 @@ __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int t
   chunk_sums<E::VEC>(f, row.NV, sc);
   st.z = (float)sc.chunk_excl[(row.NV + 31) >> 5];
   return st;
+}
+
+// row_statistics through whichever route covers the row
+template <typename T>
+__device__ RowStats row_statistics_any(Row<T> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t, PRowWeights<T> &f,
+                                       bool fast) {
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    if (fast && stage && row.off == 0 && (row.V & 7) == 0 && row.NV <= 8 * (int)blockDim.x) {
+      RowStats st;
+      if (fast_row_statistics(row, stage, sc, top_k, inv_t, f, st)) return st;
+      row.s = nullptr;
+      __syncthreads();
+    }
+  }
+  return row_statistics<T>(row, stage, sc, top_k, inv_t, f);
 }
 
 // ------------------------------------------------------------------------------------ finalize
@@ -562,8 +778,8 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step) {
 }
 
 // ------------------------------------------------------------------------------------ kernel
-template <typename T>
-__global__ void __launch_bounds__(kMaxThreads) verify_rows_kernel(const VerifyParams p) {
+template <typename T, int MAXT>
+__global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(const VerifyParams p) {
   using E = Elt<T>;
   extern __shared__ uint4 dyn_smem[];
   __shared__ Scratch sc;
@@ -605,7 +821,7 @@ __global__ void __launch_bounds__(kMaxThreads) verify_rows_kernel(const VerifyPa
       if (p.prev_stats_valid) {
         qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
       } else {
-        qs = row_statistics<T>(qrow, stage, sc, p.top_k, inv_t, qf);
+        qs = row_statistics_any<T>(qrow, stage, sc, p.top_k, inv_t, qf, p.fast != 0);
         if (tid == 0) p.stats[cur ^ 1][r] = qs;
         __syncthreads();
         qrow.s = nullptr;  // the staging buffer is about to be reused
@@ -623,7 +839,7 @@ __global__ void __launch_bounds__(kMaxThreads) verify_rows_kernel(const VerifyPa
     Row<T> prow;
     prow.init(pbase, p.V);
     PRowWeights<T> pf;
-    const RowStats ps = row_statistics<T>(prow, stage, sc, p.top_k, inv_t, pf);
+    const RowStats ps = row_statistics_any<T>(prow, stage, sc, p.top_k, inv_t, pf, p.fast != 0);
     if (tid == 0) p.stats[cur][r] = ps;
     const float p_d = d_ok ? pf.pw.one(prow.element(d), d) / ps.z : 0.0f;
 
@@ -711,11 +927,22 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
   p.staged = stage_bytes <= 160 * 1024 ? 1 : 0;
   const size_t dyn = p.staged ? stage_bytes : 0;
   int threads = nv_max <= 1024 ? 128 : nv_max <= 4096 ? 256 : nv_max <= 16384 ? 512 : 1024;
-  if (dyn > 48 * 1024)
-    SJD_CUDA(cudaFuncSetAttribute(verify_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
-  SJD_CUDA(launch_kernel(verify_rows_kernel<T>, dim3(p.B * p.W), dim3(threads), dyn, stream, p));
-  SJD_CHECK_LAUNCH();
-  return SJD_OK;
+  // rows a block can hold in registers, eight vectors per thread
+  p.fast = 0;
+  if (std::is_same<T, __nv_bfloat16>::value && p.staged && p.V % VEC == 0 && p.V / VEC <= 8 * kMaxThreads &&
+      ((uintptr_t)p.logits[0] & 15u) == 0 && ((uintptr_t)p.logits[1] & 15u) == 0) {
+    p.fast = 1;
+    threads = (p.V / VEC + 255) / 256 * 32;
+    threads = threads < 64 ? 64 : threads;
+  }
+  auto launch = [&](auto kernel) -> int {
+    if (dyn > 48 * 1024) SJD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+    SJD_CUDA(launch_kernel(kernel, dim3(p.B * p.W), dim3(threads), dyn, stream, p));
+    SJD_CHECK_LAUNCH();
+    return SJD_OK;
+  };
+  if (threads <= 256) return launch(verify_rows_kernel<T, 256>);
+  return launch(verify_rows_kernel<T, kMaxThreads>);
 }
 
 int launch_verify(const VerifyParams &p, int dtype, cudaStream_t stream) {
