@@ -936,7 +936,8 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
     threads = threads < 64 ? 64 : threads;
   }
   auto launch = [&](auto kernel) -> int {
-    if (dyn > 48 * 1024) SJD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
+    // static scratch (about 30 KB) + the staged row: opt in as soon as the sum can pass 48 KB
+    if (dyn > 16 * 1024) SJD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
     SJD_CUDA(launch_kernel(kernel, dim3(p.B * p.W), dim3(threads), dyn, stream, p));
     SJD_CHECK_LAUNCH();
     return SJD_OK;
