@@ -147,6 +147,10 @@ struct Row {
   }
   // sanitised bits of element i (0 <= i < V)
   __device__ __forceinline__ uint32_t element(int i) const {
+    if (s) {   // the staged copy is already sanitised
+      if (sizeof(T) == 2) return (uint32_t) reinterpret_cast<const unsigned short *>(s)[i + off];
+      return reinterpret_cast<const uint32_t *>(s)[i + off];
+    }
     uint32_t b = Elt<T>::load_bits(g + i);
     return Elt<T>::bad(b) ? Elt<T>::NEG_INF : b;
   }
@@ -520,6 +524,7 @@ __device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scrat
   // NaN or +inf somewhere, or no finite entry at all: the general route sanitises and flags
   if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
   row.s = stage;
+  SJD_TL(TL_VERIFY, 20, tid == 0);   // row loaded, maximum known
 
   // ---- threshold
   uint32_t tau_key = 0;
@@ -536,6 +541,7 @@ __device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scrat
       }
     }
     __syncthreads();
+    SJD_TL(TL_VERIFY, 21, tid == 0);   // 12-bit histogram complete
     for (int c = tid; c < 256; c += nt) {
       uint32_t t = 0;
 #pragma unroll
@@ -562,6 +568,7 @@ __device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scrat
     }
     __syncthreads();
     const uint32_t sel12 = sc.sel_bin, above = sc.count_above;
+    SJD_TL(TL_VERIFY, 22, tid == 0);   // bin selected
     if (sel12 == 0x7FFu || sel12 == 0x800u) {   // the bins of -0 and +0: bf16 comparison cannot tell them apart
       __syncthreads();
       return false;
@@ -605,6 +612,7 @@ __device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scrat
     }
     __syncthreads();
     tau_key = sc.sel_bin;
+    SJD_TL(TL_VERIFY, 23, tid == 0);   // threshold known
   }
 
   // ---- weights and chunk sums from registers
@@ -639,6 +647,7 @@ __device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scrat
       if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
   }
   __syncthreads();
+  SJD_TL(TL_VERIFY, 24, tid == 0);   // chunk sums written
   chunk_prefix(NC, sc);
   st.z = (float)sc.chunk_excl[NC];
   return true;
@@ -660,6 +669,66 @@ __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int t
   chunk_sums<E::VEC>(f, row.NV, sc);
   st.z = (float)sc.chunk_excl[(row.NV + 31) >> 5];
   return st;
+}
+
+// Chunk sums (and their prefix) of the residual weights max(0, p - q) of Eq. 2 with the p row read from
+// its staged copy and the q row from global memory (it was read moments ago: L2), eight vectors per
+// thread in the layout of fast_row_statistics.  Element for element the same arithmetic as
+// ResidualWeights, so sample_icdf may follow with that functor.  Requires both rows 16-byte aligned,
+// free of non-finite entries and not degenerate.
+__device__ void fast_residual_sums(const ResidualWeights<__nv_bfloat16> &rf, Scratch &sc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int NV = rf.prow.NV, NC = (NV + 31) >> 5;
+  const uint4 *pg = rf.prow.s;
+  const uint4 *qg = reinterpret_cast<const uint4 *>(rf.qrow.g);
+  const int j0 = warp * 256 + lane;
+  const float q_uniform = 1.0f / (float)rf.V;
+  float s[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    float acc = 0.0f;
+    if (j < NV) {
+      const uint4 pv = pg[j];
+      uint4 qv = make_uint4(0, 0, 0, 0);
+      if (rf.kind == SJD_Q_ROW) qv = __ldg(qg + j);
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t px = word_of(pv, w), qx = word_of(qv, w);
+        const uint32_t pk = key_pair(px), qk = key_pair(qx);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t pkey = h ? pk >> 16 : pk & 0xFFFFu;
+          const float pval = __uint_as_float(h ? px & 0xFFFF0000u : px << 16);
+          const float pp = (pkey >= rf.pw.tau_key ? exp2_neg((pval - rf.pw.xmax) * rf.pw.scale) : 0.0f) * rf.inv_zp;
+          float qq;
+          if (rf.kind == SJD_Q_ROW) {
+            const uint32_t qkey = h ? qk >> 16 : qk & 0xFFFFu;
+            const float qval = __uint_as_float(h ? qx & 0xFFFF0000u : qx << 16);
+            qq = (qkey >= rf.qw.tau_key ? exp2_neg((qval - rf.qw.xmax) * rf.qw.scale) : 0.0f) * rf.inv_zq;
+          } else if (rf.kind == SJD_Q_UNIFORM) {
+            qq = q_uniform;
+          } else {
+            qq = (j * 8 + w * 2 + h == rf.draft) ? 1.0f : 0.0f;
+          }
+          acc += fmaxf(0.0f, pp - qq);
+        }
+      }
+    }
+    s[i] = acc;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
+  }
+  __syncthreads();
+  chunk_prefix(NC, sc);
 }
 
 // row_statistics through whichever route covers the row
@@ -835,6 +904,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
       q_d = 1.0f;
     }
 
+    SJD_TL(TL_VERIFY, 10, tid == 0);   // the draft's law is known
     // ---- this iteration's distribution
     Row<T> prow;
     prow.init(pbase, p.V);
@@ -843,6 +913,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
     if (tid == 0) p.stats[cur][r] = ps;
     const float p_d = d_ok ? pf.pw.one(prow.element(d), d) / ps.z : 0.0f;
 
+    SJD_TL(TL_VERIFY, 11, tid == 0);   // this row's statistics are known
     // ---- Eq. 1
     float ratio;
     if (q_d > 0.0f) ratio = p_d / q_d;
@@ -858,6 +929,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
     const float redraft_p = sc.tok_w / ps.z;
     __syncthreads();
 
+    SJD_TL(TL_VERIFY, 12, tid == 0);   // re-draft token drawn
     // ---- Eq. 2: residual resample (used if this is the first rejected row)
     int resample_tok = -1;
     if (!accept) {
@@ -866,7 +938,14 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
       rf.inv_zp = 1.0f / ps.z; rf.inv_zq = 1.0f / qs.z;
       rf.kind = kind; rf.draft = d; rf.V = p.V;
       if (kind != SJD_Q_ROW) rf.qw = pf.pw;
-      chunk_sums<E::VEC>(rf, prow.NV, sc);
+      bool from_registers = false;
+      if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        from_registers = p.fast && prow.s && prow.off == 0 && (p.V & 7) == 0 && prow.NV <= 8 * (int)blockDim.x &&
+                         !pf.pw.degenerate &&
+                         (kind != SJD_Q_ROW || (qrow.off == 0 && qs.flags == 0 && !qf.pw.degenerate));
+        if (from_registers) fast_residual_sums(rf, sc);
+      }
+      if (!from_registers) chunk_sums<E::VEC>(rf, prow.NV, sc);
       if (sc.chunk_excl[(prow.NV + 31) >> 5] > 0.0) {
         sample_icdf<E::VEC>(rf, prow.NV, prow.off, sc, u_res);
       } else {
@@ -877,6 +956,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
       }
       resample_tok = sc.tok;
     }
+    SJD_TL(TL_VERIFY, 13, tid == 0);   // residual token drawn
     if (tid == 0) {
       RowOut ro;
       ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
@@ -893,7 +973,9 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
     sc.is_last = (old == p.W - 1);
     if (sc.is_last) {
       __threadfence();
+      SJD_TL(TL_VERIFY, 14, true);
       finalize_sequence(p, b, step);
+      SJD_TL(TL_VERIFY, 15, true);
       p.seq_counter[b] = 0;
       __threadfence();
       const int done = atomicAdd(p.done_counter, 1);
