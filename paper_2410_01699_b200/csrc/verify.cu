@@ -684,14 +684,19 @@ __device__ void fast_residual_sums(const ResidualWeights<__nv_bfloat16> &rf, Scr
   const int j0 = warp * 256 + lane;
   const float q_uniform = 1.0f / (float)rf.V;
   float s[8];
+  uint4 qall[8];   // every load of the q row in flight before the first use
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    qall[i] = (rf.kind == SJD_Q_ROW && j < NV) ? __ldg(qg + j) : make_uint4(0, 0, 0, 0);
+  }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int j = j0 + i * 32;
     float acc = 0.0f;
     if (j < NV) {
       const uint4 pv = pg[j];
-      uint4 qv = make_uint4(0, 0, 0, 0);
-      if (rf.kind == SJD_Q_ROW) qv = __ldg(qg + j);
+      const uint4 qv = qall[i];
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const uint32_t px = word_of(pv, w), qx = word_of(qv, w);
