@@ -73,7 +73,7 @@ struct GemmParams {
   int M;                  // valid token rows
   int Mp;                 // token rows of one slab, a multiple of 16 (MMA N = x_planes * Mp)
   int n_slabs;            // token slabs; CTA blockIdx.x = (weight tile / w_tiles) * n_slabs + slab
-  int w_tiles;            // adjacent weight tiles per CTA (1 or 2), each with its own accumulator
+  int w_tiles;            // adjacent weight tiles per CTA (1 or 2), each with its own accumulator (= template WT)
   int x_planes;           // 2: hi and lo planes of the activations, 1: hi only
   int x_lo_row;           // row of the lo plane inside the activation tensor map
   int k_blocks, splits;   // K / 64, K splits (gridDim.y)
@@ -196,6 +196,9 @@ __device__ __forceinline__ bool epilogue_all(bool pred) {
 }
 
 // ---------------------------------------------------------------------------------- kernel
+// WT: weight tiles per CTA, XP: activation planes multiplied (compile-time so that the common
+// shape, one tile and both planes, keeps fully unrolled issue loops)
+template <int WT, int XP>
 __global__ void __launch_bounds__(kThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant__ CUtensorMap w_map1,
                const __grid_constant__ CUtensorMap w_map2, const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
@@ -207,11 +210,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = (int)blockIdx.x / p.n_slabs, split = blockIdx.y;
-  const int tile = unit * p.w_tiles;                         // first weight tile of this CTA
+  const int tile = unit * WT;                         // first weight tile of this CTA
   const int m_base = ((int)blockIdx.x - unit * p.n_slabs) * p.Mp;   // first token row of this CTA's slab
-  const int NN = p.x_planes * p.Mp;                          // MMA N
+  const int NN = XP * p.Mp;                          // MMA N
   const int x_tile_bytes = NN * TILE_K * 2;
-  const int w_bytes = p.w_tiles * W_TILE_BYTES;
+  const int w_bytes = WT * W_TILE_BYTES;
   const int stage_bytes = w_bytes + x_tile_bytes;
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
@@ -225,7 +228,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   const int n_kb = kb_end - kb_begin;
 
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < p.w_tiles * NN) tmem_cols <<= 1;
+  while ((int)tmem_cols < WT * NN) tmem_cols <<= 1;
 
   if (tid == 0) {
     tma_prefetch_desc(w_map);
@@ -259,7 +262,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       const int pre = n_kb < p.stages ? n_kb : p.stages;
       for (int i = 0; i < pre; ++i) {
         mbar_expect_tx(&bar_full[i], (uint32_t)stage_bytes);
-        for (int j = 0; j < p.w_tiles; ++j)
+#pragma unroll
+        for (int j = 0; j < WT; ++j)
           tma_load_2d(smem + i * stage_bytes + j * W_TILE_BYTES, w_map, (kb_begin + i) * TILE_K, (tile_in_mat + j) * TILE_N,
                       &bar_full[i], policy);
       }
@@ -270,7 +274,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         uint8_t *dst = smem + i * stage_bytes;
         const int kcol = (kb_begin + i) * TILE_K;
         tma_load_2d_nohint(dst + w_bytes, &x_map, kcol, m_base, &bar_full[i]);
-        if (p.x_planes == 2)
+        if (XP == 2)
           tma_load_2d_nohint(dst + w_bytes + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[i]);
       }
       int s = pre == p.stages ? 0 : pre;
@@ -282,10 +286,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         uint8_t *dst = smem + s * stage_bytes;
         const int kcol = (kb_begin + it) * TILE_K;
         mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
-        for (int j = 0; j < p.w_tiles; ++j)
+#pragma unroll
+        for (int j = 0; j < WT; ++j)
           tma_load_2d(dst + j * W_TILE_BYTES, w_map, kcol, (tile_in_mat + j) * TILE_N, &bar_full[s], policy);
         tma_load_2d_nohint(dst + w_bytes, &x_map, kcol, m_base, &bar_full[s]);
-        if (p.x_planes == 2)
+        if (XP == 2)
           tma_load_2d_nohint(dst + w_bytes + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[s]);
         if (++s == p.stages) { s = 0; ph ^= 1u; }
       }
@@ -311,7 +316,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
 #pragma unroll
         for (int k = 0; k < TILE_K / UMMA_K; ++k) {
           const uint64_t bdesc = umma_desc_sw128(b_addr + k * UMMA_K * 2);
-          for (int j = 0; j < p.w_tiles; ++j)
+  #pragma unroll
+        for (int j = 0; j < WT; ++j)
             umma_bf16(tmem_base + j * NN, umma_desc_sw128(a_addr + j * W_TILE_BYTES + k * UMMA_K * 2), bdesc, idesc,
                       !(it == 0 && k == 0));
         }
@@ -331,13 +337,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       pdl_wait();   // the planes may still be read, and the row scales written, by the preceding kernel
       float *plane = reinterpret_cast<float *>(p.out) + (size_t)split * p.plane_stride;
       __nv_bfloat16 *out_bf16 = reinterpret_cast<__nv_bfloat16 *>(p.out);
-      for (int jm = 0; jm < p.w_tiles * p.Mp; jm += 16) {
-        const int j = jm / p.Mp, m0 = jm - j * p.Mp;            // accumulator, first token row of the chunk
+#pragma unroll
+      for (int j = 0; j < WT; ++j)                               // accumulator
+      for (int m0 = 0; m0 < p.Mp; m0 += 16) {                    // first token row of the chunk
         const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + j * NN;
         const int n = p.col_off[mat] + (tile_in_mat + j) * TILE_N + row;
         uint32_t hi[16], lo[16];
         tmem_ld16_issue(t_addr + m0, hi);
-        if (p.x_planes == 2) {
+        if (XP == 2) {
           tmem_ld16_issue(t_addr + p.Mp + m0, lo);
         } else {
 #pragma unroll
@@ -498,10 +505,21 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   SJD_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
   if (!configured[dev]) {
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
     configured[dev] = true;
   }
-  SJD_CUDA(launch_kernel(gemm_tc_kernel, dim3(ctas, g.splits), dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  const dim3 grid(ctas, g.splits);
+  if (p.w_tiles == 1 && p.x_planes == 2)
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 2>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  else if (p.w_tiles == 2 && p.x_planes == 2)
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 2>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  else if (p.w_tiles == 1)
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 1>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  else
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 1>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
