@@ -66,7 +66,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, u
                : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -190,17 +190,20 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
 #pragma unroll
     for (int ks = 0; ks < HD / 16; ++ks) {
       const int half = ks >> 2, c0 = (ks & 3) * 2;
+      // all key fragments of this k-step first, then one pass of MMAs per Q plane: consecutive MMAs
+      // go to different accumulators, so none waits for the one before it
+      uint32_t kf[KT / 8][2];
 #pragma unroll
       for (int nb = 0; nb < KT / 8; nb += 2) {
         const int row = nb * 8 + (lane & 7) + ((lane >> 4) & 1) * 8;
         const int chunkc = c0 + ((lane >> 3) & 1);
-        uint32_t b0, b1, b2, b3;
-        ldmatrix_x4(kbase + half * (KT * 128) + row * 128 + ((chunkc ^ (row & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16(sacc[nb], qh[ks], b0, b1);
-        mma_bf16(sacc[nb], ql[ks], b0, b1);
-        mma_bf16(sacc[nb + 1], qh[ks], b2, b3);
-        mma_bf16(sacc[nb + 1], ql[ks], b2, b3);
+        ldmatrix_x4(kbase + half * (KT * 128) + row * 128 + ((chunkc ^ (row & 7)) << 4), kf[nb][0], kf[nb][1], kf[nb + 1][0],
+                    kf[nb + 1][1]);
       }
+#pragma unroll
+      for (int nb = 0; nb < KT / 8; ++nb) mma_bf16(sacc[nb], qh[ks], kf[nb][0], kf[nb][1]);
+#pragma unroll
+      for (int nb = 0; nb < KT / 8; ++nb) mma_bf16(sacc[nb], ql[ks], kf[nb][0], kf[nb][1]);
     }
     // ---- mask, online softmax (base 2)
     float tmax0 = -INFINITY, tmax1 = -INFINITY;
@@ -247,15 +250,19 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
 #pragma unroll
     for (int kk = 0; kk < KT / 16; ++kk) {
 #pragma unroll
-      for (int cd = 0; cd < HD / 8; cd += 2) {
-        const int row = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const int chunkc = cd + ((lane >> 4) & 1);
-        uint32_t b0, b1, b2, b3;
-        ldmatrix_x4_trans(vbase + (chunkc >> 3) * (KT * 128) + row * 128 + (((chunkc & 7) ^ (row & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16(o[cd], ph[kk], b0, b1);
-        mma_bf16(o[cd], pl[kk], b0, b1);
-        mma_bf16(o[cd + 1], ph[kk], b2, b3);
-        mma_bf16(o[cd + 1], pl[kk], b2, b3);
+      for (int c8 = 0; c8 < HD / 8; c8 += 8) {   // eight output column blocks at a time, same ordering idea
+        uint32_t vf[8][2];
+#pragma unroll
+        for (int cd = 0; cd < 8; cd += 2) {
+          const int row = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int chunkc = c8 + cd + ((lane >> 4) & 1);
+          ldmatrix_x4_trans(vbase + (chunkc >> 3) * (KT * 128) + row * 128 + (((chunkc & 7) ^ (row & 7)) << 4), vf[cd][0],
+                            vf[cd][1], vf[cd + 1][0], vf[cd + 1][1]);
+        }
+#pragma unroll
+        for (int cd = 0; cd < 8; ++cd) mma_bf16(o[c8 + cd], ph[kk], vf[cd][0], vf[cd][1]);
+#pragma unroll
+        for (int cd = 0; cd < 8; ++cd) mma_bf16(o[c8 + cd], pl[kk], vf[cd][0], vf[cd][1]);
       }
     }
     __syncthreads();   // every warp is done with this stage
