@@ -5,7 +5,10 @@
 // by TMA (128-byte swizzle, two 64-dim boxes per 128-dim head) through a ring of mbarrier-guarded
 // stages; each warp owns 16 query rows, keeps Q (pre-scaled, split into bf16 hi + lo), the running
 // max / sum and the fp32 output accumulators in registers and runs QK^T and PV as m16n8k16 bf16
-// mma.sync with ldmatrix-fed operands.  The probabilities are split hi + lo as well, so neither
+// mma.sync with ldmatrix-fed operands.  A CTA always has four warps: with fewer than 64 query rows the
+// warps that share 16 rows split the keys of every tile between them (KG = 2 or 4 key groups, each
+// with its own running max / sum / output) and merge through shared memory at the end; one warp per
+// scheduler alone cannot keep the tensor pipe and the exponentials going at the same time.  The probabilities are split hi + lo as well, so neither
 // operand loses more than ~2^-17 relative.  The kernel is bound by streaming K/V once from HBM (GQA
 // heads of a group share their tiles through L2).  Partials (max, sum, unnormalised output) go to the
 // merge kernel of attention.cu.  Every barrier wait is bounded.
@@ -88,7 +91,7 @@ struct AttnParams {
   int plane0;            // first cache plane of this layer: planes are [b][k|v][kv_head]
 };
 
-template <int HD>
+template <int HD, int KG>
 __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
   constexpr int HALVES = HD / 64;                // 64-dim (128-byte) boxes per row
   constexpr int TILE_BYTES = KT * HD * 2;        // one of K or V
@@ -108,6 +111,10 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   const int kvh = h / (p.n_heads / p.n_kv_heads);
   const int m0 = b * W;
   const int g = lane >> 2, tq = lane & 3;
+  const int n_rw = blockDim.x / (32 * KG);   // warps along the query rows
+  const int rw = warp % n_rw, kg = warp / n_rw;   // this warp's 16 rows and its key group inside a tile
+  constexpr int NB = KT / 8 / KG;            // 8-key blocks of a tile this warp scores
+  constexpr int NK = KT / 16 / KG;           // 16-key blocks it multiplies with V
 
   if (tid < 64) s_pos[tid] = tid < W ? p.in_pos[m0 + tid] : -1;
   if (tid == 0) {
@@ -143,7 +150,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     for (int t = 0; t < n_tiles && t < kStagesAttn; ++t) issue(t);
 
   // this thread's two query rows
-  const int r0 = warp * 16 + g, r1 = r0 + 8;
+  const int r0 = rw * 16 + g, r1 = r0 + 8;
   const int pos0 = r0 < W ? s_pos[r0] : -1, pos1 = r1 < W ? s_pos[r1] : -1;
   // Q fragments, pre-scaled by log2(e) / sqrt(HD), split hi / lo
   uint32_t qh[HD / 16][4], ql[HD / 16][4];
@@ -184,32 +191,32 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     const int key0 = k_begin + t * KT;
 
     // ---- S = Q K^T  (16 rows x 64 keys per warp)
-    float sacc[KT / 8][4];
+    float sacc[NB][4];
 #pragma unroll
-    for (int i = 0; i < KT / 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.0f;
+    for (int i = 0; i < NB; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.0f;
 #pragma unroll
     for (int ks = 0; ks < HD / 16; ++ks) {
       const int half = ks >> 2, c0 = (ks & 3) * 2;
       // all key fragments of this k-step first, then one pass of MMAs per Q plane: consecutive MMAs
       // go to different accumulators, so none waits for the one before it
-      uint32_t kf[KT / 8][2];
+      uint32_t kf[NB][2];
 #pragma unroll
-      for (int nb = 0; nb < KT / 8; nb += 2) {
-        const int row = nb * 8 + (lane & 7) + ((lane >> 4) & 1) * 8;
+      for (int nb = 0; nb < NB; nb += 2) {
+        const int row = (kg * NB + nb) * 8 + (lane & 7) + ((lane >> 4) & 1) * 8;
         const int chunkc = c0 + ((lane >> 3) & 1);
         ldmatrix_x4(kbase + half * (KT * 128) + row * 128 + ((chunkc ^ (row & 7)) << 4), kf[nb][0], kf[nb][1], kf[nb + 1][0],
                     kf[nb + 1][1]);
       }
 #pragma unroll
-      for (int nb = 0; nb < KT / 8; ++nb) mma_bf16(sacc[nb], qh[ks], kf[nb][0], kf[nb][1]);
+      for (int nb = 0; nb < NB; ++nb) mma_bf16(sacc[nb], qh[ks], kf[nb][0], kf[nb][1]);
 #pragma unroll
-      for (int nb = 0; nb < KT / 8; ++nb) mma_bf16(sacc[nb], ql[ks], kf[nb][0], kf[nb][1]);
+      for (int nb = 0; nb < NB; ++nb) mma_bf16(sacc[nb], ql[ks], kf[nb][0], kf[nb][1]);
     }
     // ---- mask, online softmax (base 2)
     float tmax0 = -INFINITY, tmax1 = -INFINITY;
 #pragma unroll
-    for (int nb = 0; nb < KT / 8; ++nb) {
-      const int j = key0 + nb * 8 + tq * 2;
+    for (int nb = 0; nb < NB; ++nb) {
+      const int j = key0 + (kg * NB + nb) * 8 + tq * 2;
       if (!(j <= pos0 && j < k_end)) sacc[nb][0] = -INFINITY;
       if (!(j + 1 <= pos0 && j + 1 < k_end)) sacc[nb][1] = -INFINITY;
       if (!(j <= pos1 && j < k_end)) sacc[nb][2] = -INFINITY;
@@ -228,9 +235,9 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     m_run[0] = mn0;
     m_run[1] = mn1;
     float ls0 = 0.0f, ls1 = 0.0f;
-    uint32_t ph[KT / 16][4], pl[KT / 16][4];
+    uint32_t ph[NK][4], pl[NK][4];
 #pragma unroll
-    for (int nb = 0; nb < KT / 8; ++nb) {
+    for (int nb = 0; nb < NB; ++nb) {
       const float p0 = exp2f(sacc[nb][0] - sub0), p1 = exp2f(sacc[nb][1] - sub0);
       const float p2 = exp2f(sacc[nb][2] - sub1), p3 = exp2f(sacc[nb][3] - sub1);
       ls0 += p0 + p1;
@@ -248,13 +255,13 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     }
     // ---- O += P V
 #pragma unroll
-    for (int kk = 0; kk < KT / 16; ++kk) {
+    for (int kk = 0; kk < NK; ++kk) {
 #pragma unroll
       for (int c8 = 0; c8 < HD / 8; c8 += 8) {   // eight output column blocks at a time, same ordering idea
         uint32_t vf[8][2];
 #pragma unroll
         for (int cd = 0; cd < 8; cd += 2) {
-          const int row = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int row = (kg * NK + kk) * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
           const int chunkc = c8 + cd + ((lane >> 4) & 1);
           ldmatrix_x4_trans(vbase + (chunkc >> 3) * (KT * 128) + row * 128 + (((chunkc & 7) ^ (row & 7)) << 4), vf[cd][0],
                             vf[cd][1], vf[cd + 1][0], vf[cd + 1][1]);
@@ -277,11 +284,54 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   }
 
   SJD_TL(TL_ATTN, 2, threadIdx.x == 0);
-  // ---- partial record per (row, head, split): [max (natural log units), sum, o[HD]]
   l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
   l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
   l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
   l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+  if (KG > 1) {
+    // ---- merge the key groups of each 16-row band: groups 1.. leave (max, sum, output) in the (now
+    // idle) tile ring, group 0 folds them into its own.  Every tile was consumed before the last
+    // barrier of the loop, so the ring is free.
+    constexpr int REC = HD + 2;   // floats per row record
+    float *xch = reinterpret_cast<float *>(smem);
+    if (kg > 0) {
+      float *dst = xch + ((size_t)((kg - 1) * n_rw + rw) * 16) * REC;
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        float *row = dst + (g + rr * 8) * REC;
+        if (tq == 0) {
+          row[0] = m_run[rr];
+          row[1] = l_run[rr];
+        }
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i)
+          *reinterpret_cast<float2 *>(row + 2 + i * 8 + tq * 2) = make_float2(o[i][rr * 2], o[i][rr * 2 + 1]);
+      }
+    }
+    __syncthreads();
+    if (kg > 0) return;
+#pragma unroll
+    for (int og = 1; og < KG; ++og) {
+      const float *src = xch + ((size_t)((og - 1) * n_rw + rw) * 16) * REC;
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const float *row = src + (g + rr * 8) * REC;
+        const float m_o = row[0], l_o = row[1];
+        const float mn = fmaxf(m_run[rr], m_o);
+        const float a_s = mn > -INFINITY ? exp2f(m_run[rr] - mn) : 1.0f;   // both empty: keep zeros
+        const float a_o = mn > -INFINITY ? exp2f(m_o - mn) : 0.0f;
+        m_run[rr] = mn;
+        l_run[rr] = l_run[rr] * a_s + l_o * a_o;
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) {
+          const float2 v = *reinterpret_cast<const float2 *>(row + 2 + i * 8 + tq * 2);
+          o[i][rr * 2] = o[i][rr * 2] * a_s + v.x * a_o;
+          o[i][rr * 2 + 1] = o[i][rr * 2 + 1] * a_s + v.y * a_o;
+        }
+      }
+    }
+  }
+  // ---- partial record per (row, head, split): [max (natural log units), sum, o[HD]]
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr) {
     const int r = rr == 0 ? r0 : r1;
@@ -342,29 +392,25 @@ int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, co
   p.n_kv_heads = n_kv_heads;
   p.splits = splits;
   p.plane0 = plane0;
-  const int threads = 32 * ((rows_per_seq + 15) / 16);
+  const int threads = 128;   // four warps: 16-row bands x key groups
+  const int kg = rows_per_seq <= 16 ? 4 : rows_per_seq <= 32 ? 2 : 1;
   const dim3 grid(n_heads, M / rows_per_seq, splits);
   const CUtensorMap &km = reinterpret_cast<const CUtensorMap &>(kv_map);
   const size_t smem = (size_t)kStagesAttn * 2 * KT * head_dim * 2 + 1024;
-  static bool configured[64][2] = {};
-  int dev = 0;
-  SJD_CUDA(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
+  auto launch = [&](auto kernel) -> int {
+    SJD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    SJD_CUDA(launch_kernel(kernel, grid, dim3(threads), smem, stream, km, p));
+    SJD_CHECK_LAUNCH();
+    return SJD_OK;
+  };
   if (head_dim == 128) {
-    if (!configured[dev][1]) {
-      SJD_CUDA(cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      configured[dev][1] = true;
-    }
-    SJD_CUDA(launch_kernel(attention_mma_kernel<128>, grid, dim3(threads), smem, stream, km, p));
-  } else {
-    if (!configured[dev][0]) {
-      SJD_CUDA(cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      configured[dev][0] = true;
-    }
-    SJD_CUDA(launch_kernel(attention_mma_kernel<64>, grid, dim3(threads), smem, stream, km, p));
+    if (kg == 4) return launch(attention_mma_kernel<128, 4>);
+    if (kg == 2) return launch(attention_mma_kernel<128, 2>);
+    return launch(attention_mma_kernel<128, 1>);
   }
-  SJD_CHECK_LAUNCH();
-  return SJD_OK;
+  if (kg == 4) return launch(attention_mma_kernel<64, 4>);
+  if (kg == 2) return launch(attention_mma_kernel<64, 2>);
+  return launch(attention_mma_kernel<64, 1>);
 }
 
 }  // namespace sjd
