@@ -132,6 +132,21 @@ def test_large_shapes_two_layers(name, steps):
     assert seqs[0].max_logit_err <= 2e-2
 
 
+def test_full_depth_7b_two_steps():
+    """The benchmark's own configuration (7B shapes, all 32 layers, W = 32, the CUDA-graph step) for the
+    pre-fill and two lock-step iterations: every logit of both windows against the fp64 checker, every
+    decision re-taken by it.  Needs ~30 GB of host memory for the checker's weights and cache."""
+    import psutil
+    if psutil.virtual_memory().available < 48 * 2 ** 30:
+        pytest.skip("not enough host memory for the full-depth checker")
+    wl = WORKLOADS["7b"]
+    ctx, seqs, n, _ = run_lockstep(wl, max_steps=2, gain_jitter=0.0)
+    assert n == 2 and seqs[0].steps == 2
+    assert seqs[0].max_logit_excess <= 2e-2
+    print("full-depth 7B: max |logit diff| %.3e, beyond half a storage ulp %.3e" %
+          (seqs[0].max_logit_err, seqs[0].max_logit_excess))
+
+
 def test_api_errors_and_state():
     wl = WORKLOADS["tiny"]
     weights = B.weights_to_device(make_weights(wl))
