@@ -132,19 +132,21 @@ def test_large_shapes_two_layers(name, steps):
     assert seqs[0].max_logit_err <= 2e-2
 
 
-def test_full_depth_7b_two_steps():
-    """The benchmark's own configuration (7B shapes, all 32 layers, W = 32, the CUDA-graph step) for the
-    pre-fill and two lock-step iterations: every logit of both windows against the fp64 checker, every
-    decision re-taken by it.  Needs ~30 GB of host memory for the checker's weights and cache."""
+@pytest.mark.parametrize("name,steps", [("7b", 2), ("8b-gqa", 1)])
+def test_full_depth(name, steps):
+    """The full configurations (7B: 32 layers, vocab 65536, W = 32, the step the benchmark times; 8B with
+    grouped-query heads: 32 layers, vocab 184320, W = 64) for the pre-fill and one or two lock-step
+    iterations: every logit of the windows against the fp64 checker, every decision re-taken by it.
+    Needs ~40 GB of host memory for the checker's weights and cache."""
     import psutil
-    if psutil.virtual_memory().available < 48 * 2 ** 30:
+    if psutil.virtual_memory().available < 64 * 2 ** 30:
         pytest.skip("not enough host memory for the full-depth checker")
-    wl = WORKLOADS["7b"]
-    ctx, seqs, n, _ = run_lockstep(wl, max_steps=2, gain_jitter=0.0)
-    assert n == 2 and seqs[0].steps == 2
+    wl = WORKLOADS[name]
+    ctx, seqs, n, _ = run_lockstep(wl, max_steps=steps, gain_jitter=0.0)
+    assert n == steps and seqs[0].steps == steps
     assert seqs[0].max_logit_excess <= 2e-2
-    print("full-depth 7B: max |logit diff| %.3e, beyond half a storage ulp %.3e" %
-          (seqs[0].max_logit_err, seqs[0].max_logit_excess))
+    print("full-depth %s: max |logit diff| %.3e, beyond half a storage ulp %.3e" %
+          (name, seqs[0].max_logit_err, seqs[0].max_logit_excess))
 
 
 def test_api_errors_and_state():
