@@ -131,6 +131,10 @@ class LockStepSequence:
         self.max_logit_excess = 0.0      # largest |diff| beyond half a storage ulp
         self.steps = 0
 
+    def logit_failures(self, diff, half_ulp):
+        """Mask of logits beyond the tolerance (a test of deeper models may state a different rule)."""
+        return diff > self.tol + half_ulp
+
     def check_window(self, draft_row, kind_row, q_row, total):
         w_eff = len(self.st.drafts)
         assert int(total) == self.st.n
@@ -164,7 +168,7 @@ class LockStepSequence:
             self.max_logit_err = max(self.max_logit_err, err)
             half_ulp = storage_half_ulp(own, scfg.logits_dtype)
             self.max_logit_excess = max(self.max_logit_excess, float((diff - half_ulp).max()))
-            bad = diff > self.tol + half_ulp
+            bad = self.logit_failures(diff, half_ulp)
             assert not bad.any(), (f"step {self.steps}: {int(bad.sum())} logits off by more than {self.tol} "
                                    f"+ half a storage ulp; max |diff| {err:.3e}")
         n_before = st.n
