@@ -127,12 +127,40 @@ __global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int 
   SJD_TL(TL_SWIGLU, 0, threadIdx.x == 0);
   pdl_wait();
   SJD_TL(TL_SWIGLU, 1, threadIdx.x == 0);
-  const size_t total = (size_t)M * F;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const size_t m = i / F, f = i % F;
-    const float sc = row_scale(rs, (int)m);
-    const float g = sc * sum_planes(ps, m * ps.ld + f), u = sc * sum_planes(ps, m * ps.ld + F + f);
-    put_hilo(act, i, g / (1.0f + expf(-g)) * u);
+  if ((F & 3) == 0 && (ps.ld & 3) == 0 && (ps.plane_stride & 3) == 0) {
+    // grid (column chunks, rows): a thread handles groups of four adjacent columns of one row
+    const int m = blockIdx.y;
+    const float sc = row_scale(rs, m);
+    const float *row = ps.base + (size_t)m * ps.ld;
+    for (int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4; f < F; f += gridDim.x * blockDim.x * 4) {
+      float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+      for (int sp = 0; sp < ps.splits; ++sp) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(row + (size_t)sp * ps.plane_stride + f));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(row + (size_t)sp * ps.plane_stride + F + f));
+        g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
+        u.x += b.x; u.y += b.y; u.z += b.z; u.w += b.w;
+      }
+      const float gv[4] = {sc * g.x, sc * g.y, sc * g.z, sc * g.w}, uv[4] = {sc * u.x, sc * u.y, sc * u.z, sc * u.w};
+      __nv_bfloat16 hi[4], lo[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float v = gv[i] / (1.0f + expf(-gv[i])) * uv[i];
+        hi[i] = __float2bfloat16_rn(v);
+        lo[i] = __float2bfloat16_rn(v - __bfloat162float(hi[i]));
+      }
+      const size_t idx = (size_t)m * F + f;   // multiple of 4: 8-byte aligned stores
+      *reinterpret_cast<uint2 *>(act.base + idx) = *reinterpret_cast<const uint2 *>(hi);
+      *reinterpret_cast<uint2 *>(act.base + act.lo_offset + idx) = *reinterpret_cast<const uint2 *>(lo);
+    }
+  } else {
+    const size_t total = (size_t)M * F;
+    const size_t nthreads = (size_t)gridDim.x * gridDim.y * blockDim.x;
+    for (size_t i = ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+      const size_t m = i / F, f = i % F;
+      const float sc = row_scale(rs, (int)m);
+      const float g = sc * sum_planes(ps, m * ps.ld + f), u = sc * sum_planes(ps, m * ps.ld + F + f);
+      put_hilo(act, i, g / (1.0f + expf(-g)) * u);
+    }
   }
   SJD_TL(TL_SWIGLU, 2, threadIdx.x == 0);
 }
@@ -173,11 +201,12 @@ int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos
 }
 
 int launch_swiglu_finish(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, cudaStream_t stream) {
-  const size_t total = (size_t)M * F;
-  // at most two blocks per SM: the whole grid must be resident at once for the next kernel to be
-  // scheduled early, and it must leave thread slots for that kernel's CTAs while it waits
-  const int blocks = (int)((total + 255) / 256 < 296 ? (total + 255) / 256 : 296);
-  SJD_CUDA(launch_kernel(swiglu_finish_kernel, dim3(blocks), dim3(256), 0, stream, ps, rs, act, M, F));
+  // Few enough blocks that (for windows of a few dozen rows) the whole grid is resident at once and
+  // leaves thread slots free: only then is the next kernel scheduled early under dependent launch.
+  int per_row = (F / 4 + 255) / 256;
+  const int cap = 296 / (M < 296 ? M : 296);
+  per_row = per_row > cap ? (cap > 0 ? cap : 1) : per_row;
+  SJD_CUDA(launch_kernel(swiglu_finish_kernel, dim3(per_row, M), dim3(256), 0, stream, ps, rs, act, M, F));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }
