@@ -371,28 +371,38 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   if (!s_last) return;
   __threadfence();
   constexpr int REC = HD + 2, C4 = HD / 4;
+  // weight of every (row, key range) record, normalised: exp(max_s - max) / sum_s' l_s' exp(max_s' - max).
+  // One pass over the 2-float heads of the records; the ring is idle and holds the table.
+  float *wtab = reinterpret_cast<float *>(smem);
+  for (int r = tid; r < W; r += blockDim.x) {
+    const float *src = p.partial + ((size_t)(m0 + r) * p.n_heads + h) * p.splits * REC;
+    float gmax = -INFINITY;
+    for (int sp = 0; sp < p.splits; ++sp) gmax = fmaxf(gmax, __ldcg(src + (size_t)sp * REC));
+    float denom = 0.0f;
+    for (int sp = 0; sp < p.splits; ++sp) {
+      const float ms = __ldcg(src + (size_t)sp * REC);
+      const float wgt = ms > -INFINITY ? expf(ms - gmax) : 0.0f;
+      wtab[r * p.splits + sp] = wgt;
+      denom += __ldcg(src + (size_t)sp * REC + 1) * wgt;
+    }
+    const float inv = (s_pos[r] >= 0 && denom > 0.0f) ? 1.0f / denom : 0.0f;
+    for (int sp = 0; sp < p.splits; ++sp) wtab[r * p.splits + sp] *= inv;
+  }
+  __syncthreads();
   for (int idx = tid; idx < W * C4; idx += blockDim.x) {
     const int r = idx / C4, c = (idx - r * C4) * 4;
     const size_t obase = ((size_t)(m0 + r) * p.n_heads + h) * HD + c;
+    const float *src = p.partial + ((size_t)(m0 + r) * p.n_heads + h) * p.splits * REC + 2 + c;
+    const float *wrow = wtab + r * p.splits;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float denom = 0.0f;
-    if (s_pos[r] >= 0) {
-      const float *src = p.partial + ((size_t)(m0 + r) * p.n_heads + h) * p.splits * REC;
-      float gmax = -INFINITY;
-      for (int sp = 0; sp < p.splits; ++sp) gmax = fmaxf(gmax, __ldcg(src + (size_t)sp * REC));
-      for (int sp = 0; sp < p.splits; ++sp) {
-        const float ms = __ldcg(src + (size_t)sp * REC);
-        if (ms > -INFINITY) {
-          const float wgt = expf(ms - gmax);
-          denom += __ldcg(src + (size_t)sp * REC + 1) * wgt;
-          const float2 a = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)sp * REC + 2 + c));
-          const float2 bq = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)sp * REC + 4 + c));
-          acc.x += a.x * wgt; acc.y += a.y * wgt; acc.z += bq.x * wgt; acc.w += bq.y * wgt;
-        }
-      }
+#pragma unroll 4
+    for (int sp = 0; sp < p.splits; ++sp) {   // loads do not depend on one another: they overlap
+      const float2 a = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)sp * REC));
+      const float2 bq = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)sp * REC + 2));
+      const float wgt = wrow[sp];
+      acc.x += a.x * wgt; acc.y += a.y * wgt; acc.z += bq.x * wgt; acc.w += bq.y * wgt;
     }
-    const float inv = denom > 0.0f ? 1.0f / denom : 0.0f;
-    const float v[4] = {acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv};
+    const float v[4] = {acc.x, acc.y, acc.z, acc.w};
     *reinterpret_cast<float4 *>(p.out + obase) = make_float4(v[0], v[1], v[2], v[3]);
     if (p.hilo.base) {
       __nv_bfloat16 hi[4], lo[4];
