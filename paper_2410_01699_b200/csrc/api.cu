@@ -184,8 +184,7 @@ int attn_splits(int n_heads, int batch) {
 
 extern "C" size_t sjd_attention_workspace_bytes(int batch, int window, int n_heads, int head_dim) {
   if (batch < 1 || window < 1 || n_heads < 1 || !attention_mma_supported(head_dim, window)) return 0;
-  return up256(256 + (size_t)batch * n_heads * 4) +
-         (size_t)batch * window * n_heads * attn_splits(n_heads, batch) * (head_dim + 2) * 4;
+  return 256 + (size_t)batch * window * n_heads * attn_splits(n_heads, batch) * (head_dim + 2) * 4;
 }
 
 extern "C" int sjd_attention(int batch, int window, int n_heads, int n_kv_heads, int head_dim, int max_seq, const float *q,
@@ -202,17 +201,15 @@ extern "C" int sjd_attention(int batch, int window, int n_heads, int n_kv_heads,
   SJD_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev));
   if (cc_major < 9) return SJD_ERR_UNSUPPORTED;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  // header: status word (first 256 bytes), then one merge ticket per (sequence, head); both start at zero
-  const size_t header = up256(256 + (size_t)batch * n_heads * 4);
   int *status = (int *)ws;
-  int *tickets = (int *)((char *)ws + 256);
-  float *partial = (float *)((char *)ws + header);
-  SJD_CUDA(cudaMemsetAsync(ws, 0, header, stream));
+  float *partial = (float *)((char *)ws + 256);
+  SJD_CUDA(cudaMemsetAsync(status, 0, 256, stream));
   TensorMap kv_map;
   int rc = make_kv_tensor_map(&kv_map, kv_cache, (long)batch * 2 * n_kv_heads, max_seq, head_dim);
   if (rc != SJD_OK) return rc;
   const int splits = attn_splits(n_heads, batch);
   const int M = batch * window;
-  return launch_attention_mma(kv_map, 0, q, in_pos, partial, out, HiLoOut{nullptr, 0}, tickets, status, M, window, n_heads,
-                              n_kv_heads, head_dim, splits, stream);
+  rc = launch_attention_mma(kv_map, 0, q, in_pos, partial, status, M, window, n_heads, n_kv_heads, head_dim, splits, stream);
+  if (rc != SJD_OK) return rc;
+  return launch_attention_combine(partial, in_pos, out, M, n_heads, head_dim, splits, stream, HiLoOut{nullptr, 0});
 }

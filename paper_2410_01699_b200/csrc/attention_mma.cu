@@ -10,10 +10,8 @@
 // with its own running max / sum / output) and merge through shared memory at the end; one warp per
 // scheduler alone cannot keep the tensor pipe and the exponentials going at the same time.  The probabilities are split hi + lo as well, so neither
 // operand loses more than ~2^-17 relative.  The kernel is bound by streaming K/V once from HBM (GQA
-// heads of a group share their tiles through L2).  Every key range leaves a partial record (max, sum,
-// unnormalised output); the last CTA of a (head, sequence) to finish -- an atomic ticket, nobody
-// waits -- merges the records, normalises and writes the output rows, also as the bf16 hi/lo planes
-// the output projection reads.  Every barrier wait is bounded.
+// heads of a group share their tiles through L2).  Partials (max, sum, unnormalised output) go to the
+// merge kernel of attention.cu.  Every barrier wait is bounded.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -88,9 +86,6 @@ struct AttnParams {
   const float *q;        // [M][H*HD]
   const int32_t *in_pos; // [M]
   float *partial;        // [M][H][splits][HD + 2]
-  float *out;            // [M][H*HD]
-  HiLoOut hilo;          // optional bf16 hi/lo planes of out
-  int *tickets;          // [sequences][H], zero on entry and on exit
   int *status;
   int rows_per_seq, n_heads, n_kv_heads, splits;
   int plane0;            // first cache plane of this layer: planes are [b][k|v][kv_head]
@@ -104,7 +99,6 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ uint64_t bar_full[kStagesAttn];
   __shared__ int s_pos[64];
-  __shared__ int s_last;
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   pdl_trigger();
@@ -282,10 +276,6 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     if (tid == 0 && t + kStagesAttn < n_tiles) issue(t + kStagesAttn);
   }
   if (!ok) {
-    if (tid == 0 && p.splits > 1) {   // keep the ticket count whole for the next launch; nothing is merged
-      int *ticket = p.tickets + b * p.n_heads + h;
-      if (atomicAdd(ticket, 1) == p.splits - 1) *ticket = 0;
-    }
     if (tid == 0) atomicExch(p.status, 4);
     // leave no copy in flight: wait (bounded) for the stages that were armed
     if (tid == 0)
@@ -319,8 +309,9 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
       }
     }
     __syncthreads();
+    if (kg > 0) return;
 #pragma unroll
-    for (int og = 1; og < KG && kg == 0; ++og) {
+    for (int og = 1; og < KG; ++og) {
       const float *src = xch + ((size_t)((og - 1) * n_rw + rw) * 16) * REC;
 #pragma unroll
       for (int rr = 0; rr < 2; ++rr) {
@@ -344,7 +335,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr) {
     const int r = rr == 0 ? r0 : r1;
-    if (r >= W || kg != 0) continue;
+    if (r >= W) continue;
     float *dst = p.partial + (((size_t)(m0 + r) * p.n_heads + h) * p.splits + split) * (HD + 2);
     if (tq == 0) {
       dst[0] = m_run[rr] > -INFINITY ? m_run[rr] * 0.6931471805599453f : -INFINITY;
@@ -353,67 +344,6 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
 #pragma unroll
     for (int i = 0; i < HD / 8; ++i)
       *reinterpret_cast<float2 *>(dst + 2 + i * 8 + tq * 2) = make_float2(o[i][rr * 2], o[i][rr * 2 + 1]);
-  }
-
-  // ---- the last key range of this (head, sequence) to arrive merges all of them
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    int last = 1;
-    if (p.splits > 1) {
-      int *ticket = p.tickets + b * p.n_heads + h;
-      last = atomicAdd(ticket, 1) == p.splits - 1;
-      if (last) *ticket = 0;
-    }
-    s_last = last;
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  constexpr int REC = HD + 2, C4 = HD / 4;
-  // weight of every (row, key range) record, normalised: exp(max_s - max) / sum_s' l_s' exp(max_s' - max).
-  // One pass over the 2-float heads of the records; the ring is idle and holds the table.
-  float *wtab = reinterpret_cast<float *>(smem);
-  for (int r = tid; r < W; r += blockDim.x) {
-    const float *src = p.partial + ((size_t)(m0 + r) * p.n_heads + h) * p.splits * REC;
-    float gmax = -INFINITY;
-    for (int sp = 0; sp < p.splits; ++sp) gmax = fmaxf(gmax, __ldcg(src + (size_t)sp * REC));
-    float denom = 0.0f;
-    for (int sp = 0; sp < p.splits; ++sp) {
-      const float ms = __ldcg(src + (size_t)sp * REC);
-      const float wgt = ms > -INFINITY ? expf(ms - gmax) : 0.0f;
-      wtab[r * p.splits + sp] = wgt;
-      denom += __ldcg(src + (size_t)sp * REC + 1) * wgt;
-    }
-    const float inv = (s_pos[r] >= 0 && denom > 0.0f) ? 1.0f / denom : 0.0f;
-    for (int sp = 0; sp < p.splits; ++sp) wtab[r * p.splits + sp] *= inv;
-  }
-  __syncthreads();
-  for (int idx = tid; idx < W * C4; idx += blockDim.x) {
-    const int r = idx / C4, c = (idx - r * C4) * 4;
-    const size_t obase = ((size_t)(m0 + r) * p.n_heads + h) * HD + c;
-    const float *src = p.partial + ((size_t)(m0 + r) * p.n_heads + h) * p.splits * REC + 2 + c;
-    const float *wrow = wtab + r * p.splits;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-    for (int sp = 0; sp < p.splits; ++sp) {   // loads do not depend on one another: they overlap
-      const float2 a = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)sp * REC));
-      const float2 bq = __ldcg(reinterpret_cast<const float2 *>(src + (size_t)sp * REC + 2));
-      const float wgt = wrow[sp];
-      acc.x += a.x * wgt; acc.y += a.y * wgt; acc.z += bq.x * wgt; acc.w += bq.y * wgt;
-    }
-    const float v[4] = {acc.x, acc.y, acc.z, acc.w};
-    *reinterpret_cast<float4 *>(p.out + obase) = make_float4(v[0], v[1], v[2], v[3]);
-    if (p.hilo.base) {
-      __nv_bfloat16 hi[4], lo[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        hi[i] = __float2bfloat16_rn(v[i]);
-        lo[i] = __float2bfloat16_rn(v[i] - __bfloat162float(hi[i]));
-      }
-      *reinterpret_cast<uint2 *>(p.hilo.base + obase) = *reinterpret_cast<const uint2 *>(hi);
-      *reinterpret_cast<uint2 *>(p.hilo.base + p.hilo.lo_offset + obase) = *reinterpret_cast<const uint2 *>(lo);
-    }
   }
 }
 
@@ -447,18 +377,15 @@ int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_s
 
 bool attention_mma_supported(int head_dim, int rows_per_seq) { return (head_dim == 64 || head_dim == 128) && rows_per_seq <= 64; }
 
-// `tickets`: sequences x n_heads ints, zero on entry (the kernel leaves them zero)
+// partial kernel only; the caller merges with the combine kernel of attention.cu
 int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
-                         float *out, HiLoOut hilo, int *tickets, int *status, int M, int rows_per_seq, int n_heads,
-                         int n_kv_heads, int head_dim, int splits, cudaStream_t stream) {
+                         int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads, int head_dim, int splits,
+                         cudaStream_t stream) {
   if (!attention_mma_supported(head_dim, rows_per_seq) || M % rows_per_seq != 0) return SJD_ERR_UNSUPPORTED;
   AttnParams p;
   p.q = q;
   p.in_pos = in_pos;
   p.partial = partial;
-  p.out = out;
-  p.hilo = hilo;
-  p.tickets = tickets;
   p.status = status;
   p.rows_per_seq = rows_per_seq;
   p.n_heads = n_heads;

@@ -40,7 +40,7 @@ struct XMaps {
 struct Layout {
   size_t kv, logits[2], stats[2], row_out, counters, step, status;
   size_t x, h, qkv, q, attn, gu, act, partial, rope;
-  size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part, attn_tickets;
+  size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t total;
 };
@@ -88,7 +88,6 @@ Layout make_layout(const sjd_model_cfg &c) {
     part = need > part ? need : part;
   }
   L.partial = take(part * 4);
-  L.attn_tickets = take((size_t)c.max_batch * c.n_heads * 4);
   // bf16 hi/lo planes of the GEMM inputs, stream-K partials and tickets (tensor-core path)
   const size_t Ma = (Mx + 15) / 16 * 16;
   L.xs_h = take(2 * Ma * c.d_model * 2);
@@ -426,9 +425,10 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     const KvLayout kv = c->kv_layer(l);
     SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
     if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
-      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, attn,
-                                                hl_attn, c->at<int>(c->lay.attn_tickets), status, M, rows_per_seq,
-                                                g.n_heads, g.n_kv_heads, g.head_dim, att_splits, stream));
+      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, status, M,
+                                                rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim, att_splits, stream));
+      SJD_TR(TC_ATTENTION,
+             launch_attention_combine(partial, st.in_pos, attn, M, g.n_heads, g.head_dim, att_splits, stream, hl_attn));
     } else {
       SJD_TR(TC_ATTENTION,
              launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, att_splits, stream, hl_attn));
@@ -572,7 +572,6 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
   cudaError_t e = cudaMemcpy(c->ws + lay.rope, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.counters, 0, ((size_t)cfg->max_batch + 1) * 4);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.status, 0, 4);
-  if (e == cudaSuccess) e = cudaMemset(c->ws + lay.attn_tickets, 0, (size_t)cfg->max_batch * cfg->n_heads * 4);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     delete c;
