@@ -6,7 +6,6 @@
 namespace sjd {
 thread_local int g_last_cuda_error = 0;
 std::atomic<long long> g_launch_count{0};
-thread_local L2PrefetchSet g_prefetch = {};
 thread_local bool g_pdl = false;
 
 int check_sample_cfg(const sjd_sample_cfg *s, int vocab) {

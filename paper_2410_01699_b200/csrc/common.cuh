@@ -259,38 +259,6 @@ struct GemmTcCall {
 int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream);
 int launch_sum_planes(const float *planes, size_t plane_stride, int splits, float *out, size_t total, int accumulate,
                       cudaStream_t stream);
-// Weights the next projection will stream, fetched into L2 ahead of time by the small kernels that run
-// between two projections (their own work leaves HBM idle).  Host side: the engine fills g_prefetch
-// before launching such a kernel; the launcher takes it and passes it to the kernel.
-struct L2Span {
-  const void *base;           // 16-byte aligned
-  unsigned long long bytes;   // a multiple of 16 KB; 0: nothing
-};
-struct L2PrefetchSet {
-  L2Span s[3];
-};
-extern thread_local L2PrefetchSet g_prefetch;
-inline L2PrefetchSet take_prefetch() {
-  const L2PrefetchSet p = g_prefetch;
-  g_prefetch = L2PrefetchSet{};
-  return p;
-}
-#ifdef __CUDACC__
-// thread 0 of every block issues its share of the 16 KB chunks (asynchronous, nothing waits for them)
-__device__ __forceinline__ void l2_prefetch(const L2PrefetchSet &pf) {
-  if (threadIdx.x != 0) return;
-  const unsigned nblk = gridDim.x * gridDim.y * gridDim.z;
-  const unsigned blk = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
-#pragma unroll
-  for (int k = 0; k < 3; ++k) {
-    const unsigned long long chunks = pf.s[k].bytes >> 14;
-    const char *base = reinterpret_cast<const char *>(pf.s[k].base);
-    for (unsigned long long c = blk; c < chunks; c += nblk)
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + (c << 14)), "r"(16384u) : "memory");
-  }
-}
-#endif
-
 // The fp32 partial planes a GEMM launch left: value(m, col) = sum_s base[s * plane_stride + m * ld + col]
 struct PlaneSet {
   const float *base;

@@ -24,10 +24,6 @@ int attention_splits(int n_heads, int batch) {
   return s < 1 ? 1 : (s > 16 ? 16 : s);
 }
 
-#ifndef SJD_L2_PREFETCH_MB
-#define SJD_L2_PREFETCH_MB 48
-#endif
-constexpr size_t kL2PrefetchBytes = (size_t)SJD_L2_PREFETCH_MB << 20;   // per projection launch; 0: off
 constexpr int kMaxGemmCtas = 160;    // upper bound on the SM count used to size split-K scratch
 
 struct WMap {
@@ -415,30 +411,11 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     return r;
   };
 
-  // what the small kernels between two projections fetch into L2 for the next one: up to
-  // kL2PrefetchBytes of its weights, shared evenly between its matrices
-  auto prefetch = [&](const void *w0, size_t b0, const void *w1 = nullptr, size_t b1 = 0, const void *w2 = nullptr,
-                      size_t b2 = 0) {
-    L2PrefetchSet pf{};
-    if (kL2PrefetchBytes == 0 || tr.on) return;
-    const void *w[3] = {w0, w1, w2};
-    const size_t by[3] = {b0, b1, b2};
-    const int n = w2 ? 3 : (w1 ? 2 : 1);
-    for (int i = 0; i < n; ++i) {
-      size_t take = by[i] < kL2PrefetchBytes / n ? by[i] : kL2PrefetchBytes / n;
-      take &= ~(size_t)16383;
-      if (((uintptr_t)w[i] & 15u) == 0) pf.s[i] = L2Span{w[i], take};
-    }
-    g_prefetch = pf;
-  };
-  const size_t bq = (size_t)nq * d * 2, bk = (size_t)nk * d * 2, bo = (size_t)d * nq * 2, bf = (size_t)F * d * 2;
-
   SJD_TR(TC_OTHER, launch_embed(dt, c->tok_emb, st.in_tok, x, M, d, g.vocab, stream));
   PlaneSet pending{nullptr, 0, 0, 0};   // planes still to be added into the residual stream
   for (int l = 0; l < g.n_layers; ++l) {
     const LayerMaps &lm = c->wmaps[l];
     PlaneSet ps;
-    prefetch(c->wq[l], bq, c->wk[l], bk, c->wv[l], bk);
     SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->attn_norm[l], hl_h, ss_part, M, d, stream));
     {
       const WMap *wm[3] = {&lm.wq, &lm.wk, &lm.wv};
@@ -446,7 +423,6 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       SJD_TRY(gemm(wm, 3, n_out, xm.h, d, nqkv, planes, false, &ps));
     }
     const KvLayout kv = c->kv_layer(l);
-    prefetch(c->wo[l], bo);
     SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
     if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
       SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, status, M,
@@ -462,14 +438,12 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       const int n_out[1] = {d};
       SJD_TRY(gemm(wm, 1, n_out, xm.attn, nq, d, planes, false, &ps));
     }
-    prefetch(c->w_gate[l], bf, c->w_up[l], bf);
     SJD_TR(TC_OTHER, launch_resid_gain(dt, x, ps, c->ffn_norm[l], hl_h, ss_part, M, d, stream));
     {
       const WMap *wm[2] = {&lm.w_gate, &lm.w_up};
       const int n_out[2] = {F, F};
       SJD_TRY(gemm(wm, 2, n_out, xm.h, d, 2 * F, planes, false, &ps));
     }
-    prefetch(c->w_down[l], bf);
     SJD_TR(TC_OTHER, launch_swiglu_finish(ps, rs, hl_act, M, F, stream));
     {
       const WMap *wm[1] = {&lm.w_down};
@@ -478,7 +452,6 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     }
   }
   if (logits_out) {
-    prefetch(c->lm_head, (size_t)g.vocab * d * 2);
     SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->final_norm, hl_h, ss_part, M, d, stream));
     const WMap *wm[1] = {&c->wmap_head};
     const int n_out[1] = {g.vocab};

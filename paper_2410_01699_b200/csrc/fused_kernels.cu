@@ -44,11 +44,9 @@ constexpr int RG_COLS = RG_THREADS * 4;
 
 template <typename T>
 __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restrict__ x, PlaneSet ps, const T *__restrict__ gain,
-                                                               HiLoOut h, float *__restrict__ ss_part, int d,
-                                                               L2PrefetchSet pf) {
+                                                               HiLoOut h, float *__restrict__ ss_part, int d) {
   __shared__ float red[RG_THREADS / 32];
   pdl_trigger();
-  l2_prefetch(pf);   // weights do not depend on the preceding kernel
   SJD_TL(TL_RESID, 0, threadIdx.x == 0);
   pdl_wait();
   SJD_TL(TL_RESID, 1, threadIdx.x == 0);
@@ -84,9 +82,8 @@ __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restric
 template <typename T>
 __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__restrict__ in_pos,
                                   const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
-                                  int n_heads, L2PrefetchSet pf) {
+                                  int n_heads) {
   pdl_trigger();
-  l2_prefetch(pf);
   SJD_TL(TL_QKV, 0, threadIdx.x == 0);
   pdl_wait();
   SJD_TL(TL_QKV, 1, threadIdx.x == 0);
@@ -125,9 +122,8 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
 }
 
 // act = silu(scale * sum gate planes) * (scale * sum up planes) as bf16 hi/lo planes; planes [S][M][2F]
-__global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, L2PrefetchSet pf) {
+__global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F) {
   pdl_trigger();
-  l2_prefetch(pf);
   SJD_TL(TL_SWIGLU, 0, threadIdx.x == 0);
   pdl_wait();
   SJD_TL(TL_SWIGLU, 1, threadIdx.x == 0);
@@ -177,13 +173,12 @@ int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOu
                       cudaStream_t stream) {
   if (d % 4 != 0) return SJD_ERR_UNSUPPORTED;
   const dim3 grid(M, resid_gain_parts(d));
-  const L2PrefetchSet pf = take_prefetch();
   if (dtype == SJD_F32)
     SJD_CUDA(launch_kernel(resid_gain_kernel<float>, grid, dim3(RG_THREADS), 0, stream, x, ps,
-                           reinterpret_cast<const float *>(gain), h, ss_part, d, pf));
+                           reinterpret_cast<const float *>(gain), h, ss_part, d));
   else if (dtype == SJD_BF16)
     SJD_CUDA(launch_kernel(resid_gain_kernel<__nv_bfloat16>, grid, dim3(RG_THREADS), 0, stream, x, ps,
-                           reinterpret_cast<const __nv_bfloat16 *>(gain), h, ss_part, d, pf));
+                           reinterpret_cast<const __nv_bfloat16 *>(gain), h, ss_part, d));
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();
@@ -193,13 +188,12 @@ int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOu
 int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
   const dim3 grid(M, n_heads + 2 * kv.n_kv_heads);
-  const L2PrefetchSet pf = take_prefetch();
   if (dtype == SJD_F32)
     SJD_CUDA(launch_kernel(qkv_finish_kernel<float>, grid, dim3(64), 0, stream, ps, rs, in_pos, rope_table, q, kv,
-                           rows_per_seq, n_heads, pf));
+                           rows_per_seq, n_heads));
   else if (dtype == SJD_BF16)
     SJD_CUDA(launch_kernel(qkv_finish_kernel<__nv_bfloat16>, grid, dim3(64), 0, stream, ps, rs, in_pos, rope_table, q, kv,
-                           rows_per_seq, n_heads, pf));
+                           rows_per_seq, n_heads));
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();
@@ -212,7 +206,7 @@ int launch_swiglu_finish(PlaneSet ps, RowScale rs, HiLoOut act, int M, int F, cu
   int per_row = (F / 4 + 255) / 256;
   const int cap = 296 / (M < 296 ? M : 296);
   per_row = per_row > cap ? (cap > 0 ? cap : 1) : per_row;
-  SJD_CUDA(launch_kernel(swiglu_finish_kernel, dim3(per_row, M), dim3(256), 0, stream, ps, rs, act, M, F, take_prefetch()));
+  SJD_CUDA(launch_kernel(swiglu_finish_kernel, dim3(per_row, M), dim3(256), 0, stream, ps, rs, act, M, F));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -60,9 +60,6 @@ constexpr int kMaxStages = 8;
 #ifndef SJD_GEMM_WIDE_W_TILES
 #define SJD_GEMM_WIDE_W_TILES 1             // weight tiles per CTA in launches with several token slabs (1 or 2)
 #endif
-#ifndef SJD_GEMM_SLAB_ROWS
-#define SJD_GEMM_SLAB_ROWS 128              // most token rows per slab (per CTA); at most 256 / planes
-#endif
 #ifndef SJD_GEMM_SPLIT_MAX_M
 #define SJD_GEMM_SPLIT_MAX_M 1024           // most rows for which both the hi and the lo plane are multiplied
 #endif
@@ -435,7 +432,7 @@ bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 1024 && N % 
 GemmTcPlan gemm_tc_plan(int M, bool tiles_even) {
   GemmTcPlan pl;
   pl.x_planes = M <= SJD_GEMM_SPLIT_MAX_M ? 2 : 1;
-  const int cap = 256 / pl.x_planes < SJD_GEMM_SLAB_ROWS ? 256 / pl.x_planes : SJD_GEMM_SLAB_ROWS;
+  const int cap = 256 / pl.x_planes;
   pl.n_slabs = (M + cap - 1) / cap;
   const int per = (M + pl.n_slabs - 1) / pl.n_slabs;
   pl.slab_rows = (per + 15) / 16 * 16;
