@@ -95,6 +95,7 @@ struct Scratch {
   uint32_t hist16[16];                //   and of the last 4 bits inside the selected bin
   uint32_t hist[256];
   uint32_t redu[32];
+  uint32_t d_bits[2];                 // register-resident route: bits of the q / p row's entry at the draft token
   uint32_t sel_bin, count_above, bad;
   int sel_chunk, last_chunk;
   int tok;
@@ -653,6 +654,461 @@ __device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scrat
   return true;
 }
 
+// ------------------------------------------------------------------------------------ register-resident row, few barriers
+// The whole treatment of one window row (Eqs. 1-3) for bf16 rows a block can hold in registers, laid
+// out as in fast_row_statistics.  Every search over shared tables (histogram bins, chunk prefix) is done
+// by each warp for itself instead of by one warp between two barriers, so a row costs about a dozen
+// block barriers.  Returns false (block-uniform) when the row needs the general route; nothing it
+// has published by then differs from what that route writes.
+struct RegRow {
+  uint4 v[8];
+};
+
+__device__ __forceinline__ uint4 reg_slot(const RegRow &r, int i) {   // i is warp-uniform
+  uint4 o = r.v[0];
+#pragma unroll
+  for (int k = 1; k < 8; ++k)
+    if (i == k) o = r.v[k];
+  return o;
+}
+
+// load + maximum; publishes the entry at index d (if any) in sc.d_bits.  One barrier.  Returns the
+// block-wide maximum key; 0xFFFF if the row holds a NaN.
+__device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int d_slot, Scratch &sc, bool zero_hist) {
+  using E = Elt<__nv_bfloat16>;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
+  const int j0 = warp * 256 + lane;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    row.v[i] = j < NV ? __ldg(g + j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+  }
+  if (zero_hist)
+    for (int i = tid; i < 4096; i += nt) sc.hist12[i] = 0;
+  if (tid < 16) sc.hist16[tid] = 0;
+  __nv_bfloat162 m2 = as_bf2(row.v[0].x);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(row.v[i], w)));
+    if (d >= 0 && (d >> 3) == j0 + i * 32) {   // this thread holds entry d
+      const uint32_t wd = word_of(row.v[i], (d >> 1) & 3);
+      sc.d_bits[d_slot] = (d & 1) ? wd >> 16 : wd & 0xFFFFu;
+    }
+  }
+  const __nv_bfloat16 m1 = __hmax_nan(__low2bfloat16(m2), __high2bfloat16(m2));
+  const uint32_t mbits = (uint32_t)__bfloat16_as_ushort(m1);
+  uint32_t kmax = (mbits & 0x7FFFu) > 0x7F80u ? 0xFFFFu : E::key(mbits);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) sc.redu[warp] = kmax;
+  __syncthreads();
+  kmax = 0;
+  for (int w = 0; w < nw; ++w) kmax = max(kmax, sc.redu[w]);
+  return kmax;
+}
+
+// exact key of the K-th largest entry.  Two barriers.  false: the threshold sits in a bin next to +-0.
+__device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, Scratch &sc, uint32_t &tau_key) {
+  using E = Elt<__nv_bfloat16>;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int j0 = warp * 256 + lane;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (j0 + i * 32 < NV) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t kk = key_pair(word_of(row.v[i], w));
+        atomicAdd(&sc.hist12[(kk >> 4) & 0xFFFu], 1u);
+        atomicAdd(&sc.hist12[kk >> 20], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  // every warp walks the histogram from the row's top bin downwards, 512 bins at a time
+  uint32_t sel12 = 0, above = 0;
+  {
+    int hi = (int)(kmax >> 4);
+    uint32_t acc = 0;
+    bool found = false;
+    while (!found && hi >= 0) {
+      uint32_t c[16], t = 0;
+#pragma unroll
+      for (int jb = 0; jb < 16; ++jb) {
+        const int bin = hi - 16 * lane - jb;
+        c[jb] = bin >= 0 ? sc.hist12[bin] : 0u;
+        t += c[jb];
+      }
+      uint32_t incl = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      const uint32_t ballot = __ballot_sync(0xffffffffu, acc + incl >= K);
+      if (ballot) {
+        const int src = __ffs(ballot) - 1;
+        uint32_t a = acc + incl - t, s12 = 0, ab = 0;
+#pragma unroll
+        for (int jb = 0; jb < 16; ++jb) {
+          const uint32_t nxt = a + c[jb];
+          if (a < K && K <= nxt) {
+            s12 = (uint32_t)(hi - 16 * lane - jb);
+            ab = a;
+          }
+          a = nxt;
+        }
+        sel12 = __shfl_sync(0xffffffffu, s12, src);
+        above = __shfl_sync(0xffffffffu, ab, src);
+        found = true;
+      } else {
+        acc += __shfl_sync(0xffffffffu, incl, 31);
+        hi -= 512;
+      }
+    }
+  }
+  if (sel12 == 0x7FFu || sel12 == 0x800u) return false;
+  const uint32_t kb_lo = sel12 << 4;
+  const uint32_t v_lo = E::unkey(kb_lo), v_hi = E::unkey(kb_lo | 15u);
+  const __nv_bfloat162 lo2 = as_bf2(v_lo | (v_lo << 16)), hi2 = as_bf2(v_hi | (v_hi << 16));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (j0 + i * 32 < NV) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t x = word_of(row.v[i], w);
+        if (__hge2_mask(as_bf2(x), lo2) & __hle2_mask(as_bf2(x), hi2)) {   // rare: a few entries per warp
+          const uint32_t kk = key_pair(x);
+          if (((kk >> 4) & 0xFFFu) == sel12) atomicAdd(&sc.hist16[kk & 15u], 1u);
+          if ((kk >> 20) == sel12) atomicAdd(&sc.hist16[(kk >> 16) & 15u], 1u);
+        }
+      }
+    }
+  }
+  __syncthreads();
+  {   // every warp: largest code b of the bin with (entries of the bin with code >= b) >= K - above
+    const uint32_t need = K - above;
+    uint32_t suf = lane < 16 ? sc.hist16[lane] : 0u;
+#pragma unroll
+    for (int o = 1; o < 16; o <<= 1) {
+      const uint32_t y = __shfl_down_sync(0xffffffffu, suf, o);
+      if (lane + o < 16) suf += y;
+    }
+    const uint32_t ballot = __ballot_sync(0xffffffffu, lane < 16 && suf >= need) & 0xFFFFu;
+    tau_key = kb_lo | (ballot ? (uint32_t)(31 - __clz(ballot)) : 0u);
+  }
+  return !(tau_key == 0x7FFFu || tau_key == 0x8000u);
+}
+
+// chunk sums of a weight functor evaluated on registers -> sc.chunk_sum.  One barrier.
+template <typename F>
+__device__ __forceinline__ void rr_chunk_sums(const F &wf, int NV, Scratch &sc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int NC = (NV + 31) >> 5;
+  float s[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float w[8];
+    wf(i, w);
+    s[i] = ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
+  }
+  __syncthreads();
+}
+
+// Per-warp view of the fp64 prefix over sc.chunk_sum: lane L owns chunks [L*per, (L+1)*per).
+struct WarpPrefix {
+  double excl, incl, total;
+  int per;
+};
+__device__ __forceinline__ WarpPrefix rr_prefix(int NC, const Scratch &sc) {
+  const int lane = threadIdx.x & 31;
+  WarpPrefix wp;
+  wp.per = (NC + 31) >> 5;
+  const int lo = min(NC, lane * wp.per), hi = min(NC, lo + wp.per);
+  double loc = 0.0;
+  for (int c = lo; c < hi; ++c) loc += (double)sc.chunk_sum[c];
+  double incl = loc;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const double y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  wp.incl = incl;
+  wp.excl = incl - loc;
+  wp.total = __shfl_sync(0xffffffffu, incl, 31);
+  return wp;
+}
+
+// Inverse CDF (token order) over weights held in registers: every warp finds the chunk, the warp that
+// owns it finds the entry (same rules as sample_icdf) and publishes it.  One barrier.
+template <typename F>
+__device__ void rr_icdf(const F &wf, int NV, const WarpPrefix &wp, float u, Scratch &sc, int &tok, float &tok_w) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int NC = (NV + 31) >> 5;
+  const double target = (double)u * wp.total;
+  const int lo = min(NC, lane * wp.per), hi = min(NC, lo + wp.per);
+  // inside this lane's group: first chunk with positive mass whose interval holds the target; last positive chunk
+  int c_hit = -1, c_last = -1;
+  double base_hit = 0.0, base_last = 0.0, run = wp.excl;
+  for (int c = lo; c < hi; ++c) {
+    const float cs = sc.chunk_sum[c];
+    const double nxt = run + (double)cs;
+    if (cs > 0.0f) {
+      if (c_hit < 0 && run <= target && target < nxt) {
+        c_hit = c;
+        base_hit = run;
+      }
+      c_last = c;
+      base_last = run;
+    }
+    run = nxt;
+  }
+  const uint32_t hit = __ballot_sync(0xffffffffu, c_hit >= 0);
+  const uint32_t pos = __ballot_sync(0xffffffffu, c_last >= 0);
+  bool fallback = false;
+  int c;
+  double base;
+  if (hit) {
+    const int src = __ffs(hit) - 1;
+    c = __shfl_sync(0xffffffffu, c_hit, src);
+    base = __shfl_sync(0xffffffffu, base_hit, src);
+  } else if (pos) {
+    const int src = 31 - __clz(pos);
+    c = __shfl_sync(0xffffffffu, c_last, src);
+    base = __shfl_sync(0xffffffffu, base_last, src);
+    fallback = true;
+  } else {
+    c = -1;
+    base = 0.0;
+  }
+  if (c < 0) {
+    if (tid == 0) {
+      sc.tok = 0;
+      sc.tok_w = 0.0f;
+    }
+  } else if (warp == (c >> 3)) {
+    float w[8];
+    wf(c & 7, w);
+    float sum = 0.0f;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) sum += w[t];
+    float incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    float excl = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (lane == 0) excl = 0.0f;
+    const bool cond = !fallback && (base + (double)incl > target);
+    const uint32_t ballot = __ballot_sync(0xffffffffu, cond);
+    const uint32_t posl = __ballot_sync(0xffffffffu, sum > 0.0f);
+    int sel_lane;
+    bool take_last = false;
+    if (ballot != 0) {
+      sel_lane = __ffs(ballot) - 1;
+    } else {
+      sel_lane = posl ? 31 - __clz(posl) : 0;
+      take_last = true;
+    }
+    if (lane == sel_lane) {
+      double acc = base + (double)excl;
+      int found = -1, last = -1;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        if (w[t] > 0.0f) {
+          acc += (double)w[t];
+          last = t;
+          if (found < 0 && !take_last && acc > target) found = t;
+        }
+      }
+      const int t_sel = found >= 0 ? found : (last >= 0 ? last : 0);
+      float wsel = 0.0f;
+#pragma unroll
+      for (int t = 0; t < 8; ++t)
+        if (t == t_sel) wsel = w[t];
+      sc.tok = (c * 32 + lane) * 8 + t_sel;
+      sc.tok_w = wsel;
+    }
+  }
+  __syncthreads();
+  tok = sc.tok;
+  tok_w = sc.tok_w;
+}
+
+// weights of the eight entries of one vector under a row's statistics (value comparison: the
+// threshold is never +-0 here)
+__device__ __forceinline__ void rr_p_weights(const uint4 &v, float tau_f, float xmax, float scale, float *w) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t x = word_of(v, k);
+    const float a = __uint_as_float(x << 16), b = __uint_as_float(x & 0xFFFF0000u);
+    w[2 * k] = a >= tau_f ? exp2_neg((a - xmax) * scale) : 0.0f;
+    w[2 * k + 1] = b >= tau_f ? exp2_neg((b - xmax) * scale) : 0.0f;
+  }
+}
+
+struct RowFast {   // statistics of a row on this route
+  RowStats st;
+  float tau_f;
+  float d_weight;   // unnormalised weight of the entry at the draft token
+};
+
+// statistics of one row: 4 barriers.  false: general route.
+__device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d, int d_slot, int top_k, float inv_t,
+                              Scratch &sc, RowFast &out) {
+  using E = Elt<__nv_bfloat16>;
+  const int NV = V >> 3;
+  const bool need_select = top_k < V;
+  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select);
+  if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
+  uint32_t tau_key = 0;
+  if (need_select && !rr_select(row, NV, kmax, (uint32_t)top_k, sc, tau_key)) return false;
+  out.st.tau_key = tau_key;
+  out.st.xmax = E::val(E::unkey(kmax));
+  out.st.flags = 0;
+  out.tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
+  const float xmax = out.st.xmax, scale = inv_t * 1.4426950408889634f, tau_f = out.tau_f;
+  rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], tau_f, xmax, scale, w); }, NV, sc);
+  const float dv = E::val(sc.d_bits[d_slot]);
+  out.d_weight = (d >= 0 && dv >= tau_f) ? exp2_neg((dv - xmax) * scale) : 0.0f;
+  return true;
+}
+
+template <typename T>
+__device__ bool fast_row(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur, const T *qbase,
+                         const T *pbase, float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
+  return false;
+}
+
+template <>
+__device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
+                                        const __nv_bfloat16 *qbase, const __nv_bfloat16 *pbase, float inv_t, float u_acc,
+                                        float u_res, float u_draft, RowOut &ro) {
+  using E = Elt<__nv_bfloat16>;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
+  if (NV > 8 * (int)blockDim.x) return false;
+  const bool d_ok = d >= 0 && d < V;
+  const int dd = d_ok ? d : -1;
+  const float scale = inv_t * 1.4426950408889634f;
+  RegRow row;
+
+  // ---- the law of the draft
+  RowStats qs;
+  qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
+  float q_d;
+  if (kind == SJD_Q_ROW) {
+    if (p.prev_stats_valid) {
+      qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
+      if (qs.flags != 0 || !(qs.xmax > -FLT_MAX)) return false;
+      const uint32_t bits = d_ok ? (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(qbase) + d) : E::NEG_INF;
+      if (E::bad(bits)) return false;
+      q_d = d_ok ? (E::key(bits) >= qs.tau_key ? exp2_neg((E::val(bits) - qs.xmax) * scale) : 0.0f) / qs.z : 1.0f;
+    } else {
+      RowFast qfast;
+      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast)) return false;
+      const WarpPrefix wq = rr_prefix(NC, sc);
+      qs = qfast.st;
+      qs.z = (float)wq.total;
+      if (tid == 0) p.stats[cur ^ 1][r] = qs;
+      q_d = d_ok ? qfast.d_weight / qs.z : 1.0f;
+    }
+  } else if (kind == SJD_Q_UNIFORM) {
+    q_d = 1.0f / (float)V;
+  } else {
+    q_d = 1.0f;
+  }
+
+  // ---- this iteration's distribution
+  RowFast pfast;
+  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast)) return false;
+  const WarpPrefix wpp = rr_prefix(NC, sc);
+  RowStats ps = pfast.st;
+  ps.z = (float)wpp.total;
+  if (tid == 0) p.stats[cur][r] = ps;
+  const float p_d = d_ok ? pfast.d_weight / ps.z : 0.0f;
+  const float tau_p = pfast.tau_f, xmax_p = ps.xmax;
+
+  // ---- Eq. 1
+  float ratio;
+  if (q_d > 0.0f) ratio = p_d / q_d;
+  else ratio = p_d > 0.0f ? INFINITY : 0.0f;
+  const float thr = fminf(1.0f, ratio);
+  const bool accept = u_acc < thr;
+  uint32_t flags = 0;
+  if (thr < 1.0f && fabsf(u_acc - thr) < 1e-4f) flags |= SJD_FLAG_NEAR_TIE_ACCEPT;
+
+  // ---- Eq. 3: re-draft from p
+  auto p_w = [&](int i, float *w) { rr_p_weights(reg_slot(row, i), tau_p, xmax_p, scale, w); };
+  int redraft_tok;
+  float redraft_w;
+  rr_icdf(p_w, NV, wpp, u_draft, sc, redraft_tok, redraft_w);
+  const float redraft_p = redraft_w / ps.z;
+
+  // ---- Eq. 2: residual resample
+  int resample_tok = -1;
+  if (!accept) {
+    const float inv_zp = 1.0f / ps.z, inv_zq = 1.0f / qs.z;
+    const float q_uniform = 1.0f / (float)V;
+    const uint4 *qg = reinterpret_cast<const uint4 *>(qbase);
+    const int j0 = warp * 256 + lane;
+    const uint32_t tau_q = qs.tau_key;
+    const float xmax_q = qs.xmax;
+    auto r_w = [&](int i, float *w) {   // max(0, p - q) of the eight entries of slot i; q read through L2
+      const int j = j0 + i * 32;
+      const uint4 pv = reg_slot(row, i);
+      uint4 qv = make_uint4(0, 0, 0, 0);
+      if (kind == SJD_Q_ROW && j < NV) qv = __ldg(qg + j);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint32_t px = word_of(pv, k), qx = word_of(qv, k);
+        const uint32_t qk = key_pair(qx);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float pval = __uint_as_float(h ? px & 0xFFFF0000u : px << 16);
+          const float pp = (pval >= tau_p ? exp2_neg((pval - xmax_p) * scale) : 0.0f) * inv_zp;
+          float qq;
+          if (kind == SJD_Q_ROW) {
+            const uint32_t qkey = h ? qk >> 16 : qk & 0xFFFFu;
+            const float qval = __uint_as_float(h ? qx & 0xFFFF0000u : qx << 16);
+            qq = (qkey >= tau_q ? exp2_neg((qval - xmax_q) * scale) : 0.0f) * inv_zq;
+          } else if (kind == SJD_Q_UNIFORM) {
+            qq = q_uniform;
+          } else {
+            qq = (j * 8 + k * 2 + h == d) ? 1.0f : 0.0f;
+          }
+          w[2 * k + h] = j < NV ? fmaxf(0.0f, pp - qq) : 0.0f;
+        }
+      }
+    };
+    rr_chunk_sums(r_w, NV, sc);
+    WarpPrefix wr = rr_prefix(NC, sc);
+    float wsel;
+    if (wr.total > 0.0) {
+      rr_icdf(r_w, NV, wr, u_res, sc, resample_tok, wsel);
+    } else {
+      flags |= SJD_FLAG_RESIDUAL_EMPTY;
+      __syncthreads();
+      rr_chunk_sums(p_w, NV, sc);
+      wr = rr_prefix(NC, sc);
+      rr_icdf(p_w, NV, wr, u_res, sc, resample_tok, wsel);
+    }
+  }
+  ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
+  ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok; ro.flags = flags;
+  return true;
+}
+
 // Threshold + denominator of one row; leaves chunk sums of the row's weights in the scratch.
 template <typename T>
 __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t,
@@ -884,6 +1340,13 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
     const T *qbase = reinterpret_cast<const T *>(p.logits[cur ^ 1]) + ((size_t)b * p.W + qr) * p.V;
     const T *pbase = reinterpret_cast<const T *>(p.logits[cur]) + (size_t)r * p.V;
 
+    RowOut fast_out;
+    const bool fast_done = p.fast && (((uintptr_t)qbase | (uintptr_t)pbase) & 15u) == 0 &&
+                           fast_row<T>(p, sc, r, b, kind, d, qr, cur, qbase, pbase, inv_t, u_acc, u_res, u_draft, fast_out);
+    if (fast_done) {
+      if (tid == 0) p.row_out[r] = fast_out;
+    } else {
+    __syncthreads();
     // ---- the law of the draft
     Row<T> qrow;
     qrow.init(qbase, p.V);
@@ -968,6 +1431,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(
       ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok; ro.flags = flags;
       p.row_out[r] = ro;
     }
+    }   // general route
   }
 
   // ---- ticket: the last block of the sequence slides the window
