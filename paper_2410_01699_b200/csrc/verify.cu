@@ -31,6 +31,9 @@ namespace sjd {
 SJD_TIMELINE_TU(verify)
 namespace {
 
+#ifndef SJD_VERIFY_MIN_BLOCKS
+#define SJD_VERIFY_MIN_BLOCKS 3   // resident blocks per SM the 256-thread variant is compiled for
+#endif
 constexpr int kMaxChunks = 1024;   // 32 vectors of 16 bytes per chunk
 constexpr int kMaxThreads = 1024;
 
@@ -707,96 +710,46 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int 
   return kmax;
 }
 
-// exact key of the K-th largest entry.  Two barriers.  false: the threshold sits in a bin next to +-0.
+// Exact key of the K-th largest entry: one histogram pass over the distance (in bf16 codes) of every
+// entry below the row's maximum, exact for the 4095 codes next to the maximum (32 binades: for a
+// positive maximum, every positive value that matters) and lumped beyond; then every warp walks
+// the histogram from the top for itself.  One barrier.  false: the K-th largest lies in the lump
+// (or next to +-0), the general route decides.
 __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, Scratch &sc, uint32_t &tau_key) {
-  using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int j0 = warp * 256 + lane;
+  const uint32_t kmax2 = kmax | (kmax << 16);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     if (j0 + i * 32 < NV) {
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
-        const uint32_t kk = key_pair(word_of(row.v[i], w));
-        atomicAdd(&sc.hist12[(kk >> 4) & 0xFFFu], 1u);
-        atomicAdd(&sc.hist12[kk >> 20], 1u);
+        const uint32_t dist = kmax2 - key_pair(word_of(row.v[i], w));   // per half, no borrow: keys <= kmax
+        atomicAdd(&sc.hist12[min(dist & 0xFFFFu, 4095u)], 1u);
+        atomicAdd(&sc.hist12[min(dist >> 16, 4095u)], 1u);
       }
     }
   }
   __syncthreads();
-  // every warp walks the histogram from the row's top bin downwards, 512 bins at a time
-  uint32_t sel12 = 0, above = 0;
-  {
-    int hi = (int)(kmax >> 4);
-    uint32_t acc = 0;
-    bool found = false;
-    while (!found && hi >= 0) {
-      uint32_t c[16], t = 0;
+  uint32_t acc = 0;
+  for (int base = 0; base < 4096; base += 32) {   // 32 adjacent bins per step: conflict-free
+    const uint32_t c = sc.hist12[base + lane];
+    uint32_t incl = c;
 #pragma unroll
-      for (int jb = 0; jb < 16; ++jb) {
-        const int bin = hi - 16 * lane - jb;
-        c[jb] = bin >= 0 ? sc.hist12[bin] : 0u;
-        t += c[jb];
-      }
-      uint32_t incl = t;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      const uint32_t ballot = __ballot_sync(0xffffffffu, acc + incl >= K);
-      if (ballot) {
-        const int src = __ffs(ballot) - 1;
-        uint32_t a = acc + incl - t, s12 = 0, ab = 0;
-#pragma unroll
-        for (int jb = 0; jb < 16; ++jb) {
-          const uint32_t nxt = a + c[jb];
-          if (a < K && K <= nxt) {
-            s12 = (uint32_t)(hi - 16 * lane - jb);
-            ab = a;
-          }
-          a = nxt;
-        }
-        sel12 = __shfl_sync(0xffffffffu, s12, src);
-        above = __shfl_sync(0xffffffffu, ab, src);
-        found = true;
-      } else {
-        acc += __shfl_sync(0xffffffffu, incl, 31);
-        hi -= 512;
-      }
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
     }
-  }
-  if (sel12 == 0x7FFu || sel12 == 0x800u) return false;
-  const uint32_t kb_lo = sel12 << 4;
-  const uint32_t v_lo = E::unkey(kb_lo), v_hi = E::unkey(kb_lo | 15u);
-  const __nv_bfloat162 lo2 = as_bf2(v_lo | (v_lo << 16)), hi2 = as_bf2(v_hi | (v_hi << 16));
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    if (j0 + i * 32 < NV) {
-#pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const uint32_t x = word_of(row.v[i], w);
-        if (__hge2_mask(as_bf2(x), lo2) & __hle2_mask(as_bf2(x), hi2)) {   // rare: a few entries per warp
-          const uint32_t kk = key_pair(x);
-          if (((kk >> 4) & 0xFFFu) == sel12) atomicAdd(&sc.hist16[kk & 15u], 1u);
-          if ((kk >> 20) == sel12) atomicAdd(&sc.hist16[(kk >> 16) & 15u], 1u);
-        }
-      }
+    const uint32_t ballot = __ballot_sync(0xffffffffu, acc + incl >= K);
+    if (ballot) {
+      const uint32_t bin = (uint32_t)(base + __ffs(ballot) - 1);
+      if (bin >= 4095u) return false;
+      tau_key = kmax - bin;
+      return !(tau_key == 0x7FFFu || tau_key == 0x8000u);
     }
+    acc += __shfl_sync(0xffffffffu, incl, 31);
   }
-  __syncthreads();
-  {   // every warp: largest code b of the bin with (entries of the bin with code >= b) >= K - above
-    const uint32_t need = K - above;
-    uint32_t suf = lane < 16 ? sc.hist16[lane] : 0u;
-#pragma unroll
-    for (int o = 1; o < 16; o <<= 1) {
-      const uint32_t y = __shfl_down_sync(0xffffffffu, suf, o);
-      if (lane + o < 16) suf += y;
-    }
-    const uint32_t ballot = __ballot_sync(0xffffffffu, lane < 16 && suf >= need) & 0xFFFFu;
-    tau_key = kb_lo | (ballot ? (uint32_t)(31 - __clz(ballot)) : 0u);
-  }
-  return !(tau_key == 0x7FFFu || tau_key == 0x8000u);
+  return false;
 }
 
 // chunk sums of a weight functor evaluated on registers -> sc.chunk_sum.  One barrier.
@@ -971,14 +924,17 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d,
   const bool need_select = top_k < V;
   const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select);
   if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
+  SJD_TL(TL_VERIFY, 20, threadIdx.x == 0);   // row loaded, maximum known
   uint32_t tau_key = 0;
   if (need_select && !rr_select(row, NV, kmax, (uint32_t)top_k, sc, tau_key)) return false;
+  SJD_TL(TL_VERIFY, 23, threadIdx.x == 0);   // threshold known
   out.st.tau_key = tau_key;
   out.st.xmax = E::val(E::unkey(kmax));
   out.st.flags = 0;
   out.tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
   const float xmax = out.st.xmax, scale = inv_t * 1.4426950408889634f, tau_f = out.tau_f;
   rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], tau_f, xmax, scale, w); }, NV, sc);
+  SJD_TL(TL_VERIFY, 24, threadIdx.x == 0);   // chunk sums written
   const float dv = E::val(sc.d_bits[d_slot]);
   out.d_weight = (d >= 0 && dv >= tau_f) ? exp2_neg((dv - xmax) * scale) : 0.0f;
   return true;
@@ -1029,6 +985,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
     q_d = 1.0f;
   }
 
+  SJD_TL(TL_VERIFY, 10, tid == 0);
   // ---- this iteration's distribution
   RowFast pfast;
   if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast)) return false;
@@ -1038,6 +995,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   if (tid == 0) p.stats[cur][r] = ps;
   const float p_d = d_ok ? pfast.d_weight / ps.z : 0.0f;
   const float tau_p = pfast.tau_f, xmax_p = ps.xmax;
+  SJD_TL(TL_VERIFY, 11, tid == 0);
 
   // ---- Eq. 1
   float ratio;
@@ -1054,6 +1012,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   float redraft_w;
   rr_icdf(p_w, NV, wpp, u_draft, sc, redraft_tok, redraft_w);
   const float redraft_p = redraft_w / ps.z;
+  SJD_TL(TL_VERIFY, 12, tid == 0);
 
   // ---- Eq. 2: residual resample
   int resample_tok = -1;
@@ -1104,6 +1063,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
       rr_icdf(p_w, NV, wr, u_res, sc, resample_tok, wsel);
     }
   }
+  SJD_TL(TL_VERIFY, 13, tid == 0);
   ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
   ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok; ro.flags = flags;
   return true;
@@ -1309,7 +1269,7 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step) {
 
 // ------------------------------------------------------------------------------------ kernel
 template <typename T, int MAXT>
-__global__ void __launch_bounds__(MAXT, MAXT <= 256 ? 3 : 1) verify_rows_kernel(const VerifyParams p) {
+__global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1) verify_rows_kernel(const VerifyParams p) {
   using E = Elt<T>;
   extern __shared__ uint4 dyn_smem[];
   __shared__ Scratch sc;
