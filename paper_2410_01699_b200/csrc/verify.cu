@@ -677,7 +677,8 @@ __device__ __forceinline__ uint4 reg_slot(const RegRow &r, int i) {   // i is wa
 
 // load + maximum; publishes the entry at index d (if any) in sc.d_bits.  One barrier.  Returns the
 // block-wide maximum key; 0xFFFF if the row holds a NaN.
-__device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int d_slot, Scratch &sc, bool zero_hist) {
+__device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int d_slot, Scratch &sc, bool zero_hist,
+                                uint4 *stash) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
   const int j0 = warp * 256 + lane;
@@ -694,6 +695,7 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int 
   for (int i = 0; i < 8; ++i) {
 #pragma unroll
     for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(row.v[i], w)));
+    if (stash && j0 + i * 32 < NV) stash[j0 + i * 32] = row.v[i];
     if (d >= 0 && (d >> 3) == j0 + i * 32) {   // this thread holds entry d
       const uint32_t wd = word_of(row.v[i], (d >> 1) & 3);
       sc.d_bits[d_slot] = (d & 1) ? wd >> 16 : wd & 0xFFFFu;
@@ -918,11 +920,11 @@ struct RowFast {   // statistics of a row on this route
 
 // statistics of one row: 4 barriers.  false: general route.
 __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d, int d_slot, int top_k, float inv_t,
-                              Scratch &sc, RowFast &out) {
+                              Scratch &sc, RowFast &out, uint4 *stash) {
   using E = Elt<__nv_bfloat16>;
   const int NV = V >> 3;
   const bool need_select = top_k < V;
-  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select);
+  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select, stash);
   if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
   SJD_TL(TL_VERIFY, 20, threadIdx.x == 0);   // row loaded, maximum known
   uint32_t tau_key = 0;
@@ -941,19 +943,19 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d,
 }
 
 template <typename T>
-__device__ bool fast_row(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur, const T *qbase,
-                         const T *pbase, float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
+__device__ bool fast_row(const VerifyParams &p, Scratch &sc, uint4 *stage, int r, int b, int kind, int d, int qr, int cur,
+                         const T *qbase, const T *pbase, float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
   return false;
 }
 
 template <>
-__device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
-                                        const __nv_bfloat16 *qbase, const __nv_bfloat16 *pbase, float inv_t, float u_acc,
-                                        float u_res, float u_draft, RowOut &ro) {
+__device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint4 *stage, int r, int b, int kind, int d,
+                                        int qr, int cur, const __nv_bfloat16 *qbase, const __nv_bfloat16 *pbase,
+                                        float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
-  if (NV > 8 * (int)blockDim.x) return false;
+  if (NV > 8 * (int)blockDim.x || !stage) return false;
   const bool d_ok = d >= 0 && d < V;
   const int dd = d_ok ? d : -1;
   const float scale = inv_t * 1.4426950408889634f;
@@ -969,10 +971,16 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
       if (qs.flags != 0 || !(qs.xmax > -FLT_MAX)) return false;
       const uint32_t bits = d_ok ? (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(qbase) + d) : E::NEG_INF;
       if (E::bad(bits)) return false;
+      // the residual of Eq. 2 needs the whole q row: copy it to shared memory in the background
+      for (int j = tid; j < NV; j += blockDim.x)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(stage + j)),
+                     "l"(reinterpret_cast<const uint4 *>(qbase) + j)
+                     : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
       q_d = d_ok ? (E::key(bits) >= qs.tau_key ? exp2_neg((E::val(bits) - qs.xmax) * scale) : 0.0f) / qs.z : 1.0f;
     } else {
       RowFast qfast;
-      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast)) return false;
+      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, stage)) return false;
       const WarpPrefix wq = rr_prefix(NC, sc);
       qs = qfast.st;
       qs.z = (float)wq.total;
@@ -988,7 +996,12 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   SJD_TL(TL_VERIFY, 10, tid == 0);
   // ---- this iteration's distribution
   RowFast pfast;
-  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast)) return false;
+  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast, nullptr)) {
+    asm volatile("cp.async.wait_all;" ::: "memory");   // the general route reuses the staging buffer
+    return false;
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");   // this thread's copies of the q row have landed; the barriers
+                                                     // of the re-draft below make them visible to the block
   const WarpPrefix wpp = rr_prefix(NC, sc);
   RowStats ps = pfast.st;
   ps.z = (float)wpp.total;
@@ -1019,7 +1032,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   if (!accept) {
     const float inv_zp = 1.0f / ps.z, inv_zq = 1.0f / qs.z;
     const float q_uniform = 1.0f / (float)V;
-    const uint4 *qg = reinterpret_cast<const uint4 *>(qbase);
+    const uint4 *qg = stage;   // the q row, staged above
     const int j0 = warp * 256 + lane;
     const uint32_t tau_q = qs.tau_key;
     const float xmax_q = qs.xmax;
@@ -1027,7 +1040,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
       const int j = j0 + i * 32;
       const uint4 pv = reg_slot(row, i);
       uint4 qv = make_uint4(0, 0, 0, 0);
-      if (kind == SJD_Q_ROW && j < NV) qv = __ldg(qg + j);
+      if (kind == SJD_Q_ROW && j < NV) qv = qg[j];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const uint32_t px = word_of(pv, k), qx = word_of(qv, k);
@@ -1168,31 +1181,42 @@ __device__ RowStats row_statistics_any(Row<T> &row, uint4 *stage, Scratch &sc, i
 }
 
 // ------------------------------------------------------------------------------------ finalize
-__device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step) {
+// Run by every thread of the last block of sequence b: accept scan (warp 0), then the commit, the
+// window slide and the next inputs in parallel over the window slots.
+__device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, Scratch &sc) {
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
   const int W = p.W;
   const int w_eff = p.w_eff ? p.w_eff[b] : W;
   const RowOut *ro = p.row_out + (size_t)b * W;
   const int32_t *old_draft = p.draft + (size_t)b * W;
   const sjd_step_out &o = p.out;
-  uint32_t flags = 0;
-  int a = w_eff;
-  for (int k = 0; k < w_eff; ++k) {
-    const uint32_t rf = __ldcg(&ro[k].flags);
-    flags |= rf & SJD_FLAG_NONFINITE;
-    if (a == w_eff) {
-      flags |= rf & SJD_FLAG_NEAR_TIE_ACCEPT;
-      if (!__ldcg(&ro[k].accept)) {
-        a = k;
-        flags |= rf & SJD_FLAG_RESIDUAL_EMPTY;
-      }
+  if (tid < 32) {
+    int first = w_eff;
+    for (int k = lane; k < w_eff; k += 32)
+      if (!__ldcg(&ro[k].accept)) first = min(first, k);
+    const int a = __reduce_min_sync(0xffffffffu, first);
+    uint32_t fl = 0;
+    for (int k = lane; k < w_eff; k += 32) {
+      const uint32_t rf = __ldcg(&ro[k].flags);
+      fl |= rf & SJD_FLAG_NONFINITE;
+      if (k <= a) fl |= rf & SJD_FLAG_NEAR_TIE_ACCEPT;   // the rows the left-to-right scan looks at
+      if (k == a) fl |= rf & SJD_FLAG_RESIDUAL_EMPTY;
+    }
+    fl = __reduce_or_sync(0xffffffffu, fl);
+    if (lane == 0) {
+      sc.sel_chunk = a;
+      sc.sel_bin = fl;
     }
   }
+  __syncthreads();
+  const int a = sc.sel_chunk;
+  uint32_t flags = sc.sel_bin;
   const int m = (a < w_eff) ? a + 1 : w_eff;
   const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
   const int n2 = base + m;
 
   // fixed tokens: accepted drafts, then the resampled one
-  for (int i = 0; i < W; ++i) {
+  for (int i = tid; i < W; i += nt) {
     int tok = -1;
     if (i < a) tok = old_draft[i];
     else if (i == a && a < w_eff) tok = __ldcg(&ro[a].resample_tok);
@@ -1214,7 +1238,11 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step) {
   int32_t *nk = p.e2e ? p.st.q_kind + (size_t)b * W : nullptr;
   int32_t *nr = p.e2e ? p.st.q_row + (size_t)b * W : nullptr;
   float *nq = p.e2e ? p.st.q_draft + (size_t)b * W : nullptr;
-  for (int s = 0; s < W; ++s) {
+  // A copied slot may read a slot filled just before it (and a token fixed above), so the copy
+  // initialisations fill the window in order on one thread; everything else goes slot-parallel.
+  const bool serial = p.e2e && p.st.init != SJD_INIT_RANDOM;
+  if (serial) __syncthreads();   // the fixed tokens above are read below
+  for (int s = serial ? 0 : tid; s < W && (!serial || tid == 0); s += serial ? 1 : nt) {
     int tok = -1, kind = -1, qrow = 0;
     float q = 0.0f;
     if (s < kept) {
@@ -1250,21 +1278,26 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step) {
     if (o.q_kind) o.q_kind[(size_t)b * W + s] = kind;
     if (o.q_draft) o.q_draft[(size_t)b * W + s] = q;
   }
+  __syncthreads();   // the new window and the fixed tokens are read below
   if (p.e2e) {
-    p.st.n[b] = n2;
-    p.st.w_eff[b] = w2;
     int32_t *it = p.st.in_tok + (size_t)b * W;
     int32_t *ip = p.st.in_pos + (size_t)b * W;
-    for (int k = 0; k < W; ++k) {
+    for (int k = tid; k < W; k += nt) {
       const bool act = k < w2;
       it[k] = act ? (k == 0 ? p.st.committed[(size_t)b * p.st.max_seq + n2 - 1] : nd[k - 1]) : 0;
       ip[k] = act ? n2 - 1 + k : -1;
     }
   }
-  if (o.n_accepted) o.n_accepted[b] = a;
-  if (o.n_committed) o.n_committed[b] = m;
-  if (o.total_committed) o.total_committed[b] = n2;
-  if (o.flags) o.flags[b] = flags;
+  if (tid == 0) {
+    if (p.e2e) {
+      p.st.n[b] = n2;
+      p.st.w_eff[b] = w2;
+    }
+    if (o.n_accepted) o.n_accepted[b] = a;
+    if (o.n_committed) o.n_committed[b] = m;
+    if (o.total_committed) o.total_committed[b] = n2;
+    if (o.flags) o.flags[b] = flags;
+  }
 }
 
 // ------------------------------------------------------------------------------------ kernel
@@ -1302,7 +1335,8 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
 
     RowOut fast_out;
     const bool fast_done = p.fast && (((uintptr_t)qbase | (uintptr_t)pbase) & 15u) == 0 &&
-                           fast_row<T>(p, sc, r, b, kind, d, qr, cur, qbase, pbase, inv_t, u_acc, u_res, u_draft, fast_out);
+                           fast_row<T>(p, sc, stage, r, b, kind, d, qr, cur, qbase, pbase, inv_t, u_acc, u_res, u_draft,
+                                       fast_out);
     if (fast_done) {
       if (tid == 0) p.row_out[r] = fast_out;
     } else {
@@ -1400,18 +1434,21 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     __threadfence();
     const int old = atomicAdd(&p.seq_counter[b], 1);
     sc.is_last = (old == p.W - 1);
-    if (sc.is_last) {
-      __threadfence();
-      SJD_TL(TL_VERIFY, 14, true);
-      finalize_sequence(p, b, step);
-      SJD_TL(TL_VERIFY, 15, true);
-      p.seq_counter[b] = 0;
-      __threadfence();
-      const int done = atomicAdd(p.done_counter, 1);
-      if (done == p.B - 1) {  // every block has read the step index by now
-        *p.done_counter = 0;
-        if (p.step_ptr) *p.step_ptr = step + 1u;
-      }
+  }
+  __syncthreads();
+  if (!sc.is_last) return;
+  __threadfence();
+  SJD_TL(TL_VERIFY, 14, tid == 0);
+  finalize_sequence(p, b, step, sc);
+  SJD_TL(TL_VERIFY, 15, tid == 0);
+  __syncthreads();
+  if (tid == 0) {
+    p.seq_counter[b] = 0;
+    __threadfence();
+    const int done = atomicAdd(p.done_counter, 1);
+    if (done == p.B - 1) {  // every block has read the step index by now
+      *p.done_counter = 0;
+      if (p.step_ptr) *p.step_ptr = step + 1u;
     }
   }
 }
