@@ -15,12 +15,15 @@
 // Logits are read once from HBM; later passes hit the shared-memory copy.  Rows too large for
 // shared memory are re-read through L2.  No floating-point atomics: every sum has a fixed order.
 //
-// bf16 rows of at most 65536 entries take a leaner route through step 2: the block holds the row
-// in registers (eight 16-byte vectors per thread), finds the maximum with packed bf16 instructions,
-// histograms the top 12 key bits once, resolves the last 4 bits on the few entries of the selected
-// bin, and forms the chunk sums from registers.  Rows with NaN/+inf, without a finite entry, or
-// whose threshold lies next to +-0 (where bf16 comparison and key order differ) use the general
-// route above; both routes produce the same threshold and the same weights.
+// bf16 rows of at most 65536 entries take a leaner route (fast_row): the block holds the row in
+// registers (eight 16-byte vectors per thread), finds the maximum with packed bf16 instructions,
+// histograms once the distance of every entry below the maximum in bf16 codes (exact for the 4095
+// codes next to it), walks that histogram per warp to the exact threshold, and forms chunk sums,
+// prefix and inverse-CDF searches from registers with every table search done by each warp for itself
+// (about a dozen block barriers per row).  Rows with NaN/+inf, without a finite entry, with the
+// K-th largest entry more than 4095 codes below the maximum (e.g. a positive maximum and a negative
+// threshold) or next to +-0 use the general route above; both routes produce the same threshold and
+// the same weights.
 #include <float.h>
 
 #include <type_traits>
@@ -94,8 +97,7 @@ struct Elt<__nv_bfloat16> {
 struct Scratch {
   double chunk_excl[kMaxChunks + 1];  // exclusive prefix of chunk sums; [NC] = total
   float chunk_sum[kMaxChunks];
-  uint32_t hist12[4096];              // register-resident route: histogram of the top 12 key bits
-  uint32_t hist16[16];                //   and of the last 4 bits inside the selected bin
+  uint32_t hist12[4096];              // register-resident route: histogram of code distances below the row maximum
   uint32_t hist[256];
   uint32_t redu[32];
   uint32_t d_bits[2];                 // register-resident route: bits of the q / p row's entry at the draft token
@@ -477,7 +479,7 @@ __device__ void sample_icdf(const F &f, int NV, int off, Scratch &sc, float u) {
   __syncthreads();
 }
 
-// ------------------------------------------------------------------------------------ register-resident route
+// ------------------------------------------------------------------------------------ packed bf16 helpers
 __device__ __forceinline__ __nv_bfloat162 as_bf2(uint32_t w) { return *reinterpret_cast<__nv_bfloat162 *>(&w); }
 // order-preserving keys of both halves of a packed bf16 pair (same map as Elt<bf16>::key per half)
 __device__ __forceinline__ uint32_t key_pair(uint32_t w) {
@@ -486,180 +488,10 @@ __device__ __forceinline__ uint32_t key_pair(uint32_t w) {
 }
 __device__ __forceinline__ uint32_t word_of(const uint4 &v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 
-// Threshold, maximum and denominator of a 16-byte aligned bf16 row of NV <= 8 * blockDim.x vectors
-// held in registers: warp w owns chunks 8w .. 8w+7 (32 vectors each, the chunks of chunk_sums), lane
-// l holds vector l of each.  Leaves the staged copy, the chunk sums and their prefix exactly as
-// row_statistics does.  Returns false (block-uniform, nothing published) for rows it does not cover.
-__device__ bool fast_row_statistics(Row<__nv_bfloat16> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t,
-                                    PRowWeights<__nv_bfloat16> &f, RowStats &st) {
-  using E = Elt<__nv_bfloat16>;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
-  const int NV = row.NV, NC = (NV + 31) >> 5;
-  const bool need_select = top_k < row.V;
-  if (need_select)
-    for (int i = tid; i < 4096; i += nt) sc.hist12[i] = 0;
-  if (tid < 16) sc.hist16[tid] = 0;
-
-  // ---- load, stage, maximum
-  uint4 v[8];
-  const uint4 *g = reinterpret_cast<const uint4 *>(row.g);
-  const int j0 = warp * 256 + lane;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int j = j0 + i * 32;
-    v[i] = j < NV ? __ldg(g + j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-  }
-  __nv_bfloat162 m2 = as_bf2(v[0].x);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int j = j0 + i * 32;
-    if (j < NV) stage[j] = v[i];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(v[i], w)));
-  }
-  const __nv_bfloat16 m1 = __hmax_nan(__low2bfloat16(m2), __high2bfloat16(m2));
-  const uint32_t mbits = (uint32_t)__bfloat16_as_ushort(m1);
-  uint32_t kmax = (mbits & 0x7FFFu) > 0x7F80u ? 0xFFFFu : E::key(mbits);   // NaN sorts above everything
-  kmax = __reduce_max_sync(0xffffffffu, kmax);
-  if (lane == 0) sc.redu[warp] = kmax;
-  __syncthreads();
-  kmax = 0;
-  for (int w = 0; w < nw; ++w) kmax = max(kmax, sc.redu[w]);
-  // NaN or +inf somewhere, or no finite entry at all: the general route sanitises and flags
-  if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
-  row.s = stage;
-  SJD_TL(TL_VERIFY, 20, tid == 0);   // row loaded, maximum known
-
-  // ---- threshold
-  uint32_t tau_key = 0;
-  if (need_select) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (j0 + i * 32 < NV) {
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const uint32_t kk = key_pair(word_of(v[i], w));
-          atomicAdd(&sc.hist12[(kk >> 4) & 0xFFFu], 1u);
-          atomicAdd(&sc.hist12[kk >> 20], 1u);
-        }
-      }
-    }
-    __syncthreads();
-    SJD_TL(TL_VERIFY, 21, tid == 0);   // 12-bit histogram complete
-    for (int c = tid; c < 256; c += nt) {
-      uint32_t t = 0;
-#pragma unroll
-      for (int b = 0; b < 16; ++b) t += sc.hist12[c * 16 + b];
-      sc.hist[c] = t;
-    }
-    __syncthreads();
-    if (tid < 32) find_bin(sc, (uint32_t)top_k);
-    __syncthreads();
-    if (tid == 0) {   // the 16 fine bins of the selected coarse bin, from the top
-      const uint32_t cb = sc.sel_bin, k = (uint32_t)top_k;
-      uint32_t acc = sc.count_above, sel = cb * 16, above = acc;
-      for (int b = 15; b >= 0; --b) {
-        const uint32_t nxt = acc + sc.hist12[cb * 16 + b];
-        if (acc < k && k <= nxt) {
-          sel = cb * 16 + b;
-          above = acc;
-          break;
-        }
-        acc = nxt;
-      }
-      sc.sel_bin = sel;
-      sc.count_above = above;
-    }
-    __syncthreads();
-    const uint32_t sel12 = sc.sel_bin, above = sc.count_above;
-    SJD_TL(TL_VERIFY, 22, tid == 0);   // bin selected
-    if (sel12 == 0x7FFu || sel12 == 0x800u) {   // the bins of -0 and +0: bf16 comparison cannot tell them apart
-      __syncthreads();
-      return false;
-    }
-    // entries inside the selected bin: found with two packed comparisons per word, then counted by
-    // their last 4 key bits
-    const uint32_t kb_lo = sel12 << 4;
-    const uint32_t v_lo = E::unkey(kb_lo), v_hi = E::unkey(kb_lo | 15u);
-    const __nv_bfloat162 lo2 = as_bf2(v_lo | (v_lo << 16)), hi2 = as_bf2(v_hi | (v_hi << 16));
-    uint32_t cand = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (j0 + i * 32 < NV) {
-#pragma unroll
-        for (int w = 0; w < 4; ++w) {
-          const __nv_bfloat162 x = as_bf2(word_of(v[i], w));
-          if (__hge2_mask(x, lo2) & __hle2_mask(x, hi2)) cand |= 1u << (i * 4 + w);
-        }
-      }
-    }
-    const uint32_t *stage_w = reinterpret_cast<const uint32_t *>(stage);
-    while (cand) {
-      const int idx = __ffs(cand) - 1;
-      cand &= cand - 1;
-      const uint32_t kk = key_pair(stage_w[(size_t)(j0 + (idx >> 2) * 32) * 4 + (idx & 3)]);
-      if (((kk >> 4) & 0xFFFu) == sel12) atomicAdd(&sc.hist16[kk & 15u], 1u);
-      if ((kk >> 20) == sel12) atomicAdd(&sc.hist16[(kk >> 16) & 15u], 1u);
-    }
-    __syncthreads();
-    if (tid == 0) {
-      const uint32_t need = (uint32_t)top_k - above;   // rank inside the bin, from the top
-      uint32_t acc = 0, t = kb_lo;
-      for (int b = 15; b >= 0; --b) {
-        acc += sc.hist16[b];
-        if (acc >= need) {
-          t = kb_lo | (uint32_t)b;
-          break;
-        }
-      }
-      sc.sel_bin = t;
-    }
-    __syncthreads();
-    tau_key = sc.sel_bin;
-    SJD_TL(TL_VERIFY, 23, tid == 0);   // threshold known
-  }
-
-  // ---- weights and chunk sums from registers
-  st.tau_key = tau_key;
-  st.xmax = E::val(E::unkey(kmax));
-  st.flags = 0;
-  f.row = row;
-  f.pw.init(st, inv_t);
-  const float tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
-  const float xmax = st.xmax, scale = f.pw.scale;
-  float s[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    float acc = 0.0f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const uint32_t x = word_of(v[i], w);
-      const float a = __uint_as_float(x << 16), b = __uint_as_float(x & 0xFFFF0000u);
-      acc += a >= tau_f ? exp2_neg((a - xmax) * scale) : 0.0f;
-      acc += b >= tau_f ? exp2_neg((b - xmax) * scale) : 0.0f;
-    }
-    s[i] = acc;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
-  }
-  if (lane == 0) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
-  }
-  __syncthreads();
-  SJD_TL(TL_VERIFY, 24, tid == 0);   // chunk sums written
-  chunk_prefix(NC, sc);
-  st.z = (float)sc.chunk_excl[NC];
-  return true;
-}
-
 // ------------------------------------------------------------------------------------ register-resident row, few barriers
 // The whole treatment of one window row (Eqs. 1-3) for bf16 rows a block can hold in registers, laid
-// out as in fast_row_statistics.  Every search over shared tables (histogram bins, chunk prefix) is done
+// out warp by warp: warp w owns chunks 8w .. 8w+7 (32 vectors each, the chunks of chunk_sums), lane l
+// holds vector l of each.  Every search over shared tables (histogram bins, chunk prefix) is done
 // by each warp for itself instead of by one warp between two barriers, so a row costs about a dozen
 // block barriers.  Returns false (block-uniform) when the row needs the general route; nothing it
 // has published by then differs from what that route writes.
@@ -689,7 +521,6 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int 
   }
   if (zero_hist)
     for (int i = tid; i < 4096; i += nt) sc.hist12[i] = 0;
-  if (tid < 16) sc.hist16[tid] = 0;
   __nv_bfloat162 m2 = as_bf2(row.v[0].x);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -1100,86 +931,6 @@ __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int t
   return st;
 }
 
-// Chunk sums (and their prefix) of the residual weights max(0, p - q) of Eq. 2 with the p row read from
-// its staged copy and the q row from global memory (it was read moments ago: L2), eight vectors per
-// thread in the layout of fast_row_statistics.  Element for element the same arithmetic as
-// ResidualWeights, so sample_icdf may follow with that functor.  Requires both rows 16-byte aligned,
-// free of non-finite entries and not degenerate.
-__device__ void fast_residual_sums(const ResidualWeights<__nv_bfloat16> &rf, Scratch &sc) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int NV = rf.prow.NV, NC = (NV + 31) >> 5;
-  const uint4 *pg = rf.prow.s;
-  const uint4 *qg = reinterpret_cast<const uint4 *>(rf.qrow.g);
-  const int j0 = warp * 256 + lane;
-  const float q_uniform = 1.0f / (float)rf.V;
-  float s[8];
-  uint4 qall[8];   // every load of the q row in flight before the first use
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int j = j0 + i * 32;
-    qall[i] = (rf.kind == SJD_Q_ROW && j < NV) ? __ldg(qg + j) : make_uint4(0, 0, 0, 0);
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int j = j0 + i * 32;
-    float acc = 0.0f;
-    if (j < NV) {
-      const uint4 pv = pg[j];
-      const uint4 qv = qall[i];
-#pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const uint32_t px = word_of(pv, w), qx = word_of(qv, w);
-        const uint32_t pk = key_pair(px), qk = key_pair(qx);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint32_t pkey = h ? pk >> 16 : pk & 0xFFFFu;
-          const float pval = __uint_as_float(h ? px & 0xFFFF0000u : px << 16);
-          const float pp = (pkey >= rf.pw.tau_key ? exp2_neg((pval - rf.pw.xmax) * rf.pw.scale) : 0.0f) * rf.inv_zp;
-          float qq;
-          if (rf.kind == SJD_Q_ROW) {
-            const uint32_t qkey = h ? qk >> 16 : qk & 0xFFFFu;
-            const float qval = __uint_as_float(h ? qx & 0xFFFF0000u : qx << 16);
-            qq = (qkey >= rf.qw.tau_key ? exp2_neg((qval - rf.qw.xmax) * rf.qw.scale) : 0.0f) * rf.inv_zq;
-          } else if (rf.kind == SJD_Q_UNIFORM) {
-            qq = q_uniform;
-          } else {
-            qq = (j * 8 + w * 2 + h == rf.draft) ? 1.0f : 0.0f;
-          }
-          acc += fmaxf(0.0f, pp - qq);
-        }
-      }
-    }
-    s[i] = acc;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
-  }
-  if (lane == 0) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
-  }
-  __syncthreads();
-  chunk_prefix(NC, sc);
-}
-
-// row_statistics through whichever route covers the row
-template <typename T>
-__device__ RowStats row_statistics_any(Row<T> &row, uint4 *stage, Scratch &sc, int top_k, float inv_t, PRowWeights<T> &f,
-                                       bool fast) {
-  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-    if (fast && stage && row.off == 0 && (row.V & 7) == 0 && row.NV <= 8 * (int)blockDim.x) {
-      RowStats st;
-      if (fast_row_statistics(row, stage, sc, top_k, inv_t, f, st)) return st;
-      row.s = nullptr;
-      __syncthreads();
-    }
-  }
-  return row_statistics<T>(row, stage, sc, top_k, inv_t, f);
-}
-
 // ------------------------------------------------------------------------------------ finalize
 // Run by every thread of the last block of sequence b: accept scan (warp 0), then the commit, the
 // window slide and the next inputs in parallel over the window slots.
@@ -1352,7 +1103,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
       if (p.prev_stats_valid) {
         qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
       } else {
-        qs = row_statistics_any<T>(qrow, stage, sc, p.top_k, inv_t, qf, p.fast != 0);
+        qs = row_statistics<T>(qrow, stage, sc, p.top_k, inv_t, qf);
         if (tid == 0) p.stats[cur ^ 1][r] = qs;
         __syncthreads();
         qrow.s = nullptr;  // the staging buffer is about to be reused
@@ -1371,7 +1122,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     Row<T> prow;
     prow.init(pbase, p.V);
     PRowWeights<T> pf;
-    const RowStats ps = row_statistics_any<T>(prow, stage, sc, p.top_k, inv_t, pf, p.fast != 0);
+    const RowStats ps = row_statistics<T>(prow, stage, sc, p.top_k, inv_t, pf);
     if (tid == 0) p.stats[cur][r] = ps;
     const float p_d = d_ok ? pf.pw.one(prow.element(d), d) / ps.z : 0.0f;
 
@@ -1400,14 +1151,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
       rf.inv_zp = 1.0f / ps.z; rf.inv_zq = 1.0f / qs.z;
       rf.kind = kind; rf.draft = d; rf.V = p.V;
       if (kind != SJD_Q_ROW) rf.qw = pf.pw;
-      bool from_registers = false;
-      if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-        from_registers = p.fast && prow.s && prow.off == 0 && (p.V & 7) == 0 && prow.NV <= 8 * (int)blockDim.x &&
-                         !pf.pw.degenerate &&
-                         (kind != SJD_Q_ROW || (qrow.off == 0 && qs.flags == 0 && !qf.pw.degenerate));
-        if (from_registers) fast_residual_sums(rf, sc);
-      }
-      if (!from_registers) chunk_sums<E::VEC>(rf, prow.NV, sc);
+      chunk_sums<E::VEC>(rf, prow.NV, sc);
       if (sc.chunk_excl[(prow.NV + 31) >> 5] > 0.0) {
         sample_icdf<E::VEC>(rf, prow.NV, prow.off, sc, u_res);
       } else {
