@@ -101,6 +101,31 @@ def test_verify_temperature_and_ties():
     _check_case(case)
 
 
+@pytest.mark.parametrize("shift,top_k", [
+    (-9.0, 2000),    # positive maximum, negative threshold: more than 4095 bf16 codes apart (general route)
+    (-30.0, 2000),   # every logit negative: maximum and threshold within a few binades (register route)
+    (0.0, 8000),     # half the row kept: threshold around zero
+    (0.0, 16384),    # top_k == V: no filtering on the register route
+])
+def test_verify_threshold_far_from_the_maximum(shift, top_k):
+    """The register-resident route counts entries by their distance below the row maximum and hands rows
+    whose threshold is out of that reach to the general route; both must agree with the checker."""
+    case = make_verify_case(2, window=6, vocab=16384, top_k=top_k, seed=31)
+    case.logits_cur = round_bf16(case.logits_cur + np.float32(shift))
+    case.logits_prev = round_bf16(case.logits_prev + np.float32(shift))
+    _check_case(case, max_flag_frac=0.06)
+
+
+def test_verify_zeros_at_the_threshold():
+    """Exact zeros of both signs around the top-k threshold (bf16 comparison cannot order +0 and -0, the
+    order-preserving keys can): such rows take the general route."""
+    case = make_verify_case(2, window=4, vocab=8192, top_k=3000, seed=33)
+    for arr in (case.logits_cur, case.logits_prev):
+        small = np.abs(arr) < 0.35
+        arr[small] = np.where(arr[small] < 0, np.float32(-0.0), np.float32(0.0))
+    _check_case(case, max_flag_frac=0.06)
+
+
 def test_verify_identical_rows_accept_everything():
     """p == q bit for bit: every ratio is 1 and every draft is accepted for any uniform."""
     case = make_verify_case(2, window=12, vocab=4096, top_k=100, seed=3)
