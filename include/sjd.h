@@ -233,8 +233,9 @@ int sjd_verify_static(int batch, int window, int vocab, int logits_dtype, const 
  *     out[m][n] (+)= sum_k x[m][k] * w[n][k]      (fp32 accumulation)
  * x: device fp32 [M][K] (split internally into bf16 hi + lo parts, so activations keep ~16 bits of
  * mantissa); w: device bf16 [N][K]; out: device fp32 [M][N], overwritten (accumulate = 0) or added
- * to (accumulate != 0).  Covered shapes: 1 <= M <= 128, N a multiple of 128, K a multiple of 64,
- * compute capability 10.x; anything else returns SJD_ERR_UNSUPPORTED (sjd_step then uses its generic
+ * to (accumulate != 0).  Covered shapes: 1 <= M <= 1024 (above 128 rows the launch is cut into token
+ * slabs of at most 128 rows that share each weight tile through L2), N a multiple of 128, K a
+ * multiple of 64, compute capability 10.x; anything else returns SJD_ERR_UNSUPPORTED (sjd_step then uses its generic
  * kernel).  ws: device scratch of sjd_gemm_workspace_bytes(M, N, K), 256-byte aligned; after the stream
  * has drained its first int32 is 0, or non-zero if a bounded device-side wait ran out.
  * Errors: BAD_ARG, UNSUPPORTED, CAPACITY (ws too small), CUDA.
