@@ -174,19 +174,26 @@ __global__ void attention_combine_kernel(const float *__restrict__ partial, cons
     }
     return;
   }
-  float gmax = -INFINITY;
-  for (int s = 0; s < splits; ++s) gmax = fmaxf(gmax, src[(size_t)s * (hd + 2)]);
-  float denom = 0.0f;
-  for (int s = 0; s < splits; ++s) {
-    const float ms = src[(size_t)s * (hd + 2)];
-    if (ms > -INFINITY) denom += src[(size_t)s * (hd + 2) + 1] * expf(ms - gmax);
+  // heads of the records once (one thread per key range), then the weights from shared memory: the
+  // loads over the records below do not wait on one another
+  __shared__ float s_m[64], s_l[64], s_w[64];
+  const int ns = splits < 64 ? splits : 64;
+  if ((int)threadIdx.x < ns) {
+    s_m[threadIdx.x] = src[(size_t)threadIdx.x * (hd + 2)];
+    s_l[threadIdx.x] = src[(size_t)threadIdx.x * (hd + 2) + 1];
   }
+  __syncthreads();
+  float gmax = -INFINITY;
+  for (int s = 0; s < ns; ++s) gmax = fmaxf(gmax, s_m[s]);
+  float denom = 0.0f;
+  for (int s = 0; s < ns; ++s)
+    if (s_m[s] > -INFINITY) denom += s_l[s] * expf(s_m[s] - gmax);
+  if ((int)threadIdx.x < ns) s_w[threadIdx.x] = s_m[threadIdx.x] > -INFINITY ? expf(s_m[threadIdx.x] - gmax) : 0.0f;
+  __syncthreads();
   for (int d = threadIdx.x; d < hd; d += blockDim.x) {
     float acc = 0.0f;
-    for (int s = 0; s < splits; ++s) {
-      const float ms = src[(size_t)s * (hd + 2)];
-      if (ms > -INFINITY) acc += src[(size_t)s * (hd + 2) + 2 + d] * expf(ms - gmax);
-    }
+#pragma unroll 4
+    for (int s = 0; s < ns; ++s) acc += src[(size_t)s * (hd + 2) + 2 + d] * s_w[s];
     const float v = denom > 0.0f ? acc / denom : 0.0f;
     dst[d] = v;
     if (hilo.base) {

@@ -78,7 +78,8 @@ __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restric
 }
 
 // q,k,v = scale * sum of the QKV planes; rotate q and k (pairs i, i + hd/2) by the row's absolute
-// position; q -> fp32 [M][H*hd]; k, v -> cache row in_pos[m].  One block per (row, head slot).
+// position; q -> fp32 [M][H*hd]; k, v -> cache row in_pos[m].  64 threads per (row, head slot), four
+// slots per block.
 template <typename T>
 __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__restrict__ in_pos,
                                   const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
@@ -87,9 +88,10 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   SJD_TL(TL_QKV, 0, threadIdx.x == 0);
   pdl_wait();
   SJD_TL(TL_QKV, 1, threadIdx.x == 0);
-  const int m = blockIdx.x, slot = blockIdx.y;
+  const int m = blockIdx.x, lt = threadIdx.x & 63;
+  const int slot = blockIdx.y * (blockDim.x >> 6) + (threadIdx.x >> 6);
   const int pos = in_pos[m];
-  if (pos < 0) return;
+  if (pos < 0 || slot >= n_heads + 2 * kv.n_kv_heads) return;
   const float sc = row_scale(rs, m);
   const int b = m / rows_per_seq;
   const int hd = kv.head_dim, half = hd >> 1, nkv = kv.n_kv_heads;
@@ -100,7 +102,7 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   if (slot < n_heads + nkv) {
     const bool is_q = slot < n_heads;
     const int col0 = is_q ? slot * hd : nq + (slot - n_heads) * hd;
-    for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    for (int j = lt; j < half; j += 64) {
       const float2 c = rope[(size_t)pos * half + j];
       const float x1 = sc * sum_planes(ps, rbase + col0 + j), x2 = sc * sum_planes(ps, rbase + col0 + j + half);
       const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
@@ -116,7 +118,7 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   } else {
     const int kh = slot - n_heads - nkv;
     T *dst = vbase + ((size_t)kh * kv.max_seq + pos) * hd;
-    for (int j = threadIdx.x; j < hd; j += blockDim.x)
+    for (int j = lt; j < hd; j += 64)
       dst[j] = from_f<T>(sc * sum_planes(ps, rbase + nq + nk + kh * hd + j));
   }
 }
@@ -187,12 +189,12 @@ int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOu
 
 int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
-  const dim3 grid(M, n_heads + 2 * kv.n_kv_heads);
+  const dim3 grid(M, (n_heads + 2 * kv.n_kv_heads + 3) / 4);
   if (dtype == SJD_F32)
-    SJD_CUDA(launch_kernel(qkv_finish_kernel<float>, grid, dim3(64), 0, stream, ps, rs, in_pos, rope_table, q, kv,
+    SJD_CUDA(launch_kernel(qkv_finish_kernel<float>, grid, dim3(256), 0, stream, ps, rs, in_pos, rope_table, q, kv,
                            rows_per_seq, n_heads));
   else if (dtype == SJD_BF16)
-    SJD_CUDA(launch_kernel(qkv_finish_kernel<__nv_bfloat16>, grid, dim3(64), 0, stream, ps, rs, in_pos, rope_table, q, kv,
+    SJD_CUDA(launch_kernel(qkv_finish_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, ps, rs, in_pos, rope_table, q, kv,
                            rows_per_seq, n_heads));
   else
     return SJD_ERR_UNSUPPORTED;
