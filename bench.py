@@ -275,7 +275,7 @@ def run_library(args, wl):
     rows = batch * wl.window
     roofline = {"bound": "hbm", "kernel": "projection GEMMs (weight streaming, M = %d rows)" % rows,
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                "peak_source": "of " + peaks["source"],
+                "peak_source": "of " + peaks["source"], "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
                 "traffic": gemm_traffic_per_launch(tr["gemm_weight_bytes"] / max(1, tr["launches"]["gemm"])),
                 "algorithmic_bytes_per_launch": tr["gemm_weight_bytes"] / max(1, tr["launches"]["gemm"]),
                 "algorithmic_bytes_per_step": tr["gemm_weight_bytes"] / trace_steps,
@@ -288,6 +288,7 @@ def run_library(args, wl):
         tf = flops / (tr["ms"]["gemm"] * 1e-3) / 1e12 if tr["ms"]["gemm"] > 0 else 0.0
         roofline.update({"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": tf / peaks["bf16_tflops_sustained"], "issued_frac": 2.0 * tf / peaks["bf16_tflops_sustained"],
+                         "nominal_peak": 2250.0, "frac_of_nominal": tf / 2250.0,
                          "weight_GBps": achieved,
                          "note": "achieved counts each product once; the tensor pipe runs two MMAs per product "
                                  "(hi and lo plane of the fp32 activations): issued_frac is its utilisation"})

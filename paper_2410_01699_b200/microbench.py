@@ -32,7 +32,10 @@ def _peak():
     return 6650.0, "fallback"
 
 
-def _time(fn, iters, warmup=5, graph=False):
+NOMINAL_HBM_GBPS = 8000.0   # the data-sheet figure, printed beside the measured copy bandwidth
+
+
+def _time(fn, iters, warmup=20, graph=False):
     """Seconds per call.  graph=True records the `iters` calls into one CUDA graph and times replays of
     it, so that a kernel of a few microseconds is not timed by the speed of the Python loop."""
     for _ in range(warmup):
@@ -76,7 +79,7 @@ def bench_gemm(m, n, k, iters):
     assert int(status[0].item()) == 0, "a device-side wait ran out"
     peak, src = _peak()
     gbs = wbytes / sec / 1e9
-    return {"kernel": "sjd_gemm", "M": m, "N": n, "K": k, "us": sec * 1e6, "weight_GBps": gbs, "frac_of_hbm": gbs / peak,
+    return {"kernel": "sjd_gemm", "M": m, "N": n, "K": k, "us": sec * 1e6, "weight_GBps": gbs, "frac_of_hbm": gbs / peak, "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBPS,
             "peak_GBps": peak, "peak_source": src, "TFLOPs": 2.0 * m * n * k / sec / 1e12,
             "note": "time includes the hi/lo split and plane-sum launches of sjd_gemm"}
 
@@ -99,7 +102,7 @@ def bench_verify(batch, window, vocab, top_k, iters):
     nbytes = 2 * batch * window * vocab * 2
     gbs = nbytes / sec / 1e9
     return {"kernel": "sjd_verify", "batch": batch, "window": window, "vocab": vocab, "top_k": top_k, "us": sec * 1e6,
-            "logits_GBps": gbs, "frac_of_hbm": gbs / peak, "peak_GBps": peak, "peak_source": src,
+            "logits_GBps": gbs, "frac_of_hbm": gbs / peak, "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBPS, "peak_GBps": peak, "peak_source": src,
             "rows_per_s": batch * window / sec, "mean_accepted": float(out.host()["n_accepted"].mean())}
 
 
@@ -125,7 +128,7 @@ def bench_attention(batch, window, prefix, n_heads, n_kv_heads, head_dim, iters,
     peak, src = _peak()
     gbs = kv_bytes / sec / 1e9
     return {"kernel": "sjd_attention", "batch": batch, "window": window, "prefix": prefix, "n_heads": n_heads,
-            "n_kv_heads": n_kv_heads, "head_dim": head_dim, "us": sec * 1e6, "kv_GBps": gbs, "frac_of_hbm": gbs / peak,
+            "n_kv_heads": n_kv_heads, "head_dim": head_dim, "us": sec * 1e6, "kv_GBps": gbs, "frac_of_hbm": gbs / peak, "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBPS,
             "peak_GBps": peak, "peak_source": src, "note": "time includes the merge of the split-KV partials"}
 
 
@@ -136,13 +139,13 @@ def main():
     g.add_argument("M", type=int)
     g.add_argument("N", type=int)
     g.add_argument("K", type=int)
-    g.add_argument("--iters", type=int, default=50)
+    g.add_argument("--iters", type=int, default=100)
     v = sub.add_parser("verify")
     v.add_argument("batch", type=int)
     v.add_argument("--window", type=int, default=32)
     v.add_argument("--vocab", type=int, default=16384)
     v.add_argument("--top-k", type=int, default=2000)
-    v.add_argument("--iters", type=int, default=50)
+    v.add_argument("--iters", type=int, default=100)
     t = sub.add_parser("attention")
     t.add_argument("batch", type=int)
     t.add_argument("prefix", type=int)
@@ -150,7 +153,7 @@ def main():
     t.add_argument("--heads", type=int, default=32)
     t.add_argument("--kv-heads", type=int, default=32)
     t.add_argument("--head-dim", type=int, default=128)
-    t.add_argument("--iters", type=int, default=50)
+    t.add_argument("--iters", type=int, default=100)
     t.add_argument("--no-graph", action="store_true", help="time a plain Python loop of calls (for captures under ncu)")
     a = ap.parse_args()
     if a.cmd == "attention":
