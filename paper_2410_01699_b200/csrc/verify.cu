@@ -548,7 +548,12 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int 
 // positive maximum, every positive value that matters) and lumped beyond; then every warp walks
 // the histogram from the top for itself.  One barrier.  false: the K-th largest lies in the lump
 // (or next to +-0), the general route decides.
-__device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, Scratch &sc, uint32_t &tau_key) {
+// `z_hist` (optional): the softmax denominator from the histogram alone -- all entries of a bin share one
+// value, so Z = sum over the kept bins of count * 2^((value - max) * scale) -- for rows whose chunk
+// sums nobody needs (the previous-iteration row when its statistics are not cached).
+__device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, Scratch &sc, uint32_t &tau_key,
+                          float scale, double *z_hist) {
+  using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int j0 = warp * 256 + lane;
   const uint32_t kmax2 = kmax | (kmax << 16);
@@ -565,6 +570,8 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
   }
   __syncthreads();
   uint32_t acc = 0;
+  double zacc = 0.0;
+  const float xmax = E::val(E::unkey(kmax));
   for (int base = 0; base < 4096; base += 32) {   // 32 adjacent bins per step: conflict-free
     const uint32_t c = sc.hist12[base + lane];
     uint32_t incl = c;
@@ -574,10 +581,21 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
       if (lane >= o) incl += y;
     }
     const uint32_t ballot = __ballot_sync(0xffffffffu, acc + incl >= K);
+    if (z_hist) {   // mass of this step's bins down to (and including) the threshold bin
+      const int last = ballot ? __ffs(ballot) - 1 : 31;
+      const uint32_t bin = (uint32_t)(base + lane);
+      float zl = 0.0f;
+      if (lane <= last && c != 0 && bin <= kmax)
+        zl = (float)c * exp2_neg((E::val(E::unkey(kmax - bin)) - xmax) * scale);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) zl += __shfl_xor_sync(0xffffffffu, zl, o);
+      zacc += (double)zl;
+    }
     if (ballot) {
       const uint32_t bin = (uint32_t)(base + __ffs(ballot) - 1);
       if (bin >= 4095u) return false;
       tau_key = kmax - bin;
+      if (z_hist) *z_hist = zacc;
       return !(tau_key == 0x7FFFu || tau_key == 0x8000u);
     }
     acc += __shfl_sync(0xffffffffu, incl, 31);
@@ -747,11 +765,13 @@ struct RowFast {   // statistics of a row on this route
   RowStats st;
   float tau_f;
   float d_weight;   // unnormalised weight of the entry at the draft token
+  double z_hist;    // denominator from the histogram (rows processed without chunk sums), else < 0
 };
 
 // statistics of one row: 4 barriers.  false: general route.
+// `want_chunks`: leave the chunk sums of the row's weights in sc.chunk_sum (needed to sample from the row).
 __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d, int d_slot, int top_k, float inv_t,
-                              Scratch &sc, RowFast &out, uint4 *stash) {
+                              Scratch &sc, RowFast &out, uint4 *stash, bool want_chunks) {
   using E = Elt<__nv_bfloat16>;
   const int NV = V >> 3;
   const bool need_select = top_k < V;
@@ -759,14 +779,21 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d,
   if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
   SJD_TL(TL_VERIFY, 20, threadIdx.x == 0);   // row loaded, maximum known
   uint32_t tau_key = 0;
-  if (need_select && !rr_select(row, NV, kmax, (uint32_t)top_k, sc, tau_key)) return false;
+  const float scale = inv_t * 1.4426950408889634f;
+  const bool from_hist = need_select && !want_chunks;
+  out.z_hist = -1.0;
+  if (need_select && !rr_select(row, NV, kmax, (uint32_t)top_k, sc, tau_key, scale, from_hist ? &out.z_hist : nullptr))
+    return false;
   SJD_TL(TL_VERIFY, 23, threadIdx.x == 0);   // threshold known
   out.st.tau_key = tau_key;
   out.st.xmax = E::val(E::unkey(kmax));
   out.st.flags = 0;
   out.tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
-  const float xmax = out.st.xmax, scale = inv_t * 1.4426950408889634f, tau_f = out.tau_f;
-  rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], tau_f, xmax, scale, w); }, NV, sc);
+  const float xmax = out.st.xmax, tau_f = out.tau_f;
+  if (from_hist)
+    __syncthreads();   // sc.d_bits is read below; the walk above read the histogram the next row clears
+  else
+    rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], tau_f, xmax, scale, w); }, NV, sc);
   SJD_TL(TL_VERIFY, 24, threadIdx.x == 0);   // chunk sums written
   const float dv = E::val(sc.d_bits[d_slot]);
   out.d_weight = (d >= 0 && dv >= tau_f) ? exp2_neg((dv - xmax) * scale) : 0.0f;
@@ -811,10 +838,9 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
       q_d = d_ok ? (E::key(bits) >= qs.tau_key ? exp2_neg((E::val(bits) - qs.xmax) * scale) : 0.0f) / qs.z : 1.0f;
     } else {
       RowFast qfast;
-      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, stage)) return false;
-      const WarpPrefix wq = rr_prefix(NC, sc);
+      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, stage, false)) return false;
       qs = qfast.st;
-      qs.z = (float)wq.total;
+      qs.z = (float)(qfast.z_hist >= 0.0 ? qfast.z_hist : rr_prefix(NC, sc).total);
       if (tid == 0) p.stats[cur ^ 1][r] = qs;
       q_d = d_ok ? qfast.d_weight / qs.z : 1.0f;
     }
@@ -827,7 +853,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   SJD_TL(TL_VERIFY, 10, tid == 0);
   // ---- this iteration's distribution
   RowFast pfast;
-  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast, nullptr)) {
+  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast, nullptr, true)) {
     asm volatile("cp.async.wait_all;" ::: "memory");   // the general route reuses the staging buffer
     return false;
   }
