@@ -752,12 +752,13 @@ __device__ void rr_icdf(const F &wf, int NV, const WarpPrefix &wp, float u, Scra
 // weights of the eight entries of one vector under a row's statistics (value comparison: the
 // threshold is never +-0 here)
 __device__ __forceinline__ void rr_p_weights(const uint4 &v, float tau_f, float xmax, float scale, float *w) {
+  const float c0 = -xmax * scale;   // 2^((x - max) * scale) as one fused multiply-add per entry
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const uint32_t x = word_of(v, k);
     const float a = __uint_as_float(x << 16), b = __uint_as_float(x & 0xFFFF0000u);
-    w[2 * k] = a >= tau_f ? exp2_neg((a - xmax) * scale) : 0.0f;
-    w[2 * k + 1] = b >= tau_f ? exp2_neg((b - xmax) * scale) : 0.0f;
+    w[2 * k] = a >= tau_f ? exp2_neg(fmaf(a, scale, c0)) : 0.0f;
+    w[2 * k + 1] = b >= tau_f ? exp2_neg(fmaf(b, scale, c0)) : 0.0f;
   }
 }
 
@@ -822,11 +823,12 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   // ---- the law of the draft
   RowStats qs;
   qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
-  float q_d;
+  float q_d, tau_q = -INFINITY;   // tau_q: q's threshold as a value (the residual compares values)
   if (kind == SJD_Q_ROW) {
     if (p.prev_stats_valid) {
       qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
-      if (qs.flags != 0 || !(qs.xmax > -FLT_MAX)) return false;
+      if (qs.flags != 0 || !(qs.xmax > -FLT_MAX) || qs.tau_key == 0x7FFFu || qs.tau_key == 0x8000u) return false;
+      if (qs.tau_key != 0) tau_q = E::val(E::unkey(qs.tau_key));
       const uint32_t bits = d_ok ? (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(qbase) + d) : E::NEG_INF;
       if (E::bad(bits)) return false;
       // the residual of Eq. 2 needs the whole q row: copy it to shared memory in the background
@@ -841,6 +843,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
       if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, stage, false)) return false;
       qs = qfast.st;
       qs.z = (float)(qfast.z_hist >= 0.0 ? qfast.z_hist : rr_prefix(NC, sc).total);
+      tau_q = qfast.tau_f;
       if (tid == 0) p.stats[cur ^ 1][r] = qs;
       q_d = d_ok ? qfast.d_weight / qs.z : 1.0f;
     }
@@ -887,13 +890,13 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   // ---- Eq. 2: residual resample
   int resample_tok = -1;
   if (!accept) {
-    const float inv_zp = 1.0f / ps.z, inv_zq = 1.0f / qs.z;
+    // probabilities straight from one fused multiply-add per entry: p_i = 2^(x_i * scale + c) with
+    // c = -max * scale - log2(Z); entries below the threshold contribute nothing
+    const float cp = -xmax_p * scale - log2f(ps.z), cq = -qs.xmax * scale - log2f(qs.z);
     const float q_uniform = 1.0f / (float)V;
     const uint4 *qg = stage;   // the q row, staged above
     const int j0 = warp * 256 + lane;
-    const uint32_t tau_q = qs.tau_key;
-    const float xmax_q = qs.xmax;
-    auto r_w = [&](int i, float *w) {   // max(0, p - q) of the eight entries of slot i; q read through L2
+    auto r_w = [&](int i, float *w) {   // max(0, p - q) of the eight entries of slot i
       const int j = j0 + i * 32;
       const uint4 pv = reg_slot(row, i);
       uint4 qv = make_uint4(0, 0, 0, 0);
@@ -901,22 +904,20 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const uint32_t px = word_of(pv, k), qx = word_of(qv, k);
-        const uint32_t qk = key_pair(qx);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const float pval = __uint_as_float(h ? px & 0xFFFF0000u : px << 16);
-          const float pp = (pval >= tau_p ? exp2_neg((pval - xmax_p) * scale) : 0.0f) * inv_zp;
+          const float pp = pval >= tau_p ? exp2_neg(fmaf(pval, scale, cp)) : 0.0f;   // fillers (-inf) give 0
           float qq;
           if (kind == SJD_Q_ROW) {
-            const uint32_t qkey = h ? qk >> 16 : qk & 0xFFFFu;
             const float qval = __uint_as_float(h ? qx & 0xFFFF0000u : qx << 16);
-            qq = (qkey >= tau_q ? exp2_neg((qval - xmax_q) * scale) : 0.0f) * inv_zq;
+            qq = qval >= tau_q ? exp2_neg(fmaf(qval, scale, cq)) : 0.0f;
           } else if (kind == SJD_Q_UNIFORM) {
             qq = q_uniform;
           } else {
             qq = (j * 8 + k * 2 + h == d) ? 1.0f : 0.0f;
           }
-          w[2 * k + h] = j < NV ? fmaxf(0.0f, pp - qq) : 0.0f;
+          w[2 * k + h] = fmaxf(0.0f, pp - qq);
         }
       }
     };
