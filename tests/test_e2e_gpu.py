@@ -132,6 +132,22 @@ def test_large_shapes_two_layers(name, steps):
     assert seqs[0].max_logit_err <= 2e-2
 
 
+@pytest.mark.parametrize("batch,window,prompt_len,init,steps", [
+    (4, 8, 64, INIT_COPY_ABOVE, 3),    # small window, spatial initialisation (grid stride 49), 32 rows per pass
+    (2, 64, 64, INIT_RANDOM, 2),       # widest window: 128 rows per pass, attention with four row bands per CTA
+    (8, 32, 64, INIT_RANDOM, 2),       # 256 rows per pass: two token slabs per weight tile at the 7B widths
+    (1, 32, 700, INIT_COPY_ABOVE, 2),  # long prefix: several key tiles per split-KV range, pre-fill in 22 chunks
+])
+def test_sweep_points_two_layers(batch, window, prompt_len, init, steps):
+    """Points of the batch / window / prefix / initialisation sweep on the 7B layer shapes (two layers so
+    that the checker stays affordable), in lock-step with the checker."""
+    wl = WORKLOADS["7b-2l"].with_(prompt_len=prompt_len)
+    ctx, seqs, n, _ = run_lockstep(wl, batch=batch, window=window, init=init, max_steps=steps, gain_jitter=0.0)
+    assert n == steps
+    for s in seqs:
+        assert s.max_logit_excess <= 2e-2
+
+
 @pytest.mark.parametrize("name,steps", [("7b", 2), ("8b-gqa", 1)])
 def test_full_depth(name, steps):
     """The full configurations (7B: 32 layers, vocab 65536, W = 32, the step the benchmark times; 8B with
