@@ -74,13 +74,6 @@ __device__ __forceinline__ void mma_bf16(float *c, const uint32_t *a, uint32_t b
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// 2^x for x <= 0 (arguments are scores minus their running maximum): the hardware approximation
-// (2 ulp), results below the normal range flush to 0, 2^-inf = 0
-__device__ __forceinline__ float exp2_le0(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 // two floats -> packed bf16 hi pair and bf16 lo pair (lo = value - hi, rounded)
 __device__ __forceinline__ void split_pair(float x, float y, uint32_t &hi, uint32_t &lo) {
   const __nv_bfloat16 hx = __float2bfloat16_rn(x), hy = __float2bfloat16_rn(y);
@@ -245,8 +238,8 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     uint32_t ph[NK][4], pl[NK][4];
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb) {
-      const float p0 = exp2_le0(sacc[nb][0] - sub0), p1 = exp2_le0(sacc[nb][1] - sub0);
-      const float p2 = exp2_le0(sacc[nb][2] - sub1), p3 = exp2_le0(sacc[nb][3] - sub1);
+      const float p0 = exp2f(sacc[nb][0] - sub0), p1 = exp2f(sacc[nb][1] - sub0);
+      const float p2 = exp2f(sacc[nb][2] - sub1), p3 = exp2f(sacc[nb][3] - sub1);
       ls0 += p0 + p1;
       ls1 += p2 + p3;
       const int kk = nb >> 1, hi8 = (nb & 1) * 2;   // A fragment regs: {row g, row g+8} x {keys 0-7, keys 8-15}
