@@ -36,16 +36,28 @@ __device__ __forceinline__ float row_scale(const RowScale &rs, int m) {
   for (int j = 0; j < rs.n_part; ++j) tot += __ldg(rs.ss_part + (size_t)m * rs.n_part + j);
   return rsqrtf(tot * rs.inv_d + rs.eps);
 }
+// the same for a row index that is uniform over the (full) warp: lanes share the loads.  The partials
+// are added in a fixed tree order, so every caller gets the same bits.
+__device__ __forceinline__ float row_scale_warp(const RowScale &rs, int m) {
+  if (!rs.ss_part) return 1.0f;
+  const int lane = threadIdx.x & 31;
+  float tot = 0.0f;
+  for (int j = lane; j < rs.n_part; j += 32) tot += __ldg(rs.ss_part + (size_t)m * rs.n_part + j);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+  return rsqrtf(tot * rs.inv_d + rs.eps);
+}
 
 // x[m][:] += sum_s P[s][m][:]  (residual connection); emits x * gain as bf16 hi/lo planes (the RMS
-// scale is applied downstream) and this block's share of sum(x^2).  Grid (rows, column chunks of 1024).
+// scale is applied downstream) and one partial of sum(x^2) per 128 columns (= per warp, = per weight
+// tile of the projections, which write the same partials when they fold this step into their
+// epilogue).  Grid (rows, column chunks of 1024).
 constexpr int RG_THREADS = 256;
 constexpr int RG_COLS = RG_THREADS * 4;
 
 template <typename T>
 __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restrict__ x, PlaneSet ps, const T *__restrict__ gain,
                                                                HiLoOut h, float *__restrict__ ss_part, int d) {
-  __shared__ float red[RG_THREADS / 32];
   pdl_trigger();
   SJD_TL(TL_RESID, 0, threadIdx.x == 0);
   pdl_wait();
@@ -66,14 +78,8 @@ __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restric
   }
   float ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
   ss = warp_sum(ss);
-  if ((tid & 31) == 0) red[tid >> 5] = ss;
-  __syncthreads();
-  if (tid == 0) {
-    float tot = 0.0f;
-#pragma unroll
-    for (int w = 0; w < RG_THREADS / 32; ++w) tot += red[w];
-    ss_part[(size_t)m * gridDim.y + chunk] = tot;
-  }
+  const int part = chunk * (RG_THREADS / 32) + (tid >> 5), n_part = (d + 127) / 128;
+  if ((tid & 31) == 0 && part < n_part) ss_part[(size_t)m * n_part + part] = ss;
   SJD_TL(TL_RESID, 2, threadIdx.x == 0);
 }
 
@@ -91,8 +97,8 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   const int m = blockIdx.x, lt = threadIdx.x & 63;
   const int slot = blockIdx.y * (blockDim.x >> 6) + (threadIdx.x >> 6);
   const int pos = in_pos[m];
+  const float sc = row_scale_warp(rs, m);   // before any thread leaves: the warp shares the loads
   if (pos < 0 || slot >= n_heads + 2 * kv.n_kv_heads) return;
-  const float sc = row_scale(rs, m);
   const int b = m / rows_per_seq;
   const int hd = kv.head_dim, half = hd >> 1, nkv = kv.n_kv_heads;
   const int nq = n_heads * hd, nk = nkv * hd;
@@ -132,7 +138,7 @@ __global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int 
   if ((F & 3) == 0 && (ps.ld & 3) == 0 && (ps.plane_stride & 3) == 0) {
     // grid (column chunks, rows): a thread handles groups of four adjacent columns of one row
     const int m = blockIdx.y;
-    const float sc = row_scale(rs, m);
+    const float sc = row_scale_warp(rs, m);
     const float *row = ps.base + (size_t)m * ps.ld;
     for (int f = (blockIdx.x * blockDim.x + threadIdx.x) * 4; f < F; f += gridDim.x * blockDim.x * 4) {
       float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
@@ -169,12 +175,12 @@ __global__ void swiglu_finish_kernel(PlaneSet ps, RowScale rs, HiLoOut act, int 
 
 }  // namespace
 
-int resid_gain_parts(int d) { return (d + RG_COLS - 1) / RG_COLS; }
+int resid_gain_parts(int d) { return (d + 127) / 128; }
 
 int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOut h, float *ss_part, int M, int d,
                       cudaStream_t stream) {
   if (d % 4 != 0) return SJD_ERR_UNSUPPORTED;
-  const dim3 grid(M, resid_gain_parts(d));
+  const dim3 grid(M, (d + RG_COLS - 1) / RG_COLS);
   if (dtype == SJD_F32)
     SJD_CUDA(launch_kernel(resid_gain_kernel<float>, grid, dim3(RG_THREADS), 0, stream, x, ps,
                            reinterpret_cast<const float *>(gain), h, ss_part, d));

@@ -205,6 +205,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full;
   __shared__ uint32_t s_tmem_base;
+  __shared__ float s_scale[TILE_N];   // per-row output scales of this CTA's token slab (epilogue)
 
   pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
   SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
@@ -337,6 +338,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       pdl_wait();   // the planes may still be read, and the row scales written, by the preceding kernel
       float *plane = reinterpret_cast<float *>(p.out) + (size_t)split * p.plane_stride;
       __nv_bfloat16 *out_bf16 = reinterpret_cast<__nv_bfloat16 *>(p.out);
+      if (p.ss_part) {   // RMS scale of each token row, once per CTA (epilogue thread e: row m_base + e)
+        const int e = tid - 64, m = m_base + e;
+        float sc = 1.0f;
+        if (e < p.Mp && m < p.M) {
+          float tot = 0.0f;
+          for (int jj = 0; jj < p.n_part; ++jj) tot += __ldg(p.ss_part + (size_t)m * p.n_part + jj);
+          sc = rsqrtf(tot * p.inv_d + p.eps);
+        }
+        s_scale[e] = sc;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
 #pragma unroll
       for (int j = 0; j < WT; ++j)                               // accumulator
       for (int m0 = 0; m0 < p.Mp; m0 += 16) {                    // first token row of the chunk
@@ -356,11 +368,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
           const int m = m_base + m0 + i;
           if (m < p.M) {
             float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
-            if (p.ss_part) {
-              float tot = 0.0f;
-              for (int jj = 0; jj < p.n_part; ++jj) tot += __ldg(p.ss_part + (size_t)m * p.n_part + jj);
-              v *= rsqrtf(tot * p.inv_d + p.eps);
-            }
+            if (p.ss_part) v *= s_scale[m0 + i];
             if (p.store_bf16) out_bf16[(size_t)m * p.ldc + n] = __float2bfloat16_rn(v);
             else plane[(size_t)m * p.ldc + n] = v;
           }
