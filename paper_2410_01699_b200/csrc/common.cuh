@@ -255,16 +255,6 @@ struct GemmTcCall {
   int n_part;
   float inv_d, eps;
   int n_sms;
-  // Optional (single matrix, at most 64 rows, fp32 planes): the residual step folded into the epilogue.
-  // The last K split of a weight tile to finish (atomic ticket, nobody waits) adds the split planes
-  // of its 128 columns in split order into resid_x, writes (x * gain) as bf16 hi/lo planes and the
-  // tile's partial of sum(x^2) per row -- what resid_gain_kernel does, without a launch of its own.
-  float *resid_x;                  // [M][ldc] residual stream, updated in place; null: off
-  const __nv_bfloat16 *resid_gain; // [n_out[0]] gain of the normalisation that follows
-  __nv_bfloat16 *resid_h;          // hi plane [rows][ldc]; the lo plane starts resid_h_lo elements later
-  size_t resid_h_lo;
-  float *resid_ss;                 // [M][n_out[0] / 128]
-  int *resid_tickets;              // [n_out[0] / 128], zero on entry, left zero
 };
 int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream);
 int launch_sum_planes(const float *planes, size_t plane_stride, int splits, float *out, size_t total, int accumulate,

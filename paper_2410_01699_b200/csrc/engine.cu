@@ -40,7 +40,7 @@ struct XMaps {
 struct Layout {
   size_t kv, logits[2], stats[2], row_out, counters, step, status;
   size_t x, h, qkv, q, attn, gu, act, partial, rope;
-  size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part, gemm_tickets;
+  size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t total;
 };
@@ -112,7 +112,6 @@ Layout make_layout(const sjd_model_cfg &c) {
     L.gemm_planes = take(need * 4);
   }
   L.ss_part = take(Mx * (size_t)resid_gain_parts(c.d_model) * 4);
-  L.gemm_tickets = take((size_t)resid_gain_parts(c.d_model) * 4);
   L.rope = take((size_t)c.max_seq * (c.head_dim / 2) * sizeof(float2));
   L.committed = take((size_t)c.max_batch * c.max_seq * 4);
   L.n = take((size_t)c.max_batch * 4);
@@ -371,11 +370,8 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
   Tracer &tr = c->tracer;
 
   // one GEMM launch over n_mats matrices sharing the activation operand; returns the planes it wrote
-  // With at most 64 rows the residual step (x += projection; next normalisation's gain; hi/lo planes;
-  // sum of squares) runs inside the epilogue of the O and down projections instead of a kernel of its own.
-  const bool fold_resid = M <= 64 && d % 128 == 0;
   auto gemm = [&](const WMap *const *wm, int n_mats, const int *n_out, const TensorMap &x_map, int k_in, int ldc, void *out,
-                  bool bf16_out, PlaneSet *ps, const void *fold_gain = nullptr) -> int {
+                  bool bf16_out, PlaneSet *ps) -> int {
     GemmTcCall call;
     memset(&call, 0, sizeof(call));
     int tiles = 0, col = 0;
@@ -408,14 +404,6 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       call.inv_d = rs.inv_d;
       call.eps = rs.eps;
     }
-    if (fold_gain) {
-      call.resid_x = x;
-      call.resid_gain = reinterpret_cast<const __nv_bfloat16 *>(fold_gain);
-      call.resid_h = hl_h.base;
-      call.resid_h_lo = hl_h.lo_offset;
-      call.resid_ss = ss_part;
-      call.resid_tickets = c->at<int>(c->lay.gemm_tickets);
-    }
     if (ps) *ps = PlaneSet{reinterpret_cast<const float *>(out), call.plane_stride, ldc, call.splits};
     tr.begin(TC_GEMM, stream);
     const int r = launch_gemm_tc(call, stream);
@@ -428,8 +416,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
   for (int l = 0; l < g.n_layers; ++l) {
     const LayerMaps &lm = c->wmaps[l];
     PlaneSet ps;
-    if (!(fold_resid && l > 0))
-      SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->attn_norm[l], hl_h, ss_part, M, d, stream));
+    SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->attn_norm[l], hl_h, ss_part, M, d, stream));
     {
       const WMap *wm[3] = {&lm.wq, &lm.wk, &lm.wv};
       const int n_out[3] = {nq, nk, nk};
@@ -449,9 +436,9 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     {
       const WMap *wm[1] = {&lm.wo};
       const int n_out[1] = {d};
-      SJD_TRY(gemm(wm, 1, n_out, xm.attn, nq, d, planes, false, &ps, fold_resid ? c->ffn_norm[l] : nullptr));
+      SJD_TRY(gemm(wm, 1, n_out, xm.attn, nq, d, planes, false, &ps));
     }
-    if (!fold_resid) SJD_TR(TC_OTHER, launch_resid_gain(dt, x, ps, c->ffn_norm[l], hl_h, ss_part, M, d, stream));
+    SJD_TR(TC_OTHER, launch_resid_gain(dt, x, ps, c->ffn_norm[l], hl_h, ss_part, M, d, stream));
     {
       const WMap *wm[2] = {&lm.w_gate, &lm.w_up};
       const int n_out[2] = {F, F};
@@ -461,12 +448,11 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     {
       const WMap *wm[1] = {&lm.w_down};
       const int n_out[1] = {d};
-      const void *next_gain = l + 1 < g.n_layers ? c->attn_norm[l + 1] : c->final_norm;
-      SJD_TRY(gemm(wm, 1, n_out, xm.act, F, d, planes, false, &pending, fold_resid ? next_gain : nullptr));
+      SJD_TRY(gemm(wm, 1, n_out, xm.act, F, d, planes, false, &pending));
     }
   }
   if (logits_out) {
-    if (!fold_resid) SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->final_norm, hl_h, ss_part, M, d, stream));
+    SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->final_norm, hl_h, ss_part, M, d, stream));
     const WMap *wm[1] = {&c->wmap_head};
     const int n_out[1] = {g.vocab};
     SJD_TRY(gemm(wm, 1, n_out, xm.h, d, g.vocab, logits_out, true, nullptr));
@@ -586,7 +572,6 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
   cudaError_t e = cudaMemcpy(c->ws + lay.rope, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.counters, 0, ((size_t)cfg->max_batch + 1) * 4);
   if (e == cudaSuccess) e = cudaMemset(c->ws + lay.status, 0, 4);
-  if (e == cudaSuccess) e = cudaMemset(c->ws + lay.gemm_tickets, 0, (size_t)resid_gain_parts(cfg->d_model) * 4);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     delete c;

@@ -85,13 +85,6 @@ struct GemmParams {
   const float *ss_part;   // optional [M][n_part] partial sums of squares: rows are scaled by
   int n_part;             //   1 / sqrt(sum_j ss_part[m][j] * inv_d + eps) before they are stored
   float inv_d, eps;
-  float *resid_x;         // residual step folded into the epilogue (see GemmTcCall); null: off
-  const __nv_bfloat16 *resid_gain;
-  __nv_bfloat16 *resid_h;
-  size_t resid_h_lo;
-  float *resid_ss;
-  int *resid_tickets;
-  int n_tiles;            // weight tiles of the launch
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -213,8 +206,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   __shared__ uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full;
   __shared__ uint32_t s_tmem_base;
   __shared__ float s_scale[TILE_N];   // per-row output scales of this CTA's token slab (epilogue)
-  __shared__ float s_red[4][64];      // folded residual step: per-warp partials of sum(x^2) per row
-  __shared__ int s_last;
 
   pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
   SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
@@ -383,45 +374,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
           }
         }
       }
-      if (p.resid_x) {
-        // ---- folded residual step: the last split of this tile to get here finishes its 128 columns
-        __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (tid == 64) {
-          int last = 1;
-          if (p.splits > 1) {
-            last = atomicAdd(&p.resid_tickets[tile], 1) == p.splits - 1;
-            if (last) p.resid_tickets[tile] = 0;
-          }
-          s_last = last;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (s_last) {
-          __threadfence();
-          const int n = p.col_off[mat] + tile_in_mat * TILE_N + row;
-          const float gn = __bfloat162float(p.resid_gain[n]);
-          const float *planes = reinterpret_cast<const float *>(p.out);
-          for (int m = 0; m < p.M; ++m) {
-            const size_t idx = (size_t)m * p.ldc + n;
-            float tot = 0.0f;
-            for (int sp = 0; sp < p.splits; ++sp) tot += __ldcg(planes + (size_t)sp * p.plane_stride + idx);
-            const float xv = p.resid_x[idx] + tot;
-            p.resid_x[idx] = xv;
-            const float hv = xv * gn;
-            const __nv_bfloat16 hi = __float2bfloat16_rn(hv);
-            p.resid_h[idx] = hi;
-            p.resid_h[p.resid_h_lo + idx] = __float2bfloat16_rn(hv - __bfloat162float(hi));
-            float sq = xv * xv;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-            if (lane == 0) s_red[quarter][m] = sq;
-          }
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          const int e = tid - 64;
-          if (e < p.M)
-            p.resid_ss[(size_t)e * p.n_tiles + tile] = (s_red[0][e] + s_red[1][e]) + (s_red[2][e] + s_red[3][e]);
-        }
-      }
     } else if (tid == 64) {
       atomicExch(p.status, 3);
     }
@@ -539,16 +491,6 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.status = g.status;
   p.ss_part = g.ss_part;
   p.n_part = g.n_part;
-  p.resid_x = g.resid_x;
-  p.resid_gain = g.resid_gain;
-  p.resid_h = g.resid_h;
-  p.resid_h_lo = g.resid_h_lo;
-  p.resid_ss = g.resid_ss;
-  p.resid_tickets = g.resid_tickets;
-  p.n_tiles = tiles;
-  if (g.resid_x && (g.n_mats != 1 || g.M > 64 || g.store_bf16 || pl.n_slabs != 1 || pl.w_tiles != 1 || !g.resid_gain ||
-                    !g.resid_h || !g.resid_ss || !g.resid_tickets))
-    return SJD_ERR_BAD_ARG;
   p.inv_d = g.inv_d;
   p.eps = g.eps;
   const int stage_bytes = p.w_tiles * W_TILE_BYTES + p.x_planes * p.Mp * TILE_K * 2;
