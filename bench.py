@@ -33,10 +33,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # DRAM traffic of the dominant kernel (gemm_tc_kernel) from an ncu capture of the gate|up-sized launch
-# (profiles/gemm_tc_dram_traffic.md): 186.38 MB read + written for 180.36 MB of weights.  Traffic grows
+# (profiles/gemm_tc_dram_traffic.md): 184.98 MB read + written for 180.36 MB of weights.  Traffic grows
 # in proportion to the weight bytes of a launch, so a step's launches scale by that ratio.  Valid only
 # for the kernel source the counters were taken with.
-GEMM_TRAFFIC = {"source_sha256_16": "260ad485c835081f", "dram_bytes_per_weight_byte": 186.38 / 180.36}
+GEMM_TRAFFIC = {"source_sha256_16": "c6eab8e298c7d034", "dram_bytes_per_weight_byte": 184.98 / 180.36}
 
 
 def gemm_traffic_per_launch(algorithmic_bytes_per_launch):
