@@ -19,8 +19,11 @@ inline size_t esize(int dtype) { return dtype == SJD_F32 ? 4 : 2; }
 
 // Key-range splits of the attention grid: heads * batch * splits CTAs, two of which fit one SM (their
 // K/V rings take ~99 KB each), so the grid is sized to fill one wave of 2 * 148 slots and no more.
+#ifndef SJD_ATTN_SLOTS
+#define SJD_ATTN_SLOTS (2 * 148)
+#endif
 int attention_splits(int n_heads, int batch) {
-  int s = (2 * 148) / (n_heads * batch);
+  int s = SJD_ATTN_SLOTS / (n_heads * batch);
   return s < 1 ? 1 : (s > 16 ? 16 : s);
 }
 
