@@ -175,11 +175,11 @@ extern "C" size_t sjd_timeline_bytes(void) { return sizeof(TimelineBuf); }
 #endif
 
 // ---- the window attention of Step 2 in isolation (tensor-core split-KV kernel, bf16 cache)
-namespace {
-int attn_splits(int n_heads, int batch) {
-  int s = (2 * 148) / (n_heads * batch);
-  return s < 1 ? 1 : (s > 16 ? 16 : s);
+namespace sjd {
+int attention_splits(int n_heads, int batch);   // engine.cu
 }
+namespace {
+int attn_splits(int n_heads, int batch) { return sjd::attention_splits(n_heads, batch); }
 }  // namespace
 
 extern "C" size_t sjd_attention_workspace_bytes(int batch, int window, int n_heads, int head_dim) {

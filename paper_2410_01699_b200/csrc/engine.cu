@@ -12,11 +12,6 @@
 #include "common.cuh"
 
 namespace sjd {
-namespace {
-
-inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
-inline size_t esize(int dtype) { return dtype == SJD_F32 ? 4 : 2; }
-
 // Key-range splits of the attention grid: heads * batch * splits CTAs, two of which fit one SM (their
 // K/V rings take ~99 KB each), so the grid is sized to fill one wave of 2 * 148 slots and no more.
 #ifndef SJD_ATTN_SLOTS
@@ -26,6 +21,11 @@ int attention_splits(int n_heads, int batch) {
   int s = SJD_ATTN_SLOTS / (n_heads * batch);
   return s < 1 ? 1 : (s > 16 ? 16 : s);
 }
+
+namespace {
+
+inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+inline size_t esize(int dtype) { return dtype == SJD_F32 ? 4 : 2; }
 
 constexpr int kMaxGemmCtas = 160;    // upper bound on the SM count used to size split-K scratch
 
