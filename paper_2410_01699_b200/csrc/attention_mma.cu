@@ -86,6 +86,8 @@ struct AttnParams {
   const float *q;        // [M][H*HD]
   const int32_t *in_pos; // [M]
   float *partial;        // [M][H][splits][HD + 2]
+  float *out;            // [M][H*HD]: written here when splits == 1 (no merge launch needed)
+  HiLoOut hilo;          // optional bf16 hi/lo planes of out (same case)
   int *status;
   int rows_per_seq, n_heads, n_kv_heads, splits;
   int plane0;            // first cache plane of this layer: planes are [b][k|v][kv_head]
@@ -331,6 +333,29 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
       }
     }
   }
+  if (p.splits == 1) {
+    // ---- a single key range: normalise and write the output rows (and their hi/lo planes) directly
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int r = rr == 0 ? r0 : r1;
+      if (r >= W) continue;
+      const float inv = l_run[rr] > 0.0f ? 1.0f / l_run[rr] : 0.0f;   // inactive rows: zeros
+      const size_t base = ((size_t)(m0 + r) * p.n_heads + h) * HD;
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) {
+        const float v0 = o[i][rr * 2] * inv, v1 = o[i][rr * 2 + 1] * inv;
+        const size_t idx = base + i * 8 + tq * 2;
+        *reinterpret_cast<float2 *>(p.out + idx) = make_float2(v0, v1);
+        if (p.hilo.base) {
+          uint32_t hi, lo;
+          split_pair(v0, v1, hi, lo);
+          *reinterpret_cast<uint32_t *>(p.hilo.base + idx) = hi;
+          *reinterpret_cast<uint32_t *>(p.hilo.base + p.hilo.lo_offset + idx) = lo;
+        }
+      }
+    }
+    return;
+  }
   // ---- partial record per (row, head, split): [max (natural log units), sum, o[HD]]
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr) {
@@ -377,15 +402,18 @@ int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_s
 
 bool attention_mma_supported(int head_dim, int rows_per_seq) { return (head_dim == 64 || head_dim == 128) && rows_per_seq <= 64; }
 
-// partial kernel only; the caller merges with the combine kernel of attention.cu
+// With splits > 1 the kernel leaves partial records and the caller merges them with the combine kernel of
+// attention.cu; with a single key range it writes `out` (and `hilo`) itself and no merge is needed.
 int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
-                         int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads, int head_dim, int splits,
-                         cudaStream_t stream) {
+                         float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads,
+                         int head_dim, int splits, cudaStream_t stream) {
   if (!attention_mma_supported(head_dim, rows_per_seq) || M % rows_per_seq != 0) return SJD_ERR_UNSUPPORTED;
   AttnParams p;
   p.q = q;
   p.in_pos = in_pos;
   p.partial = partial;
+  p.out = out;
+  p.hilo = hilo;
   p.status = status;
   p.rows_per_seq = rows_per_seq;
   p.n_heads = n_heads;

@@ -317,7 +317,7 @@ int launch_attention_combine(const float *partial, const int32_t *in_pos, float 
 int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_seq, int head_dim);
 bool attention_mma_supported(int head_dim, int rows_per_seq);
 int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
-                         int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads, int head_dim, int splits,
-                         cudaStream_t stream);
+                         float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads,
+                         int head_dim, int splits, cudaStream_t stream);
 
 }  // namespace sjd

@@ -428,10 +428,12 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     const KvLayout kv = c->kv_layer(l);
     SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
     if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
-      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, status, M,
-                                                rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim, att_splits, stream));
-      SJD_TR(TC_ATTENTION,
-             launch_attention_combine(partial, st.in_pos, attn, M, g.n_heads, g.head_dim, att_splits, stream, hl_attn));
+      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, attn,
+                                                hl_attn, status, M, rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim,
+                                                att_splits, stream));
+      if (att_splits > 1)
+        SJD_TR(TC_ATTENTION,
+               launch_attention_combine(partial, st.in_pos, attn, M, g.n_heads, g.head_dim, att_splits, stream, hl_attn));
     } else {
       SJD_TR(TC_ATTENTION,
              launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, att_splits, stream, hl_attn));

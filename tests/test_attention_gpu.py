@@ -34,6 +34,8 @@ def _reference(q, kv, pos, window, n_kv_heads):
     (3, 16, 70, 8, 2, 64),        # head_dim 64
     (1, 5, 1, 4, 4, 64),          # first step after a one-token prompt: query k sees k + 1 rows
     (1, 24, 64, 4, 1, 128),       # window not a multiple of 16, one kv head
+    (5, 16, 90, 32, 8, 64),       # 160 (head, sequence) pairs: one key range each, output written without a merge
+    (10, 32, 130, 32, 32, 128),   # the same at the 7B head shape, W = 32
 ])
 def test_attention_matches_definition(batch, window, prefix, heads, kv_heads, hd):
     g = torch.Generator().manual_seed(prefix + window)
