@@ -95,16 +95,19 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   pdl_wait();
   SJD_TL(TL_QKV, 1, threadIdx.x == 0);
   const int m = blockIdx.x, lt = threadIdx.x & 63;
-  const int slot = blockIdx.y * (blockDim.x >> 6) + (threadIdx.x >> 6);
   const int pos = in_pos[m];
   const float sc = row_scale_warp(rs, m);   // before any thread leaves: the warp shares the loads
-  if (pos < 0 || slot >= n_heads + 2 * kv.n_kv_heads) return;
+  if (pos < 0) return;
   const int b = m / rows_per_seq;
   const int hd = kv.head_dim, half = hd >> 1, nkv = kv.n_kv_heads;
   const int nq = n_heads * hd, nk = nkv * hd;
   const size_t rbase = (size_t)m * ps.ld;
   T *kbase = reinterpret_cast<T *>(kv.base) + (size_t)b * 2 * nkv * kv.max_seq * hd;
   T *vbase = kbase + (size_t)nkv * kv.max_seq * hd;
+  // the block's 64-thread groups walk over the head slots of the row (one pass when the grid has a
+  // block for every four slots, several when many rows share fewer blocks per row)
+  const int stride = gridDim.y * (blockDim.x >> 6);
+  for (int slot = blockIdx.y * (blockDim.x >> 6) + (threadIdx.x >> 6); slot < n_heads + 2 * nkv; slot += stride) {
   if (slot < n_heads + nkv) {
     const bool is_q = slot < n_heads;
     const int col0 = is_q ? slot * hd : nq + (slot - n_heads) * hd;
@@ -126,6 +129,7 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
     T *dst = vbase + ((size_t)kh * kv.max_seq + pos) * hd;
     for (int j = lt; j < hd; j += 64)
       dst[j] = from_f<T>(sc * sum_planes(ps, rbase + nq + nk + kh * hd + j));
+  }
   }
 }
 
@@ -195,7 +199,12 @@ int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOu
 
 int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
-  const dim3 grid(M, (n_heads + 2 * kv.n_kv_heads + 3) / 4);
+  // a block per four head slots for a few dozen rows; fewer blocks per row (each walking more slots) as
+  // the rows grow, about eight blocks per SM in all
+  int per_row = (n_heads + 2 * kv.n_kv_heads + 3) / 4;
+  const int cap = 1184 / M > 0 ? 1184 / M : 1;
+  per_row = per_row < cap ? per_row : cap;
+  const dim3 grid(M, per_row);
   if (dtype == SJD_F32)
     SJD_CUDA(launch_kernel(qkv_finish_kernel<float>, grid, dim3(256), 0, stream, ps, rs, in_pos, rope_table, q, kv,
                            rows_per_seq, n_heads));
