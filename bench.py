@@ -186,7 +186,7 @@ def run_reference(args, wl):
 
 
 def workload_config(wl, batch_per_gpu):
-    return {"workload": "7B-shaped decoder, one SJD iteration per step (BASELINE configs[2])", "name": wl.name,
+    return {"workload": "7B-shaped decoder, one SJD iteration per step (7B Llama-style decoder, W=32, top-k 2000, batch 1)", "name": wl.name,
             "n_layers": wl.n_layers, "d_model": wl.d_model, "n_heads": wl.n_heads, "n_kv_heads": wl.n_kv_heads,
             "ffn_hidden": wl.ffn_hidden, "vocab": wl.vocab, "prompt_len": wl.prompt_len, "n_generate": wl.n_generate,
             "window": wl.window, "top_k": wl.top_k, "temperature": wl.temperature, "init": "random",
