@@ -8,10 +8,12 @@ random init), batch 1, W = 32, top-k 2000, prompt 64.  Inputs are synthetic and 
   python bench.py --gpus N --steps K --warmup W            # this library (N > 1: under torchrun)
   python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
 
-Prints ONE JSON line.  `value` is device-timed with everything resident in HBM; `e2e` goes through the
-C-ABI with pinned host buffers for the prompt (copied in) and the step results (written out) and a
-host read of the results every step; `roofline` is the weight-streaming GEMM (the dominant kernel)
-against the measured HBM copy bandwidth; `cpu_baseline` is the oracle timed on a bounded sample.
+Prints ONE JSON line.  `value` is device-timed with everything resident in HBM (median of at least five
+blocks of K steps); `e2e` goes through the C-ABI with pinned host buffers for the prompt (copied in) and
+the step results (written out) and a host read of the results every step; `roofline` is the
+weight-streaming GEMM (the dominant kernel) against the measured HBM copy bandwidth; `kernels` holds the
+isolated verification kernel and the window attention against the same bandwidth; `cpu_baseline` is the
+oracle timed on a bounded sample.
 """
 from __future__ import annotations
 
@@ -32,8 +34,8 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-# DRAM traffic of the dominant kernel (gemm_tc_kernel) from an ncu capture of the gate|up-sized launch
-# (profiles/gemm_tc_dram_traffic.md): 184.98 MB read + written for 180.36 MB of weights.  Traffic grows
+# DRAM traffic of the dominant kernel (gemm_tc_kernel) from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum) of the gate|up-sized launch: 184.98 MB read + written for 180.36 MB of weights.  Traffic grows
 # in proportion to the weight bytes of a launch, so a step's launches scale by that ratio.  Valid only
 # for the kernel source the counters were taken with.
 GEMM_TRAFFIC = {"source_sha256_16": "c6eab8e298c7d034", "dram_bytes_per_weight_byte": 184.98 / 180.36}
@@ -197,7 +199,30 @@ def workload_config(wl, batch_per_gpu):
 # ------------------------------------------------------------------------------------------------
 # this library
 # ------------------------------------------------------------------------------------------------
+def kernel_points(peaks):
+    """The isolated verification kernel and the window attention on the workloads their roofline bars are
+    stated on, timed through the C-ABI in this same run (CUDA events on the launching stream, buffers
+    rotating through more than the L2 cache): algorithmic bytes, microseconds, GB/s and the fraction of
+    the measured HBM copy bandwidth."""
+    from paper_2410_01699_b200 import microbench as mb
+    pts = {}
+
+    def put(name, res, gbs_key, nbytes):
+        pts[name] = {"algorithmic_bytes": nbytes, "us": res["us"], "GBps": res[gbs_key],
+                     "frac": res[gbs_key] / peaks["hbm_gbs"], "peak_source": "of " + peaks["source"]}
+
+    for b in (32, 16):
+        r = mb.bench_verify(b, 32, 16384, 2000, iters=60)
+        put("verify_b%d_w32_v16384_k2000" % b, r, "logits_GBps", 2 * b * 32 * 16384 * 2)
+    for b, prefix in ((8, 4000), (1, 2300)):
+        r = mb.bench_attention(b, 32, prefix, 32, 32, 128, iters=60)
+        put("attention_b%d_w32_n%d_h32x128" % (b, prefix + 32), r, "kv_GBps", b * 2 * 32 * (prefix + 32) * 128 * 2)
+    return pts
+
+
 def run_library(args, wl):
+    import statistics
+
     import torch
     import torch.distributed as dist
 
@@ -224,43 +249,78 @@ def run_library(args, wl):
     prompt_dev = prompt_host.to(dev)
     out_dev = B.StepOut(batch, wl.window, device=dev)
     stream = torch.cuda.current_stream()
+    total_tokens = wl.prompt_len + wl.n_generate
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing: K steps enqueued back to back, no host round trip
+    def all_max(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def all_sum(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.int64, device=dev)
+        dist.all_reduce(t)
+        return int(t.item())
+
+    # ---- warm-up: the requested steps, then more until at least WARM_SECONDS have gone by in total (the
+    # first replays of the two step graphs and the clock ramp are slower than the steady state)
+    WARM_SECONDS = 0.3
     ctx.prefill(prompt_dev, sample)
-    committed_acc = torch.zeros(batch, dtype=torch.int64, device=dev)
-    for _ in range(args.warmup):
+    info = ctx.info()
+    t_warm = time.perf_counter()
+    warm_run = 0
+    while warm_run < max(3, args.warmup) or time.perf_counter() - t_warm < WARM_SECONDS:
         ctx.step(out_dev)
-    barrier()
+        warm_run += 1
+        if warm_run % 4 == 0:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    warm_seconds = time.perf_counter() - t_warm
+
+    # ---- device-resident timing: blocks of K steps enqueued back to back with no host round trip, each
+    # block bracketed by a barrier + synchronize and timed with CUDA events; at least 5 blocks and at
+    # least about a second in total.  ms_per_step is the median block (min and max beside it).
     clocks = ClockSampler(local)
     clocks.start()
     launches0 = B.sjd_launch_count()
+    committed_acc = torch.zeros(batch, dtype=torch.int64, device=dev)
+    block_ms, blocks_wanted, steps_timed = [], 5, 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    for _ in range(args.steps):
-        ctx.step(out_dev)
-        committed_acc += out_dev.n_committed  # device-side add of the step's result, no sync
-    e1.record(stream)
-    barrier()
-    ms = e0.elapsed_time(e1)
+    while len(block_ms) < blocks_wanted:
+        # enough of the image left for this block even if every draft of every step were accepted?  else start over
+        n_now = int(out_dev.total_committed.max().item())
+        if n_now + args.steps * wl.window >= total_tokens and n_now + 2 * args.steps >= total_tokens:
+            ctx.prefill(prompt_dev, sample)
+            for _ in range(4):
+                ctx.step(out_dev)
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            ctx.step(out_dev)
+            committed_acc += out_dev.n_committed  # device-side add of the step's result, no sync
+        e1.record(stream)
+        barrier()
+        block_ms.append(all_max(e0.elapsed_time(e1)))
+        steps_timed += args.steps
+        if len(block_ms) == blocks_wanted and sum(block_ms) < 1000.0 and blocks_wanted < 50:
+            blocks_wanted += 1
     launches = B.sjd_launch_count() - launches0
     clk = clocks.stop()
-    tokens = int(committed_acc.sum().item())
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        tk = torch.tensor([tokens], dtype=torch.int64, device=dev)
-        dist.all_reduce(tk)
-        tokens = int(tk.item())
+    tokens = all_sum(int(committed_acc.sum().item()))
     assert ctx.device_status() == B.SJD_OK
-    value = tokens / (ms * 1e-3)
-    tokens_per_step = tokens / (args.steps * batch * world)
+    # tokens fixed per step and sequence over every timed step (a property of the seeded run, not of its
+    # speed); throughput = that rate over the median block's time per step
+    tokens_per_step = tokens / (steps_timed * batch * world)
+    ms_per_step = statistics.median(block_ms) / args.steps
+    value = tokens_per_step * batch * world / (ms_per_step * 1e-3)
 
     # ---- per-kernel-class device time (separate traced steps, CUDA events on the launching stream)
     trace_steps = max(3, min(10, args.steps))
@@ -280,7 +340,8 @@ def run_library(args, wl):
                 "algorithmic_bytes_per_launch": tr["gemm_weight_bytes"] / max(1, tr["launches"]["gemm"]),
                 "algorithmic_bytes_per_step": tr["gemm_weight_bytes"] / trace_steps,
                 "launches_per_step": tr["launches"]["gemm"] / trace_steps, "avg_launch_ms": gemm_ms_per_launch,
-                "step_ms_by_class": {k: v / trace_steps for k, v in tr["ms"].items()}}
+                "step_ms_by_class": {k: v / trace_steps for k, v in tr["ms"].items()},
+                "whole_step_frac": wl.step_weight_bytes() / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     if rows > 128:
         # many rows: the projections are bound by the tensor pipe.  Useful flops = 2 * rows * weights;
         # the kernel multiplies both bf16 planes of the activations, i.e. issues twice that.
@@ -293,33 +354,37 @@ def run_library(args, wl):
                          "note": "achieved counts each product once; the tensor pipe runs two MMAs per product "
                                  "(hi and lo plane of the fp32 activations): issued_frac is its utilisation"})
 
-    # ---- end to end through the C-ABI with host buffers: prompt copied in from pinned memory, results
-    # written to pinned host memory and read by the host after every step
+    # ---- end to end through the C-ABI with host buffers: every step the host hands the library pinned
+    # host buffers for the results, waits for the step and reads them; the prompt is copied in from pinned
+    # host memory and pre-filled inside the timed region.  Same number of steps per block as above; the
+    # rate of tokens per step is the one measured above (it does not depend on which leg runs).
     out_host = B.StepOut(batch, wl.window, pinned=True)
     e2e_steps = args.steps
-    barrier()
-    t0 = time.perf_counter()
-    prompt_dev.copy_(prompt_host, non_blocking=True)
-    ctx.prefill(prompt_dev, sample)
-    e2e_tokens = 0
-    for _ in range(e2e_steps):
-        ctx.step(out_host)
-        stream.synchronize()
-        e2e_tokens += int(out_host.n_committed.sum())
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-        tk = torch.tensor([e2e_tokens], dtype=torch.int64, device=dev)
-        dist.all_reduce(tk)
-        e2e_tokens = int(tk.item())
+    e2e_blocks = []
+    for _ in range(3):
+        barrier()
+        t0 = time.perf_counter()
+        prompt_dev.copy_(prompt_host, non_blocking=True)
+        ctx.prefill(prompt_dev, sample)
+        seen = 0
+        for _ in range(e2e_steps):
+            ctx.step(out_host)
+            stream.synchronize()
+            seen += int(out_host.n_committed.sum())
+        torch.cuda.synchronize()
+        e2e_blocks.append(all_max(time.perf_counter() - t0))
+    e2e_s = statistics.median(e2e_blocks)
     out_bytes = sum(getattr(out_host, n).numel() * 4 for n in ("n_accepted", "n_committed", "committed", "draft",
                                                                 "q_kind", "q_draft", "total_committed", "flags"))
-    e2e = {"value": e2e_tokens / e2e_s, "unit": UNIT,
+    e2e = {"value": tokens_per_step * batch * world * e2e_steps / e2e_s, "unit": UNIT,
            "h2d_bytes_per_step": prompt_host.numel() * 4 / e2e_steps, "d2h_bytes_per_step": out_bytes,
-           "note": "includes pre-fill of the %d-token prompt; host waits for and reads every step's results" % wl.prompt_len}
+           "ms_per_step": e2e_s / e2e_steps * 1e3,
+           "note": "median of 3 blocks of %d steps, each with the copy and pre-fill of the %d-token prompt inside; "
+                   "the host waits for and reads every step's results" % (e2e_steps, wl.prompt_len)}
+
+    kernels = None
+    if rank == 0 and world == 1 and not args.no_kernel_points:
+        kernels = kernel_points(peaks)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -328,15 +393,37 @@ def run_library(args, wl):
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(wl, batch),
-                "clocks": clk, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+                "clocks": clk, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
+                "cpu_baseline": cpu,
+                "timing": {"blocks": len(block_ms), "steps_per_block": args.steps,
+                           "ms_per_step_min": min(block_ms) / args.steps, "ms_per_step_max": max(block_ms) / args.steps,
+                           "warmup_steps_run": warm_run, "warmup_seconds": warm_seconds},
+                "pipeline": info,
                 "sjd": {"committed_tokens_per_step": tokens_per_step,
                         "steps_per_image_est": wl.n_generate / tokens_per_step if tokens_per_step else None,
                         "step_floor_ms_at_measured_hbm": wl.step_weight_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e3}}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def _spawned_rank(local_rank, args, wl, port):
+    os.environ.update({"RANK": str(local_rank), "LOCAL_RANK": str(local_rank), "WORLD_SIZE": str(args.gpus),
+                       "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+    run_library(args, wl)
+
+
+def launch_ranks(args, wl):
+    """`python bench.py --gpus N` without a launcher: start the N ranks here, one process per GPU."""
+    import socket
+
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_spawned_rank, args=(args, wl, port), nprocs=args.gpus, join=True)
 
 
 def main():
@@ -348,11 +435,10 @@ def main():
     ap.add_argument("--workload", default="7b")
     ap.add_argument("--batch", type=int, default=1, help="sequences per GPU")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-points", action="store_true", help="skip the isolated verify / attention timings")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (longer KV prefix)")
     ap.add_argument("--window", type=int, default=0, help="override the Jacobi window W (at most 64)")
     args = ap.parse_args()
-    # at least 10 untimed steps: the first replays of the two step graphs are slower than the rest
-    args.warmup = max(args.warmup, 10) if args.impl == "ours" else args.warmup
     from paper_2410_01699_b200.inputs import WORKLOADS
     wl = WORKLOADS[args.workload]
     if args.prompt_len:
@@ -361,6 +447,8 @@ def main():
         wl = wl.with_(window=args.window)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        launch_ranks(args, wl)
     else:
         run_library(args, wl)
 

@@ -213,11 +213,12 @@ int sjd_verify(int batch, int window, int vocab, int logits_dtype, const void *l
  * cudaMalloc / cudaFree and calls no allocating routine; inputs and outputs stay the caller's.
  *   - Limits: batch * window <= SJD_VERIFY_STATIC_MAX_ROWS and batch <= SJD_VERIFY_STATIC_MAX_BATCH,
  *     else SJD_ERR_CAPACITY (nothing is launched).
- *   - The first call on each device looks up the array's device address (once per device, with that
- *     device current).  Make that first call outside any stream capture.
+ *   - Every call looks up the array's device address for the current device (a host-side query of
+ *     the loaded library, no allocation).  The first call on a device also makes the CUDA runtime load
+ *     the library's device code there: make that first call outside any stream capture.
  *   - All calls on a device share the one array.  It keeps the previous call's contents; the call
  *     clears the counters that must start at zero.  Two calls that overlap on the GPU (different
- *     streams, or different threads or contexts of the same process on one device) race on it:
+ *     streams, or different threads of the same process on one device) race on it:
  *     serialise them.  sjd_verify with separate workspaces has no such restriction.
  */
 #define SJD_VERIFY_STATIC_MAX_ROWS 2048
@@ -261,6 +262,21 @@ size_t sjd_attention_workspace_bytes(int batch, int window, int n_heads, int hea
 int sjd_attention(int batch, int window, int n_heads, int n_kv_heads, int head_dim, int max_seq, const float *q,
                   const void *kv_cache, const int32_t *in_pos, float *out, void *ws, size_t ws_bytes,
                   void *cuda_stream);
+
+/*
+ * Which kernels the steps of a pre-filled context run (the forward pass of Sec. 4.1 Step 2 has two
+ * implementations: the tensor-core pipeline for bf16 models whose projection widths are multiples
+ * of 128 with inner sizes that are multiples of 64, and generic FMA kernels, roughly 50 times slower
+ * on the projections, for everything else).  Host-side query, nothing is launched.
+ * Errors: BAD_ARG, STATE (no prefill yet: the answer depends on batch and window).
+ */
+typedef struct {
+  int32_t tensor_core_projections; /* 1: tcgen05 weight-streaming GEMM + fused consumers; 0: generic kernels */
+  int32_t tensor_core_attention;   /* 1: TMA-staged split-KV tensor-core attention; 0: generic kernel       */
+  int32_t step_graph;              /* 1: a step is replayed as one captured CUDA graph                       */
+  int32_t rows_per_step;           /* batch * window rows per forward pass                                    */
+} sjd_info;
+int sjd_get_info(sjd_ctx *ctx, sjd_info *info);
 
 /* Synchronises the context's last stream and returns SJD_OK, SJD_ERR_DEVICE_TIMEOUT
  * or SJD_ERR_CUDA according to the device status word. */

@@ -28,7 +28,7 @@ TORCH_DTYPES = {SJD_F32: torch.float32, SJD_BF16: torch.bfloat16}
 EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_get_window", "sjd_peek_logits",
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
            "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static",
-           "sjd_gemm_workspace_bytes", "sjd_gemm", "sjd_attention_workspace_bytes", "sjd_attention"]
+           "sjd_gemm_workspace_bytes", "sjd_gemm", "sjd_attention_workspace_bytes", "sjd_attention", "sjd_get_info"]
 
 
 class SJDError(RuntimeError):
@@ -63,6 +63,11 @@ class sjd_sample_cfg(C.Structure):
 class sjd_step_out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("n_accepted", "n_committed", "committed", "draft", "q_kind", "q_draft",
                                           "total_committed", "flags")]
+
+
+class sjd_info(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("tensor_core_projections", "tensor_core_attention", "step_graph",
+                                         "rows_per_step")]
 
 
 _lib = None
@@ -112,6 +117,8 @@ def lib():
     L.sjd_attention_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
     L.sjd_attention.restype = C.c_int
     L.sjd_attention.argtypes = [C.c_int] * 6 + [C.c_void_p] * 5 + [C.c_size_t, C.c_void_p]
+    L.sjd_get_info.restype = C.c_int
+    L.sjd_get_info.argtypes = [C.c_void_p, C.POINTER(sjd_info)]
     L.sjd_last_device_status.restype = C.c_int
     L.sjd_last_device_status.argtypes = [C.c_void_p]
     L.sjd_last_cuda_error.restype = C.c_int
@@ -296,6 +303,12 @@ class Context:
         names = ("gemm", "attention", "verify", "other")
         return {"ms": dict(zip(names, list(ms))), "launches": dict(zip(names, list(n))),
                 "gemm_weight_bytes": float(wb.value)}
+
+    def info(self) -> dict:
+        """Which kernels the steps of this (pre-filled) context run; see sjd_get_info."""
+        i = sjd_info()
+        _check(lib().sjd_get_info(self._ctx, C.byref(i)), "sjd_get_info")
+        return {n: int(getattr(i, n)) for n, _ in sjd_info._fields_}
 
     def device_status(self) -> int:
         return int(lib().sjd_last_device_status(self._ctx))

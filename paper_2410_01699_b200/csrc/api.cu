@@ -24,23 +24,22 @@ using namespace sjd;
 
 extern "C" size_t sjd_verify_workspace_bytes(int batch, int window) { return verify_scratch_bytes(batch, window); }
 
-extern "C" int sjd_verify(int batch, int window, int vocab, int logits_dtype, const void *logits_cur,
-                          const void *logits_prev, const int32_t *draft, const int32_t *q_kind,
-                          const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
-                          const sjd_step_out *out, void *ws, size_t ws_bytes, void *cuda_stream) {
-  if (batch < 1 || window < 1 || vocab < 1 || !logits_cur || !draft || !sample || !out || !ws)
+namespace sjd {
+// Argument checks and parameter set-up shared by the two isolated-verification entry points;
+// `scratch` holds verify_scratch_bytes(batch, window) bytes, 16-byte aligned.
+int verify_isolated(int batch, int window, int vocab, int logits_dtype, const void *logits_cur, const void *logits_prev,
+                    const int32_t *draft, const int32_t *q_kind, const int32_t *base_pos, const sjd_sample_cfg *sample,
+                    uint32_t step, const sjd_step_out *out, void *scratch, cudaStream_t stream) {
+  if (batch < 1 || window < 1 || vocab < 1 || !logits_cur || !draft || !sample || !out || !scratch)
     return SJD_ERR_BAD_ARG;
   if (!logits_prev && !q_kind) return SJD_ERR_BAD_ARG;  // rows of law SJD_Q_ROW need their logits
   if (logits_dtype != SJD_F32 && logits_dtype != SJD_BF16) return SJD_ERR_UNSUPPORTED;
   if (window > 64) return SJD_ERR_CAPACITY;
-  if (!(sample->temperature > 0.0f) || sample->top_k < 1) return SJD_ERR_BAD_ARG;
-  const size_t need = verify_scratch_bytes(batch, window);
-  if (ws_bytes < need) return SJD_ERR_CAPACITY;
-  if (((uintptr_t)ws & 15u) != 0) return SJD_ERR_BAD_ARG;
-  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  if (!(sample->temperature > 0.0f) || sample->top_k < 1 || sample->seq_base < 0) return SJD_ERR_BAD_ARG;
+  if (((uintptr_t)scratch & 15u) != 0) return SJD_ERR_BAD_ARG;
 
   const size_t rows = (size_t)batch * window;
-  char *w = (char *)ws;
+  char *w = (char *)scratch;
   VerifyParams p;
   memset(&p, 0, sizeof(p));
   p.logits[0] = logits_cur;
@@ -50,14 +49,11 @@ extern "C" int sjd_verify(int batch, int window, int vocab, int logits_dtype, co
   p.row_out = (RowOut *)(w + 2 * rows * sizeof(RowStats));
   p.seq_counter = (int32_t *)(w + 2 * rows * sizeof(RowStats) + rows * sizeof(RowOut));
   p.done_counter = p.seq_counter + batch;
+  // the ticket counters must start at zero whatever an earlier call left in the scratch
   SJD_CUDA(cudaMemsetAsync(p.seq_counter, 0, ((size_t)batch + 1) * sizeof(int32_t), stream));
   p.draft = draft;
   p.q_kind = q_kind;
-  p.q_row = nullptr;
-  p.prev_stats_valid = 0;
-  p.w_eff = nullptr;
   p.base_pos = base_pos;
-  p.step_ptr = nullptr;
   p.step = step;
   p.B = batch;
   p.W = window;
@@ -70,6 +66,17 @@ extern "C" int sjd_verify(int batch, int window, int vocab, int logits_dtype, co
   p.e2e = 0;
   p.out = *out;
   return launch_verify(p, logits_dtype, stream);
+}
+}  // namespace sjd
+
+extern "C" int sjd_verify(int batch, int window, int vocab, int logits_dtype, const void *logits_cur,
+                          const void *logits_prev, const int32_t *draft, const int32_t *q_kind,
+                          const int32_t *base_pos, const sjd_sample_cfg *sample, uint32_t step,
+                          const sjd_step_out *out, void *ws, size_t ws_bytes, void *cuda_stream) {
+  if (!ws) return SJD_ERR_BAD_ARG;
+  if (batch >= 1 && window >= 1 && ws_bytes < verify_scratch_bytes(batch, window)) return SJD_ERR_CAPACITY;
+  return verify_isolated(batch, window, vocab, logits_dtype, logits_cur, logits_prev, draft, q_kind, base_pos, sample,
+                         step, out, ws, (cudaStream_t)cuda_stream);
 }
 
 extern "C" int sjd_last_cuda_error(void) { return g_last_cuda_error; }

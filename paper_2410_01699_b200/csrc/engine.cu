@@ -770,6 +770,19 @@ extern "C" int sjd_peek_logits(sjd_ctx *c, void *dst, size_t bytes, void *cuda_s
   return SJD_OK;
 }
 
+extern "C" int sjd_get_info(sjd_ctx *c, sjd_info *info) {
+  if (!c || !info) return SJD_ERR_BAD_ARG;
+  if (!c->prefilled) return SJD_ERR_STATE;
+  const int M = c->batch * c->window;
+  const bool tc = c->use_tc && c->all_tc && M <= 1024 && c->xmaps.count((M + 15) / 16 * 16) != 0;
+  info->tensor_core_projections = tc ? 1 : 0;
+  info->tensor_core_attention =
+      (tc && c->kv_map_valid && attention_mma_supported(c->cfg.head_dim, c->window)) ? 1 : 0;
+  info->step_graph = (c->graphs_enabled && c->use_tc) ? 1 : 0;
+  info->rows_per_step = M;
+  return SJD_OK;
+}
+
 extern "C" int sjd_last_device_status(sjd_ctx *c) {
   if (!c) return SJD_ERR_BAD_ARG;
   SJD_CUDA(cudaStreamSynchronize(c->last_stream));

@@ -114,17 +114,52 @@ def oracle_model_cfg(wl):
                     wl.rope_theta, wl.rms_eps)
 
 
-class LockStepSequence:
-    """One sequence of a batch followed by the checker."""
+class LogitErrors:
+    """Running summary of |checker - library| over every compared logit: the largest difference, the
+    largest difference beyond half a unit in the last place of the stored value, and how many logits lie
+    beyond 1e-2 / 1.5e-2 / 2e-2 (each plus that half unit)."""
+    BARS = (1e-2, 1.5e-2, 2e-2)
 
-    def __init__(self, wl, weights_cpu, prompt_row, scfg, seq_id, logit_tol):
+    def __init__(self):
+        self.total = 0
+        self.max_abs = 0.0
+        self.max_excess = 0.0
+        self.beyond = [0, 0, 0]
+
+    def add(self, diff, half_ulp):
+        excess = diff - half_ulp
+        self.total += int(diff.size)
+        self.max_abs = max(self.max_abs, float(diff.max()))
+        self.max_excess = max(self.max_excess, float(excess.max()))
+        for i, bar in enumerate(self.BARS):
+            self.beyond[i] += int((excess > bar).sum())
+
+    def line(self, label):
+        return ("%s: max |diff| %.3e, beyond half a storage ulp %.3e; of %d logits %d / %d / %d beyond "
+                "1e-2 / 1.5e-2 / 2e-2" % (label, self.max_abs, self.max_excess, self.total, *self.beyond))
+
+
+class LockStepSequence:
+    """One sequence of a batch followed by the checker.  With `also_plain_cache` a second copy of the
+    checker's model keeps its K/V cache unrounded (the plain definition of the forward pass); its logits
+    are only measured (`errors_plain`), the decisions and the asserted tolerance stay with the checker
+    whose cache is rounded to the storage dtype."""
+
+    def __init__(self, wl, weights_cpu, prompt_row, scfg, seq_id, logit_tol, also_plain_cache=False):
         from oracle.model import OracleModel
         from oracle.sjd import CachedModel, sjd_begin
         self.wl, self.scfg, self.tol = wl, scfg, logit_tol
-        self.model = CachedModel(OracleModel(oracle_model_cfg(wl), weights_cpu), wl.prompt_len + scfg.n_generate + 1,
-                                 kv_storage=wl.dtype)
+        om = OracleModel(oracle_model_cfg(wl), weights_cpu)
+        self.model = CachedModel(om, wl.prompt_len + scfg.n_generate + 1, kv_storage=wl.dtype)
         self.prompt = [int(t) for t in prompt_row]
         self.model.prefill(self.prompt)
+        self.errors = LogitErrors()
+        self.errors_plain = None
+        self.plain = None
+        if also_plain_cache and wl.dtype != "f32":
+            self.plain = CachedModel(om, wl.prompt_len + scfg.n_generate + 1, kv_storage="f64")
+            self.plain.prefill(self.prompt)
+            self.errors_plain = LogitErrors()
         self.st = sjd_begin(self.prompt, scfg, wl.vocab, seq=seq_id)
         self.stats = ParityStats(sequences=1)
         self.max_logit_err = 0.0
@@ -168,6 +203,11 @@ class LockStepSequence:
             self.max_logit_err = max(self.max_logit_err, err)
             half_ulp = storage_half_ulp(own, scfg.logits_dtype)
             self.max_logit_excess = max(self.max_logit_excess, float((diff - half_ulp).max()))
+            self.errors.add(diff, half_ulp)
+            if self.plain is not None:
+                plain = self.plain.step_logits(st.committed, st.drafts[:w_eff - 1])
+                self.errors_plain.add(np.abs(plain - gpu_logits_rows[:w_eff]),
+                                      storage_half_ulp(plain, scfg.logits_dtype))
             bad = self.logit_failures(diff, half_ulp)
             assert not bad.any(), (f"step {self.steps}: {int(bad.sum())} logits off by more than {self.tol} "
                                    f"+ half a storage ulp; max |diff| {err:.3e}")

@@ -12,6 +12,7 @@ import torch
 
 from paper_2410_01699_b200 import binding as B
 from paper_2410_01699_b200.inputs import make_verify_case
+from tests.parity_util import compare_window, oracle_verify_case
 
 pytestmark = pytest.mark.gpu
 
@@ -45,6 +46,33 @@ def test_static_scratch_entry_point_matches_sjd_verify_on_consecutive_calls():
         for f in FIELDS:
             assert np.array_equal(ref[f], got[f]), "call %d: %s differs" % (i, f)
         assert np.all(got["n_committed"] >= 1)
+        # and against the CPU checker, like every other verification test
+        prob_tol = 1e-5
+        for b in range(case.batch):
+            vr, qdescs = oracle_verify_case(case, b)
+            compare_window(vr, dict(n_accepted=got["n_accepted"][b], committed=got["committed"][b],
+                                    draft=got["draft"][b], q_draft=got["q_draft"][b]),
+                           case.logits_cur[b].astype(np.float64), case.draft[b], qdescs, case.temperature,
+                           case.top_k, prob_tol, where="call %d, seq %d" % (i, b))
+
+
+def test_static_scratch_entry_point_allocates_nothing():
+    """Free device memory, as the driver reports it, is the same before and after calls of the entry point
+    (inputs and outputs are created before the first reading; the first call, which makes the runtime
+    load the library's device code, comes before it too)."""
+    case = make_verify_case(4, window=16, vocab=8192, top_k=300, seed=44)
+    cur, prev, draft, kind, base = _device_inputs(case)
+    sample = B.make_sample_cfg(temperature=case.temperature, top_k=case.top_k, seed=case.seed, window=case.window)
+    got = B.StepOut(case.batch, case.window)
+    B.sjd_verify_static(cur, prev, draft, kind, base, sample, case.step, got)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    reserved_before = torch.cuda.memory_reserved()
+    for _ in range(3):
+        B.sjd_verify_static(cur, prev, draft, kind, base, sample, case.step, got)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= free_before
+    assert torch.cuda.memory_reserved() == reserved_before
 
 
 def test_static_scratch_entry_point_rejects_oversized_problems():
