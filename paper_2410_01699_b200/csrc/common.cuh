@@ -255,6 +255,14 @@ struct GemmTcCall {
   int n_part;
   float inv_d, eps;
   int n_sms;
+  // weight rows per tile (0: 128).  Fewer rows make more, smaller tiles (their tensor maps must have been
+  // made with that box height); the unused rows of the 128-row MMA cost nothing on a bandwidth-bound launch.
+  int tile_rows;
+  // gate|up mode (act_hi != null): n_mats == 2, matrices gate and up of n_out[0] rows each, tile_rows <= 64,
+  // splits == 1; instead of planes the launch stores silu(gate) * up (both under the row scale) as bf16
+  // hi/lo planes [M][n_out[0]], the lo plane act_lo_off elements after the hi plane.
+  __nv_bfloat16 *act_hi;
+  size_t act_lo_off;
 };
 int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream);
 int launch_sum_planes(const float *planes, size_t plane_stride, int splits, float *out, size_t total, int accumulate,

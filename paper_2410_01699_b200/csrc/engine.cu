@@ -3,6 +3,7 @@
 // counters, step index) lives in device memory, so consecutive steps are enqueued back to back with
 // no host round trip.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -35,6 +36,7 @@ struct WMap {
 };
 struct LayerMaps {
   WMap wq, wk, wv, wo, w_gate, w_up, w_down;
+  WMap gate_gu, up_gu;   // gate and up matrices in boxes of gu_rows rows: the gate|up launch that applies SwiGLU itself
 };
 struct XMaps {
   TensorMap h, attn, act;
@@ -251,6 +253,10 @@ struct sjd_ctx {
   Tracer tracer;
   bool use_tc = false;   // bf16 model on a device with tensor memory: tensor-core GEMM path
   bool all_tc = false;   // every projection of the model is covered by it
+  bool gu_fused = false; // gate|up projection with SwiGLU in its epilogue (every layer has the maps for it)
+  int gu_rows = 0;       // feature rows of the gate (and of the up) matrix per CTA of that launch
+  int head_rows = 0;     // weight rows per CTA of the logits projection (0: 128)
+  WMap wmap_head_r;      // lm_head in boxes of head_rows rows
   int n_ctas = 0;
   std::vector<LayerMaps> wmaps;
   WMap wmap_head;
@@ -374,9 +380,14 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
 
   // one GEMM launch over n_mats matrices sharing the activation operand; returns the planes it wrote
   auto gemm = [&](const WMap *const *wm, int n_mats, const int *n_out, const TensorMap &x_map, int k_in, int ldc, void *out,
-                  bool bf16_out, PlaneSet *ps) -> int {
+                  bool bf16_out, PlaneSet *ps, int tile_rows = 0, const HiLoOut *act = nullptr) -> int {
     GemmTcCall call;
     memset(&call, 0, sizeof(call));
+    call.tile_rows = tile_rows;
+    if (act) {
+      call.act_hi = act->base;
+      call.act_lo_off = act->lo_offset;
+    }
     int tiles = 0, col = 0;
     bool tiles_even = true;
     for (int j = 0; j < n_mats; ++j) {
@@ -394,14 +405,14 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     call.x_lo_row = Ma;
     call.M = M;
     call.K = k_in;
-    call.splits = bf16_out ? 1 : gemm_tc_splits(gemm_tc_plan(M, tiles_even), tiles, k_in / 64, c->n_ctas);
+    call.splits = (bf16_out || act) ? 1 : gemm_tc_splits(gemm_tc_plan(M, tiles_even), tiles, k_in / 64, c->n_ctas);
     call.out = out;
     call.plane_stride = (size_t)M * ldc;
     call.ldc = ldc;
     call.store_bf16 = bf16_out ? 1 : 0;
     call.status = status;
     call.n_sms = c->n_ctas;
-    if (bf16_out) {   // the logits projection applies the final norm's row scale itself
+    if (bf16_out || act) {   // the logits projection and the gate|up launch apply the pending row scale themselves
       call.ss_part = rs.ss_part;
       call.n_part = rs.n_part;
       call.inv_d = rs.inv_d;
@@ -444,12 +455,16 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       SJD_TRY(gemm(wm, 1, n_out, xm.attn, nq, d, planes, false, &ps));
     }
     SJD_TR(TC_OTHER, launch_resid_gain(dt, x, ps, c->ffn_norm[l], hl_h, ss_part, M, d, stream));
-    {
+    if (c->gu_fused) {
+      const WMap *wm[2] = {&lm.gate_gu, &lm.up_gu};
+      const int n_out[2] = {F, F};
+      SJD_TRY(gemm(wm, 2, n_out, xm.h, d, F, nullptr, false, nullptr, c->gu_rows, &hl_act));
+    } else {
       const WMap *wm[2] = {&lm.w_gate, &lm.w_up};
       const int n_out[2] = {F, F};
       SJD_TRY(gemm(wm, 2, n_out, xm.h, d, 2 * F, planes, false, &ps));
+      SJD_TR(TC_OTHER, launch_swiglu_finish(ps, rs, hl_act, M, F, stream));
     }
-    SJD_TR(TC_OTHER, launch_swiglu_finish(ps, rs, hl_act, M, F, stream));
     {
       const WMap *wm[1] = {&lm.w_down};
       const int n_out[1] = {d};
@@ -458,9 +473,10 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
   }
   if (logits_out) {
     SJD_TR(TC_OTHER, launch_resid_gain(dt, x, pending, c->final_norm, hl_h, ss_part, M, d, stream));
-    const WMap *wm[1] = {&c->wmap_head};
+    const int head_rows = M <= 128 ? c->head_rows : 0;   // several token slabs share 128-row tiles through L2
+    const WMap *wm[1] = {head_rows ? &c->wmap_head_r : &c->wmap_head};
     const int n_out[1] = {g.vocab};
-    SJD_TRY(gemm(wm, 1, n_out, xm.h, d, g.vocab, logits_out, true, nullptr));
+    SJD_TRY(gemm(wm, 1, n_out, xm.h, d, g.vocab, logits_out, true, nullptr, head_rows));
   }
   return SJD_OK;
 }
@@ -608,6 +624,31 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
     }
     mk(c->wmap_head, c->lm_head, cfg->vocab, d);
     c->all_tc = c->wmap_head.valid;
+    // gate|up with SwiGLU in the epilogue: 64 gate rows and the same 64 up rows per CTA, one K split.
+    // (Measured on the 7B shapes: 40 rows per CTA, which fills one wave of two CTAs per SM exactly, is no
+    // faster than 64: every CTA reads the whole activation operand, so smaller tiles raise that traffic.)
+    {
+      int r = 64;
+      if (const char *e = getenv("SJD_GU_ROWS")) r = atoi(e);   // tuning: 0 switches the fused launch off, else 8..64
+      c->gu_rows = r;
+      c->gu_fused = r >= 8 && r <= 64 && d % 64 == 0;
+      for (int l = 0; l < L && c->gu_fused; ++l) {
+        LayerMaps &lm = c->wmaps[l];
+        lm.gate_gu.valid = make_tensor_map_bf16(&lm.gate_gu.map, c->w_gate[l], F, d, r) == SJD_OK;
+        lm.up_gu.valid = make_tensor_map_bf16(&lm.up_gu.map, c->w_up[l], F, d, r) == SJD_OK;
+        c->gu_fused = lm.gate_gu.valid && lm.up_gu.valid;
+      }
+    }
+    // logits projection: optional tile height below 128 rows (SJD_HEAD_ROWS; measured on the 7B shapes: 112
+    // rows = two full waves of CTAs is 4 % slower than 128 rows in 1.7 waves, so the default stays 128)
+    if (const char *e = getenv("SJD_HEAD_ROWS")) {
+      const int r = atoi(e);
+      if (r >= 8 && r < 128 && c->wmap_head.valid &&
+          make_tensor_map_bf16(&c->wmap_head_r.map, c->lm_head, cfg->vocab, d, r) == SJD_OK) {
+        c->wmap_head_r.valid = true;
+        c->head_rows = r;
+      }
+    }
     // the cache as one 3-D tensor map for the tensor-core attention; unwritten rows must read as finite
     // numbers (a masked probability of 0 times NaN would poison the output), so the cache starts at zero
     const long planes = (long)L * cfg->max_batch * 2 * cfg->n_kv_heads;

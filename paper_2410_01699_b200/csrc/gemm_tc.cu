@@ -28,6 +28,7 @@
 //   * Every wait is bounded: after ~2 s a role records an error in the status word and leaves; the
 //     CTA still frees its TMEM.
 #include <cuda.h>
+#include <string.h>
 
 #include "common.cuh"
 
@@ -41,7 +42,7 @@ constexpr int UMMA_K = 16;
 constexpr int W_TILE_BYTES = TILE_N * TILE_K * 2;
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
-// tunables (defaults chosen by measurement on B200; see profiles/)
+// tunables (defaults chosen by measurement on B200)
 #ifndef SJD_GEMM_SMEM_BUDGET
 #define SJD_GEMM_SMEM_BUDGET (100 * 1024)   // ring bytes per CTA when two CTAs share an SM
 #endif
@@ -85,6 +86,14 @@ struct GemmParams {
   const float *ss_part;   // optional [M][n_part] partial sums of squares: rows are scaled by
   int n_part;             //   1 / sqrt(sum_j ss_part[m][j] * inv_d + eps) before they are stored
   float inv_d, eps;
+  int tile_rows;          // weight rows a tile really holds (<= 128; the rest of the MMA's 128 rows is idle)
+  int n_out[3];           // output features of matrix j (the last tile of a matrix may be partial)
+  // gate|up mode (template GU): tile t holds rows [t*tile_rows, (t+1)*tile_rows) of the gate matrix in MMA
+  // rows 0.. and the same rows of the up matrix in MMA rows 64..; the epilogue stores
+  // silu(gate) * up as bf16 hi/lo planes [M][F]
+  __nv_bfloat16 *act_hi;
+  size_t act_lo_off;
+  int F;
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -198,7 +207,7 @@ __device__ __forceinline__ bool epilogue_all(bool pred) {
 // ---------------------------------------------------------------------------------- kernel
 // WT: weight tiles per CTA, XP: activation planes multiplied (compile-time so that the common
 // shape, one tile and both planes, keeps fully unrolled issue loops)
-template <int WT, int XP>
+template <int WT, int XP, bool GU>
 __global__ void __launch_bounds__(kThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant__ CUtensorMap w_map1,
                const __grid_constant__ CUtensorMap w_map2, const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
@@ -217,10 +226,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   const int x_tile_bytes = NN * TILE_K * 2;
   const int w_bytes = WT * W_TILE_BYTES;
   const int stage_bytes = w_bytes + x_tile_bytes;
+  const int R = p.tile_rows;
+  const uint32_t stage_tx = (uint32_t)((GU ? 2 : WT) * R * TILE_K * 2 + x_tile_bytes);   // bytes the copies of a stage deliver
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
   // which weight matrix this tile belongs to
-  const int mat = tile < p.tile_end[0] ? 0 : (tile < p.tile_end[1] ? 1 : 2);
+  const int mat = GU ? 0 : (tile < p.tile_end[0] ? 0 : (tile < p.tile_end[1] ? 1 : 2));
   const CUtensorMap *w_map = mat == 0 ? &w_map0 : (mat == 1 ? &w_map1 : &w_map2);
   const int tile_in_mat = tile - (mat == 0 ? 0 : p.tile_end[mat - 1]);
   // this CTA's k-blocks
@@ -262,11 +273,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       // then wait for the predecessor before fetching the activation tiles it produced.
       const int pre = n_kb < p.stages ? n_kb : p.stages;
       for (int i = 0; i < pre; ++i) {
-        mbar_expect_tx(&bar_full[i], (uint32_t)stage_bytes);
+        mbar_expect_tx(&bar_full[i], stage_tx);
+        if (GU) {
+          tma_load_2d(smem + i * stage_bytes, &w_map0, (kb_begin + i) * TILE_K, tile * R, &bar_full[i], policy);
+          tma_load_2d(smem + i * stage_bytes + W_TILE_BYTES / 2, &w_map1, (kb_begin + i) * TILE_K, tile * R, &bar_full[i],
+                      policy);
+        } else {
 #pragma unroll
-        for (int j = 0; j < WT; ++j)
-          tma_load_2d(smem + i * stage_bytes + j * W_TILE_BYTES, w_map, (kb_begin + i) * TILE_K, (tile_in_mat + j) * TILE_N,
-                      &bar_full[i], policy);
+          for (int j = 0; j < WT; ++j)
+            tma_load_2d(smem + i * stage_bytes + j * W_TILE_BYTES, w_map, (kb_begin + i) * TILE_K, (tile_in_mat + j) * R,
+                        &bar_full[i], policy);
+        }
       }
       SJD_TL(TL_GEMM, 3, true);
       pdl_wait();
@@ -286,10 +303,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         if (!mbar_wait(&bar_empty[s], ph ^ 1u)) { ok = false; break; }
         uint8_t *dst = smem + s * stage_bytes;
         const int kcol = (kb_begin + it) * TILE_K;
-        mbar_expect_tx(&bar_full[s], (uint32_t)stage_bytes);
+        mbar_expect_tx(&bar_full[s], stage_tx);
+        if (GU) {
+          tma_load_2d(dst, &w_map0, kcol, tile * R, &bar_full[s], policy);
+          tma_load_2d(dst + W_TILE_BYTES / 2, &w_map1, kcol, tile * R, &bar_full[s], policy);
+        } else {
 #pragma unroll
-        for (int j = 0; j < WT; ++j)
-          tma_load_2d(dst + j * W_TILE_BYTES, w_map, kcol, (tile_in_mat + j) * TILE_N, &bar_full[s], policy);
+          for (int j = 0; j < WT; ++j)
+            tma_load_2d(dst + j * W_TILE_BYTES, w_map, kcol, (tile_in_mat + j) * R, &bar_full[s], policy);
+        }
         tma_load_2d_nohint(dst + w_bytes, &x_map, kcol, m_base, &bar_full[s]);
         if (XP == 2)
           tma_load_2d_nohint(dst + w_bytes + x_tile_bytes / 2, &x_map, kcol, p.x_lo_row + m_base, &bar_full[s]);
@@ -338,10 +360,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
       pdl_wait();   // the planes may still be read, and the row scales written, by the preceding kernel
       float *plane = reinterpret_cast<float *>(p.out) + (size_t)split * p.plane_stride;
       __nv_bfloat16 *out_bf16 = reinterpret_cast<__nv_bfloat16 *>(p.out);
-      if (p.ss_part) {   // RMS scale of each token row, once per CTA (epilogue thread e: row m_base + e)
+      if (p.ss_part || GU) {   // RMS scale of each token row, once per CTA (epilogue thread e: row m_base + e)
         const int e = tid - 64, m = m_base + e;
         float sc = 1.0f;
-        if (e < p.Mp && m < p.M) {
+        if (p.ss_part && e < p.Mp && m < p.M) {
           float tot = 0.0f;
           for (int jj = 0; jj < p.n_part; ++jj) tot += __ldg(p.ss_part + (size_t)m * p.n_part + jj);
           sc = rsqrtf(tot * p.inv_d + p.eps);
@@ -349,11 +371,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         s_scale[e] = sc;
         asm volatile("bar.sync 1, 128;" ::: "memory");
       }
+      if (GU) {
+        // MMA rows 0..63 hold gate features, rows 64..127 the same features of the up matrix.  The warps
+        // that read the up rows (TMEM lane quarters 2, 3) pass their values through shared memory (the
+        // ring is idle by now) to the warps that read the gate rows, which finish the activation.
+        float *ex = reinterpret_cast<float *>(smem);   // [64][Mp + 1]
+        const int ldx = p.Mp + 1;
+        const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int f = tile * R + (row & 63);
+        const bool live = (row & 63) < R && f < p.F;
+        if (quarter >= 2) {
+          for (int m0 = 0; m0 < p.Mp; m0 += 16) {
+            uint32_t hi[16], lo[16];
+            tmem_ld16_issue(t_addr + m0, hi);
+            tmem_ld16_issue(t_addr + p.Mp + m0, lo);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              ex[(row - 64) * ldx + m0 + i] = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * s_scale[m0 + i];
+          }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // the up values are in place
+        if (quarter < 2) {
+          for (int m0 = 0; m0 < p.Mp; m0 += 16) {
+            uint32_t hi[16], lo[16];
+            tmem_ld16_issue(t_addr + m0, hi);
+            tmem_ld16_issue(t_addr + p.Mp + m0, lo);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int m = m_base + m0 + i;
+              if (live && m < p.M) {
+                const float g = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * s_scale[m0 + i];
+                const float u = ex[row * ldx + m0 + i];
+                const float v = g / (1.0f + expf(-g)) * u;
+                const __nv_bfloat16 vh = __float2bfloat16_rn(v);
+                p.act_hi[(size_t)m * p.F + f] = vh;
+                p.act_hi[p.act_lo_off + (size_t)m * p.F + f] = __float2bfloat16_rn(v - __bfloat162float(vh));
+              }
+            }
+          }
+        }
+      } else {
 #pragma unroll
       for (int j = 0; j < WT; ++j)                               // accumulator
       for (int m0 = 0; m0 < p.Mp; m0 += 16) {                    // first token row of the chunk
         const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + j * NN;
-        const int n = p.col_off[mat] + (tile_in_mat + j) * TILE_N + row;
+        const int n_local = (tile_in_mat + j) * R + row;
+        const int n = p.col_off[mat] + n_local;
+        const bool live = row < R && n_local < p.n_out[mat];
         uint32_t hi[16], lo[16];
         tmem_ld16_issue(t_addr + m0, hi);
         if (XP == 2) {
@@ -366,13 +432,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           const int m = m_base + m0 + i;
-          if (m < p.M) {
+          if (live && m < p.M) {
             float v = __uint_as_float(hi[i]) + __uint_as_float(lo[i]);
             if (p.ss_part) v *= s_scale[m0 + i];
             if (p.store_bf16) out_bf16[(size_t)m * p.ldc + n] = __float2bfloat16_rn(v);
             else plane[(size_t)m * p.ldc + n] = v;
           }
         }
+      }
       }
     } else if (tid == 64) {
       atomicExch(p.status, 3);
@@ -463,22 +530,32 @@ int gemm_tc_splits(const GemmTcPlan &pl, int tiles, int k_blocks, int n_sms) {
 int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   if (g.n_mats < 1 || g.n_mats > 3 || g.splits < 1) return SJD_ERR_BAD_ARG;
   GemmParams p;
+  memset(&p, 0, sizeof(p));
+  const bool gu = g.act_hi != nullptr;
+  const int R = g.tile_rows > 0 ? g.tile_rows : TILE_N;
+  if (R > TILE_N || (gu && (R > TILE_N / 2 || g.n_mats != 2 || g.n_out[0] != g.n_out[1] || g.splits != 1)))
+    return SJD_ERR_BAD_ARG;
   int tiles = 0;
   bool tiles_even = true;
   for (int j = 0; j < 3; ++j) {
-    if (j < g.n_mats) {
-      if (!gemm_tc_supported(g.M, g.n_out[j], g.K)) return SJD_ERR_UNSUPPORTED;
-      tiles += g.n_out[j] / TILE_N;
-      tiles_even = tiles_even && (g.n_out[j] / TILE_N) % 2 == 0;
+    if (j < g.n_mats && !(gu && j == 1)) {
+      if (g.M < 1 || g.M > 1024 || g.K % TILE_K != 0 || g.n_out[j] < 1) return SJD_ERR_UNSUPPORTED;
+      if (R == TILE_N && g.n_out[j] % TILE_N != 0) return SJD_ERR_UNSUPPORTED;
+      const int t = (g.n_out[j] + R - 1) / R;
+      tiles += t;
+      tiles_even = tiles_even && t % 2 == 0;
     }
     p.tile_end[j] = tiles;
     p.col_off[j] = j < g.n_mats ? g.col_off[j] : 0;
+    p.n_out[j] = j < g.n_mats ? g.n_out[j] : 0;
   }
   if (g.store_bf16 && g.splits != 1) return SJD_ERR_BAD_ARG;
   p.out = g.out;
   p.plane_stride = g.plane_stride;
   p.ldc = g.ldc;
-  const GemmTcPlan pl = gemm_tc_plan(g.M, tiles_even);
+  GemmTcPlan pl = gemm_tc_plan(g.M, tiles_even);
+  if (gu || R != TILE_N) pl.w_tiles = 1;
+  if (gu && pl.x_planes != 2) return SJD_ERR_UNSUPPORTED;
   p.M = g.M;
   p.Mp = pl.slab_rows;
   p.n_slabs = pl.n_slabs;
@@ -493,6 +570,10 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.n_part = g.n_part;
   p.inv_d = g.inv_d;
   p.eps = g.eps;
+  p.tile_rows = R;
+  p.act_hi = g.act_hi;
+  p.act_lo_off = g.act_lo_off;
+  p.F = gu ? g.n_out[0] : 0;
   const int stage_bytes = p.w_tiles * W_TILE_BYTES + p.x_planes * p.Mp * TILE_K * 2;
   const int ctas = tiles / p.w_tiles * p.n_slabs;
   // one CTA per SM or fewer: give each the deeper ring
@@ -513,21 +594,25 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   SJD_CUDA(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
   if (!configured[dev]) {
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * kSmemBudget + 2048));
+    const int max_dyn = 2 * kSmemBudget + 2048;
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
     configured[dev] = true;
   }
   const dim3 grid(ctas, g.splits);
-  if (p.w_tiles == 1 && p.x_planes == 2)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 2>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  if (gu)
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 2, true>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+  else if (p.w_tiles == 1 && p.x_planes == 2)
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 2, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   else if (p.w_tiles == 2 && p.x_planes == 2)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 2>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 2, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   else if (p.w_tiles == 1)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 1>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 1, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   else
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 1>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 1, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

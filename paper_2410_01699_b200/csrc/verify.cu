@@ -35,7 +35,7 @@ SJD_TIMELINE_TU(verify)
 namespace {
 
 #ifndef SJD_VERIFY_MIN_BLOCKS
-#define SJD_VERIFY_MIN_BLOCKS 3   // resident blocks per SM the 256-thread variant is compiled for
+#define SJD_VERIFY_MIN_BLOCKS 4   // resident blocks per SM the 256-thread variant is compiled for (64 registers)
 #endif
 constexpr int kMaxChunks = 1024;   // 32 vectors of 16 bytes per chunk
 constexpr int kMaxThreads = 1024;
@@ -563,6 +563,9 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
 #pragma unroll
       for (int w = 0; w < 4; ++w) {
         const uint32_t dist = kmax2 - key_pair(word_of(row.v[i], w));   // per half, no borrow: keys <= kmax
+        // every entry is counted, the far ones in the last bin (skipping them under a predicate was measured
+        // slower: the predicate becomes a branch, and the cost of a shared-memory reduction does not depend
+        // on how many lanes take part or on how many of them hit the same counter)
         atomicAdd(&sc.hist12[min(dist & 0xFFFFu, 4095u)], 1u);
         atomicAdd(&sc.hist12[min(dist >> 16, 4095u)], 1u);
       }
@@ -604,6 +607,8 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
 }
 
 // chunk sums of a weight functor evaluated on registers -> sc.chunk_sum.  One barrier.
+// Every lane holds eight slot sums; the warp adds them up transposed (each exchange halves the number of
+// slots a lane still carries: 4 + 2 + 1 + 1 + 1 shuffles instead of 8 x 5), in a fixed order.
 template <typename F>
 __device__ __forceinline__ void rr_chunk_sums(const F &wf, int NV, Scratch &sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -615,16 +620,27 @@ __device__ __forceinline__ void rr_chunk_sums(const F &wf, int NV, Scratch &sc) 
     wf(i, w);
     s[i] = ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
   }
+  const bool b4 = (lane & 16) != 0, b3 = (lane & 8) != 0, b2 = (lane & 4) != 0;
+  float a[4], c[2];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
+  for (int k = 0; k < 4; ++k) {   // lanes 16..31 keep slots 4..7, lanes 0..15 slots 0..3
+    const float send = b4 ? s[k] : s[k + 4], keep = b4 ? s[k + 4] : s[k];
+    a[k] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
   }
-  if (lane == 0) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (warp * 8 + i < NC) sc.chunk_sum[warp * 8 + i] = s[i];
+  for (int k = 0; k < 2; ++k) {
+    const float send = b3 ? a[k] : a[k + 2], keep = b3 ? a[k + 2] : a[k];
+    c[k] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
   }
+  float e;
+  {
+    const float send = b2 ? c[0] : c[1], keep = b2 ? c[1] : c[0];
+    e = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+  e += __shfl_xor_sync(0xffffffffu, e, 2);
+  e += __shfl_xor_sync(0xffffffffu, e, 1);
+  const int slot = (lane >> 2) & 7;   // bit 4 -> slot bit 2, bit 3 -> bit 1, bit 2 -> bit 0
+  if ((lane & 3) == 0 && warp * 8 + slot < NC) sc.chunk_sum[warp * 8 + slot] = e;
   __syncthreads();
 }
 
@@ -749,16 +765,30 @@ __device__ void rr_icdf(const F &wf, int NV, const WarpPrefix &wp, float u, Scra
   tok_w = sc.tok_w;
 }
 
-// weights of the eight entries of one vector under a row's statistics (value comparison: the
-// threshold is never +-0 here)
-__device__ __forceinline__ void rr_p_weights(const uint4 &v, float tau_f, float xmax, float scale, float *w) {
-  const float c0 = -xmax * scale;   // 2^((x - max) * scale) as one fused multiply-add per entry
+// weights of the eight entries of one vector whose entries below the threshold have been replaced by
+// -inf (rr_mask_below): 2^((x - max) * scale) as one fused multiply-add and one exp2 per entry
+__device__ __forceinline__ void rr_p_weights(const uint4 &v, float xmax, float scale, float *w) {
+  const float c0 = -xmax * scale;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const uint32_t x = word_of(v, k);
-    const float a = __uint_as_float(x << 16), b = __uint_as_float(x & 0xFFFF0000u);
-    w[2 * k] = a >= tau_f ? exp2_neg(fmaf(a, scale, c0)) : 0.0f;
-    w[2 * k + 1] = b >= tau_f ? exp2_neg(fmaf(b, scale, c0)) : 0.0f;
+    w[2 * k] = exp2_neg(fmaf(__uint_as_float(x << 16), scale, c0));
+    w[2 * k + 1] = exp2_neg(fmaf(__uint_as_float(x & 0xFFFF0000u), scale, c0));
+  }
+}
+
+// entries below the threshold (a value other than +-0) become -inf, two per instruction pair
+__device__ __forceinline__ void rr_mask_below(RegRow &row, float tau_f) {
+  const __nv_bfloat16 t1 = __float2bfloat16_rn(tau_f);   // exact: the threshold is an entry of the row
+  const __nv_bfloat162 t2 = __halves2bfloat162(t1, t1);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    uint32_t *w = reinterpret_cast<uint32_t *>(&row.v[i]);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t m = __hge2_mask(as_bf2(w[k]), t2);
+      w[k] = (w[k] & m) | (0xFF80FF80u & ~m);
+    }
   }
 }
 
@@ -770,13 +800,14 @@ struct RowFast {   // statistics of a row on this route
 };
 
 // statistics of one row: 4 barriers.  false: general route.
-// `want_chunks`: leave the chunk sums of the row's weights in sc.chunk_sum (needed to sample from the row).
+// `want_chunks`: mask the entries below the threshold in `row` and leave the chunk sums of the row's
+// weights in sc.chunk_sum (needed to sample from the row).
 __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d, int d_slot, int top_k, float inv_t,
-                              Scratch &sc, RowFast &out, uint4 *stash, bool want_chunks) {
+                              Scratch &sc, RowFast &out, bool want_chunks) {
   using E = Elt<__nv_bfloat16>;
   const int NV = V >> 3;
   const bool need_select = top_k < V;
-  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select, stash);
+  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select, nullptr);
   if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
   SJD_TL(TL_VERIFY, 20, threadIdx.x == 0);   // row loaded, maximum known
   uint32_t tau_key = 0;
@@ -791,10 +822,12 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d,
   out.st.flags = 0;
   out.tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
   const float xmax = out.st.xmax, tau_f = out.tau_f;
-  if (from_hist)
+  if (from_hist) {
     __syncthreads();   // sc.d_bits is read below; the walk above read the histogram the next row clears
-  else
-    rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], tau_f, xmax, scale, w); }, NV, sc);
+  } else {
+    if (need_select) rr_mask_below(row, tau_f);
+    rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], xmax, scale, w); }, NV, sc);
+  }
   SJD_TL(TL_VERIFY, 24, threadIdx.x == 0);   // chunk sums written
   const float dv = E::val(sc.d_bits[d_slot]);
   out.d_weight = (d >= 0 && dv >= tau_f) ? exp2_neg((dv - xmax) * scale) : 0.0f;
@@ -807,14 +840,16 @@ __device__ bool fast_row(const VerifyParams &p, Scratch &sc, uint4 *stage, int r
   return false;
 }
 
+constexpr int kResampleDeferred = -2;   // RowOut.resample_tok of a rejected row whose Eq. 2 draw is still to be made
+
 template <>
 __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint4 *stage, int r, int b, int kind, int d,
                                         int qr, int cur, const __nv_bfloat16 *qbase, const __nv_bfloat16 *pbase,
                                         float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
   using E = Elt<__nv_bfloat16>;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
-  if (NV > 8 * (int)blockDim.x || !stage) return false;
+  if (NV > 8 * (int)blockDim.x) return false;
   const bool d_ok = d >= 0 && d < V;
   const int dd = d_ok ? d : -1;
   const float scale = inv_t * 1.4426950408889634f;
@@ -823,27 +858,19 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   // ---- the law of the draft
   RowStats qs;
   qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
-  float q_d, tau_q = -INFINITY;   // tau_q: q's threshold as a value (the residual compares values)
+  float q_d;
   if (kind == SJD_Q_ROW) {
     if (p.prev_stats_valid) {
       qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
       if (qs.flags != 0 || !(qs.xmax > -FLT_MAX) || qs.tau_key == 0x7FFFu || qs.tau_key == 0x8000u) return false;
-      if (qs.tau_key != 0) tau_q = E::val(E::unkey(qs.tau_key));
       const uint32_t bits = d_ok ? (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(qbase) + d) : E::NEG_INF;
       if (E::bad(bits)) return false;
-      // the residual of Eq. 2 needs the whole q row: copy it to shared memory in the background
-      for (int j = tid; j < NV; j += blockDim.x)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(stage + j)),
-                     "l"(reinterpret_cast<const uint4 *>(qbase) + j)
-                     : "memory");
-      asm volatile("cp.async.commit_group;" ::: "memory");
       q_d = d_ok ? (E::key(bits) >= qs.tau_key ? exp2_neg((E::val(bits) - qs.xmax) * scale) : 0.0f) / qs.z : 1.0f;
     } else {
       RowFast qfast;
-      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, stage, false)) return false;
+      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, false)) return false;
       qs = qfast.st;
       qs.z = (float)(qfast.z_hist >= 0.0 ? qfast.z_hist : rr_prefix(NC, sc).total);
-      tau_q = qfast.tau_f;
       if (tid == 0) p.stats[cur ^ 1][r] = qs;
       q_d = d_ok ? qfast.d_weight / qs.z : 1.0f;
     }
@@ -854,20 +881,15 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   }
 
   SJD_TL(TL_VERIFY, 10, tid == 0);
-  // ---- this iteration's distribution
+  // ---- this iteration's distribution (entries below the threshold are -inf in `row` from here on)
   RowFast pfast;
-  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast, nullptr, true)) {
-    asm volatile("cp.async.wait_all;" ::: "memory");   // the general route reuses the staging buffer
-    return false;
-  }
-  asm volatile("cp.async.wait_all;" ::: "memory");   // this thread's copies of the q row have landed; the barriers
-                                                     // of the re-draft below make them visible to the block
+  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast, true)) return false;
   const WarpPrefix wpp = rr_prefix(NC, sc);
   RowStats ps = pfast.st;
   ps.z = (float)wpp.total;
   if (tid == 0) p.stats[cur][r] = ps;
   const float p_d = d_ok ? pfast.d_weight / ps.z : 0.0f;
-  const float tau_p = pfast.tau_f, xmax_p = ps.xmax;
+  const float xmax_p = ps.xmax;
   SJD_TL(TL_VERIFY, 11, tid == 0);
 
   // ---- Eq. 1
@@ -880,64 +902,139 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   if (thr < 1.0f && fabsf(u_acc - thr) < 1e-4f) flags |= SJD_FLAG_NEAR_TIE_ACCEPT;
 
   // ---- Eq. 3: re-draft from p
-  auto p_w = [&](int i, float *w) { rr_p_weights(reg_slot(row, i), tau_p, xmax_p, scale, w); };
+  auto p_w = [&](int i, float *w) { rr_p_weights(reg_slot(row, i), xmax_p, scale, w); };
   int redraft_tok;
   float redraft_w;
   rr_icdf(p_w, NV, wpp, u_draft, sc, redraft_tok, redraft_w);
   const float redraft_p = redraft_w / ps.z;
   SJD_TL(TL_VERIFY, 12, tid == 0);
 
-  // ---- Eq. 2: residual resample
-  int resample_tok = -1;
-  if (!accept) {
-    // probabilities straight from one fused multiply-add per entry: p_i = 2^(x_i * scale + c) with
-    // c = -max * scale - log2(Z); entries below the threshold contribute nothing
-    const float cp = -xmax_p * scale - log2f(ps.z), cq = -qs.xmax * scale - log2f(qs.z);
-    const float q_uniform = 1.0f / (float)V;
-    const uint4 *qg = stage;   // the q row, staged above
-    const int j0 = warp * 256 + lane;
-    auto r_w = [&](int i, float *w) {   // max(0, p - q) of the eight entries of slot i
-      const int j = j0 + i * 32;
+  // ---- Eq. 2 is left to the block that scans the sequence: only the first rejected row needs it
+  ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
+  ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = accept ? -1 : kResampleDeferred;
+  ro.flags = flags;
+  return true;
+}
+
+// Eq. 2 for the first rejected row of sequence b, when that row left it open (register-resident route):
+// run by every thread of the sequence's last block before the window slide.  The row's statistics and
+// those of its draft's law were published by the block that verified it; the two logits rows are read
+// again (they are still in L2): p into registers, q vector by vector as it is needed.
+template <typename T>
+__device__ void deferred_residual(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {}
+
+template <>
+__device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {
+  using E = Elt<__nv_bfloat16>;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int W = p.W, V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
+  const int w_eff = p.w_eff ? p.w_eff[b] : W;
+  RowOut *ro = p.row_out + (size_t)b * W;
+  if (tid < 32) {
+    int first = w_eff;
+    for (int k = lane; k < w_eff; k += 32)
+      if (!__ldcg(&ro[k].accept)) first = min(first, k);
+    first = __reduce_min_sync(0xffffffffu, first);
+    if (lane == 0) sc.sel_chunk = (first < w_eff && __ldcg(&ro[first].resample_tok) == kResampleDeferred) ? first : -1;
+  }
+  __syncthreads();
+  const int a = sc.sel_chunk;
+  __syncthreads();
+  if (a < 0) return;
+  const int r = b * W + a;
+  const int kind = p.q_kind ? p.q_kind[r] : SJD_Q_ROW;
+  const int d = p.draft[r];
+  const int qr = p.q_row ? p.q_row[r] : a;
+  const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
+  const Philox4 rnd = philox4x32_10((uint32_t)(base + a), step, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo,
+                                    p.seed_hi);
+  const float u_res = u24(rnd.w[1]);
+  const float scale = (1.0f / p.temperature) * 1.4426950408889634f;
+  const __nv_bfloat16 *qbase = reinterpret_cast<const __nv_bfloat16 *>(p.logits[cur ^ 1]) + ((size_t)b * W + qr) * V;
+  const __nv_bfloat16 *pbase = reinterpret_cast<const __nv_bfloat16 *>(p.logits[cur]) + (size_t)r * V;
+  auto load_stats = [](const RowStats *g) {
+    const uint4 u = __ldcg(reinterpret_cast<const uint4 *>(g));
+    RowStats st;
+    st.tau_key = u.x; st.xmax = __uint_as_float(u.y); st.z = __uint_as_float(u.z); st.flags = u.w;
+    return st;
+  };
+  const RowStats ps = load_stats(&p.stats[cur][r]);
+  RowStats qs;
+  qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
+  if (kind == SJD_Q_ROW) {
+    qs = load_stats(&p.stats[cur ^ 1][(size_t)b * W + qr]);
+  }
+  const float tau_p = ps.tau_key ? E::val(E::unkey(ps.tau_key)) : -INFINITY;
+  const float tau_q = qs.tau_key ? E::val(E::unkey(qs.tau_key)) : -INFINITY;
+  RegRow row;
+  const int j0 = warp * 256 + lane;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    row.v[i] = j < NV ? __ldg(reinterpret_cast<const uint4 *>(pbase) + j)
+                      : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+  }
+
+  // probabilities straight from one fused multiply-add per entry: p_i = 2^(x_i * scale + c) with
+  // c = -max * scale - log2(Z); entries below the threshold contribute nothing
+  const float cp = -ps.xmax * scale - log2f(ps.z), cq = -qs.xmax * scale - log2f(qs.z);
+  const float q_uniform = 1.0f / (float)V;
+  auto r_w = [&](int i, float *w) {   // max(0, p - q) of the eight entries of slot i
+    const int j = j0 + i * 32;
+    const uint4 pv = reg_slot(row, i);
+    uint4 qv = make_uint4(0, 0, 0, 0);
+    if (kind == SJD_Q_ROW && j < NV) qv = __ldg(reinterpret_cast<const uint4 *>(qbase) + j);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t px = word_of(pv, k), qx = word_of(qv, k);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float pval = __uint_as_float(h ? px & 0xFFFF0000u : px << 16);
+        const float pp = pval >= tau_p ? exp2_neg(fmaf(pval, scale, cp)) : 0.0f;   // fillers (-inf) give 0
+        float qq;
+        if (kind == SJD_Q_ROW) {
+          const float qval = __uint_as_float(h ? qx & 0xFFFF0000u : qx << 16);
+          qq = qval >= tau_q ? exp2_neg(fmaf(qval, scale, cq)) : 0.0f;
+        } else if (kind == SJD_Q_UNIFORM) {
+          qq = q_uniform;
+        } else {
+          qq = (j * 8 + k * 2 + h == d) ? 1.0f : 0.0f;
+        }
+        w[2 * k + h] = fmaxf(0.0f, pp - qq);
+      }
+    }
+  };
+  uint32_t flags = 0;
+  int tok;
+  float wsel;
+  rr_chunk_sums(r_w, NV, sc);
+  WarpPrefix wr = rr_prefix(NC, sc);
+  if (wr.total > 0.0) {
+    rr_icdf(r_w, NV, wr, u_res, sc, tok, wsel);
+  } else {
+    flags |= SJD_FLAG_RESIDUAL_EMPTY;
+    const float c0 = ps.xmax;
+    auto p_w = [&](int i, float *w) {
       const uint4 pv = reg_slot(row, i);
-      uint4 qv = make_uint4(0, 0, 0, 0);
-      if (kind == SJD_Q_ROW && j < NV) qv = qg[j];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const uint32_t px = word_of(pv, k), qx = word_of(qv, k);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const float pval = __uint_as_float(h ? px & 0xFFFF0000u : px << 16);
-          const float pp = pval >= tau_p ? exp2_neg(fmaf(pval, scale, cp)) : 0.0f;   // fillers (-inf) give 0
-          float qq;
-          if (kind == SJD_Q_ROW) {
-            const float qval = __uint_as_float(h ? qx & 0xFFFF0000u : qx << 16);
-            qq = qval >= tau_q ? exp2_neg(fmaf(qval, scale, cq)) : 0.0f;
-          } else if (kind == SJD_Q_UNIFORM) {
-            qq = q_uniform;
-          } else {
-            qq = (j * 8 + k * 2 + h == d) ? 1.0f : 0.0f;
-          }
-          w[2 * k + h] = fmaxf(0.0f, pp - qq);
-        }
+        const uint32_t px = word_of(pv, k);
+        const float lo = __uint_as_float(px << 16), hi = __uint_as_float(px & 0xFFFF0000u);
+        w[2 * k] = lo >= tau_p ? exp2_neg((lo - c0) * scale) : 0.0f;
+        w[2 * k + 1] = hi >= tau_p ? exp2_neg((hi - c0) * scale) : 0.0f;
       }
     };
-    rr_chunk_sums(r_w, NV, sc);
-    WarpPrefix wr = rr_prefix(NC, sc);
-    float wsel;
-    if (wr.total > 0.0) {
-      rr_icdf(r_w, NV, wr, u_res, sc, resample_tok, wsel);
-    } else {
-      flags |= SJD_FLAG_RESIDUAL_EMPTY;
-      __syncthreads();
-      rr_chunk_sums(p_w, NV, sc);
-      wr = rr_prefix(NC, sc);
-      rr_icdf(p_w, NV, wr, u_res, sc, resample_tok, wsel);
-    }
+    __syncthreads();
+    rr_chunk_sums(p_w, NV, sc);
+    wr = rr_prefix(NC, sc);
+    rr_icdf(p_w, NV, wr, u_res, sc, tok, wsel);
   }
-  SJD_TL(TL_VERIFY, 13, tid == 0);
-  ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
-  ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok; ro.flags = flags;
-  return true;
+  if (tid == 0) {
+    ro[a].resample_tok = tok;
+    ro[a].flags = __ldcg(&ro[a].flags) | flags;
+    __threadfence();
+  }
+  __syncthreads();
 }
 
 // Threshold + denominator of one row; leaves chunk sums of the row's weights in the scratch.
@@ -1210,6 +1307,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   if (!sc.is_last) return;
   __threadfence();
   SJD_TL(TL_VERIFY, 14, tid == 0);
+  if (p.fast) deferred_residual<T>(p, b, step, cur, sc);
   finalize_sequence(p, b, step, sc);
   SJD_TL(TL_VERIFY, 15, tid == 0);
   __syncthreads();
@@ -1244,7 +1342,6 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
   if ((nv_max + 31) / 32 > kMaxChunks) return SJD_ERR_CAPACITY;
   const size_t stage_bytes = (size_t)nv_max * 16;
   p.staged = stage_bytes <= 160 * 1024 ? 1 : 0;
-  const size_t dyn = p.staged ? stage_bytes : 0;
   int threads = nv_max <= 1024 ? 128 : nv_max <= 4096 ? 256 : nv_max <= 16384 ? 512 : 1024;
   // rows a block can hold in registers, eight vectors per thread
   p.fast = 0;
@@ -1253,7 +1350,11 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
     p.fast = 1;
     threads = (p.V / VEC + 255) / 256 * 32;
     threads = threads < 64 ? 64 : threads;
+    // no staging buffer: the rows live in registers; the odd row that needs the general route (a NaN, a
+    // threshold out of the histogram's reach) re-reads global memory instead, and more blocks fit an SM
+    p.staged = 0;
   }
+  const size_t dyn = p.staged ? stage_bytes : 0;
   auto launch = [&](auto kernel) -> int {
     // static scratch (about 30 KB) + the staged row: opt in as soon as the sum can pass 48 KB
     if (dyn > 16 * 1024) SJD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn));
