@@ -95,6 +95,41 @@ def icdf(weights, u: float):
     return i, margin
 
 
+def guided_logits(logits_cond, logits_uncond, weight: float, storage: str = "f64"):
+    """Classifier-free guidance (Sec. 5.1, implementation details: guidance weight 3.0 on every run):
+    one logits row from the conditional and the unconditional stream of the same image,
+
+        l = l_u + w * (l_c - l_u).
+
+    w = 1 gives the conditional row, w = 0 the unconditional one.  The inputs are stored logits.
+    `storage` names the dtype the mixed row is stored in before verification:
+      'f64'          the plain formula in fp64;
+      'f32', 'bf16'  the stored code is a decision taken from floating point, so it is taken in the
+                     precision of the library's arithmetic: d = fl32(l_c - l_u), l = fl32(w * d + l_u)
+                     with a single rounding (a fused multiply-add), then rounded to the storage dtype.
+                     The product w * d of two fp32 numbers and its sum with a bf16 / fp32 value are
+                     exact in fp64 for any logits of ordinary magnitude, so rounding the fp64 result to
+                     fp32 is that single rounding.
+    Returns fp64 values."""
+    lc = np.asarray(logits_cond, dtype=np.float64)
+    lu = np.asarray(logits_uncond, dtype=np.float64)
+    if storage == "f64":
+        return lu + float(weight) * (lc - lu)
+    w32 = np.float64(np.float32(weight))
+    with np.errstate(invalid="ignore", over="ignore"):
+        d = (lc - lu).astype(np.float32).astype(np.float64)
+        mixed = (w32 * d + lu).astype(np.float32)
+    if storage == "f32":
+        return mixed.astype(np.float64)
+    if storage == "bf16":
+        bits = np.ascontiguousarray(mixed).view(np.uint32).astype(np.uint64)
+        rounded = ((bits + np.uint64(0x7FFF) + ((bits >> np.uint64(16)) & np.uint64(1)))
+                   >> np.uint64(16)) << np.uint64(16)
+        out = rounded.astype(np.uint32).view(np.float32).astype(np.float64)
+        return np.where(np.isfinite(mixed), out, mixed.astype(np.float64))
+    raise ValueError(storage)
+
+
 @dataclass
 class QDesc:
     """The law a draft token was drawn from (Step 1: each draft carries the

@@ -24,7 +24,7 @@ import numpy as np
 
 from . import philox
 from .model import KVCache, OracleModel, round_to_storage
-from .sampling import (FLAG_DONE, Q_ONEHOT, Q_ROW, Q_UNIFORM, QDesc, VerifyResult, icdf,
+from .sampling import (FLAG_DONE, Q_ONEHOT, Q_ROW, Q_UNIFORM, QDesc, VerifyResult, guided_logits, icdf,
                        verify_window, warp)
 
 INIT_RANDOM = 0       # Sec. 4.2: uniform random candidate
@@ -106,6 +106,37 @@ class RecomputeModel:
     def step_logits(self, committed, drafts_in):
         full = self.model.forward_full(list(committed) + list(drafts_in))
         return full[len(committed) - 1:]
+
+
+class GuidedModel:
+    """Two streams of one image under classifier-free guidance (Sec. 5.1): the conditional stream
+    sees the text prompt, the unconditional one a prompt of its own (same length); both see the same
+    image tokens.  Every stream's logits are stored in `storage` first, then mixed row by row
+    (sampling.guided_logits) and stored again; drafts, uniforms and every decision are shared, since
+    there is one verification per image, on the mixed rows."""
+
+    def __init__(self, model_cond, model_uncond, prompt_uncond, weight: float, storage: str = "f32"):
+        self.mc, self.mu = model_cond, model_uncond
+        self.prompt_u = [int(t) for t in prompt_uncond]
+        self.weight, self.storage = float(weight), storage
+        self.p_len = None
+
+    def prefill(self, prompt):
+        assert len(prompt) == len(self.prompt_u), "both streams use prompts of one length"
+        self.p_len = len(prompt)
+        self.mc.prefill(list(prompt))
+        self.mu.prefill(list(self.prompt_u))
+
+    def stream_logits(self, committed, drafts_in):
+        """Stored logits of the two streams, (conditional, unconditional)."""
+        image = list(committed[self.p_len:])
+        lc = round_to_storage(self.mc.step_logits(list(committed), drafts_in), self.storage)
+        lu = round_to_storage(self.mu.step_logits(self.prompt_u + image, drafts_in), self.storage)
+        return lc, lu
+
+    def step_logits(self, committed, drafts_in):
+        lc, lu = self.stream_logits(committed, drafts_in)
+        return guided_logits(lc, lu, self.weight, self.storage)
 
 
 class TableModel:
