@@ -110,6 +110,14 @@ typedef struct {
   int32_t n_generate;  /* N, image tokens to generate per sequence                              */
   int32_t seq_base;    /* global id of sequence 0 of this batch (Philox counter word 2): a batch    */
                        /* sharded over several GPUs draws the same numbers wherever a sequence runs  */
+  float guidance;      /* classifier-free guidance weight w (Sec. 5.1 uses 3.0); 0 = no guidance.   */
+                       /* With w != 0 the batch holds two streams per image: sequence 2i is image   */
+                       /* i's conditional stream, 2i+1 its unconditional one (prompts of one length, */
+                       /* different tokens); both share drafts, uniforms and decisions.  Each        */
+                       /* stream's logits are stored in cfg.dtype; verification reads every row as   */
+                       /* l_u + w (l_c - l_u), evaluated in fp32 as fma(w, l_c - l_u, l_u) and       */
+                       /* rounded to cfg.dtype.  Outputs then have batch / 2 entries (one per image)  */
+                       /* and the Philox sequence id is seq_base + i.  sjd_verify(_static): must be 0 */
 } sjd_sample_cfg;
 
 /* Results of one step.  Any pointer may be NULL (that output is skipped). */

@@ -57,7 +57,8 @@ class sjd_weights(C.Structure):
 
 class sjd_sample_cfg(C.Structure):
     _fields_ = [("temperature", C.c_float), ("top_k", C.c_int32), ("seed", C.c_uint64), ("window", C.c_int32),
-                ("init", C.c_int32), ("grid_stride", C.c_int32), ("n_generate", C.c_int32), ("seq_base", C.c_int32)]
+                ("init", C.c_int32), ("grid_stride", C.c_int32), ("n_generate", C.c_int32), ("seq_base", C.c_int32),
+                ("guidance", C.c_float)]
 
 
 class sjd_step_out(C.Structure):
@@ -155,9 +156,9 @@ def make_model_cfg(wl, max_batch: int, max_seq: int, max_window: int) -> sjd_mod
 
 
 def make_sample_cfg(temperature=1.0, top_k=2000, seed=0, window=16, init=SJD_INIT_RANDOM, grid_stride=0,
-                    n_generate=0, seq_base=0) -> sjd_sample_cfg:
+                    n_generate=0, seq_base=0, guidance=0.0) -> sjd_sample_cfg:
     return sjd_sample_cfg(float(temperature), int(top_k), int(seed), int(window), int(init), int(grid_stride),
-                          int(n_generate), int(seq_base))
+                          int(n_generate), int(seq_base), float(guidance))
 
 
 class StepOut:

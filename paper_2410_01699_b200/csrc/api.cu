@@ -15,6 +15,7 @@ int check_sample_cfg(const sjd_sample_cfg *s, int vocab) {
   if (s->init < SJD_INIT_RANDOM || s->init > SJD_INIT_COPY_LEFT) return SJD_ERR_BAD_ARG;
   if (s->init == SJD_INIT_COPY_ABOVE && s->grid_stride < 1) return SJD_ERR_BAD_ARG;
   if (s->seq_base < 0) return SJD_ERR_BAD_ARG;
+  if (!(s->guidance == s->guidance) || s->guidance > 1e6f || s->guidance < -1e6f) return SJD_ERR_BAD_ARG;
   (void)vocab;
   return SJD_OK;
 }
@@ -36,6 +37,7 @@ int verify_isolated(int batch, int window, int vocab, int logits_dtype, const vo
   if (logits_dtype != SJD_F32 && logits_dtype != SJD_BF16) return SJD_ERR_UNSUPPORTED;
   if (window > 64) return SJD_ERR_CAPACITY;
   if (!(sample->temperature > 0.0f) || sample->top_k < 1 || sample->seq_base < 0) return SJD_ERR_BAD_ARG;
+  if (sample->guidance != 0.0f) return SJD_ERR_UNSUPPORTED;   // guidance pairs the streams of a context (sjd_step)
   if (((uintptr_t)scratch & 15u) != 0) return SJD_ERR_BAD_ARG;
 
   const size_t rows = (size_t)batch * window;

@@ -204,6 +204,11 @@ struct VerifyParams {
   uint32_t seed_lo, seed_hi;
   uint32_t seq_base;       // global id of sequence 0 (batch sharded across GPUs)
   int e2e;                 // 1: update SeqState (window slide); 0: isolated verification
+  // Classifier-free guidance (paired != 0): sequences 2i and 2i + 1 of the forward pass are the conditional
+  // and the unconditional stream of image i; B counts images; every logits row is read as
+  // l_u + guidance * (l_c - l_u) rounded to the storage dtype, and the slide writes both streams' state.
+  int paired;
+  float guidance;
   SeqState st;
   sjd_step_out out;
 };

@@ -203,15 +203,16 @@ __global__ void prefill_inputs_kernel(const int32_t *prompt, int P, int c0, int 
   }
 }
 
-__global__ void get_window_kernel(SeqState st, sjd_step_out o, int W) {
-  const int b = blockIdx.x;
+// one block per image; `streams` sequences per image hold the same window (2 under guidance), the first is read
+__global__ void get_window_kernel(SeqState st, sjd_step_out o, int W, int streams) {
+  const int b = blockIdx.x, sb = b * streams;
   for (int k = threadIdx.x; k < W; k += blockDim.x) {
-    const int i = b * W + k;
-    if (o.draft) o.draft[i] = st.draft[i];
-    if (o.q_kind) o.q_kind[i] = st.q_kind[i];
-    if (o.q_draft) o.q_draft[i] = st.q_draft[i];
+    const int i = b * W + k, si = sb * W + k;
+    if (o.draft) o.draft[i] = st.draft[si];
+    if (o.q_kind) o.q_kind[i] = st.q_kind[si];
+    if (o.q_draft) o.q_draft[i] = st.q_draft[si];
   }
-  if (threadIdx.x == 0 && o.total_committed) o.total_committed[b] = st.n[b];
+  if (threadIdx.x == 0 && o.total_committed) o.total_committed[b] = st.n[sb];
 }
 
 }  // namespace
@@ -526,6 +527,12 @@ int run_verify(sjd_ctx *c, const sjd_step_out *out, cudaStream_t stream) {
   p.seq_base = (uint32_t)c->sample.seq_base;
   p.e2e = 1;
   p.st = st;
+  if (c->sample.guidance != 0.0f) {   // sequences 2i, 2i + 1 = conditional and unconditional stream of image i
+    p.paired = 1;
+    p.guidance = c->sample.guidance;
+    p.B = c->batch / 2;
+    p.done_counter = p.seq_counter + p.B;
+  }
   if (out) p.out = *out;
   return launch_verify(p, c->cfg.dtype, stream);
 }
@@ -674,6 +681,7 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
   if (sample->n_generate < 0) return SJD_ERR_BAD_ARG;
   if (batch > c->cfg.max_batch || sample->window > c->cfg.max_window) return SJD_ERR_CAPACITY;
   if ((long)prompt_len + sample->n_generate > c->cfg.max_seq) return SJD_ERR_CAPACITY;
+  if (sample->guidance != 0.0f && batch % 2 != 0) return SJD_ERR_BAD_ARG;   // streams come in pairs
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   c->sample = *sample;
   c->batch = batch;
@@ -796,7 +804,8 @@ extern "C" int sjd_step(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) 
 extern "C" int sjd_get_window(sjd_ctx *c, const sjd_step_out *out, void *cuda_stream) {
   if (!c || !out) return SJD_ERR_BAD_ARG;
   if (!c->prefilled) return SJD_ERR_STATE;
-  get_window_kernel<<<c->batch, 64, 0, (cudaStream_t)cuda_stream>>>(c->state(), *out, c->window);
+  const int streams = c->sample.guidance != 0.0f ? 2 : 1;
+  get_window_kernel<<<c->batch / streams, 64, 0, (cudaStream_t)cuda_stream>>>(c->state(), *out, c->window, streams);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -62,6 +62,7 @@ struct Elt<float> {
   __device__ static __forceinline__ uint32_t key(uint32_t b) { return (b & 0x80000000u) ? ~b : (b | 0x80000000u); }
   __device__ static __forceinline__ uint32_t unkey(uint32_t k) { return (k & 0x80000000u) ? (k ^ 0x80000000u) : ~k; }
   __device__ static __forceinline__ float val(uint32_t b) { return __uint_as_float(b); }
+  __device__ static __forceinline__ uint32_t bits(float x) { return __float_as_uint(x); }
 };
 
 template <>
@@ -91,6 +92,7 @@ struct Elt<__nv_bfloat16> {
   __device__ static __forceinline__ uint32_t key(uint32_t b) { return (b & 0x8000u) ? (~b & 0xFFFFu) : (b | 0x8000u); }
   __device__ static __forceinline__ uint32_t unkey(uint32_t k) { return (k & 0x8000u) ? (k ^ 0x8000u) : (~k & 0xFFFFu); }
   __device__ static __forceinline__ float val(uint32_t b) { return __uint_as_float(b << 16); }
+  __device__ static __forceinline__ uint32_t bits(float x) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x)); }
 };
 
 // ------------------------------------------------------------------------------------ scratch
@@ -113,29 +115,41 @@ struct Scratch {
 template <typename T>
 struct Row {
   const T *g;
+  const T *g2;   // classifier-free guidance: the unconditional stream's row (g is the conditional one), or null
+  float gw;      // guidance weight
   int V, off, NV;
   const uint4 *s;  // shared-memory copy (sanitised), or null
 
-  __device__ void init(const T *row, int v) {
+  __device__ void init(const T *row, int v, const T *row_uncond = nullptr, float weight = 0.0f) {
     g = row;
+    g2 = row_uncond;
+    gw = weight;
     V = v;
     off = (int)(((uintptr_t)row & 15u) / sizeof(T));
     NV = (off + v + Elt<T>::VEC - 1) / Elt<T>::VEC;
     s = nullptr;
+  }
+  // bits of element i as the verification sees it: the stored logit, or under guidance the mix
+  // l_u + w * (l_c - l_u) (one subtraction, one fused multiply-add in fp32) rounded to the storage dtype
+  __device__ __forceinline__ uint32_t raw_bits(int i) const {
+    const uint32_t b = Elt<T>::load_bits(g + i);
+    if (!g2) return b;
+    const float c = Elt<T>::val(b), u = Elt<T>::val(Elt<T>::load_bits(g2 + i));
+    return Elt<T>::bits(fmaf(gw, c - u, u));
   }
   // sanitised vector straight from global memory
   __device__ __forceinline__ uint4 load_global(int j, uint32_t &bad) const {
     using E = Elt<T>;
     const int i0 = j * E::VEC - off;
     uint4 v;
-    if (i0 >= 0 && i0 + E::VEC <= V) {
+    if (!g2 && i0 >= 0 && i0 + E::VEC <= V) {
       v = __ldg(reinterpret_cast<const uint4 *>(g + i0));
     } else {
       v = make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int t = 0; t < E::VEC; ++t) {
         const int i = i0 + t;
-        E::set(v, t, (i >= 0 && i < V) ? E::load_bits(g + i) : E::NEG_INF);
+        E::set(v, t, (i >= 0 && i < V) ? raw_bits(i) : E::NEG_INF);
       }
     }
 #pragma unroll
@@ -157,7 +171,7 @@ struct Row {
       if (sizeof(T) == 2) return (uint32_t) reinterpret_cast<const unsigned short *>(s)[i + off];
       return reinterpret_cast<const uint32_t *>(s)[i + off];
     }
-    uint32_t b = Elt<T>::load_bits(g + i);
+    const uint32_t b = raw_bits(i);
     return Elt<T>::bad(b) ? Elt<T>::NEG_INF : b;
   }
 };
@@ -488,6 +502,26 @@ __device__ __forceinline__ uint32_t key_pair(uint32_t w) {
 }
 __device__ __forceinline__ uint32_t word_of(const uint4 &v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
 
+// One 16-byte vector of a row under classifier-free guidance: per entry l_u + w * (l_c - l_u) with one
+// subtraction and one fused multiply-add in fp32, rounded to bf16 (the same arithmetic as Row::raw_bits).
+__device__ __forceinline__ uint4 mix_vec_bf16(const uint4 &c, const uint4 &u, float w) {
+  uint32_t o[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t cx = word_of(c, k), ux = word_of(u, k);
+    const float c0 = __uint_as_float(cx << 16), c1 = __uint_as_float(cx & 0xFFFF0000u);
+    const float u0 = __uint_as_float(ux << 16), u1 = __uint_as_float(ux & 0xFFFF0000u);
+    const __nv_bfloat162 m = __floats2bfloat162_rn(fmaf(w, c0 - u0, u0), fmaf(w, c1 - u1, u1));
+    o[k] = *reinterpret_cast<const uint32_t *>(&m);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+// vector j of a bf16 row (16-byte aligned), mixed with the unconditional stream's row when there is one
+__device__ __forceinline__ uint4 rr_load_vec(const uint4 *g, const uint4 *g2, float w, int j) {
+  const uint4 c = __ldg(g + j);
+  return g2 ? mix_vec_bf16(c, __ldg(g2 + j), w) : c;
+}
+
 // ------------------------------------------------------------------------------------ register-resident row, few barriers
 // The whole treatment of one window row (Eqs. 1-3) for bf16 rows a block can hold in registers, laid
 // out warp by warp: warp w owns chunks 8w .. 8w+7 (32 vectors each, the chunks of chunk_sums), lane l
@@ -509,15 +543,15 @@ __device__ __forceinline__ uint4 reg_slot(const RegRow &r, int i) {   // i is wa
 
 // load + maximum; publishes the entry at index d (if any) in sc.d_bits.  One barrier.  Returns the
 // block-wide maximum key; 0xFFFF if the row holds a NaN.
-__device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int d_slot, Scratch &sc, bool zero_hist,
-                                uint4 *stash) {
+__device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, const uint4 *g2, float gw, int NV, int d, int d_slot,
+                                Scratch &sc, bool zero_hist) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
   const int j0 = warp * 256 + lane;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int j = j0 + i * 32;
-    row.v[i] = j < NV ? __ldg(g + j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+    row.v[i] = j < NV ? rr_load_vec(g, g2, gw, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
   }
   if (zero_hist)
     for (int i = tid; i < 4096; i += nt) sc.hist12[i] = 0;
@@ -526,7 +560,6 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, int NV, int d, int 
   for (int i = 0; i < 8; ++i) {
 #pragma unroll
     for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(row.v[i], w)));
-    if (stash && j0 + i * 32 < NV) stash[j0 + i * 32] = row.v[i];
     if (d >= 0 && (d >> 3) == j0 + i * 32) {   // this thread holds entry d
       const uint32_t wd = word_of(row.v[i], (d >> 1) & 3);
       sc.d_bits[d_slot] = (d & 1) ? wd >> 16 : wd & 0xFFFFu;
@@ -802,12 +835,13 @@ struct RowFast {   // statistics of a row on this route
 // statistics of one row: 4 barriers.  false: general route.
 // `want_chunks`: mask the entries below the threshold in `row` and leave the chunk sums of the row's
 // weights in sc.chunk_sum (needed to sample from the row).
-__device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d, int d_slot, int top_k, float inv_t,
-                              Scratch &sc, RowFast &out, bool want_chunks) {
+__device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, const __nv_bfloat16 *g2, float gw, int V, int d,
+                              int d_slot, int top_k, float inv_t, Scratch &sc, RowFast &out, bool want_chunks) {
   using E = Elt<__nv_bfloat16>;
   const int NV = V >> 3;
   const bool need_select = top_k < V;
-  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), NV, d, d_slot, sc, need_select, nullptr);
+  const uint32_t kmax = rr_load_max(row, reinterpret_cast<const uint4 *>(g), reinterpret_cast<const uint4 *>(g2), gw, NV, d,
+                                    d_slot, sc, need_select);
   if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
   SJD_TL(TL_VERIFY, 20, threadIdx.x == 0);   // row loaded, maximum known
   uint32_t tau_key = 0;
@@ -834,18 +868,35 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, int V, int d,
   return true;
 }
 
+// The logits rows of window slot k of image b: this iteration's (p) and the one the draft was drawn from
+// (q, row qr of the other buffer); under guidance the unconditional stream's rows beside them (else null).
 template <typename T>
-__device__ bool fast_row(const VerifyParams &p, Scratch &sc, uint4 *stage, int r, int b, int kind, int d, int qr, int cur,
-                         const T *qbase, const T *pbase, float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
+struct RowRefs {
+  const T *p, *p2, *q, *q2;
+};
+template <typename T>
+__device__ __forceinline__ RowRefs<T> row_refs(const VerifyParams &p, int b, int k, int qr, int cur) {
+  const int sb = p.paired ? 2 * b : b;
+  RowRefs<T> rr;
+  rr.p = reinterpret_cast<const T *>(p.logits[cur]) + ((size_t)sb * p.W + k) * p.V;
+  rr.q = reinterpret_cast<const T *>(p.logits[cur ^ 1]) + ((size_t)sb * p.W + qr) * p.V;
+  rr.p2 = p.paired ? rr.p + (size_t)p.W * p.V : nullptr;
+  rr.q2 = p.paired ? rr.q + (size_t)p.W * p.V : nullptr;
+  return rr;
+}
+
+template <typename T>
+__device__ bool fast_row(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
+                         const RowRefs<T> &rows, float inv_t, float u_acc, float u_draft, RowOut &ro) {
   return false;
 }
 
 constexpr int kResampleDeferred = -2;   // RowOut.resample_tok of a rejected row whose Eq. 2 draw is still to be made
 
 template <>
-__device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint4 *stage, int r, int b, int kind, int d,
-                                        int qr, int cur, const __nv_bfloat16 *qbase, const __nv_bfloat16 *pbase,
-                                        float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
+__device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
+                                        const RowRefs<__nv_bfloat16> &rows, float inv_t, float u_acc, float u_draft,
+                                        RowOut &ro) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x;
   const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
@@ -863,12 +914,19 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
     if (p.prev_stats_valid) {
       qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
       if (qs.flags != 0 || !(qs.xmax > -FLT_MAX) || qs.tau_key == 0x7FFFu || qs.tau_key == 0x8000u) return false;
-      const uint32_t bits = d_ok ? (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(qbase) + d) : E::NEG_INF;
+      uint32_t bits = E::NEG_INF;
+      if (d_ok) {
+        bits = E::load_bits(rows.q + d);
+        if (rows.q2) {
+          const float cq = E::val(bits), uq = E::val(E::load_bits(rows.q2 + d));
+          bits = E::bits(fmaf(p.guidance, cq - uq, uq));
+        }
+      }
       if (E::bad(bits)) return false;
       q_d = d_ok ? (E::key(bits) >= qs.tau_key ? exp2_neg((E::val(bits) - qs.xmax) * scale) : 0.0f) / qs.z : 1.0f;
     } else {
       RowFast qfast;
-      if (!rr_statistics(row, qbase, V, dd, 0, p.top_k, inv_t, sc, qfast, false)) return false;
+      if (!rr_statistics(row, rows.q, rows.q2, p.guidance, V, dd, 0, p.top_k, inv_t, sc, qfast, false)) return false;
       qs = qfast.st;
       qs.z = (float)(qfast.z_hist >= 0.0 ? qfast.z_hist : rr_prefix(NC, sc).total);
       if (tid == 0) p.stats[cur ^ 1][r] = qs;
@@ -883,7 +941,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, uint
   SJD_TL(TL_VERIFY, 10, tid == 0);
   // ---- this iteration's distribution (entries below the threshold are -inf in `row` from here on)
   RowFast pfast;
-  if (!rr_statistics(row, pbase, V, dd, 1, p.top_k, inv_t, sc, pfast, true)) return false;
+  if (!rr_statistics(row, rows.p, rows.p2, p.guidance, V, dd, 1, p.top_k, inv_t, sc, pfast, true)) return false;
   const WarpPrefix wpp = rr_prefix(NC, sc);
   RowStats ps = pfast.st;
   ps.z = (float)wpp.total;
@@ -928,7 +986,7 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int W = p.W, V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
-  const int w_eff = p.w_eff ? p.w_eff[b] : W;
+  const int w_eff = p.w_eff ? p.w_eff[p.paired ? 2 * b : b] : W;
   RowOut *ro = p.row_out + (size_t)b * W;
   if (tid < 32) {
     int first = w_eff;
@@ -942,16 +1000,18 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
   __syncthreads();
   if (a < 0) return;
   const int r = b * W + a;
-  const int kind = p.q_kind ? p.q_kind[r] : SJD_Q_ROW;
-  const int d = p.draft[r];
-  const int qr = p.q_row ? p.q_row[r] : a;
-  const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
+  const int sb = p.paired ? 2 * b : b;   // the sequence whose state holds the window (both streams hold the same)
+  const int kind = p.q_kind ? p.q_kind[sb * W + a] : SJD_Q_ROW;
+  const int d = p.draft[sb * W + a];
+  const int qr = p.q_row ? p.q_row[sb * W + a] : a;
+  const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
   const Philox4 rnd = philox4x32_10((uint32_t)(base + a), step, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo,
                                     p.seed_hi);
   const float u_res = u24(rnd.w[1]);
   const float scale = (1.0f / p.temperature) * 1.4426950408889634f;
-  const __nv_bfloat16 *qbase = reinterpret_cast<const __nv_bfloat16 *>(p.logits[cur ^ 1]) + ((size_t)b * W + qr) * V;
-  const __nv_bfloat16 *pbase = reinterpret_cast<const __nv_bfloat16 *>(p.logits[cur]) + (size_t)r * V;
+  const RowRefs<__nv_bfloat16> rows = row_refs<__nv_bfloat16>(p, b, a, qr, cur);
+  const uint4 *pg = reinterpret_cast<const uint4 *>(rows.p), *pg2 = reinterpret_cast<const uint4 *>(rows.p2);
+  const uint4 *qg = reinterpret_cast<const uint4 *>(rows.q), *qg2 = reinterpret_cast<const uint4 *>(rows.q2);
   auto load_stats = [](const RowStats *g) {
     const uint4 u = __ldcg(reinterpret_cast<const uint4 *>(g));
     RowStats st;
@@ -971,8 +1031,7 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int j = j0 + i * 32;
-    row.v[i] = j < NV ? __ldg(reinterpret_cast<const uint4 *>(pbase) + j)
-                      : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+    row.v[i] = j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
   }
 
   // probabilities straight from one fused multiply-add per entry: p_i = 2^(x_i * scale + c) with
@@ -983,7 +1042,7 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
     const int j = j0 + i * 32;
     const uint4 pv = reg_slot(row, i);
     uint4 qv = make_uint4(0, 0, 0, 0);
-    if (kind == SJD_Q_ROW && j < NV) qv = __ldg(reinterpret_cast<const uint4 *>(qbase) + j);
+    if (kind == SJD_Q_ROW && j < NV) qv = rr_load_vec(qg, qg2, p.guidance, j);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const uint32_t px = word_of(pv, k), qx = word_of(qv, k);
@@ -1057,13 +1116,17 @@ __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int t
 
 // ------------------------------------------------------------------------------------ finalize
 // Run by every thread of the last block of sequence b: accept scan (warp 0), then the commit, the
-// window slide and the next inputs in parallel over the window slots.
+// window slide and the next inputs in parallel over the window slots.  Under guidance "sequence b" is
+// image b: its window is kept twice, in the state of the conditional stream (sequence 2b) and of the
+// unconditional one (2b + 1); both copies are read from the first and written identically, except that
+// each stream's fixed tokens (and so its next first input) go to its own token array.
 __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, Scratch &sc) {
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
   const int W = p.W;
-  const int w_eff = p.w_eff ? p.w_eff[b] : W;
+  const int sb = p.paired ? 2 * b : b, n_streams = p.paired ? 2 : 1;
+  const int w_eff = p.w_eff ? p.w_eff[sb] : W;
   const RowOut *ro = p.row_out + (size_t)b * W;
-  const int32_t *old_draft = p.draft + (size_t)b * W;
+  const int32_t *old_draft = p.draft + (size_t)sb * W;
   const sjd_step_out &o = p.out;
   if (tid < 32) {
     int first = w_eff;
@@ -1087,7 +1150,7 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
   const int a = sc.sel_chunk;
   uint32_t flags = sc.sel_bin;
   const int m = (a < w_eff) ? a + 1 : w_eff;
-  const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
+  const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
   const int n2 = base + m;
 
   // fixed tokens: accepted drafts, then the resampled one
@@ -1096,7 +1159,8 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
     if (i < a) tok = old_draft[i];
     else if (i == a && a < w_eff) tok = __ldcg(&ro[a].resample_tok);
     if (o.committed) o.committed[(size_t)b * W + i] = tok;
-    if (p.e2e && i < m) p.st.committed[(size_t)b * p.st.max_seq + base + i] = tok;
+    if (p.e2e && i < m)
+      for (int s2 = 0; s2 < n_streams; ++s2) p.st.committed[(size_t)(sb + s2) * p.st.max_seq + base + i] = tok;
   }
 
   int w2 = 0, kept = 0;
@@ -1109,10 +1173,7 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
     kept = (a < w_eff) ? (w_eff - a - 1) : 0;
     w2 = kept;
   }
-  int32_t *nd = p.e2e ? p.st.draft + (size_t)b * W : nullptr;
-  int32_t *nk = p.e2e ? p.st.q_kind + (size_t)b * W : nullptr;
-  int32_t *nr = p.e2e ? p.st.q_row + (size_t)b * W : nullptr;
-  float *nq = p.e2e ? p.st.q_draft + (size_t)b * W : nullptr;
+  int32_t *nd = p.e2e ? p.st.draft + (size_t)sb * W : nullptr;
   // A copied slot may read a slot filled just before it (and a token fixed above), so the copy
   // initialisations fill the window in order on one thread; everything else goes slot-parallel.
   const bool serial = p.e2e && p.st.init != SJD_INIT_RANDOM;
@@ -1132,7 +1193,7 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
                          : p.st.init == SJD_INIT_COPY_LEFT ? 1 : 0;
       const int src = t_pos - stride;
       if (p.st.init != SJD_INIT_RANDOM && stride > 0 && src >= p.st.prompt_len) {
-        tok = src < n2 ? p.st.committed[(size_t)b * p.st.max_seq + src] : nd[src - n2];
+        tok = src < n2 ? p.st.committed[(size_t)sb * p.st.max_seq + src] : nd[src - n2];
         kind = SJD_Q_ONEHOT;
         q = 1.0f;
       } else {
@@ -1144,10 +1205,13 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
       }
     }
     if (p.e2e) {
-      nd[s] = tok;
-      nk[s] = kind;
-      nr[s] = qrow;
-      nq[s] = q;
+      for (int s2 = 0; s2 < n_streams; ++s2) {
+        const size_t at = (size_t)(sb + s2) * W + s;
+        p.st.draft[at] = tok;
+        p.st.q_kind[at] = kind;
+        p.st.q_row[at] = qrow;
+        p.st.q_draft[at] = q;
+      }
     }
     if (o.draft) o.draft[(size_t)b * W + s] = tok;
     if (o.q_kind) o.q_kind[(size_t)b * W + s] = kind;
@@ -1155,18 +1219,22 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
   }
   __syncthreads();   // the new window and the fixed tokens are read below
   if (p.e2e) {
-    int32_t *it = p.st.in_tok + (size_t)b * W;
-    int32_t *ip = p.st.in_pos + (size_t)b * W;
-    for (int k = tid; k < W; k += nt) {
-      const bool act = k < w2;
-      it[k] = act ? (k == 0 ? p.st.committed[(size_t)b * p.st.max_seq + n2 - 1] : nd[k - 1]) : 0;
-      ip[k] = act ? n2 - 1 + k : -1;
+    for (int s2 = 0; s2 < n_streams; ++s2) {
+      int32_t *it = p.st.in_tok + (size_t)(sb + s2) * W;
+      int32_t *ip = p.st.in_pos + (size_t)(sb + s2) * W;
+      for (int k = tid; k < W; k += nt) {
+        const bool act = k < w2;
+        it[k] = act ? (k == 0 ? p.st.committed[(size_t)(sb + s2) * p.st.max_seq + n2 - 1] : nd[k - 1]) : 0;
+        ip[k] = act ? n2 - 1 + k : -1;
+      }
     }
   }
   if (tid == 0) {
     if (p.e2e) {
-      p.st.n[b] = n2;
-      p.st.w_eff[b] = w2;
+      for (int s2 = 0; s2 < n_streams; ++s2) {
+        p.st.n[sb + s2] = n2;
+        p.st.w_eff[sb + s2] = w2;
+      }
     }
     if (o.n_accepted) o.n_accepted[b] = a;
     if (o.n_committed) o.n_committed[b] = m;
@@ -1189,36 +1257,35 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
 
   const int r = blockIdx.x;
   const int b = r / p.W, k = r % p.W;
+  const int sb = p.paired ? 2 * b : b;   // sequence whose state describes the window (under guidance both streams' do)
+  const int rs = sb * p.W + k;
   const int tid = threadIdx.x;
-  const int w_eff = p.w_eff ? p.w_eff[b] : p.W;
+  const int w_eff = p.w_eff ? p.w_eff[sb] : p.W;
   const uint32_t step = p.step_ptr ? *p.step_ptr : p.step;
   const int cur = p.step_ptr ? (int)(step & 1u) : 0;
   const float inv_t = 1.0f / p.temperature;
 
   if (k < w_eff) {
-    const int kind = p.q_kind ? p.q_kind[r] : SJD_Q_ROW;
-    const int d = p.draft[r];
+    const int kind = p.q_kind ? p.q_kind[rs] : SJD_Q_ROW;
+    const int d = p.draft[rs];
     const bool d_ok = d >= 0 && d < p.V;
-    const int qr = p.q_row ? p.q_row[r] : k;
-    const int base = p.e2e ? p.st.n[b] : (p.base_pos ? p.base_pos[b] : 0);
+    const int qr = p.q_row ? p.q_row[rs] : k;
+    const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
     const Philox4 rnd = philox4x32_10((uint32_t)(base + k), step, p.seq_base + (uint32_t)b, kStreamVerify,
                                       p.seed_lo, p.seed_hi);
     const float u_acc = u24(rnd.w[0]), u_res = u24(rnd.w[1]), u_draft = u24(rnd.w[2]);
-
-    const T *qbase = reinterpret_cast<const T *>(p.logits[cur ^ 1]) + ((size_t)b * p.W + qr) * p.V;
-    const T *pbase = reinterpret_cast<const T *>(p.logits[cur]) + (size_t)r * p.V;
+    const RowRefs<T> rows = row_refs<T>(p, b, k, qr, cur);
 
     RowOut fast_out;
-    const bool fast_done = p.fast && (((uintptr_t)qbase | (uintptr_t)pbase) & 15u) == 0 &&
-                           fast_row<T>(p, sc, stage, r, b, kind, d, qr, cur, qbase, pbase, inv_t, u_acc, u_res, u_draft,
-                                       fast_out);
+    const bool fast_done = p.fast && (((uintptr_t)rows.q | (uintptr_t)rows.p) & 15u) == 0 &&
+                           fast_row<T>(p, sc, r, b, kind, d, qr, cur, rows, inv_t, u_acc, u_draft, fast_out);
     if (fast_done) {
       if (tid == 0) p.row_out[r] = fast_out;
     } else {
     __syncthreads();
     // ---- the law of the draft
     Row<T> qrow;
-    qrow.init(qbase, p.V);
+    qrow.init(rows.q, p.V, rows.q2, p.guidance);
     RowStats qs;
     qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
     PRowWeights<T> qf;
@@ -1244,7 +1311,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     SJD_TL(TL_VERIFY, 10, tid == 0);   // the draft's law is known
     // ---- this iteration's distribution
     Row<T> prow;
-    prow.init(pbase, p.V);
+    prow.init(rows.p, p.V, rows.p2, p.guidance);
     PRowWeights<T> pf;
     const RowStats ps = row_statistics<T>(prow, stage, sc, p.top_k, inv_t, pf);
     if (tid == 0) p.stats[cur][r] = ps;

@@ -145,12 +145,21 @@ class LockStepSequence:
     are only measured (`errors_plain`), the decisions and the asserted tolerance stay with the checker
     whose cache is rounded to the storage dtype."""
 
-    def __init__(self, wl, weights_cpu, prompt_row, scfg, seq_id, logit_tol, also_plain_cache=False):
+    def __init__(self, wl, weights_cpu, prompt_row, scfg, seq_id, logit_tol, also_plain_cache=False, guidance=0.0,
+                 prompt_uncond=None):
+        """With guidance != 0 the sequence is an image with two streams (prompt_row: the conditional
+        prompt, prompt_uncond: the unconditional one); `step` then takes the library's stored logits of
+        both streams, checks each against the checker's stream and re-takes the decisions from their
+        mix (oracle.sampling.guided_logits in the storage dtype)."""
         from oracle.model import OracleModel
-        from oracle.sjd import CachedModel, sjd_begin
+        from oracle.sjd import CachedModel, GuidedModel, sjd_begin
         self.wl, self.scfg, self.tol = wl, scfg, logit_tol
         om = OracleModel(oracle_model_cfg(wl), weights_cpu)
         self.model = CachedModel(om, wl.prompt_len + scfg.n_generate + 1, kv_storage=wl.dtype)
+        self.guidance = float(guidance)
+        if self.guidance != 0.0:
+            uncond = CachedModel(om, wl.prompt_len + scfg.n_generate + 1, kv_storage=wl.dtype)
+            self.model = GuidedModel(self.model, uncond, prompt_uncond, self.guidance, wl.dtype)
         self.prompt = [int(t) for t in prompt_row]
         self.model.prefill(self.prompt)
         self.errors = LogitErrors()
@@ -194,6 +203,21 @@ class LockStepSequence:
             return
         self.steps += 1
         drafts, qdescs = list(st.drafts), list(st.qdescs)
+        if self.guidance != 0.0:
+            from oracle.sampling import guided_logits
+            gpu_c, gpu_u = gpu_logits_rows
+            if check_logits:
+                own_c, own_u = self.model.stream_logits(st.committed, st.drafts[:w_eff - 1])
+                for own, got in ((own_c, gpu_c), (own_u, gpu_u)):
+                    # (the checker's streams are already rounded to the storage dtype: compare values)
+                    diff = np.abs(own - got[:w_eff])
+                    self.max_logit_err = max(self.max_logit_err, float(diff.max()))
+                    half_ulp = storage_half_ulp(own, scfg.logits_dtype)
+                    self.max_logit_excess = max(self.max_logit_excess, float((diff - half_ulp).max()))
+                    self.errors.add(diff, half_ulp)
+                    assert not self.logit_failures(diff, half_ulp).any(), f"step {self.steps}: stream logits off"
+            gpu_logits_rows = guided_logits(gpu_c[:w_eff], gpu_u[:w_eff], self.guidance, scfg.logits_dtype)
+            check_logits = False
         if check_logits:
             own = self.model.step_logits(st.committed, st.drafts[:w_eff - 1])
             # the library's value is its fp32 result rounded to the storage dtype: allow the stated

@@ -105,6 +105,62 @@ def test_tiny_top1_is_greedy_decoding():
     assert steps <= 48
 
 
+def run_lockstep_guided(wl, images, guidance, max_steps=None, init=INIT_RANDOM, window=None, n_generate=None):
+    """Lock-step under classifier-free guidance: 2 * images sequences in the library (conditional and
+    unconditional stream of each image, prompts of one length with different tokens), one checker per image."""
+    window = window or wl.window
+    n_generate = wl.n_generate if n_generate is None else n_generate
+    weights = make_weights(wl, gain_jitter=0.1)
+    prompt = make_prompt(wl, 2 * images)       # rows 2i / 2i+1: conditional / unconditional prompt of image i
+    cfg = B.make_model_cfg(wl, max_batch=2 * images, max_seq=wl.prompt_len + n_generate + 8, max_window=window)
+    ctx = B.Context(cfg, B.weights_to_device(weights))
+    sample = B.make_sample_cfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window,
+                               init=init, grid_stride=wl.grid_stride, n_generate=n_generate, guidance=guidance)
+    scfg = SampleCfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window, init=init,
+                     grid_stride=wl.grid_stride, n_generate=n_generate, logits_dtype=wl.dtype)
+    ctx.prefill(torch.from_numpy(prompt).cuda(), sample)
+    out = B.StepOut(images, window)
+    ctx.get_window(out)
+    h = out.host()
+    seqs = [LockStepSequence(wl, weights, prompt[2 * i], scfg, i, LOGIT_TOL[wl.dtype], guidance=guidance,
+                             prompt_uncond=prompt[2 * i + 1]) for i in range(images)]
+    for i, s in enumerate(seqs):
+        s.check_window(h["draft"][i], h["q_kind"][i], h["q_draft"][i], h["total_committed"][i])
+    steps, total = 0, wl.prompt_len + n_generate
+    while any(s.st.n < total for s in seqs):
+        ctx.step(out)
+        logits = ctx.peek_logits().to(torch.float64).cpu().numpy()
+        h = out.host()
+        for i, s in enumerate(seqs):
+            s.step((logits[2 * i], logits[2 * i + 1]), {k: v[i] for k, v in h.items()})
+        steps += 1
+        assert steps <= n_generate
+        if max_steps and steps >= max_steps:
+            break
+    assert ctx.device_status() == B.SJD_OK
+    return seqs, steps
+
+
+def test_tiny_guided_generation():
+    """Classifier-free guidance (weight 3.0) on the tiny fp32 model: two streams per image, one shared
+    verification on the mixed rows; two images, 60 tokens each, copied-token initialisation."""
+    wl = WORKLOADS["tiny"]
+    seqs, steps = run_lockstep_guided(wl, images=2, guidance=3.0, n_generate=60, init=INIT_COPY_LEFT)
+    for s in seqs:
+        assert s.st.n == wl.prompt_len + 60
+        assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
+
+
+def test_small_bf16_guided_generation():
+    """The same on the small bf16 model (tensor-core pipeline, register-resident verification route):
+    the mixed row is rounded to bf16 before the top-k threshold is taken."""
+    wl = WORKLOADS["small-bf16"]
+    seqs, steps = run_lockstep_guided(wl, images=2, guidance=3.0, n_generate=80)
+    for s in seqs:
+        assert s.max_logit_err <= 2e-2
+        assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
+
+
 def test_small_bf16_gqa_generation():
     """bf16 storage, grouped-query attention, sizes that are not multiples of the tile sizes."""
     wl = WORKLOADS["small-bf16"]
