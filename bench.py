@@ -237,15 +237,17 @@ def run_library(args, wl):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    batch = args.batch
+    batch = args.batch                                   # images per GPU
+    streams = 2 if args.guidance != 0.0 else 1           # classifier-free guidance: two sequences per image
     seq_base, _ = shard_sequences(batch * world, world, rank)
 
     weights = make_weights(wl, device=dev)
     max_seq = wl.prompt_len + wl.n_generate + 8
-    ctx = B.Context(B.make_model_cfg(wl, batch, max_seq, wl.window), weights, device=dev)
+    ctx = B.Context(B.make_model_cfg(wl, batch * streams, max_seq, wl.window), weights, device=dev)
     sample = B.make_sample_cfg(wl.temperature, wl.top_k, wl.philox_seed, wl.window, B.SJD_INIT_RANDOM,
-                               wl.grid_stride, wl.n_generate, seq_base=seq_base)
-    prompt_host = torch.from_numpy(make_prompt(wl, batch * world)[seq_base:seq_base + batch].copy()).pin_memory()
+                               wl.grid_stride, wl.n_generate, seq_base=seq_base, guidance=args.guidance)
+    prompt_host = torch.from_numpy(make_prompt(wl, batch * streams * world)[seq_base * streams:(seq_base + batch) * streams]
+                                   .copy()).pin_memory()
     prompt_dev = prompt_host.to(dev)
     out_dev = B.StepOut(batch, wl.window, device=dev)
     stream = torch.cuda.current_stream()
@@ -332,7 +334,7 @@ def run_library(args, wl):
     peaks = measured_peaks()
     gemm_ms_per_launch = tr["ms"]["gemm"] / max(1, tr["launches"]["gemm"])
     achieved = tr["gemm_weight_bytes"] / (tr["ms"]["gemm"] * 1e-3) / 1e9 if tr["ms"]["gemm"] > 0 else 0.0
-    rows = batch * wl.window
+    rows = batch * streams * wl.window
     roofline = {"bound": "hbm", "kernel": "projection GEMMs (weight streaming, M = %d rows)" % rows,
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                 "peak_source": "of " + peaks["source"], "nominal_peak": 8000.0, "frac_of_nominal": achieved / 8000.0,
@@ -394,7 +396,7 @@ def run_library(args, wl):
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(wl, batch),
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(wl, batch), guidance=args.guidance, rows_per_step=rows),
                 "clocks": clk, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
                 "cpu_baseline": cpu,
                 "timing": {"blocks": len(block_ms), "steps_per_block": args.steps,
@@ -438,6 +440,8 @@ def main():
     ap.add_argument("--no-kernel-points", action="store_true", help="skip the isolated verify / attention timings")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (longer KV prefix)")
     ap.add_argument("--window", type=int, default=0, help="override the Jacobi window W (at most 64)")
+    ap.add_argument("--guidance", type=float, default=0.0,
+                    help="classifier-free guidance weight (the paper runs 3.0): two streams per image, 2 x batch x W rows")
     args = ap.parse_args()
     from paper_2410_01699_b200.inputs import WORKLOADS
     wl = WORKLOADS[args.workload]

@@ -31,6 +31,10 @@ INIT_RANDOM = 0       # Sec. 4.2: uniform random candidate
 INIT_COPY_ABOVE = 1   # Sec. 4.2 (b): repeat the token one grid row above
 INIT_COPY_LEFT = 2    # Sec. 4.2 (a): repeat the left neighbour
 
+SCHEDULE_SJD = 0        # Sec. 4.1: probabilistic criterion (Eqs. 1-3)
+SCHEDULE_JACOBI = 1     # Sec. 3.2: every slot re-drawn each pass, a slot is fixed once its token no longer changes
+SCHEDULE_NO_REFINE = 2  # appendix "effectiveness" ablation: Eqs. 1-2 only, unaccepted slots are re-initialised
+
 
 @dataclass
 class SampleCfg:
@@ -42,6 +46,7 @@ class SampleCfg:
     grid_stride: int = 0       # tokens per image row (incl. any row-end token)
     n_generate: int = 0
     logits_dtype: str = "f32"  # storage dtype of the logits: 'f32' or 'bf16'
+    schedule: int = SCHEDULE_SJD
 
 
 @dataclass
@@ -222,8 +227,15 @@ def sjd_step(state: SJDState, model, scfg: SampleCfg, vocab: int, logits_overrid
         stored = round_to_storage(raw, scfg.logits_dtype)
 
     # Step 3: verification scan, calibrated resample, refinement
-    uniforms = [philox.verify_uniforms(scfg.seed, n + k, j, state.seq) for k in range(w_eff)]
-    vr = verify_window(stored, state.drafts, state.qdescs, uniforms, scfg.temperature, scfg.top_k)
+    if scfg.schedule == SCHEDULE_JACOBI:
+        vr = jacobi_window(stored, state.drafts, scfg, n, state.seq)
+    else:
+        uniforms = [philox.verify_uniforms(scfg.seed, n + k, j, state.seq) for k in range(w_eff)]
+        vr = verify_window(stored, state.drafts, state.qdescs, uniforms, scfg.temperature, scfg.top_k)
+        if scfg.schedule == SCHEDULE_NO_REFINE:
+            # no refinement: the slots after the rejection are not re-drawn from this pass's rows (Eq. 3) but
+            # replaced by newly initialised tokens, like the slots that enter the window
+            vr.redraft, vr.redraft_rows, vr.redraft_margin = [], [], []
 
     # fixed tokens grow by the accepted prefix (+ the resampled token)
     state.committed.extend(vr.committed)
@@ -242,6 +254,38 @@ def sjd_step(state: SJDState, model, scfg: SampleCfg, vocab: int, logits_overrid
         q_draft=[q_of_draft(qd, d, vocab, scfg) for qd, d in zip(state.qdescs, state.drafts)])
 
 
+def jacobi_window(stored, drafts, scfg: SampleCfg, n: int, seq: int) -> VerifyResult:
+    """One pass of Jacobi decoding with sampling (Sec. 3.2): every slot k is re-drawn from this pass's
+    row, x'_k = icdf(warp(row_k), u_k); the longest prefix of slots whose token did not change is fixed
+    (the deterministic criterion), and so is the first changed slot, whose context is fixed by then.
+    Reading: the draw of a position uses the same uniform in every pass (a function of the position,
+    not of the pass: the re-draft word of the Philox block with step index 0), which is what makes
+    "unchanged between consecutive iterations" a fixed point: the iteration then converges to the
+    image ordinary sampling would produce from the same per-position uniforms."""
+    w_eff = len(drafts)
+    res = VerifyResult(accept=[], n_accepted=w_eff, committed=[], redraft=[], redraft_rows=[])
+    new, margins = [], []
+    for k in range(w_eff):
+        u = philox.verify_uniforms(scfg.seed, n + k, 0, seq)[2]
+        t, margin = icdf(warp(stored[k], scfg.temperature, scfg.top_k), u)
+        new.append(int(t))
+        margins.append(margin)
+    a = 0
+    while a < w_eff and new[a] == int(drafts[a]):
+        a += 1
+    res.n_accepted = a
+    res.accept = [True] * a + ([False] if a < w_eff else [])
+    res.accept_margin = margins[:a + 1]        # a changed token is a changed inverse-CDF draw
+    res.ratio = [1.0] * a + ([0.0] if a < w_eff else [])
+    res.committed = [int(d) for d in drafts[:a]] + ([new[a]] if a < w_eff else [])
+    if a < w_eff:
+        res.resample_margin = margins[a]
+    res.redraft = new[a + 1:]
+    res.redraft_rows = list(range(a + 1, w_eff))
+    res.redraft_margin = margins[a + 1:]
+    return res
+
+
 def sjd_generate(prompt, model, scfg: SampleCfg, vocab: int, seq: int = 0, max_steps=None):
     """Run SJD until N tokens are fixed.  Returns (generated tokens, number of
     forward passes, per-step committed counts)."""
@@ -258,15 +302,16 @@ def sjd_generate(prompt, model, scfg: SampleCfg, vocab: int, seq: int = 0, max_s
     return st.committed[len(prompt):], steps, accepted
 
 
-def ar_generate(prompt, model, scfg: SampleCfg, vocab: int, seq: int = 0):
+def ar_generate(prompt, model, scfg: SampleCfg, vocab: int, seq: int = 0, fixed_step=None):
     """Ordinary next-token sampling (Sec. 3.1): one forward pass per token.
-    Token at position t uses the re-draft uniform of (t, step = t - P)."""
+    Token at position t uses the re-draft uniform of (t, step = t - P), or of (t, fixed_step) when
+    a fixed step index is given (the per-position uniforms of the Jacobi schedule)."""
     model.prefill(list(prompt))
     c = [int(t) for t in prompt]
     p_len = len(prompt)
     for i in range(scfg.n_generate):
         row = round_to_storage(model.step_logits(c, []), scfg.logits_dtype)[0]
-        u = philox.verify_uniforms(scfg.seed, len(c), i, seq)[2]
+        u = philox.verify_uniforms(scfg.seed, len(c), i if fixed_step is None else fixed_step, seq)[2]
         tok, _ = icdf(warp(row, scfg.temperature, scfg.top_k), u)
         c.append(tok)
     return c[p_len:], scfg.n_generate

@@ -12,9 +12,9 @@ from scipy import stats
 from oracle import philox
 from oracle.model import ModelCfg, OracleModel
 from oracle.sampling import Q_ONEHOT, Q_ROW, Q_UNIFORM, warp
-from oracle.sjd import (INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, CachedModel, RecomputeModel,
-                        SampleCfg, TableModel, ar_generate, greedy_ar_generate, jacobi_generate,
-                        sjd_begin, sjd_generate, sjd_step)
+from oracle.sjd import (INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, SCHEDULE_JACOBI, SCHEDULE_NO_REFINE,
+                        CachedModel, RecomputeModel, SampleCfg, TableModel, ar_generate, greedy_ar_generate,
+                        jacobi_generate, sjd_begin, sjd_generate, sjd_step)
 
 
 def _tiny_model(seed=0, vocab=96):
@@ -186,3 +186,61 @@ def test_step_bound_on_transformer_with_sampling():
         toks, steps, accepted = sjd_generate(prompt, CachedModel(model, 64), scfg, cfg.vocab)
         assert len(toks) == 40 and sum(accepted) == 40 and steps <= 40
         assert all(1 <= a <= 8 for a in accepted)
+
+
+# ---------------------------------------------------------------------------------------------
+# baseline schedules on the same state machine (Sec. 3.2; the no-refinement ablation of the appendix)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("window,init", [(1, INIT_RANDOM), (5, INIT_RANDOM), (8, INIT_COPY_LEFT)])
+def test_jacobi_with_sampling_converges_to_ordinary_sampling_with_the_same_uniforms(window, init):
+    """With one uniform per position, the Jacobi iteration is a fixed-point iteration of a triangular
+    system: whatever the window and the initial guesses, it ends at the image that one-token-at-a-time
+    sampling draws from the same uniforms, in at most as many passes as tokens."""
+    cfg, model = _tiny_model(seed=3)
+    prompt = [7, 1, 50, 12]
+    n_gen = 20
+    for seed in range(5):
+        scfg = SampleCfg(temperature=1.0, top_k=8, seed=seed, window=window, init=init, grid_stride=4,
+                         n_generate=n_gen, schedule=SCHEDULE_JACOBI)
+        toks, steps, accepted = sjd_generate(prompt, CachedModel(model, 64), scfg, cfg.vocab)
+        plain, _ = ar_generate(prompt, CachedModel(model, 64), scfg, cfg.vocab, fixed_step=0)
+        assert toks == plain
+        assert steps <= n_gen and sum(accepted) == n_gen
+        if window == 1:
+            assert steps == n_gen
+
+
+def test_jacobi_schedule_with_top1_is_greedy_jacobi_decoding():
+    cfg, model = _tiny_model(seed=1)
+    prompt = [5, 9, 2, 77, 31]
+    n_gen, window = 24, 6
+    greedy = greedy_ar_generate(prompt, CachedModel(model, 64), n_gen)
+    for seed in range(3):
+        scfg = SampleCfg(temperature=1.0, top_k=1, seed=seed, window=window, n_generate=n_gen, schedule=SCHEDULE_JACOBI)
+        toks, steps, _ = sjd_generate(prompt, CachedModel(model, 64), scfg, cfg.vocab)
+        jtoks, jpasses = jacobi_generate(prompt, CachedModel(model, 64), n_gen, window, cfg.vocab, seed=seed)
+        assert toks == greedy == jtoks and steps == jpasses
+
+
+def test_without_refinement_the_law_is_still_exact_but_nothing_is_kept():
+    """Eqs. 1-2 alone (slots after a rejection re-initialised instead of re-drawn by Eq. 3): the images
+    still follow the model's law, and every slot of the window after a rejection is a fresh one."""
+    vocab, n_gen, n_runs = 4, 4, 12000
+    table = TableModel(vocab, order=2, seed=11)
+    prompt = [1, 3]
+    joint = _exact_joint(table, prompt, n_gen, 1.0, 3)
+    counts = {}
+    for seed in range(n_runs):
+        scfg = SampleCfg(temperature=1.0, top_k=3, seed=seed, window=3, n_generate=n_gen, schedule=SCHEDULE_NO_REFINE)
+        toks, steps, accepted = sjd_generate(prompt, table, scfg, vocab)
+        assert steps <= n_gen and sum(accepted) == n_gen
+        counts[tuple(toks)] = counts.get(tuple(toks), 0) + 1
+    assert _chi_square_joint(counts, joint, n_runs) > 1e-4
+    scfg = SampleCfg(temperature=1.0, top_k=3, seed=5, window=3, n_generate=12, schedule=SCHEDULE_NO_REFINE)
+    st = sjd_begin(prompt, scfg, vocab)
+    for _ in range(6):
+        if not st.drafts:
+            break
+        rec = sjd_step(st, table, scfg, vocab)
+        assert all(k == Q_UNIFORM for k in rec.kinds)
+        assert rec.verify.redraft == []
