@@ -63,6 +63,17 @@ typedef enum {
   SJD_INIT_COPY_LEFT = 2   /* token at position - 1 (strategy (a)); q = point mass           */
 } sjd_init_kind;
 
+/* Which decoding schedule a step runs: the paper's method, or one of the baselines it is compared with
+ * (Table 1 rows A-D: plain next-token sampling is SJD with window 1; Sec. 3.2; the no-refinement ablation). */
+typedef enum {
+  SJD_SCHEDULE_SJD = 0,       /* Sec. 4.1: accept with min(1, p/q), resample the first rejection, re-draft the rest */
+  SJD_SCHEDULE_JACOBI = 1,    /* Sec. 3.2: every slot re-drawn from this pass's row with the uniform of its      */
+                              /* position (re-draft word, step index 0); the unchanged prefix and the first    */
+                              /* changed slot are fixed; no q is used                                            */
+  SJD_SCHEDULE_NO_REFINE = 2  /* Eqs. 1-2 only: the slots after the first rejection are re-initialised (Sec. 4.2) */
+                              /* instead of re-drawn by Eq. 3                                                     */
+} sjd_schedule_kind;
+
 /* The law a draft token was drawn from (Step 1: "the probability corresponding to the draft"). */
 typedef enum {
   SJD_Q_ROW = 0,     /* top-k softmax of the logits row that produced it one iteration ago */
@@ -118,6 +129,7 @@ typedef struct {
                        /* l_u + w (l_c - l_u), evaluated in fp32 as fma(w, l_c - l_u, l_u) and       */
                        /* rounded to cfg.dtype.  Outputs then have batch / 2 entries (one per image)  */
                        /* and the Philox sequence id is seq_base + i.  sjd_verify(_static): must be 0 */
+  int32_t schedule;    /* sjd_schedule_kind; 0 = the paper's method                                  */
 } sjd_sample_cfg;
 
 /* Results of one step.  Any pointer may be NULL (that output is skipped). */

@@ -20,6 +20,7 @@ SJD_ERR_CUDA, SJD_ERR_DEVICE_TIMEOUT, SJD_ERR_STATE = -4, -5, -6
 SJD_F32, SJD_BF16 = 0, 1
 SJD_INIT_RANDOM, SJD_INIT_COPY_ABOVE, SJD_INIT_COPY_LEFT = 0, 1, 2
 SJD_Q_ROW, SJD_Q_UNIFORM, SJD_Q_ONEHOT = 0, 1, 2
+SJD_SCHEDULE_SJD, SJD_SCHEDULE_JACOBI, SJD_SCHEDULE_NO_REFINE = 0, 1, 2
 SJD_FLAG_NEAR_TIE_ACCEPT, SJD_FLAG_RESIDUAL_EMPTY, SJD_FLAG_NONFINITE, SJD_FLAG_DONE = 1, 4, 8, 16
 
 DTYPES = {"f32": SJD_F32, "bf16": SJD_BF16}
@@ -58,7 +59,7 @@ class sjd_weights(C.Structure):
 class sjd_sample_cfg(C.Structure):
     _fields_ = [("temperature", C.c_float), ("top_k", C.c_int32), ("seed", C.c_uint64), ("window", C.c_int32),
                 ("init", C.c_int32), ("grid_stride", C.c_int32), ("n_generate", C.c_int32), ("seq_base", C.c_int32),
-                ("guidance", C.c_float)]
+                ("guidance", C.c_float), ("schedule", C.c_int32)]
 
 
 class sjd_step_out(C.Structure):
@@ -156,9 +157,9 @@ def make_model_cfg(wl, max_batch: int, max_seq: int, max_window: int) -> sjd_mod
 
 
 def make_sample_cfg(temperature=1.0, top_k=2000, seed=0, window=16, init=SJD_INIT_RANDOM, grid_stride=0,
-                    n_generate=0, seq_base=0, guidance=0.0) -> sjd_sample_cfg:
+                    n_generate=0, seq_base=0, guidance=0.0, schedule=0) -> sjd_sample_cfg:
     return sjd_sample_cfg(float(temperature), int(top_k), int(seed), int(window), int(init), int(grid_stride),
-                          int(n_generate), int(seq_base), float(guidance))
+                          int(n_generate), int(seq_base), float(guidance), int(schedule))
 
 
 class StepOut:

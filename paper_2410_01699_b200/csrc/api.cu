@@ -16,6 +16,7 @@ int check_sample_cfg(const sjd_sample_cfg *s, int vocab) {
   if (s->init == SJD_INIT_COPY_ABOVE && s->grid_stride < 1) return SJD_ERR_BAD_ARG;
   if (s->seq_base < 0) return SJD_ERR_BAD_ARG;
   if (!(s->guidance == s->guidance) || s->guidance > 1e6f || s->guidance < -1e6f) return SJD_ERR_BAD_ARG;
+  if (s->schedule < SJD_SCHEDULE_SJD || s->schedule > SJD_SCHEDULE_NO_REFINE) return SJD_ERR_BAD_ARG;
   (void)vocab;
   return SJD_OK;
 }
@@ -38,6 +39,7 @@ int verify_isolated(int batch, int window, int vocab, int logits_dtype, const vo
   if (window > 64) return SJD_ERR_CAPACITY;
   if (!(sample->temperature > 0.0f) || sample->top_k < 1 || sample->seq_base < 0) return SJD_ERR_BAD_ARG;
   if (sample->guidance != 0.0f) return SJD_ERR_UNSUPPORTED;   // guidance pairs the streams of a context (sjd_step)
+  if (sample->schedule < SJD_SCHEDULE_SJD || sample->schedule > SJD_SCHEDULE_NO_REFINE) return SJD_ERR_BAD_ARG;
   if (((uintptr_t)scratch & 15u) != 0) return SJD_ERR_BAD_ARG;
 
   const size_t rows = (size_t)batch * window;
@@ -66,6 +68,7 @@ int verify_isolated(int batch, int window, int vocab, int logits_dtype, const vo
   p.seed_hi = (uint32_t)(sample->seed >> 32);
   p.seq_base = (uint32_t)sample->seq_base;
   p.e2e = 0;
+  p.schedule = sample->schedule;
   p.out = *out;
   return launch_verify(p, logits_dtype, stream);
 }

@@ -209,6 +209,7 @@ struct VerifyParams {
   // l_u + guidance * (l_c - l_u) rounded to the storage dtype, and the slide writes both streams' state.
   int paired;
   float guidance;
+  int schedule;            // sjd_schedule_kind
   SeqState st;
   sjd_step_out out;
 };

@@ -526,6 +526,7 @@ int run_verify(sjd_ctx *c, const sjd_step_out *out, cudaStream_t stream) {
   p.seed_hi = (uint32_t)(c->sample.seed >> 32);
   p.seq_base = (uint32_t)c->sample.seq_base;
   p.e2e = 1;
+  p.schedule = c->sample.schedule;
   p.st = st;
   if (c->sample.guidance != 0.0f) {   // sequences 2i, 2i + 1 = conditional and unconditional stream of image i
     p.paired = 1;

@@ -971,6 +971,13 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
   ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = accept ? -1 : kResampleDeferred;
   ro.flags = flags;
+  if (p.schedule == SJD_SCHEDULE_JACOBI) {   // deterministic criterion: the slot is fixed if its token did not change
+    const bool same = d_ok && redraft_tok == d;
+    ro.thr = same ? 1.0f : 0.0f;
+    ro.accept = same ? 1 : 0;
+    ro.resample_tok = same ? -1 : redraft_tok;   // the first changed slot is fixed to its new token
+    ro.flags = 0;
+  }
   return true;
 }
 
@@ -1168,9 +1175,10 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
     const int total = p.st.prompt_len + p.st.n_generate;
     w2 = max(0, min(W, total - n2));
     kept = (a < w_eff) ? min(w_eff - a - 1, w2) : 0;
+    if (p.schedule == SJD_SCHEDULE_NO_REFINE) kept = 0;   // every slot of the new window is initialised afresh
     if (n2 >= total) flags |= SJD_FLAG_DONE;
   } else {
-    kept = (a < w_eff) ? (w_eff - a - 1) : 0;
+    kept = (a < w_eff && p.schedule != SJD_SCHEDULE_NO_REFINE) ? (w_eff - a - 1) : 0;
     w2 = kept;
   }
   int32_t *nd = p.e2e ? p.st.draft + (size_t)sb * W : nullptr;
@@ -1266,14 +1274,19 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   const float inv_t = 1.0f / p.temperature;
 
   if (k < w_eff) {
-    const int kind = p.q_kind ? p.q_kind[rs] : SJD_Q_ROW;
+    // (the Jacobi schedule compares tokens and uses no q: treat every draft as a copied one)
+    const int kind = p.schedule == SJD_SCHEDULE_JACOBI ? SJD_Q_ONEHOT : (p.q_kind ? p.q_kind[rs] : SJD_Q_ROW);
     const int d = p.draft[rs];
     const bool d_ok = d >= 0 && d < p.V;
     const int qr = p.q_row ? p.q_row[rs] : k;
     const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
     const Philox4 rnd = philox4x32_10((uint32_t)(base + k), step, p.seq_base + (uint32_t)b, kStreamVerify,
                                       p.seed_lo, p.seed_hi);
-    const float u_acc = u24(rnd.w[0]), u_res = u24(rnd.w[1]), u_draft = u24(rnd.w[2]);
+    const float u_acc = u24(rnd.w[0]), u_res = u24(rnd.w[1]);
+    float u_draft = u24(rnd.w[2]);
+    const bool jacobi = p.schedule == SJD_SCHEDULE_JACOBI;
+    if (jacobi)   // Sec. 3.2: the draw of a position uses the same uniform in every pass (step index 0)
+      u_draft = u24(philox4x32_10((uint32_t)(base + k), 0u, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo, p.seed_hi).w[2]);
     const RowRefs<T> rows = row_refs<T>(p, b, k, qr, cur);
 
     RowOut fast_out;
@@ -1322,8 +1335,8 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     float ratio;
     if (q_d > 0.0f) ratio = p_d / q_d;
     else ratio = p_d > 0.0f ? INFINITY : 0.0f;
-    const float thr = fminf(1.0f, ratio);
-    const bool accept = u_acc < thr;
+    float thr = fminf(1.0f, ratio);
+    bool accept = u_acc < thr;
     uint32_t flags = ps.flags | (kind == SJD_Q_ROW ? qs.flags : 0u);
     if (thr < 1.0f && fabsf(u_acc - thr) < 1e-4f) flags |= SJD_FLAG_NEAR_TIE_ACCEPT;
 
@@ -1336,7 +1349,12 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     SJD_TL(TL_VERIFY, 12, tid == 0);   // re-draft token drawn
     // ---- Eq. 2: residual resample (used if this is the first rejected row)
     int resample_tok = -1;
-    if (!accept) {
+    if (jacobi) {   // deterministic criterion instead of Eqs. 1-2
+      accept = d_ok && redraft_tok == d;
+      thr = accept ? 1.0f : 0.0f;
+      flags &= ~SJD_FLAG_NEAR_TIE_ACCEPT;
+      resample_tok = accept ? -1 : redraft_tok;
+    } else if (!accept) {
       ResidualWeights<T> rf;
       rf.prow = prow; rf.qrow = qrow; rf.pw = pf.pw; rf.qw = qf.pw;
       rf.inv_zp = 1.0f / ps.z; rf.inv_zq = 1.0f / qs.z;

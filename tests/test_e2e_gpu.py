@@ -17,7 +17,7 @@ LOGIT_TOL = {"f32": 1e-4, "bf16": 2e-2}
 
 
 def run_lockstep(wl, batch=1, max_steps=None, init=INIT_RANDOM, check_logits_every=1, gain_jitter=0.1, window=None,
-                 n_generate=None, seq_base=0, top_k=None, also_plain_cache=False):
+                 n_generate=None, seq_base=0, top_k=None, also_plain_cache=False, schedule=0):
     window = window or wl.window
     n_generate = wl.n_generate if n_generate is None else n_generate
     top_k = top_k or wl.top_k
@@ -26,9 +26,10 @@ def run_lockstep(wl, batch=1, max_steps=None, init=INIT_RANDOM, check_logits_eve
     cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=wl.prompt_len + n_generate + 8, max_window=window)
     ctx = B.Context(cfg, B.weights_to_device(weights))
     sample = B.make_sample_cfg(temperature=wl.temperature, top_k=top_k, seed=wl.philox_seed, window=window,
-                               init=init, grid_stride=wl.grid_stride, n_generate=n_generate, seq_base=seq_base)
+                               init=init, grid_stride=wl.grid_stride, n_generate=n_generate, seq_base=seq_base,
+                               schedule=schedule)
     scfg = SampleCfg(temperature=wl.temperature, top_k=top_k, seed=wl.philox_seed, window=window, init=init,
-                     grid_stride=wl.grid_stride, n_generate=n_generate, logits_dtype=wl.dtype)
+                     grid_stride=wl.grid_stride, n_generate=n_generate, logits_dtype=wl.dtype, schedule=schedule)
     ctx.prefill(torch.from_numpy(prompt).cuda(), sample)
     out = B.StepOut(batch, window)
     ctx.get_window(out)
@@ -159,6 +160,36 @@ def test_small_bf16_guided_generation():
     for s in seqs:
         assert s.max_logit_err <= 2e-2
         assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
+
+
+@pytest.mark.parametrize("name,batch", [("tiny", 1), ("small-bf16", 2)])
+def test_jacobi_schedule(name, batch):
+    """Sec. 3.2 on the same kernels: every slot re-drawn each pass with the uniform of its position, the
+    unchanged prefix fixed.  Lock-step with the checker; on the fp32 model the finished image must also
+    be the one ordinary sampling draws from the same uniforms."""
+    from oracle.model import OracleModel
+    from oracle.sjd import SCHEDULE_JACOBI, CachedModel, ar_generate
+    from tests.parity_util import oracle_model_cfg
+    wl = WORKLOADS[name]
+    n_gen = 48
+    ctx, seqs, steps, _ = run_lockstep(wl, batch=batch, n_generate=n_gen, schedule=SCHEDULE_JACOBI, gain_jitter=0.0)
+    assert steps <= n_gen
+    if wl.dtype == "f32" and seqs[0].stats.flagged == 0:
+        scfg = SampleCfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, n_generate=n_gen,
+                         logits_dtype=wl.dtype)
+        model = CachedModel(OracleModel(oracle_model_cfg(wl), make_weights(wl)), wl.prompt_len + n_gen + 1)
+        plain, _ = ar_generate(list(make_prompt(wl)[0]), model, scfg, wl.vocab, fixed_step=0)
+        assert seqs[0].st.committed[wl.prompt_len:] == plain
+
+
+@pytest.mark.parametrize("name,init", [("tiny", INIT_RANDOM), ("small-bf16", INIT_COPY_LEFT)])
+def test_no_refinement_schedule(name, init):
+    """The ablation without Eq. 3: after the first rejection every remaining slot is initialised afresh."""
+    from oracle.sjd import SCHEDULE_NO_REFINE
+    wl = WORKLOADS[name]
+    ctx, seqs, steps, out = run_lockstep(wl, n_generate=40, schedule=SCHEDULE_NO_REFINE, init=init)
+    assert steps <= 40
+    assert not np.any(out.host()["q_kind"] == B.SJD_Q_ROW)
 
 
 def test_small_bf16_gqa_generation():
