@@ -411,6 +411,64 @@ def run_library(args, wl):
         dist.destroy_process_group()
 
 
+def run_table(args, wl):
+    """The structure of the paper's Table 1 (rows A-D) and of its no-refinement ablation on this library's
+    kernels: whole images generated by next-token sampling (A: window 1), Jacobi decoding with the
+    deterministic criterion (B), SJD with random initialisation (C), SJD with the spatial prior (D: token
+    one grid row above) and SJD without refinement; forward passes per image, latency, ratios against A.
+    Random-init weights accept almost nothing, so the ratios say nothing about trained models."""
+    import torch
+
+    from paper_2410_01699_b200 import binding as B
+    from paper_2410_01699_b200.inputs import make_prompt, make_weights
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    weights = make_weights(wl, device=dev)
+    n_gen = args.n_generate or wl.n_generate
+    max_seq = wl.prompt_len + n_gen + 8
+    prompt = torch.from_numpy(make_prompt(wl, 1)).to(dev)
+    ctx = B.Context(B.make_model_cfg(wl, 1, max_seq, wl.window), weights, device=dev)
+    rows = [("A", "next-token sampling (window 1)", 1, B.SJD_SCHEDULE_SJD, B.SJD_INIT_RANDOM),
+            ("B", "Jacobi decoding, unchanged-token criterion", wl.window, B.SJD_SCHEDULE_JACOBI, B.SJD_INIT_RANDOM),
+            ("C", "SJD, random initialisation", wl.window, B.SJD_SCHEDULE_SJD, B.SJD_INIT_RANDOM),
+            ("D", "SJD, token one grid row above", wl.window, B.SJD_SCHEDULE_SJD, B.SJD_INIT_COPY_ABOVE),
+            ("no-refinement", "SJD without Eq. 3", wl.window, B.SJD_SCHEDULE_NO_REFINE, B.SJD_INIT_RANDOM)]
+    table, chunk = [], 64
+    for tag, name, window, schedule, init in rows:
+        sample = B.make_sample_cfg(wl.temperature, wl.top_k, wl.philox_seed, window, init, wl.grid_stride, n_gen,
+                                   schedule=schedule)
+        out = B.StepOut(1, window, device=dev)
+        ctx.prefill(prompt, sample)
+        for _ in range(4):   # first replays of freshly captured step graphs
+            ctx.step(out)
+        ctx.prefill(prompt, sample)
+        busy = torch.zeros(1, dtype=torch.int64, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        run = 0
+        while True:
+            for _ in range(chunk):
+                ctx.step(out)
+                busy += (out.n_committed > 0).to(torch.int64)   # device-side count of passes that fixed a token
+            run += chunk
+            if int(out.total_committed.item()) >= wl.prompt_len + n_gen:
+                break
+        e1.record()
+        torch.cuda.synchronize()
+        steps = int(busy.item())
+        ms = e0.elapsed_time(e1) * steps / run     # passes after the image is complete are not counted
+        table.append({"row": tag, "config": name, "window": window, "steps_per_image": steps,
+                      "tokens_per_step": n_gen / steps, "latency_s": ms * 1e-3, "ms_per_step": ms / steps})
+    base = table[0]
+    for r in table:
+        r["step_ratio_vs_A"] = base["steps_per_image"] / r["steps_per_image"]
+        r["latency_ratio_vs_A"] = base["latency_s"] / r["latency_s"]
+    print(json.dumps({"table": table, "workload": wl.name, "n_generate": n_gen, "data": "synthetic",
+                      "note": "random-init weights: acceptance statistics are not those of a trained model"}), flush=True)
+
+
 def _spawned_rank(local_rank, args, wl, port):
     os.environ.update({"RANK": str(local_rank), "LOCAL_RANK": str(local_rank), "WORLD_SIZE": str(args.gpus),
                        "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
@@ -440,6 +498,9 @@ def main():
     ap.add_argument("--no-kernel-points", action="store_true", help="skip the isolated verify / attention timings")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (longer KV prefix)")
     ap.add_argument("--window", type=int, default=0, help="override the Jacobi window W (at most 64)")
+    ap.add_argument("--table", action="store_true",
+                    help="whole-image generation under the baseline schedules and SJD (rows A-D and no-refinement)")
+    ap.add_argument("--n-generate", type=int, default=0, help="image tokens per image for --table (default: the workload's)")
     ap.add_argument("--guidance", type=float, default=0.0,
                     help="classifier-free guidance weight (the paper runs 3.0): two streams per image, 2 x batch x W rows")
     args = ap.parse_args()
@@ -451,6 +512,8 @@ def main():
         wl = wl.with_(window=args.window)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.table:
+        run_table(args, wl)
     elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         launch_ranks(args, wl)
     else:
