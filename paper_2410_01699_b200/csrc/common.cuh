@@ -219,6 +219,7 @@ struct VerifyParams {
   uint32_t step;           // used when step_ptr == null
   int B, W, V;
   int staged;              // row fits the dynamic shared buffer
+  int defer_residual;      // register route: rejected rows leave the Eq. 2 draw to the sequence's last block
   int fast;                // bf16 rows, 16-byte aligned, V % 8 == 0, V / 8 <= 8 * blockDim.x: a block may keep a row in registers
   float temperature;
   int top_k;

@@ -885,9 +885,12 @@ __device__ __forceinline__ RowRefs<T> row_refs(const VerifyParams &p, int b, int
   return rr;
 }
 
+__device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowRefs<__nv_bfloat16> &rows, int kind, int d,
+                            const RowStats &ps, const RowStats &qs, float u_res, Scratch &sc, int &tok, uint32_t &flags);
+
 template <typename T>
 __device__ bool fast_row(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
-                         const RowRefs<T> &rows, float inv_t, float u_acc, float u_draft, RowOut &ro) {
+                         const RowRefs<T> &rows, float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
   return false;
 }
 
@@ -895,8 +898,8 @@ constexpr int kResampleDeferred = -2;   // RowOut.resample_tok of a rejected row
 
 template <>
 __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
-                                        const RowRefs<__nv_bfloat16> &rows, float inv_t, float u_acc, float u_draft,
-                                        RowOut &ro) {
+                                        const RowRefs<__nv_bfloat16> &rows, float inv_t, float u_acc, float u_res,
+                                        float u_draft, RowOut &ro) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x;
   const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
@@ -967,9 +970,17 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   const float redraft_p = redraft_w / ps.z;
   SJD_TL(TL_VERIFY, 12, tid == 0);
 
-  // ---- Eq. 2 is left to the block that scans the sequence: only the first rejected row needs it
+  // ---- Eq. 2.  Only the first rejected row of a sequence needs it.  In a grid of several waves a rejected row
+  // leaves it to the block that scans the sequence (32 draws per launch instead of up to B * W); in a grid
+  // that is resident at once (one sequence: latency matters, throughput does not) every rejected row draws
+  // its token now, in parallel with the others.
+  int resample_tok = accept ? -1 : kResampleDeferred;
+  if (!accept && !p.defer_residual && p.schedule != SJD_SCHEDULE_JACOBI) {
+    __syncthreads();
+    rr_residual(p, row, rows, kind, d, ps, qs, u_res, sc, resample_tok, flags);
+  }
   ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
-  ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = accept ? -1 : kResampleDeferred;
+  ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok;
   ro.flags = flags;
   if (p.schedule == SJD_SCHEDULE_JACOBI) {   // deterministic criterion: the slot is fixed if its token did not change
     const bool same = d_ok && redraft_tok == d;
@@ -981,66 +992,19 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   return true;
 }
 
-// Eq. 2 for the first rejected row of sequence b, when that row left it open (register-resident route):
-// run by every thread of the sequence's last block before the window slide.  The row's statistics and
-// those of its draft's law were published by the block that verified it; the two logits rows are read
-// again (they are still in L2): p into registers, q vector by vector as it is needed.
-template <typename T>
-__device__ void deferred_residual(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {}
-
-template <>
-__device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {
+// Eq. 2 on a p row held in registers (entries below its threshold may already have been replaced by
+// -inf): residual weights max(0, p - q), their chunk sums and the inverse-CDF draw; the q row is read
+// from global memory (L2) vector by vector as it is needed.  Block-wide; returns the token and flags.
+__device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowRefs<__nv_bfloat16> &rows, int kind, int d,
+                            const RowStats &ps, const RowStats &qs, float u_res, Scratch &sc, int &tok, uint32_t &flags) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int W = p.W, V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
-  const int w_eff = p.w_eff ? p.w_eff[p.paired ? 2 * b : b] : W;
-  RowOut *ro = p.row_out + (size_t)b * W;
-  if (tid < 32) {
-    int first = w_eff;
-    for (int k = lane; k < w_eff; k += 32)
-      if (!__ldcg(&ro[k].accept)) first = min(first, k);
-    first = __reduce_min_sync(0xffffffffu, first);
-    if (lane == 0) sc.sel_chunk = (first < w_eff && __ldcg(&ro[first].resample_tok) == kResampleDeferred) ? first : -1;
-  }
-  __syncthreads();
-  const int a = sc.sel_chunk;
-  __syncthreads();
-  if (a < 0) return;
-  const int r = b * W + a;
-  const int sb = p.paired ? 2 * b : b;   // the sequence whose state holds the window (both streams hold the same)
-  const int kind = p.q_kind ? p.q_kind[sb * W + a] : SJD_Q_ROW;
-  const int d = p.draft[sb * W + a];
-  const int qr = p.q_row ? p.q_row[sb * W + a] : a;
-  const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
-  const Philox4 rnd = philox4x32_10((uint32_t)(base + a), step, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo,
-                                    p.seed_hi);
-  const float u_res = u24(rnd.w[1]);
+  const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
   const float scale = (1.0f / p.temperature) * 1.4426950408889634f;
-  const RowRefs<__nv_bfloat16> rows = row_refs<__nv_bfloat16>(p, b, a, qr, cur);
-  const uint4 *pg = reinterpret_cast<const uint4 *>(rows.p), *pg2 = reinterpret_cast<const uint4 *>(rows.p2);
   const uint4 *qg = reinterpret_cast<const uint4 *>(rows.q), *qg2 = reinterpret_cast<const uint4 *>(rows.q2);
-  auto load_stats = [](const RowStats *g) {
-    const uint4 u = __ldcg(reinterpret_cast<const uint4 *>(g));
-    RowStats st;
-    st.tau_key = u.x; st.xmax = __uint_as_float(u.y); st.z = __uint_as_float(u.z); st.flags = u.w;
-    return st;
-  };
-  const RowStats ps = load_stats(&p.stats[cur][r]);
-  RowStats qs;
-  qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
-  if (kind == SJD_Q_ROW) {
-    qs = load_stats(&p.stats[cur ^ 1][(size_t)b * W + qr]);
-  }
   const float tau_p = ps.tau_key ? E::val(E::unkey(ps.tau_key)) : -INFINITY;
   const float tau_q = qs.tau_key ? E::val(E::unkey(qs.tau_key)) : -INFINITY;
-  RegRow row;
   const int j0 = warp * 256 + lane;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int j = j0 + i * 32;
-    row.v[i] = j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-  }
-
   // probabilities straight from one fused multiply-add per entry: p_i = 2^(x_i * scale + c) with
   // c = -max * scale - log2(Z); entries below the threshold contribute nothing
   const float cp = -ps.xmax * scale - log2f(ps.z), cq = -qs.xmax * scale - log2f(qs.z);
@@ -1070,8 +1034,6 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
       }
     }
   };
-  uint32_t flags = 0;
-  int tok;
   float wsel;
   rr_chunk_sums(r_w, NV, sc);
   WarpPrefix wr = rr_prefix(NC, sc);
@@ -1095,6 +1057,63 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
     wr = rr_prefix(NC, sc);
     rr_icdf(p_w, NV, wr, u_res, sc, tok, wsel);
   }
+}
+
+// Eq. 2 for the first rejected row of sequence b, when that row left it open (register-resident route,
+// grids of more than one wave): run by every thread of the sequence's last block before the window slide.
+// The row's statistics and those of its draft's law were published by the block that verified it; the p
+// row is read again into registers (it is still in L2).
+template <typename T>
+__device__ void deferred_residual(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {}
+
+template <>
+__device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int W = p.W, NV = p.V >> 3;
+  const int w_eff = p.w_eff ? p.w_eff[p.paired ? 2 * b : b] : W;
+  RowOut *ro = p.row_out + (size_t)b * W;
+  if (tid < 32) {
+    int first = w_eff;
+    for (int k = lane; k < w_eff; k += 32)
+      if (!__ldcg(&ro[k].accept)) first = min(first, k);
+    first = __reduce_min_sync(0xffffffffu, first);
+    if (lane == 0) sc.sel_chunk = (first < w_eff && __ldcg(&ro[first].resample_tok) == kResampleDeferred) ? first : -1;
+  }
+  __syncthreads();
+  const int a = sc.sel_chunk;
+  __syncthreads();
+  if (a < 0) return;
+  const int r = b * W + a;
+  const int sb = p.paired ? 2 * b : b;   // the sequence whose state holds the window (both streams hold the same)
+  const int kind = p.q_kind ? p.q_kind[sb * W + a] : SJD_Q_ROW;
+  const int d = p.draft[sb * W + a];
+  const int qr = p.q_row ? p.q_row[sb * W + a] : a;
+  const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
+  const Philox4 rnd = philox4x32_10((uint32_t)(base + a), step, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo,
+                                    p.seed_hi);
+  const float u_res = u24(rnd.w[1]);
+  const RowRefs<__nv_bfloat16> rows = row_refs<__nv_bfloat16>(p, b, a, qr, cur);
+  const uint4 *pg = reinterpret_cast<const uint4 *>(rows.p), *pg2 = reinterpret_cast<const uint4 *>(rows.p2);
+  auto load_stats = [](const RowStats *g) {
+    const uint4 u = __ldcg(reinterpret_cast<const uint4 *>(g));
+    RowStats st;
+    st.tau_key = u.x; st.xmax = __uint_as_float(u.y); st.z = __uint_as_float(u.z); st.flags = u.w;
+    return st;
+  };
+  const RowStats ps = load_stats(&p.stats[cur][r]);
+  RowStats qs;
+  qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
+  if (kind == SJD_Q_ROW) qs = load_stats(&p.stats[cur ^ 1][(size_t)b * W + qr]);
+  RegRow row;
+  const int j0 = warp * 256 + lane;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    row.v[i] = j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+  }
+  uint32_t flags = 0;
+  int tok;
+  rr_residual(p, row, rows, kind, d, ps, qs, u_res, sc, tok, flags);
   if (tid == 0) {
     ro[a].resample_tok = tok;
     ro[a].flags = __ldcg(&ro[a].flags) | flags;
@@ -1291,7 +1310,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
 
     RowOut fast_out;
     const bool fast_done = p.fast && (((uintptr_t)rows.q | (uintptr_t)rows.p) & 15u) == 0 &&
-                           fast_row<T>(p, sc, r, b, kind, d, qr, cur, rows, inv_t, u_acc, u_draft, fast_out);
+                           fast_row<T>(p, sc, r, b, kind, d, qr, cur, rows, inv_t, u_acc, u_res, u_draft, fast_out);
     if (fast_done) {
       if (tid == 0) p.row_out[r] = fast_out;
     } else {
@@ -1392,7 +1411,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   if (!sc.is_last) return;
   __threadfence();
   SJD_TL(TL_VERIFY, 14, tid == 0);
-  if (p.fast) deferred_residual<T>(p, b, step, cur, sc);
+  if (p.fast && p.defer_residual) deferred_residual<T>(p, b, step, cur, sc);
   finalize_sequence(p, b, step, sc);
   SJD_TL(TL_VERIFY, 15, tid == 0);
   __syncthreads();
@@ -1438,6 +1457,15 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
     // no staging buffer: the rows live in registers; the odd row that needs the general route (a NaN, a
     // threshold out of the histogram's reach) re-reads global memory instead, and more blocks fit an SM
     p.staged = 0;
+    // more blocks than can be resident at once: rejected rows leave the Eq. 2 draw to the sequence's last block
+    static int n_sms = 0;
+    if (n_sms == 0) {
+      int dev = 0, v = 0;
+      if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
+        n_sms = v;
+    }
+    const int resident = (n_sms > 0 ? n_sms : 148) * (threads <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1);
+    p.defer_residual = p.B * p.W > resident ? 1 : 0;
   }
   const size_t dyn = p.staged ? stage_bytes : 0;
   auto launch = [&](auto kernel) -> int {
