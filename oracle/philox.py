@@ -86,6 +86,13 @@ def verify_uniforms(seed: int, position: int, step: int, seq: int):
     return u24(w[0]), u24(w[1]), u24(w[2])
 
 
+def init_uniform(seed: int, position: int, step: int, seq: int) -> float:
+    """The uniform a freshly initialised slot is drawn with when its token comes from a neighbour's
+    predicted distribution (Sec. 4.2 (c), (d)): the same Philox word as init_token, as a 24-bit uniform."""
+    w = philox4x32_10((position, step, seq, STREAM_INIT), split_seed(seed))
+    return u24(w[0])
+
+
 def init_token(seed: int, position: int, step: int, seq: int, vocab: int) -> int:
     """Uniform token in [0, vocab) for a freshly initialised window slot
     (Sec. 4.2: candidates drawn from a uniform distribution): floor(word*V/2^32)."""

@@ -30,6 +30,8 @@ from .sampling import (FLAG_DONE, Q_ONEHOT, Q_ROW, Q_UNIFORM, QDesc, VerifyResul
 INIT_RANDOM = 0       # Sec. 4.2: uniform random candidate
 INIT_COPY_ABOVE = 1   # Sec. 4.2 (b): repeat the token one grid row above
 INIT_COPY_LEFT = 2    # Sec. 4.2 (a): repeat the left neighbour
+INIT_RESAMPLE_LEFT = 3   # Sec. 4.2 (c): draw from the distribution predicted at the left neighbour
+INIT_RESAMPLE_ABOVE = 4  # Sec. 4.2 (d): draw from the distribution predicted one grid row above
 
 SCHEDULE_SJD = 0        # Sec. 4.1: probabilistic criterion (Eqs. 1-3)
 SCHEDULE_JACOBI = 1     # Sec. 3.2: every slot re-drawn each pass, a slot is fixed once its token no longer changes
@@ -58,6 +60,7 @@ class SJDState:
     step: int = 0
     seq: int = 0
     flags: int = 0
+    rows: dict = field(default_factory=dict)   # position -> the most recent stored logits row that predicted it
 
     @property
     def n(self) -> int:
@@ -174,7 +177,28 @@ class TableModel:
 # ----------------------------------------------------------------------------------------------
 def _fresh_slot(state: SJDState, drafts, scfg: SampleCfg, vocab: int, t_pos: int, step_tag: int):
     """Token and q descriptor for a newly initialised slot at absolute position t_pos.
-    `drafts` are the slots of the new window already filled (positions n .. t_pos-1)."""
+    `drafts` are the slots of the new window already filled (positions n .. t_pos-1).
+
+    Strategies (c) and (d) draw the token from the distribution the model predicted at a neighbour's
+    position.  Reading: "predicted" is the most recent logits row computed for that position (the pass in
+    which the position was last inside the window); the slot's law is then that row's top-k softmax,
+    which is what Theorem 1 needs as q.  (c): the neighbour is the nearest position to the left that has
+    ever been through a pass (a slot appended in this very step has not); (d): the position one grid row
+    above.  Without such a row (the first window, the first image row) the slot is a uniform random token."""
+    if scfg.init in (INIT_RESAMPLE_LEFT, INIT_RESAMPLE_ABOVE):
+        if scfg.init == INIT_RESAMPLE_LEFT:
+            src = t_pos - 1
+            while src >= state.prompt_len and src not in state.rows:
+                src -= 1
+        else:
+            src = t_pos - scfg.grid_stride
+        row = state.rows.get(src) if src >= state.prompt_len else None
+        if row is not None:
+            u = philox.init_uniform(scfg.seed, t_pos, step_tag, state.seq)
+            tok, _ = icdf(warp(row, scfg.temperature, scfg.top_k), u)
+            return int(tok), QDesc(Q_ROW, row=row.copy())
+        tok = philox.init_token(scfg.seed, t_pos, step_tag, state.seq, vocab)
+        return int(tok), QDesc(Q_UNIFORM)
     stride = {INIT_COPY_ABOVE: scfg.grid_stride, INIT_COPY_LEFT: 1}.get(scfg.init, 0)
     src = t_pos - stride
     if scfg.init != INIT_RANDOM and stride > 0 and src >= state.prompt_len:
@@ -226,6 +250,8 @@ def sjd_step(state: SJDState, model, scfg: SampleCfg, vocab: int, logits_overrid
         raw = model.step_logits(state.committed, state.drafts[:w_eff - 1])
         stored = round_to_storage(raw, scfg.logits_dtype)
 
+    for k in range(w_eff):   # the most recent prediction for every position of the window (Sec. 4.2 (c), (d))
+        state.rows[n + k] = stored[k]
     # Step 3: verification scan, calibrated resample, refinement
     if scfg.schedule == SCHEDULE_JACOBI:
         vr = jacobi_window(stored, state.drafts, scfg, n, state.seq)

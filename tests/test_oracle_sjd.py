@@ -12,7 +12,8 @@ from scipy import stats
 from oracle import philox
 from oracle.model import ModelCfg, OracleModel
 from oracle.sampling import Q_ONEHOT, Q_ROW, Q_UNIFORM, warp
-from oracle.sjd import (INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, SCHEDULE_JACOBI, SCHEDULE_NO_REFINE,
+from oracle.sjd import (INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, INIT_RESAMPLE_ABOVE, INIT_RESAMPLE_LEFT,
+                        SCHEDULE_JACOBI, SCHEDULE_NO_REFINE,
                         CachedModel, RecomputeModel, SampleCfg, TableModel, ar_generate, greedy_ar_generate,
                         jacobi_generate, sjd_begin, sjd_generate, sjd_step)
 
@@ -54,7 +55,8 @@ def _chi_square_joint(counts: dict, joint: dict, n_runs: int):
 
 
 @pytest.mark.parametrize("window,init", [(1, INIT_RANDOM), (3, INIT_RANDOM), (4, INIT_RANDOM),
-                                         (3, INIT_COPY_LEFT), (4, INIT_COPY_ABOVE)])
+                                         (3, INIT_COPY_LEFT), (4, INIT_COPY_ABOVE),
+                                         (3, INIT_RESAMPLE_LEFT), (2, INIT_RESAMPLE_ABOVE)])
 def test_joint_distribution_is_exact_by_enumeration(window, init):
     """Theorem 1 for whole sequences: over many seeds the generated 4-token sequences follow
     prod_i p(x_i | x_<i), whatever the window and the initialisation."""
@@ -244,3 +246,40 @@ def test_without_refinement_the_law_is_still_exact_but_nothing_is_kept():
         rec = sjd_step(st, table, scfg, vocab)
         assert all(k == Q_UNIFORM for k in rec.kinds)
         assert rec.verify.redraft == []
+
+
+def test_resampled_initialisation_draws_from_the_neighbours_prediction():
+    """Sec. 4.2 (c), (d) on a hand-built case: a model whose rows are (almost) point masses makes the
+    draw from "the distribution predicted at the neighbour" visible as the neighbour row's arg-max, and the
+    slot carries that row as its law; without a row (first window) the slot is a uniform random token."""
+    vocab = 6
+
+    class Peaked:
+        def prefill(self, prompt):
+            pass
+
+        def step_logits(self, committed, drafts_in):
+            seq = list(committed) + list(drafts_in)
+            n = len(committed)
+            out = np.full((len(drafts_in) + 1, vocab), -30.0)
+            for k in range(len(drafts_in) + 1):
+                out[k, (n + k) % vocab] = 5.0      # the row that predicts position n + k peaks at (n + k) % vocab
+            return out
+
+    for init, stride in ((INIT_RESAMPLE_LEFT, 3), (INIT_RESAMPLE_ABOVE, 3)):
+        scfg = SampleCfg(temperature=1.0, top_k=vocab, seed=3, window=3, init=init, grid_stride=stride, n_generate=12)
+        st = sjd_begin([0, 1], scfg, vocab)
+        assert [q.kind for q in st.qdescs] == [Q_UNIFORM] * 3          # nothing predicted yet
+        rec = sjd_step(st, Peaked(), scfg, vocab)
+        n0, n1 = 2, st.n
+        kept = len(rec.verify.redraft)
+        fresh_positions = [n1 + s for s in range(kept, len(st.drafts))]
+        assert fresh_positions, "the first step fixes at least one token, so at least one slot is new"
+        for t in fresh_positions:
+            tok, qd = st.drafts[t - n1], st.qdescs[t - n1]
+            src = min(t - 1, n0 + 2) if init == INIT_RESAMPLE_LEFT else t - stride
+            if src >= 2 and src in st.rows:
+                assert qd.kind == Q_ROW and tok == src % vocab          # the neighbour's own prediction
+                assert np.array_equal(qd.row, st.rows[src])
+            else:
+                assert qd.kind == Q_UNIFORM
