@@ -60,7 +60,11 @@ typedef enum { SJD_F32 = 0, SJD_BF16 = 1 } sjd_dtype;
 typedef enum {
   SJD_INIT_RANDOM = 0,     /* uniform random token; carries q = 1/V                         */
   SJD_INIT_COPY_ABOVE = 1, /* token at position - grid_stride (strategy (b)); q = point mass */
-  SJD_INIT_COPY_LEFT = 2   /* token at position - 1 (strategy (a)); q = point mass           */
+  SJD_INIT_COPY_LEFT = 2,  /* token at position - 1 (strategy (a)); q = point mass           */
+  SJD_INIT_RESAMPLE_LEFT = 3 /* strategy (c): drawn from the distribution predicted at the left neighbour, */
+                           /* i.e. from the most recent logits row of the nearest position to the left   */
+                           /* that has been through a pass (row min(t - 1 - n, W_eff - 1) of this pass);  */
+                           /* q = that row's top-k softmax; first window: uniform random token            */
 } sjd_init_kind;
 
 /* Which decoding schedule a step runs: the paper's method, or one of the baselines it is compared with

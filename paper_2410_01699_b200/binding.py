@@ -18,7 +18,7 @@ SJD_OK = 0
 SJD_ERR_BAD_ARG, SJD_ERR_CAPACITY, SJD_ERR_UNSUPPORTED = -1, -2, -3
 SJD_ERR_CUDA, SJD_ERR_DEVICE_TIMEOUT, SJD_ERR_STATE = -4, -5, -6
 SJD_F32, SJD_BF16 = 0, 1
-SJD_INIT_RANDOM, SJD_INIT_COPY_ABOVE, SJD_INIT_COPY_LEFT = 0, 1, 2
+SJD_INIT_RANDOM, SJD_INIT_COPY_ABOVE, SJD_INIT_COPY_LEFT, SJD_INIT_RESAMPLE_LEFT = 0, 1, 2, 3
 SJD_Q_ROW, SJD_Q_UNIFORM, SJD_Q_ONEHOT = 0, 1, 2
 SJD_SCHEDULE_SJD, SJD_SCHEDULE_JACOBI, SJD_SCHEDULE_NO_REFINE = 0, 1, 2
 SJD_FLAG_NEAR_TIE_ACCEPT, SJD_FLAG_RESIDUAL_EMPTY, SJD_FLAG_NONFINITE, SJD_FLAG_DONE = 1, 4, 8, 16

@@ -108,6 +108,10 @@ struct Scratch {
   int tok;
   float tok_w;
   int is_last;
+  // new window slots whose token is drawn from a logits row of this pass (Sec. 4.2 (c)): filled by
+  // draw_fresh_slots, consumed by finalize_sequence; row -1: no row, the slot is a uniform random token
+  int fresh_tok[64], fresh_row[64];
+  float fresh_q[64];
 };
 
 // A logits row seen as 16-byte vectors aligned in global memory: vector j holds elements
@@ -1140,6 +1144,67 @@ __device__ RowStats row_statistics(Row<T> &row, uint4 *stage, Scratch &sc, int t
   return st;
 }
 
+// ------------------------------------------------------------------------------------ initialisation (c)
+// Sec. 4.2 (c): every slot that enters the window draws its token from the distribution predicted at its left
+// neighbour: the most recent logits row of the nearest position to the left that has been through a pass,
+// which is row min(t - 1 - n, W_eff - 1) of this pass (n: fixed tokens before the pass).  Run by every
+// thread of the sequence's last block before the slide; one inverse-CDF draw over the row per new slot
+// (the chunk sums are shared by consecutive slots that draw from the same row).
+template <typename T>
+__device__ void draw_fresh_slots(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {
+  using E = Elt<T>;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int W = p.W;
+  const int sb = p.paired ? 2 * b : b;
+  const int w_eff = p.w_eff ? p.w_eff[sb] : W;
+  const RowOut *ro = p.row_out + (size_t)b * W;
+  if (tid < 32) {
+    int first = w_eff;
+    for (int k = lane; k < w_eff; k += 32)
+      if (!__ldcg(&ro[k].accept)) first = min(first, k);
+    first = __reduce_min_sync(0xffffffffu, first);
+    if (lane == 0) sc.sel_chunk = first;
+  }
+  __syncthreads();
+  const int a = sc.sel_chunk;
+  __syncthreads();
+  const int m = (a < w_eff) ? a + 1 : w_eff;
+  const int base = p.st.n[sb], n2 = base + m;
+  const int w2 = max(0, min(W, p.st.prompt_len + p.st.n_generate - n2));
+  int kept = (a < w_eff) ? min(w_eff - a - 1, w2) : 0;
+  if (p.schedule == SJD_SCHEDULE_NO_REFINE) kept = 0;
+  const float inv_t = 1.0f / p.temperature;
+  int have = -1;   // row whose chunk sums are in the scratch
+  for (int s = kept; s < w2; ++s) {
+    const int t_pos = n2 + s;
+    const int k = w_eff > 0 ? min(t_pos - 1 - base, w_eff - 1) : -1;
+    if (k < 0) {
+      if (tid == 0) sc.fresh_row[s] = -1;
+      continue;
+    }
+    const RowRefs<T> rows = row_refs<T>(p, b, k, 0, cur);
+    const uint4 su = __ldcg(reinterpret_cast<const uint4 *>(&p.stats[cur][(size_t)b * W + k]));
+    RowStats st;
+    st.tau_key = su.x; st.xmax = __uint_as_float(su.y); st.z = __uint_as_float(su.z); st.flags = su.w;
+    PRowWeights<T> f;
+    f.row.init(rows.p, p.V, rows.p2, p.guidance);
+    f.pw.init(st, inv_t);
+    if (k != have) {
+      chunk_sums<E::VEC>(f, f.row.NV, sc);
+      have = k;
+    }
+    const Philox4 rnd = philox4x32_10((uint32_t)t_pos, step, p.seq_base + (uint32_t)b, kStreamInit, p.seed_lo, p.seed_hi);
+    sample_icdf<E::VEC>(f, f.row.NV, f.row.off, sc, u24(rnd.w[0]));
+    if (tid == 0) {
+      sc.fresh_tok[s] = sc.tok;
+      sc.fresh_q[s] = sc.tok_w / st.z;
+      sc.fresh_row[s] = k;
+    }
+    __syncthreads();
+  }
+  __syncthreads();
+}
+
 // ------------------------------------------------------------------------------------ finalize
 // Run by every thread of the last block of sequence b: accept scan (warp 0), then the commit, the
 // window slide and the next inputs in parallel over the window slots.  Under guidance "sequence b" is
@@ -1214,6 +1279,11 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
       q = __ldcg(&ro[k].redraft_p);
       kind = SJD_Q_ROW;
       qrow = k;
+    } else if (s < w2 && p.st.init == SJD_INIT_RESAMPLE_LEFT && sc.fresh_row[s] >= 0) {  // Sec. 4.2 (c)
+      tok = sc.fresh_tok[s];
+      q = sc.fresh_q[s];
+      kind = SJD_Q_ROW;
+      qrow = sc.fresh_row[s];
     } else if (s < w2) {  // freshly initialised slot (end-to-end mode only), Sec. 4.2
       const int t_pos = n2 + s;
       const int stride = p.st.init == SJD_INIT_COPY_ABOVE ? p.st.grid_stride
@@ -1412,6 +1482,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   __threadfence();
   SJD_TL(TL_VERIFY, 14, tid == 0);
   if (p.fast && p.defer_residual) deferred_residual<T>(p, b, step, cur, sc);
+  if (p.e2e && p.st.init == SJD_INIT_RESAMPLE_LEFT) draw_fresh_slots<T>(p, b, step, cur, sc);
   finalize_sequence(p, b, step, sc);
   SJD_TL(TL_VERIFY, 15, tid == 0);
   __syncthreads();

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle.sjd import INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, SampleCfg
+from oracle.sjd import INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, INIT_RESAMPLE_LEFT, SampleCfg
 from paper_2410_01699_b200 import binding as B
 from paper_2410_01699_b200.inputs import WORKLOADS, make_prompt, make_weights
 from tests.parity_util import LockStepSequence
@@ -74,10 +74,21 @@ def test_tiny_fp32_full_generation():
     assert h["total_committed"][0] == wl.prompt_len + wl.n_generate
 
 
-@pytest.mark.parametrize("init", [INIT_COPY_ABOVE, INIT_COPY_LEFT])
+@pytest.mark.parametrize("init", [INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RESAMPLE_LEFT])
 def test_tiny_spatial_initialisation(init):
     wl = WORKLOADS["tiny"]
     run_lockstep(wl, init=init, n_generate=100)
+
+
+@pytest.mark.parametrize("schedule", [0, 2])
+def test_small_bf16_initialisation_from_the_left_neighbours_prediction(schedule):
+    """Sec. 4.2 (c) on the bf16 model (rows verified on the register-resident route, new slots drawn from
+    them by the sequence's last block), with and without refinement: without it every slot after the
+    rejection is new and draws from the row that predicted its own left neighbour."""
+    wl = WORKLOADS["small-bf16"]
+    ctx, seqs, steps, out = run_lockstep(wl, batch=2, init=INIT_RESAMPLE_LEFT, n_generate=60, schedule=schedule)
+    kinds = out.host()["q_kind"]
+    assert steps <= 60
 
 
 def test_tiny_batch_of_three_and_ragged_window():
