@@ -223,6 +223,6 @@ extern "C" int sjd_attention(int batch, int window, int n_heads, int n_kv_heads,
   const int M = batch * window;
   rc = launch_attention_mma(kv_map, 0, q, in_pos, partial, out, HiLoOut{nullptr, 0}, status, M, window, n_heads, n_kv_heads,
                             head_dim, splits, stream);
-  if (rc != SJD_OK || splits <= 8) return rc;   // up to 8 key ranges merge inside the kernel (one cluster)
+  if (rc != SJD_OK || splits == 1) return rc;
   return launch_attention_combine(partial, in_pos, out, M, n_heads, head_dim, splits, stream, HiLoOut{nullptr, 0});
 }

@@ -20,7 +20,7 @@ namespace sjd {
 #endif
 int attention_splits(int n_heads, int batch) {
   int s = SJD_ATTN_SLOTS / (n_heads * batch);
-  return s < 1 ? 1 : (s > 8 ? 8 : s);   // at most 8: the key ranges of a head form one thread-block cluster
+  return s < 1 ? 1 : (s > 16 ? 16 : s);
 }
 
 namespace {
@@ -443,7 +443,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, attn,
                                                 hl_attn, status, M, rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim,
                                                 att_splits, stream));
-      if (att_splits > 8)   // (not reached: the split rule stays within one cluster, which merges by itself)
+      if (att_splits > 1)
         SJD_TR(TC_ATTENTION,
                launch_attention_combine(partial, st.in_pos, attn, M, g.n_heads, g.head_dim, att_splits, stream, hl_attn));
     } else {
