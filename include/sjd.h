@@ -61,10 +61,15 @@ typedef enum {
   SJD_INIT_RANDOM = 0,     /* uniform random token; carries q = 1/V                         */
   SJD_INIT_COPY_ABOVE = 1, /* token at position - grid_stride (strategy (b)); q = point mass */
   SJD_INIT_COPY_LEFT = 2,  /* token at position - 1 (strategy (a)); q = point mass           */
-  SJD_INIT_RESAMPLE_LEFT = 3 /* strategy (c): drawn from the distribution predicted at the left neighbour, */
+  SJD_INIT_RESAMPLE_LEFT = 3, /* strategy (c): drawn from the distribution predicted at the left neighbour, */
                            /* i.e. from the most recent logits row of the nearest position to the left   */
                            /* that has been through a pass (row min(t - 1 - n, W_eff - 1) of this pass);  */
                            /* q = that row's top-k softmax; first window: uniform random token            */
+  SJD_INIT_RESAMPLE_ABOVE = 4 /* strategy (d): drawn from the distribution predicted at position -        */
+                           /* grid_stride, i.e. from the most recent logits row of that position, which   */
+                           /* the context retains in a ring of cfg.max_ring rows (the rows as the         */
+                           /* verification saw them: mixed under guidance); no such row (first image      */
+                           /* row): uniform random token                                                   */
 } sjd_init_kind;
 
 /* Which decoding schedule a step runs: the paper's method, or one of the baselines it is compared with
@@ -82,7 +87,8 @@ typedef enum {
 typedef enum {
   SJD_Q_ROW = 0,     /* top-k softmax of the logits row that produced it one iteration ago */
   SJD_Q_UNIFORM = 1, /* 1/V                                                                */
-  SJD_Q_ONEHOT = 2   /* point mass on the draft itself                                     */
+  SJD_Q_ONEHOT = 2,  /* point mass on the draft itself                                     */
+  SJD_Q_RING = 3     /* top-k softmax of a retained logits row (SJD_INIT_RESAMPLE_ABOVE)   */
 } sjd_q_kind;
 
 /* bits of sjd_step_out.flags */
@@ -97,6 +103,9 @@ typedef struct {
   float rms_eps;
   int32_t dtype;    /* sjd_dtype of weights, activations, KV cache and stored logits */
   int32_t max_batch, max_seq, max_window;
+  int32_t max_ring; /* logits rows retained per image for SJD_INIT_RESAMPLE_ABOVE: at least grid_stride +   */
+                    /* window (each costs vocab elements of dtype in the workspace); 0 if that strategy is  */
+                    /* not used                                                                            */
 } sjd_model_cfg;
 
 /* Device pointers, borrowed.  Per-layer entries are HOST arrays of n_layers device pointers. */

@@ -18,8 +18,8 @@ SJD_OK = 0
 SJD_ERR_BAD_ARG, SJD_ERR_CAPACITY, SJD_ERR_UNSUPPORTED = -1, -2, -3
 SJD_ERR_CUDA, SJD_ERR_DEVICE_TIMEOUT, SJD_ERR_STATE = -4, -5, -6
 SJD_F32, SJD_BF16 = 0, 1
-SJD_INIT_RANDOM, SJD_INIT_COPY_ABOVE, SJD_INIT_COPY_LEFT, SJD_INIT_RESAMPLE_LEFT = 0, 1, 2, 3
-SJD_Q_ROW, SJD_Q_UNIFORM, SJD_Q_ONEHOT = 0, 1, 2
+SJD_INIT_RANDOM, SJD_INIT_COPY_ABOVE, SJD_INIT_COPY_LEFT, SJD_INIT_RESAMPLE_LEFT, SJD_INIT_RESAMPLE_ABOVE = 0, 1, 2, 3, 4
+SJD_Q_ROW, SJD_Q_UNIFORM, SJD_Q_ONEHOT, SJD_Q_RING = 0, 1, 2, 3
 SJD_SCHEDULE_SJD, SJD_SCHEDULE_JACOBI, SJD_SCHEDULE_NO_REFINE = 0, 1, 2
 SJD_FLAG_NEAR_TIE_ACCEPT, SJD_FLAG_RESIDUAL_EMPTY, SJD_FLAG_NONFINITE, SJD_FLAG_DONE = 1, 4, 8, 16
 
@@ -45,7 +45,7 @@ class sjd_model_cfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "ffn_hidden",
                                          "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32),
-                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_window", C.c_int32)]
+                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_window", C.c_int32), ("max_ring", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -150,10 +150,10 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_model_cfg(wl, max_batch: int, max_seq: int, max_window: int) -> sjd_model_cfg:
+def make_model_cfg(wl, max_batch: int, max_seq: int, max_window: int, max_ring: int = 0) -> sjd_model_cfg:
     """wl: anything with the model fields of inputs.Workload."""
     return sjd_model_cfg(wl.n_layers, wl.d_model, wl.n_heads, wl.n_kv_heads, wl.head_dim, wl.ffn_hidden, wl.vocab,
-                         wl.rope_theta, wl.rms_eps, DTYPES[wl.dtype], max_batch, max_seq, max_window)
+                         wl.rope_theta, wl.rms_eps, DTYPES[wl.dtype], max_batch, max_seq, max_window, max_ring)
 
 
 def make_sample_cfg(temperature=1.0, top_k=2000, seed=0, window=16, init=SJD_INIT_RANDOM, grid_stride=0,

@@ -12,8 +12,8 @@ int check_sample_cfg(const sjd_sample_cfg *s, int vocab) {
   if (!s) return SJD_ERR_BAD_ARG;
   if (!(s->temperature > 0.0f) || s->top_k < 1 || s->window < 1) return SJD_ERR_BAD_ARG;
   if (s->window > 64) return SJD_ERR_CAPACITY;
-  if (s->init < SJD_INIT_RANDOM || s->init > SJD_INIT_RESAMPLE_LEFT) return SJD_ERR_BAD_ARG;
-  if (s->init == SJD_INIT_COPY_ABOVE && s->grid_stride < 1) return SJD_ERR_BAD_ARG;
+  if (s->init < SJD_INIT_RANDOM || s->init > SJD_INIT_RESAMPLE_ABOVE) return SJD_ERR_BAD_ARG;
+  if ((s->init == SJD_INIT_COPY_ABOVE || s->init == SJD_INIT_RESAMPLE_ABOVE) && s->grid_stride < 1) return SJD_ERR_BAD_ARG;
   if (s->seq_base < 0) return SJD_ERR_BAD_ARG;
   if (!(s->guidance == s->guidance) || s->guidance > 1e6f || s->guidance < -1e6f) return SJD_ERR_BAD_ARG;
   if (s->schedule < SJD_SCHEDULE_SJD || s->schedule > SJD_SCHEDULE_NO_REFINE) return SJD_ERR_BAD_ARG;

@@ -211,12 +211,21 @@ struct VerifyParams {
   int paired;
   float guidance;
   int schedule;            // sjd_schedule_kind
+  // Sec. 4.2 (d): ring of retained rows [image][ring_len][V] (storage dtype, as verification saw them) with
+  // their statistics; slot = position % ring_len.  n_prev / w_prev [image]: fixed tokens and window size
+  // before the slide of the last verification (what the retaining copy goes by).  ring == null: not in use.
+  void *ring;
+  RowStats *ring_stats;
+  int ring_len;
+  int32_t *n_prev, *w_prev;
   SeqState st;
   sjd_step_out out;
 };
 
 // kernel launchers (each returns an sjd_status)
 int launch_verify(const VerifyParams &p, int dtype, cudaStream_t stream);
+// after a verification: copy the rows of the window it verified (and their statistics) into the ring
+int launch_retain_rows(const VerifyParams &p, int dtype, cudaStream_t stream);
 size_t verify_scratch_bytes(int batch, int window);
 int check_sample_cfg(const sjd_sample_cfg *s, int vocab);
 

@@ -47,6 +47,7 @@ struct Layout {
   size_t x, h, qkv, q, attn, gu, act, partial, rope;
   size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
+  size_t ring, ring_stats, n_prev, w_prev;   // Sec. 4.2 (d): retained logits rows (max_ring > 0)
   size_t total;
 };
 
@@ -57,6 +58,7 @@ bool cfg_valid(const sjd_model_cfg *c) {
     return false;
   if (c->head_dim % 2 != 0 || c->n_heads % c->n_kv_heads != 0) return false;
   if (!(c->rms_eps > 0.0f) || !(c->rope_theta > 0.0f)) return false;
+  if (c->max_ring < 0) return false;
   return true;
 }
 
@@ -127,6 +129,11 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.q_draft = take(Mx * 4);
   L.in_tok = take(Mx * 4);
   L.in_pos = take(Mx * 4);
+  const size_t ring_rows = (size_t)c.max_batch * (c.max_ring > 0 ? c.max_ring : 0);
+  L.ring = take(ring_rows * c.vocab * es);
+  L.ring_stats = take(ring_rows * sizeof(RowStats));
+  L.n_prev = take((size_t)c.max_batch * 4);
+  L.w_prev = take((size_t)c.max_batch * 4);
   L.total = off;
   return L;
 }
@@ -535,6 +542,15 @@ int run_verify(sjd_ctx *c, const sjd_step_out *out, cudaStream_t stream) {
     p.done_counter = p.seq_counter + p.B;
   }
   if (out) p.out = *out;
+  if (c->sample.init == SJD_INIT_RESAMPLE_ABOVE) {   // retained rows: read by this launch, refreshed after it
+    p.ring = c->ws + c->lay.ring;
+    p.ring_stats = c->at<RowStats>(c->lay.ring_stats);
+    p.ring_len = c->cfg.max_ring;
+    p.n_prev = c->at<int32_t>(c->lay.n_prev);
+    p.w_prev = c->at<int32_t>(c->lay.w_prev);
+    const int rc = launch_verify(p, c->cfg.dtype, stream);
+    return rc != SJD_OK ? rc : launch_retain_rows(p, c->cfg.dtype, stream);
+  }
   return launch_verify(p, c->cfg.dtype, stream);
 }
 
@@ -683,6 +699,8 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
   if (batch > c->cfg.max_batch || sample->window > c->cfg.max_window) return SJD_ERR_CAPACITY;
   if ((long)prompt_len + sample->n_generate > c->cfg.max_seq) return SJD_ERR_CAPACITY;
   if (sample->guidance != 0.0f && batch % 2 != 0) return SJD_ERR_BAD_ARG;   // streams come in pairs
+  if (sample->init == SJD_INIT_RESAMPLE_ABOVE && c->cfg.max_ring < sample->grid_stride + sample->window)
+    return SJD_ERR_CAPACITY;   // a retained row must outlive the window that draws from it
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   c->sample = *sample;
   c->batch = batch;

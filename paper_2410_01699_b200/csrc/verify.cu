@@ -108,9 +108,10 @@ struct Scratch {
   int tok;
   float tok_w;
   int is_last;
-  // new window slots whose token is drawn from a logits row of this pass (Sec. 4.2 (c)): filled by
-  // draw_fresh_slots, consumed by finalize_sequence; row -1: no row, the slot is a uniform random token
-  int fresh_tok[64], fresh_row[64];
+  // new window slots whose token is drawn from a logits row (Sec. 4.2 (c), (d)): filled by draw_fresh_slots,
+  // consumed by finalize_sequence; row -1: no row, the slot is a uniform random token; kind SJD_Q_ROW: a row
+  // of this pass's buffer, SJD_Q_RING: a slot of the ring of retained rows
+  int fresh_tok[64], fresh_row[64], fresh_kind[64];
   float fresh_q[64];
 };
 
@@ -877,15 +878,25 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, const __nv_bf
 template <typename T>
 struct RowRefs {
   const T *p, *p2, *q, *q2;
+  const RowStats *qstats;   // statistics of the q row (valid when the launch has them cached)
 };
+// q_ring: the draft's law is a retained row (Sec. 4.2 (d)): qr is then a slot of the ring, whose rows are
+// stored as the verification saw them (already mixed under guidance)
 template <typename T>
-__device__ __forceinline__ RowRefs<T> row_refs(const VerifyParams &p, int b, int k, int qr, int cur) {
+__device__ __forceinline__ RowRefs<T> row_refs(const VerifyParams &p, int b, int k, int qr, int cur, bool q_ring = false) {
   const int sb = p.paired ? 2 * b : b;
   RowRefs<T> rr;
   rr.p = reinterpret_cast<const T *>(p.logits[cur]) + ((size_t)sb * p.W + k) * p.V;
-  rr.q = reinterpret_cast<const T *>(p.logits[cur ^ 1]) + ((size_t)sb * p.W + qr) * p.V;
   rr.p2 = p.paired ? rr.p + (size_t)p.W * p.V : nullptr;
-  rr.q2 = p.paired ? rr.q + (size_t)p.W * p.V : nullptr;
+  if (q_ring) {
+    rr.q = reinterpret_cast<const T *>(p.ring) + ((size_t)b * p.ring_len + qr) * p.V;
+    rr.q2 = nullptr;
+    rr.qstats = p.ring_stats + (size_t)b * p.ring_len + qr;
+  } else {
+    rr.q = reinterpret_cast<const T *>(p.logits[cur ^ 1]) + ((size_t)sb * p.W + qr) * p.V;
+    rr.q2 = p.paired ? rr.q + (size_t)p.W * p.V : nullptr;
+    rr.qstats = p.stats[cur ^ 1] + (size_t)b * p.W + qr;
+  }
   return rr;
 }
 
@@ -919,7 +930,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   float q_d;
   if (kind == SJD_Q_ROW) {
     if (p.prev_stats_valid) {
-      qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
+      qs = *rows.qstats;
       if (qs.flags != 0 || !(qs.xmax > -FLT_MAX) || qs.tau_key == 0x7FFFu || qs.tau_key == 0x8000u) return false;
       uint32_t bits = E::NEG_INF;
       if (d_ok) {
@@ -1089,14 +1100,15 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
   if (a < 0) return;
   const int r = b * W + a;
   const int sb = p.paired ? 2 * b : b;   // the sequence whose state holds the window (both streams hold the same)
-  const int kind = p.q_kind ? p.q_kind[sb * W + a] : SJD_Q_ROW;
+  const int kind_raw = p.q_kind ? p.q_kind[sb * W + a] : SJD_Q_ROW;
+  const int kind = kind_raw == SJD_Q_RING ? SJD_Q_ROW : kind_raw;
   const int d = p.draft[sb * W + a];
   const int qr = p.q_row ? p.q_row[sb * W + a] : a;
   const int base = p.e2e ? p.st.n[sb] : (p.base_pos ? p.base_pos[b] : 0);
   const Philox4 rnd = philox4x32_10((uint32_t)(base + a), step, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo,
                                     p.seed_hi);
   const float u_res = u24(rnd.w[1]);
-  const RowRefs<__nv_bfloat16> rows = row_refs<__nv_bfloat16>(p, b, a, qr, cur);
+  const RowRefs<__nv_bfloat16> rows = row_refs<__nv_bfloat16>(p, b, a, qr, cur, kind_raw == SJD_Q_RING);
   const uint4 *pg = reinterpret_cast<const uint4 *>(rows.p), *pg2 = reinterpret_cast<const uint4 *>(rows.p2);
   auto load_stats = [](const RowStats *g) {
     const uint4 u = __ldcg(reinterpret_cast<const uint4 *>(g));
@@ -1107,7 +1119,7 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
   const RowStats ps = load_stats(&p.stats[cur][r]);
   RowStats qs;
   qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
-  if (kind == SJD_Q_ROW) qs = load_stats(&p.stats[cur ^ 1][(size_t)b * W + qr]);
+  if (kind == SJD_Q_ROW) qs = load_stats(rows.qstats);
   RegRow row;
   const int j0 = warp * 256 + lane;
 #pragma unroll
@@ -1177,17 +1189,32 @@ __device__ void draw_fresh_slots(const VerifyParams &p, int b, uint32_t step, in
   int have = -1;   // row whose chunk sums are in the scratch
   for (int s = kept; s < w2; ++s) {
     const int t_pos = n2 + s;
-    const int k = w_eff > 0 ? min(t_pos - 1 - base, w_eff - 1) : -1;
-    if (k < 0) {
+    // k: row of this pass's buffer (>= 0), or -2 - slot for a slot of the ring, or -1: no row
+    int k = -1;
+    if (p.st.init == SJD_INIT_RESAMPLE_LEFT) {
+      if (w_eff > 0) k = min(t_pos - 1 - base, w_eff - 1);
+    } else {   // (d): the position one grid row above; its most recent row is in this pass's buffer if it was
+               // inside the window just verified, else in the ring (every image position passes through a window)
+      const int src = t_pos - p.st.grid_stride;
+      if (src >= p.st.prompt_len) {
+        if (src >= base) k = src - base < w_eff ? src - base : -1;
+        else if (p.ring) k = -2 - src % p.ring_len;
+      }
+    }
+    if (k == -1) {
       if (tid == 0) sc.fresh_row[s] = -1;
       continue;
     }
-    const RowRefs<T> rows = row_refs<T>(p, b, k, 0, cur);
-    const uint4 su = __ldcg(reinterpret_cast<const uint4 *>(&p.stats[cur][(size_t)b * W + k]));
+    const bool from_ring = k < -1;
+    const int slot = from_ring ? -2 - k : k;
+    const RowRefs<T> rows = row_refs<T>(p, b, from_ring ? 0 : slot, from_ring ? slot : 0, cur, from_ring);
+    const RowStats *sp = from_ring ? rows.qstats : &p.stats[cur][(size_t)b * W + slot];
+    const uint4 su = __ldcg(reinterpret_cast<const uint4 *>(sp));
     RowStats st;
     st.tau_key = su.x; st.xmax = __uint_as_float(su.y); st.z = __uint_as_float(su.z); st.flags = su.w;
     PRowWeights<T> f;
-    f.row.init(rows.p, p.V, rows.p2, p.guidance);
+    if (from_ring) f.row.init(rows.q, p.V);
+    else f.row.init(rows.p, p.V, rows.p2, p.guidance);
     f.pw.init(st, inv_t);
     if (k != have) {
       chunk_sums<E::VEC>(f, f.row.NV, sc);
@@ -1198,7 +1225,8 @@ __device__ void draw_fresh_slots(const VerifyParams &p, int b, uint32_t step, in
     if (tid == 0) {
       sc.fresh_tok[s] = sc.tok;
       sc.fresh_q[s] = sc.tok_w / st.z;
-      sc.fresh_row[s] = k;
+      sc.fresh_row[s] = slot;
+      sc.fresh_kind[s] = from_ring ? SJD_Q_RING : SJD_Q_ROW;
     }
     __syncthreads();
   }
@@ -1279,10 +1307,11 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
       q = __ldcg(&ro[k].redraft_p);
       kind = SJD_Q_ROW;
       qrow = k;
-    } else if (s < w2 && p.st.init == SJD_INIT_RESAMPLE_LEFT && sc.fresh_row[s] >= 0) {  // Sec. 4.2 (c)
+    } else if (s < w2 && (p.st.init == SJD_INIT_RESAMPLE_LEFT || p.st.init == SJD_INIT_RESAMPLE_ABOVE) &&
+               sc.fresh_row[s] >= 0) {  // Sec. 4.2 (c), (d)
       tok = sc.fresh_tok[s];
       q = sc.fresh_q[s];
-      kind = SJD_Q_ROW;
+      kind = sc.fresh_kind[s];
       qrow = sc.fresh_row[s];
     } else if (s < w2) {  // freshly initialised slot (end-to-end mode only), Sec. 4.2
       const int t_pos = n2 + s;
@@ -1333,6 +1362,10 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
         p.st.w_eff[sb + s2] = w2;
       }
     }
+    if (p.n_prev) {   // what the retaining copy after this launch goes by (Sec. 4.2 (d))
+      p.n_prev[b] = base;
+      p.w_prev[b] = w_eff;
+    }
     if (o.n_accepted) o.n_accepted[b] = a;
     if (o.n_committed) o.n_committed[b] = m;
     if (o.total_committed) o.total_committed[b] = n2;
@@ -1364,7 +1397,9 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
 
   if (k < w_eff) {
     // (the Jacobi schedule compares tokens and uses no q: treat every draft as a copied one)
-    const int kind = p.schedule == SJD_SCHEDULE_JACOBI ? SJD_Q_ONEHOT : (p.q_kind ? p.q_kind[rs] : SJD_Q_ROW);
+    const int kind_raw = p.q_kind ? p.q_kind[rs] : SJD_Q_ROW;
+    const bool q_ring = kind_raw == SJD_Q_RING;   // a retained row: the same law as a row of the other buffer
+    const int kind = p.schedule == SJD_SCHEDULE_JACOBI ? SJD_Q_ONEHOT : (q_ring ? SJD_Q_ROW : kind_raw);
     const int d = p.draft[rs];
     const bool d_ok = d >= 0 && d < p.V;
     const int qr = p.q_row ? p.q_row[rs] : k;
@@ -1376,7 +1411,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     const bool jacobi = p.schedule == SJD_SCHEDULE_JACOBI;
     if (jacobi)   // Sec. 3.2: the draw of a position uses the same uniform in every pass (step index 0)
       u_draft = u24(philox4x32_10((uint32_t)(base + k), 0u, p.seq_base + (uint32_t)b, kStreamVerify, p.seed_lo, p.seed_hi).w[2]);
-    const RowRefs<T> rows = row_refs<T>(p, b, k, qr, cur);
+    const RowRefs<T> rows = row_refs<T>(p, b, k, qr, cur, q_ring);
 
     RowOut fast_out;
     const bool fast_done = p.fast && (((uintptr_t)rows.q | (uintptr_t)rows.p) & 15u) == 0 &&
@@ -1394,7 +1429,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
     float q_d;
     if (kind == SJD_Q_ROW) {
       if (p.prev_stats_valid) {
-        qs = p.stats[cur ^ 1][(size_t)b * p.W + qr];
+        qs = *rows.qstats;
       } else {
         qs = row_statistics<T>(qrow, stage, sc, p.top_k, inv_t, qf);
         if (tid == 0) p.stats[cur ^ 1][r] = qs;
@@ -1482,7 +1517,8 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   __threadfence();
   SJD_TL(TL_VERIFY, 14, tid == 0);
   if (p.fast && p.defer_residual) deferred_residual<T>(p, b, step, cur, sc);
-  if (p.e2e && p.st.init == SJD_INIT_RESAMPLE_LEFT) draw_fresh_slots<T>(p, b, step, cur, sc);
+  if (p.e2e && (p.st.init == SJD_INIT_RESAMPLE_LEFT || p.st.init == SJD_INIT_RESAMPLE_ABOVE))
+    draw_fresh_slots<T>(p, b, step, cur, sc);
   finalize_sequence(p, b, step, sc);
   SJD_TL(TL_VERIFY, 15, tid == 0);
   __syncthreads();
@@ -1497,7 +1533,42 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   }
 }
 
+// Sec. 4.2 (d): keep the rows of the window just verified (as the verification saw them: mixed under
+// guidance) and their statistics in the ring, slot = position % ring_len; one block per (row, image).
+template <typename T>
+__global__ void retain_rows_kernel(const VerifyParams p) {
+  pdl_trigger();
+  pdl_wait();
+  const int k = blockIdx.x, b = blockIdx.y;
+  if (k >= p.w_prev[b]) return;
+  const uint32_t step = *p.step_ptr - 1u;          // the verification before this kernel has bumped the index
+  const int cur = (int)(step & 1u);
+  const int slot = (p.n_prev[b] + k) % p.ring_len;
+  Row<T> row;
+  const RowRefs<T> rows = row_refs<T>(p, b, k, 0, cur);
+  row.init(rows.p, p.V, rows.p2, p.guidance);
+  T *dst = reinterpret_cast<T *>(p.ring) + ((size_t)b * p.ring_len + slot) * p.V;
+  unsigned short *d16 = reinterpret_cast<unsigned short *>(dst);
+  uint32_t *d32 = reinterpret_cast<uint32_t *>(dst);
+  for (int i = threadIdx.x; i < p.V; i += blockDim.x) {
+    const uint32_t bits = row.raw_bits(i);
+    if (sizeof(T) == 2) d16[i] = (unsigned short)bits;
+    else d32[i] = bits;
+  }
+  if (threadIdx.x == 0) p.ring_stats[(size_t)b * p.ring_len + slot] = p.stats[cur][(size_t)b * p.W + k];
+}
+
 }  // namespace
+
+int launch_retain_rows(const VerifyParams &p, int dtype, cudaStream_t stream) {
+  if (!p.ring || !p.ring_stats || p.ring_len < 1 || !p.n_prev || !p.w_prev || !p.step_ptr) return SJD_ERR_BAD_ARG;
+  const dim3 grid(p.W, p.B);
+  if (dtype == SJD_F32) SJD_CUDA(launch_kernel(retain_rows_kernel<float>, grid, dim3(256), 0, stream, p));
+  else if (dtype == SJD_BF16) SJD_CUDA(launch_kernel(retain_rows_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, p));
+  else return SJD_ERR_UNSUPPORTED;
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
 
 size_t verify_scratch_bytes(int batch, int window) {
   if (batch <= 0 || window <= 0) return 0;

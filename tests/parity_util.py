@@ -183,7 +183,9 @@ class LockStepSequence:
         w_eff = len(self.st.drafts)
         assert int(total) == self.st.n
         assert [int(t) for t in draft_row[:w_eff]] == self.st.drafts, "window drafts differ"
-        assert [int(t) for t in kind_row[:w_eff]] == [q.kind for q in self.st.qdescs], "window laws differ"
+        # (the library tells a row of the other logits buffer, 0, from a retained row, 3: the same kind of law)
+        assert [0 if int(t) == 3 else int(t) for t in kind_row[:w_eff]] == [q.kind for q in self.st.qdescs], \
+            "window laws differ"
         assert all(int(t) == -1 for t in draft_row[w_eff:])
         from oracle.sjd import q_of_draft
         for k in range(w_eff):
@@ -256,13 +258,11 @@ class LockStepSequence:
         a = int(out_b["n_accepted"])
         st.committed = st.committed[:n_before] + [int(t) for t in out_b["committed"][:m]]
         new_w = max(0, min(scfg.window, self.wl.prompt_len + scfg.n_generate - st.n))
-        st.drafts = [int(t) for t in out_b["draft"][:new_w]]
-        st.qdescs = []
-        kept = 0
-        for s in range(new_w):
-            kind = int(out_b["q_kind"][s])
-            if kind == Q_ROW:
-                st.qdescs.append(QDesc(Q_ROW, row=np.array(gpu_logits_rows[a + 1 + s], dtype=np.float64)))
-                kept += 1
-            else:
-                st.qdescs.append(QDesc(kind))
+        # the slots re-drawn by Eq. 3 follow the library (rows a+1 ..); the slots that enter the window are
+        # a function of the state alone, so the checker initialises them itself and the windows are compared
+        from oracle.sjd import SCHEDULE_NO_REFINE, _fill_window
+        redrawn = 0 if scfg.schedule == SCHEDULE_NO_REFINE else max(0, min(w_eff - a - 1, new_w))
+        st.drafts = [int(t) for t in out_b["draft"][:redrawn]]
+        st.qdescs = [QDesc(Q_ROW, row=np.array(gpu_logits_rows[a + 1 + s], dtype=np.float64)) for s in range(redrawn)]
+        _fill_window(st, scfg, vocab, st.step - 1)
+        self.check_window(out_b["draft"], out_b["q_kind"], out_b["q_draft"], out_b["total_committed"])

@@ -6,7 +6,8 @@ import numpy as np
 import pytest
 import torch
 
-from oracle.sjd import INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, INIT_RESAMPLE_LEFT, SampleCfg
+from oracle.sjd import (INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RANDOM, INIT_RESAMPLE_ABOVE, INIT_RESAMPLE_LEFT,
+                        SampleCfg)
 from paper_2410_01699_b200 import binding as B
 from paper_2410_01699_b200.inputs import WORKLOADS, make_prompt, make_weights
 from tests.parity_util import LockStepSequence
@@ -23,7 +24,8 @@ def run_lockstep(wl, batch=1, max_steps=None, init=INIT_RANDOM, check_logits_eve
     top_k = top_k or wl.top_k
     weights = make_weights(wl, gain_jitter=gain_jitter)
     prompt = make_prompt(wl, batch)
-    cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=wl.prompt_len + n_generate + 8, max_window=window)
+    cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=wl.prompt_len + n_generate + 8, max_window=window,
+                           max_ring=wl.grid_stride + window if init == INIT_RESAMPLE_ABOVE else 0)
     ctx = B.Context(cfg, B.weights_to_device(weights))
     sample = B.make_sample_cfg(temperature=wl.temperature, top_k=top_k, seed=wl.philox_seed, window=window,
                                init=init, grid_stride=wl.grid_stride, n_generate=n_generate, seq_base=seq_base,
@@ -74,10 +76,31 @@ def test_tiny_fp32_full_generation():
     assert h["total_committed"][0] == wl.prompt_len + wl.n_generate
 
 
-@pytest.mark.parametrize("init", [INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RESAMPLE_LEFT])
+@pytest.mark.parametrize("init", [INIT_COPY_ABOVE, INIT_COPY_LEFT, INIT_RESAMPLE_LEFT, INIT_RESAMPLE_ABOVE])
 def test_tiny_spatial_initialisation(init):
     wl = WORKLOADS["tiny"]
     run_lockstep(wl, init=init, n_generate=100)
+
+
+def test_small_bf16_initialisation_from_the_prediction_above():
+    """Sec. 4.2 (d) on the bf16 model with a grid row shorter than the window (stride 5, W = 16): the row
+    above is sometimes a row of the pass just verified and sometimes a retained row of the ring, and a
+    retained row serves as the draft's law on the register-resident verification route."""
+    wl = WORKLOADS["small-bf16"].with_(grid_stride=5)
+    ctx, seqs, steps, out = run_lockstep(wl, batch=2, init=INIT_RESAMPLE_ABOVE, n_generate=60)
+    assert steps <= 60
+    wl = WORKLOADS["small-bf16"]    # stride 16 = W: every source row comes from the ring
+    ctx, seqs, steps, out = run_lockstep(wl, init=INIT_RESAMPLE_ABOVE, n_generate=60, schedule=2)
+    assert steps <= 60
+
+
+def test_resample_above_needs_a_ring():
+    wl = WORKLOADS["tiny"]
+    ctx = B.Context(B.make_model_cfg(wl, 1, 64, 8, max_ring=10), B.weights_to_device(make_weights(wl)))
+    with pytest.raises(B.SJDError) as e:
+        ctx.prefill(torch.from_numpy(make_prompt(wl, 1)).cuda(),
+                    B.make_sample_cfg(top_k=10, window=8, n_generate=20, init=B.SJD_INIT_RESAMPLE_ABOVE, grid_stride=16))
+    assert e.value.status == B.SJD_ERR_CAPACITY
 
 
 @pytest.mark.parametrize("schedule", [0, 2])
