@@ -99,7 +99,7 @@ struct Elt<__nv_bfloat16> {
 struct Scratch {
   double chunk_excl[kMaxChunks + 1];  // exclusive prefix of chunk sums; [NC] = total
   float chunk_sum[kMaxChunks];
-  uint32_t hist12[4096];              // register-resident route: histogram of code distances below the row maximum
+  alignas(16) uint32_t hist12[4096];              // register-resident route: histogram of code distances below the row maximum
   uint32_t hist[256];
   uint32_t redu[32];
   uint32_t d_bits[2];                 // register-resident route: bits of the q / p row's entry at the draft token
@@ -559,7 +559,7 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, const uint4 *g2, fl
     row.v[i] = j < NV ? rr_load_vec(g, g2, gw, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
   }
   if (zero_hist)
-    for (int i = tid; i < 4096; i += nt) sc.hist12[i] = 0;
+    for (int i = tid; i < 1024; i += nt) reinterpret_cast<uint4 *>(sc.hist12)[i] = make_uint4(0u, 0u, 0u, 0u);
   __nv_bfloat162 m2 = as_bf2(row.v[0].x);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -610,36 +610,39 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
     }
   }
   __syncthreads();
+  // The walk: 32 adjacent bins per step (conflict-free).  A step that does not reach the K-th entry costs one
+  // load and one warp-wide integer sum; only the step that does is scanned.  For z_hist every lane
+  // accumulates the mass of its own bins and the warp adds the lanes up once, at the end.
   uint32_t acc = 0;
-  double zacc = 0.0;
+  float zl = 0.0f;
   const float xmax = E::val(E::unkey(kmax));
-  for (int base = 0; base < 4096; base += 32) {   // 32 adjacent bins per step: conflict-free
+  for (int base = 0; base < 4096; base += 32) {
     const uint32_t c = sc.hist12[base + lane];
+    const uint32_t bin = (uint32_t)(base + lane);
+    const uint32_t tot = __reduce_add_sync(0xffffffffu, c);
+    if (acc + tot < K) {
+      if (z_hist && c != 0 && bin <= kmax) zl += (float)c * exp2_neg((E::val(E::unkey(kmax - bin)) - xmax) * scale);
+      acc += tot;
+      continue;
+    }
     uint32_t incl = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += y;
     }
-    const uint32_t ballot = __ballot_sync(0xffffffffu, acc + incl >= K);
+    const uint32_t ballot = __ballot_sync(0xffffffffu, acc + incl >= K);   // non-zero: this step reaches K
+    const int last = __ffs(ballot) - 1;
     if (z_hist) {   // mass of this step's bins down to (and including) the threshold bin
-      const int last = ballot ? __ffs(ballot) - 1 : 31;
-      const uint32_t bin = (uint32_t)(base + lane);
-      float zl = 0.0f;
-      if (lane <= last && c != 0 && bin <= kmax)
-        zl = (float)c * exp2_neg((E::val(E::unkey(kmax - bin)) - xmax) * scale);
+      if (lane <= last && c != 0 && bin <= kmax) zl += (float)c * exp2_neg((E::val(E::unkey(kmax - bin)) - xmax) * scale);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) zl += __shfl_xor_sync(0xffffffffu, zl, o);
-      zacc += (double)zl;
+      *z_hist = (double)zl;
     }
-    if (ballot) {
-      const uint32_t bin = (uint32_t)(base + __ffs(ballot) - 1);
-      if (bin >= 4095u) return false;
-      tau_key = kmax - bin;
-      if (z_hist) *z_hist = zacc;
-      return !(tau_key == 0x7FFFu || tau_key == 0x8000u);
-    }
-    acc += __shfl_sync(0xffffffffu, incl, 31);
+    const uint32_t tbin = (uint32_t)(base + last);
+    if (tbin >= 4095u) return false;
+    tau_key = kmax - tbin;
+    return !(tau_key == 0x7FFFu || tau_key == 0x8000u);
   }
   return false;
 }
