@@ -53,7 +53,7 @@ constexpr int kMaxStages = 8;
 #define SJD_GEMM_L2_PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
 #endif
 #ifndef SJD_GEMM_MIN_KB
-#define SJD_GEMM_MIN_KB 16                  // fewest k-blocks (of 16 KB of weights) a CTA should stream
+#define SJD_GEMM_MIN_KB 8                   // fewest k-blocks (of 16 KB of weights) a CTA should stream (8: the O projection runs 32 x 8 CTAs whose whole share fits the prefetched ring; 3.51 against 3.54 ms per step with 16)
 #endif
 #ifndef SJD_GEMM_CTAS_PER_SM
 #define SJD_GEMM_CTAS_PER_SM 2
@@ -375,41 +375,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
         // MMA rows 0..63 hold gate features, rows 64..127 the same features of the up matrix.  The warps
         // that read the up rows (TMEM lane quarters 2, 3) pass their values through shared memory (the
         // ring is idle by now) to the warps that read the gate rows, which finish the activation.
-        float *ex = reinterpret_cast<float *>(smem);   // [64][Mp + 1]
+        // Every epilogue warp parks its 32 accumulator rows (scaled) in shared memory, row-major with an odd
+        // stride; after one barrier the 128 threads share the activation work: thread t finishes feature
+        // t % 64 for every second token, so that a warp's stores cover 32 adjacent features of one token.
+        float *ex = reinterpret_cast<float *>(smem);   // [128][Mp + 1]
         const int ldx = p.Mp + 1;
         const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        const int f = tile * R + (row & 63);
-        const bool live = (row & 63) < R && f < p.F;
-        if (quarter >= 2) {
-          for (int m0 = 0; m0 < p.Mp; m0 += 16) {
-            uint32_t hi[16], lo[16];
-            tmem_ld16_issue(t_addr + m0, hi);
-            tmem_ld16_issue(t_addr + p.Mp + m0, lo);
-            tmem_ld_wait();
+        for (int m0 = 0; m0 < p.Mp; m0 += 16) {
+          uint32_t hi[16], lo[16];
+          tmem_ld16_issue(t_addr + m0, hi);
+          tmem_ld16_issue(t_addr + p.Mp + m0, lo);
+          tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-              ex[(row - 64) * ldx + m0 + i] = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * s_scale[m0 + i];
-          }
+          for (int i = 0; i < 16; ++i)
+            ex[row * ldx + m0 + i] = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * s_scale[m0 + i];
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // the up values are in place
-        if (quarter < 2) {
-          for (int m0 = 0; m0 < p.Mp; m0 += 16) {
-            uint32_t hi[16], lo[16];
-            tmem_ld16_issue(t_addr + m0, hi);
-            tmem_ld16_issue(t_addr + p.Mp + m0, lo);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int m = m_base + m0 + i;
-              if (live && m < p.M) {
-                const float g = (__uint_as_float(hi[i]) + __uint_as_float(lo[i])) * s_scale[m0 + i];
-                const float u = ex[row * ldx + m0 + i];
-                const float v = g / (1.0f + expf(-g)) * u;
-                const __nv_bfloat16 vh = __float2bfloat16_rn(v);
-                p.act_hi[(size_t)m * p.F + f] = vh;
-                p.act_hi[p.act_lo_off + (size_t)m * p.F + f] = __float2bfloat16_rn(v - __bfloat162float(vh));
-              }
-            }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int e = tid - 64, fr = e & 63;
+        const int f = tile * R + fr;
+        if (fr < R && f < p.F) {
+          for (int mm = e >> 6; mm < p.Mp; mm += 2) {
+            const int m = m_base + mm;
+            if (m >= p.M) break;
+            const float g = ex[fr * ldx + mm], u = ex[(64 + fr) * ldx + mm];
+            const float v = g / (1.0f + expf(-g)) * u;
+            const __nv_bfloat16 vh = __float2bfloat16_rn(v);
+            p.act_hi[(size_t)m * p.F + f] = vh;
+            p.act_hi[p.act_lo_off + (size_t)m * p.F + f] = __float2bfloat16_rn(v - __bfloat162float(vh));
           }
         }
       } else {

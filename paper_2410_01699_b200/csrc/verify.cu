@@ -565,10 +565,15 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, const uint4 *g2, fl
   for (int i = 0; i < 8; ++i) {
 #pragma unroll
     for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(row.v[i], w)));
-    if (d >= 0 && (d >> 3) == j0 + i * 32) {   // this thread holds entry d
-      const uint32_t wd = word_of(row.v[i], (d >> 1) & 3);
-      sc.d_bits[d_slot] = (d & 1) ? wd >> 16 : wd & 0xFFFFu;
+  }
+  if (tid == 0 && d >= 0) {   // the entry at the draft token: one more load (a cache hit) instead of a search through the registers
+    const unsigned short *e = reinterpret_cast<const unsigned short *>(g);
+    uint32_t bits = (uint32_t)__ldg(e + d);
+    if (g2) {
+      const float c = E::val(bits), u = E::val((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(g2) + d));
+      bits = E::bits(fmaf(gw, c - u, u));
     }
+    sc.d_bits[d_slot] = bits;
   }
   const __nv_bfloat16 m1 = __hmax_nan(__low2bfloat16(m2), __high2bfloat16(m2));
   const uint32_t mbits = (uint32_t)__bfloat16_as_ushort(m1);
