@@ -122,6 +122,11 @@ typedef struct {
   const void *const *w_gate;    /* [ffn_hidden][d_model]      */
   const void *const *w_up;      /* [ffn_hidden][d_model]      */
   const void *const *w_down;    /* [d_model][ffn_hidden]      */
+  /* QK-norm variant (the Chameleon family of Sec. 5.1): per-layer gains [head_dim]; every head of q and of k  */
+  /* is RMS-normalised over its head_dim entries (eps = rms_eps) and multiplied by the gain before the rotary */
+  /* step.  Both NULL: the plain model.                                                                        */
+  const void *const *q_norm;
+  const void *const *k_norm;
 } sjd_weights;
 
 typedef struct {

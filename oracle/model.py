@@ -10,6 +10,10 @@ Sec. 3.2, Sec. 4.1 Step 2); its models are 7B Llama/Chameleon-style decoders
   per layer:
     h    = rmsnorm(x; attn_norm)            h_i = x_i * g_i / sqrt(mean(x^2) + eps)
     q,k,v= h Wq^T, h Wk^T, h Wv^T           (no bias; W stored [out][in])
+    [QK-norm variant, the Chameleon family the paper's models derive from (Sec. 5.1): when the layer
+         has gains q_norm / k_norm (length hd), every head of q and of k is normalised over its hd
+         dimensions before the rotary step, q_h = rmsnorm(q_h; q_norm), k_h = rmsnorm(k_h; k_norm).
+         Reading: the RMS form without bias, like every other normalisation of this block.]
     RoPE on q and k, half-split pairing: dims i and i + hd/2 rotate together
          by angle pos * theta^(-2i/hd), pos = absolute index from 0
     a    = causal softmax(q k^T / sqrt(hd)) v;  kv head j serves the H/KVh
@@ -143,6 +147,9 @@ class OracleModel:
         q = (h @ _f64(lw["wq"]).T).reshape(t_len, cfg.n_heads, cfg.head_dim)
         k = (h @ _f64(lw["wk"]).T).reshape(t_len, cfg.n_kv_heads, cfg.head_dim)
         v = (h @ _f64(lw["wv"]).T).reshape(t_len, cfg.n_kv_heads, cfg.head_dim)
+        if lw.get("q_norm") is not None:      # QK-norm variant: per head, over the head dimension
+            q = rmsnorm(q, lw["q_norm"], cfg.rms_eps)
+            k = rmsnorm(k, lw["k_norm"], cfg.rms_eps)
         q = rope(q, positions, cfg.rope_theta)
         k = rope(k, positions, cfg.rope_theta)
         if cache is not None:

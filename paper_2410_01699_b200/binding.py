@@ -53,7 +53,8 @@ _PP = C.POINTER(C.c_void_p)
 
 class sjd_weights(C.Structure):
     _fields_ = [("tok_emb", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)] + \
-               [(n, _PP) for n in ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")]
+               [(n, _PP) for n in ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down",
+                                   "q_norm", "k_norm")]
 
 
 class sjd_sample_cfg(C.Structure):
@@ -267,7 +268,10 @@ class Context:
         self._arrays = {}
         w = sjd_weights()
         w.tok_emb, w.final_norm, w.lm_head = (weights[k].data_ptr() for k in ("tok_emb", "final_norm", "lm_head"))
-        for name in ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down"):
+        names = ["attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down"]
+        if n_layers and "q_norm" in weights["layers"][0]:   # QK-norm variant
+            names += ["q_norm", "k_norm"]
+        for name in names:
             arr = (C.c_void_p * n_layers)(*[weights["layers"][l][name].data_ptr() for l in range(n_layers)])
             self._arrays[name] = arr
             setattr(w, name, C.cast(arr, _PP))

@@ -323,10 +323,16 @@ struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
   void *base;
   int n_kv_heads, max_seq, head_dim;
 };
+// QK-norm variant: every head of q and of k is RMS-normalised over its head_dim entries (gains of `dtype`,
+// length head_dim) before the rotary step; null gains: the plain model.
+struct QkNorm {
+  const void *q_gain, *k_gain;
+  float eps;
+};
 int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
-                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
+                       KvLayout kv, int M, int rows_per_seq, int n_heads, QkNorm qkn, cudaStream_t stream);
 int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
-                      KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream);
+                      KvLayout kv, int M, int rows_per_seq, int n_heads, QkNorm qkn, cudaStream_t stream);
 // act[m][f] = silu(gu[m][f]) * gu[m][F + f]
 int launch_swiglu(const float *gu, float *act, int M, int F, cudaStream_t stream, HiLoOut hilo = HiLoOut{nullptr, 0});
 // Window-causal attention: query row m (sequence m / rows_per_seq, position in_pos[m]) attends cache rows

@@ -233,6 +233,8 @@ struct sjd_ctx {
   char *ws;
   const void *tok_emb, *final_norm, *lm_head;
   std::vector<const void *> attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down;
+  std::vector<const void *> q_norm, k_norm;   // QK-norm gains per layer (null entries: the plain model)
+  QkNorm qk_norm(int l) const { return QkNorm{q_norm[l], k_norm[l], cfg.rms_eps}; }
   sjd_sample_cfg sample;
   int batch, prompt_len, window;
   bool prefilled;
@@ -346,7 +348,7 @@ int forward_generic(sjd_ctx *c, int rows_per_seq, void *logits_out, cudaStream_t
     SJD_TRY(gemm(c->wk[l], h, d, qkv + nq, nqkv, nk, d, EPI_STORE_F32));
     SJD_TRY(gemm(c->wv[l], h, d, qkv + nq + nk, nqkv, nk, d, EPI_STORE_F32));
     const KvLayout kv = c->kv_layer(l);
-    SJD_TR(TC_OTHER, launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
+    SJD_TR(TC_OTHER, launch_rope_append(dt, qkv, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, c->qk_norm(l), stream));
     SJD_TR(TC_ATTENTION, launch_attention(dt, q, kv, st.in_pos, attn, partial, M, rows_per_seq, g.n_heads, splits, stream));
     SJD_TRY(gemm(c->wo[l], attn, nq, x, d, d, nq, EPI_ADD_F32));
     SJD_TR(TC_OTHER, launch_rmsnorm(dt, x, c->ffn_norm[l], h, M, d, g.rms_eps, stream));
@@ -445,7 +447,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       SJD_TRY(gemm(wm, 3, n_out, xm.h, d, nqkv, planes, false, &ps));
     }
     const KvLayout kv = c->kv_layer(l);
-    SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, stream));
+    SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, c->qk_norm(l), stream));
     if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
       SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, attn,
                                                 hl_attn, status, M, rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim,
@@ -598,6 +600,12 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
   c->w_gate.assign(w->w_gate, w->w_gate + L);
   c->w_up.assign(w->w_up, w->w_up + L);
   c->w_down.assign(w->w_down, w->w_down + L);
+  c->q_norm.assign(L, nullptr);
+  c->k_norm.assign(L, nullptr);
+  if (w->q_norm && w->k_norm) {
+    c->q_norm.assign(w->q_norm, w->q_norm + L);
+    c->k_norm.assign(w->k_norm, w->k_norm + L);
+  }
   c->prefilled = false;
   c->batch = c->prompt_len = c->window = 0;
   c->host_step = 0;

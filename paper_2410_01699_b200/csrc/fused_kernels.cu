@@ -89,7 +89,8 @@ __global__ void __launch_bounds__(RG_THREADS) resid_gain_kernel(float *__restric
 template <typename T>
 __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__restrict__ in_pos,
                                   const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
-                                  int n_heads) {
+                                  int n_heads, QkNorm qkn) {
+  __shared__ float s_ss[8];   // QK-norm: per-warp sums of squares of a head (two warps per 64-thread group)
   pdl_trigger();
   SJD_TL(TL_QKV, 0, threadIdx.x == 0);
   pdl_wait();
@@ -111,9 +112,30 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   if (slot < n_heads + nkv) {
     const bool is_q = slot < n_heads;
     const int col0 = is_q ? slot * hd : nq + (slot - n_heads) * hd;
-    for (int j = lt; j < half; j += 64) {
+    // head_dim <= 128: a thread of the group owns at most one rotary pair (j, j + half) of the head
+    {
+      const int j = lt;
+      const bool has = j < half;
+      float x1 = 0.0f, x2 = 0.0f;
+      if (has) {
+        x1 = sc * sum_planes(ps, rbase + col0 + j);
+        x2 = sc * sum_planes(ps, rbase + col0 + j + half);
+      }
+      if (qkn.q_gain) {   // QK-norm: RMS over the head's entries, held by the 64 threads of this group
+        const int grp = threadIdx.x >> 6;
+        const float ws = warp_sum(x1 * x1 + x2 * x2);
+        if ((threadIdx.x & 31) == 0) s_ss[threadIdx.x >> 5] = ws;
+        asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory");
+        const float rinv = rsqrtf((s_ss[2 * grp] + s_ss[2 * grp + 1]) / (float)hd + qkn.eps);
+        asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory");   // the sums are reused by the group's next head
+        if (has) {
+          const T *gain = reinterpret_cast<const T *>(is_q ? qkn.q_gain : qkn.k_gain);
+          x1 *= rinv * to_f<T>(gain[j]);
+          x2 *= rinv * to_f<T>(gain[j + half]);
+        }
+      }
+      if (!has) continue;
       const float2 c = rope[(size_t)pos * half + j];
-      const float x1 = sc * sum_planes(ps, rbase + col0 + j), x2 = sc * sum_planes(ps, rbase + col0 + j + half);
       const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
       if (is_q) {
         q[(size_t)m * nq + slot * hd + j] = r1;
@@ -198,7 +220,8 @@ int launch_resid_gain(int dtype, float *x, PlaneSet ps, const void *gain, HiLoOu
 }
 
 int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos, const float2 *rope_table, float *q,
-                      KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
+                      KvLayout kv, int M, int rows_per_seq, int n_heads, QkNorm qkn, cudaStream_t stream) {
+  if (kv.head_dim > 128) return SJD_ERR_UNSUPPORTED;
   // a block per four head slots for a few dozen rows; fewer blocks per row (each walking more slots) as
   // the rows grow, about eight blocks per SM in all
   int per_row = (n_heads + 2 * kv.n_kv_heads + 3) / 4;
@@ -207,10 +230,10 @@ int launch_qkv_finish(int dtype, PlaneSet ps, RowScale rs, const int32_t *in_pos
   const dim3 grid(M, per_row);
   if (dtype == SJD_F32)
     SJD_CUDA(launch_kernel(qkv_finish_kernel<float>, grid, dim3(256), 0, stream, ps, rs, in_pos, rope_table, q, kv,
-                           rows_per_seq, n_heads));
+                           rows_per_seq, n_heads, qkn));
   else if (dtype == SJD_BF16)
     SJD_CUDA(launch_kernel(qkv_finish_kernel<__nv_bfloat16>, grid, dim3(256), 0, stream, ps, rs, in_pos, rope_table, q, kv,
-                           rows_per_seq, n_heads));
+                           rows_per_seq, n_heads, qkn));
   else
     return SJD_ERR_UNSUPPORTED;
   SJD_CHECK_LAUNCH();

@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
 template <typename T>
 __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t *__restrict__ in_pos,
                                    const float2 *__restrict__ rope, float *__restrict__ q, KvLayout kv, int rows_per_seq,
-                                   int n_heads) {
+                                   int n_heads, QkNorm qkn) {
   const int m = blockIdx.x;
   const int pos = in_pos[m];
   if (pos < 0) return;
@@ -144,13 +144,23 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t 
   for (int i = threadIdx.x; i < (n_heads + nkv) * half; i += blockDim.x) {
     const int head = i / half, j = i % half;
     const float2 c = cs[j];
+    float g1 = 1.0f, g2 = 1.0f;
+    if (qkn.q_gain) {   // QK-norm: this head's RMS over its hd entries (every thread of the head sums them itself)
+      const float *hv = row + (head < n_heads ? head * hd : nq + (head - n_heads) * hd);
+      float ss = 0.0f;
+      for (int t = 0; t < hd; ++t) ss += hv[t] * hv[t];
+      const float rinv = rsqrtf(ss / (float)hd + qkn.eps);
+      const T *gain = reinterpret_cast<const T *>(head < n_heads ? qkn.q_gain : qkn.k_gain);
+      g1 = rinv * to_f<T>(gain[j]);
+      g2 = rinv * to_f<T>(gain[j + half]);
+    }
     if (head < n_heads) {
-      const float x1 = row[head * hd + j], x2 = row[head * hd + j + half];
+      const float x1 = g1 * row[head * hd + j], x2 = g2 * row[head * hd + j + half];
       q[(size_t)m * nq + head * hd + j] = x1 * c.x - x2 * c.y;
       q[(size_t)m * nq + head * hd + j + half] = x2 * c.x + x1 * c.y;
     } else {
       const int kh = head - n_heads;
-      const float x1 = row[nq + kh * hd + j], x2 = row[nq + kh * hd + j + half];
+      const float x1 = g1 * row[nq + kh * hd + j], x2 = g2 * row[nq + kh * hd + j + half];
       T *dst = kbase + ((size_t)kh * kv.max_seq + pos) * hd;
       dst[j] = from_f<T>(x1 * c.x - x2 * c.y);
       dst[j + half] = from_f<T>(x2 * c.x + x1 * c.y);
@@ -205,9 +215,9 @@ int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M,
 }
 
 int launch_rope_append(int dtype, const float *qkv, const int32_t *in_pos, const float2 *rope_table, float *q,
-                       KvLayout kv, int M, int rows_per_seq, int n_heads, cudaStream_t stream) {
+                       KvLayout kv, int M, int rows_per_seq, int n_heads, QkNorm qkn, cudaStream_t stream) {
   SJD_DISPATCH(dtype, (rope_append_kernel<T><<<M, 256, 0, stream>>>(qkv, in_pos, rope_table, q, kv, rows_per_seq,
-                                                                   n_heads)));
+                                                                   n_heads, qkn)));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -87,11 +87,13 @@ def _randn(shape, std, gen, dtype):
     return (torch.randn(shape, generator=gen, dtype=torch.float32, device=gen.device) * std).to(dtype)
 
 
-def make_weights(wl: Workload, gain_jitter: float = 0.0, std: float = 0.02, device="cpu"):
+def make_weights(wl: Workload, gain_jitter: float = 0.0, std: float = 0.02, device="cpu", qk_norm: bool = False):
     """Random-init weights N(0, std^2) rounded to the workload dtype.  Matrices are
     [out_features][in_features].  Norm gains are 1 (+ optional jitter so tests exercise the
     gain path).  Generated on `device` with that device's generator: CPU tensors are what
-    parity tests feed to both sides; the benchmark generates its 7B weights on the GPU."""
+    parity tests feed to both sides; the benchmark generates its 7B weights on the GPU.
+    qk_norm: add per-layer gains q_norm / k_norm [head_dim] (1 + 0.2 N(0, 1)) for the QK-norm variant of
+    the Chameleon family; they are drawn after everything else, so the other weights do not change."""
     dt = torch_dtype(wl.dtype)
     gen = torch.Generator(device=device).manual_seed(wl.weight_seed)
     d, hd = wl.d_model, wl.head_dim
@@ -117,6 +119,11 @@ def make_weights(wl: Workload, gain_jitter: float = 0.0, std: float = 0.02, devi
         })
     w["final_norm"] = gain()
     w["lm_head"] = _randn((wl.vocab, d), std, gen, dt)
+    if qk_norm:
+        for lw in w["layers"]:
+            for name in ("q_norm", "k_norm"):
+                lw[name] = (torch.ones(hd, dtype=torch.float32, device=gen.device)
+                            + 0.2 * torch.randn(hd, generator=gen, device=gen.device)).to(dt)
     return w
 
 

@@ -29,7 +29,7 @@ def test_library_exports_every_declared_function():
 
 def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(B.sjd_model_cfg) == 14 * 4
-    assert C.sizeof(B.sjd_weights) == 12 * 8
+    assert C.sizeof(B.sjd_weights) == 14 * 8
     assert C.sizeof(B.sjd_sample_cfg) == 48
     assert B.sjd_sample_cfg.guidance.offset == 36 and B.sjd_sample_cfg.schedule.offset == 40
     assert B.sjd_sample_cfg.seed.offset == 8 and B.sjd_sample_cfg.window.offset == 16

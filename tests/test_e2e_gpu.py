@@ -18,11 +18,11 @@ LOGIT_TOL = {"f32": 1e-4, "bf16": 2e-2}
 
 
 def run_lockstep(wl, batch=1, max_steps=None, init=INIT_RANDOM, check_logits_every=1, gain_jitter=0.1, window=None,
-                 n_generate=None, seq_base=0, top_k=None, also_plain_cache=False, schedule=0):
+                 n_generate=None, seq_base=0, top_k=None, also_plain_cache=False, schedule=0, qk_norm=False):
     window = window or wl.window
     n_generate = wl.n_generate if n_generate is None else n_generate
     top_k = top_k or wl.top_k
-    weights = make_weights(wl, gain_jitter=gain_jitter)
+    weights = make_weights(wl, gain_jitter=gain_jitter, qk_norm=qk_norm)
     prompt = make_prompt(wl, batch)
     cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=wl.prompt_len + n_generate + 8, max_window=window,
                            max_ring=wl.grid_stride + window if init == INIT_RESAMPLE_ABOVE else 0)
@@ -224,6 +224,20 @@ def test_no_refinement_schedule(name, init):
     ctx, seqs, steps, out = run_lockstep(wl, n_generate=40, schedule=SCHEDULE_NO_REFINE, init=init)
     assert steps <= 40
     assert not np.any(out.host()["q_kind"] == B.SJD_Q_ROW)
+
+
+@pytest.mark.parametrize("name,n_generate", [("tiny", 60), ("small-bf16", 80), ("7b-2l", 0)])
+def test_qk_norm_variant(name, n_generate):
+    """The QK-norm variant of the decoder (per-head RMS normalisation of q and k before the rotary step, the
+    Chameleon family): generic kernels (tiny fp32), tensor-core pipeline with head_dim 64 (small bf16) and
+    with head_dim 128 (7B layer shapes, two layers, three steps)."""
+    wl = WORKLOADS[name]
+    if n_generate:
+        ctx, seqs, steps, _ = run_lockstep(wl, batch=2 if name != "tiny" else 1, n_generate=n_generate, qk_norm=True)
+    else:
+        ctx, seqs, steps, _ = run_lockstep(wl, max_steps=3, gain_jitter=0.0, qk_norm=True)
+    for s in seqs:
+        assert s.max_logit_excess <= LOGIT_TOL[wl.dtype]
 
 
 def test_small_bf16_gqa_generation():

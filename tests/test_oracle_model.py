@@ -83,8 +83,12 @@ def _torch_forward(cfg: ModelCfg, w, tokens, kv_cast=None):
 
     for lw in w["layers"]:
         h = F.rms_norm(x, (cfg.d_model,), t(lw["attn_norm"]), eps=cfg.rms_eps)
-        q = rot((h @ t(lw["wq"]).T).view(T, cfg.n_heads, hd))
-        k = rot((h @ t(lw["wk"]).T).view(T, cfg.n_kv_heads, hd))
+        q = (h @ t(lw["wq"]).T).view(T, cfg.n_heads, hd)
+        k = (h @ t(lw["wk"]).T).view(T, cfg.n_kv_heads, hd)
+        if lw.get("q_norm") is not None:
+            q = F.rms_norm(q, (hd,), t(lw["q_norm"]), eps=cfg.rms_eps)
+            k = F.rms_norm(k, (hd,), t(lw["k_norm"]), eps=cfg.rms_eps)
+        q, k = rot(q), rot(k)
         v = (h @ t(lw["wv"]).T).view(T, cfg.n_kv_heads, hd)
         if kv_cast is not None:
             k, v = k.to(kv_cast).to(torch.float64), v.to(kv_cast).to(torch.float64)
@@ -195,3 +199,30 @@ def test_torch_tensor_weights_are_accepted():
     tokens = [3, 1, 4, 1, 5]
     np.testing.assert_allclose(OracleModel(CFG, tw).forward_full(tokens),
                                OracleModel(CFG, nw).forward_full(tokens), rtol=1e-12)
+
+
+def _with_qk_norm(w, cfg, seed=5):
+    rng = np.random.default_rng(seed)
+    out = dict(w, layers=[dict(lw, q_norm=1 + 0.2 * rng.normal(size=cfg.head_dim),
+                               k_norm=1 + 0.2 * rng.normal(size=cfg.head_dim)) for lw in w["layers"]])
+    return out
+
+
+def test_qk_norm_variant_against_torch_and_its_scale_invariance():
+    """The QK-norm variant: (1) equals an independent forward built from torch's rms_norm applied per head
+    before the rotary step; (2) differs from the plain model; (3) its logits do not change when W_q or W_k
+    is scaled by a positive constant (each head is normalised; eps is made negligible for this check);
+    (4) with a cache it still equals the full causal forward."""
+    cfg = ModelCfg(n_layers=2, d_model=48, n_heads=6, n_kv_heads=2, head_dim=8, ffn_hidden=77, vocab=53, rms_eps=1e-12)
+    w = _with_qk_norm(_weights(cfg, seed=3), cfg)
+    tokens = [3, 17, 5, 44, 9, 9, 30]
+    model = OracleModel(cfg, w)
+    got = model.forward_full(tokens)
+    np.testing.assert_allclose(got, _torch_forward(cfg, w, tokens), rtol=1e-9, atol=1e-11)
+    plain = OracleModel(cfg, _weights(cfg, seed=3)).forward_full(tokens)
+    assert np.abs(got - plain).max() > 1e-2
+    scaled = dict(w, layers=[dict(lw, wq=3.0 * lw["wq"], wk=0.25 * lw["wk"]) for lw in w["layers"]])
+    np.testing.assert_allclose(OracleModel(cfg, scaled).forward_full(tokens), got, rtol=1e-7, atol=1e-9)
+    cache = model.new_cache(16)
+    model.forward_window(cache, tokens[:4], 0, want_logits=False)
+    np.testing.assert_allclose(model.forward_window(cache, tokens[4:], 4), got[4:], rtol=1e-10, atol=1e-12)
