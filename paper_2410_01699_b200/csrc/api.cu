@@ -110,7 +110,7 @@ constexpr int kGemmSmsMax = 160;
 extern "C" size_t sjd_gemm_workspace_bytes(int M, int N, int K) {
   if (!gemm_tc_supported(M, N, K)) return 0;
   const int mp = (M + 15) / 16 * 16;
-  const int splits = gemm_tc_splits(gemm_tc_plan(M, (N / 128) % 2 == 0), N / 128, K / 64, kGemmSmsMax);
+  const int splits = gemm_tc_splits(gemm_tc_plan(M), N / 128, K / 64, kGemmSmsMax);
   return 256 + up256((size_t)splits * M * N * 4) + up256((size_t)2 * mp * K * 2);
 }
 
@@ -128,7 +128,7 @@ extern "C" int sjd_gemm(int M, int N, int K, const float *x, const void *w, floa
   sms = sms < kGemmSmsMax ? sms : kGemmSmsMax;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   const int mp = (M + 15) / 16 * 16;
-  const GemmTcPlan plan = gemm_tc_plan(M, (N / 128) % 2 == 0);
+  const GemmTcPlan plan = gemm_tc_plan(M);
   const int splits = gemm_tc_splits(plan, N / 128, K / 64, sms);
   const int splits_max = gemm_tc_splits(plan, N / 128, K / 64, kGemmSmsMax);
   char *p = (char *)ws;

@@ -243,12 +243,12 @@ struct alignas(64) TensorMap {   // an encoded TMA descriptor (same size and ali
 // bf16 row-major [rows][cols] matrix cut into boxes of box_rows x 64 columns, 128-byte swizzle
 int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols, int box_rows);
 bool gemm_tc_supported(int M, int N, int K);
-// Shape of a launch of M rows: activation planes multiplied (2: hi and lo, 1: hi only), token slabs,
-// rows per slab (a multiple of 16: the box height of the activation tensor map), weight tiles per CTA.
+// Shape of a launch of M rows: token slabs and rows per slab (a multiple of 16: the box height of the
+// activation tensor map).
 struct GemmTcPlan {
-  int x_planes, n_slabs, slab_rows, w_tiles;
+  int n_slabs, slab_rows;
 };
-GemmTcPlan gemm_tc_plan(int M, bool tiles_even);
+GemmTcPlan gemm_tc_plan(int M);
 int gemm_tc_splits(const GemmTcPlan &pl, int tiles, int k_blocks, int n_sms);   // tiles: 128-row weight tiles of the launch
 // One launch over up to three weight matrices that share the activation operand X (two bf16 planes:
 // hi at row 0, lo at row x_lo_row of x_map, each [rows][K]).  Matrix j has n_out[j] rows and writes

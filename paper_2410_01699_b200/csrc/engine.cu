@@ -103,15 +103,13 @@ Layout make_layout(const sjd_model_cfg &c) {
   {
     // fp32 partial planes of one GEMM launch: the largest splits * rows * columns over the launches
     const int tiles[4] = {(int)((nq + 2 * nk) / 128), c.d_model / 128, 2 * c.ffn_hidden / 128, c.d_model / 128};
-    const bool even[4] = {(nq / 128) % 2 == 0 && (nk / 128) % 2 == 0, (c.d_model / 128) % 2 == 0,
-                          (c.ffn_hidden / 128) % 2 == 0, (c.d_model / 128) % 2 == 0};
     const int kbs[4] = {c.d_model / 64, (int)(nq / 64), c.d_model / 64, c.ffn_hidden / 64};
     const size_t cols[4] = {nq + 2 * nk, (size_t)c.d_model, (size_t)2 * c.ffn_hidden, (size_t)c.d_model};
     size_t need = 0;
     for (int i = 0; i < 4; ++i) {
       for (size_t rows = 16; rows < Mx + 16 && rows <= 1024; rows += 16) {   // splits shrink as the token slabs grow
         const size_t m = rows < Mx ? rows : Mx;
-        const size_t n = (size_t)gemm_tc_splits(gemm_tc_plan((int)m, even[i]), tiles[i] > 0 ? tiles[i] : 1, kbs[i],
+        const size_t n = (size_t)gemm_tc_splits(gemm_tc_plan((int)m), tiles[i] > 0 ? tiles[i] : 1, kbs[i],
                                                  kMaxGemmCtas) * m * cols[i];
         need = n > need ? n : need;
       }
@@ -399,9 +397,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
       call.act_lo_off = act->lo_offset;
     }
     int tiles = 0, col = 0;
-    bool tiles_even = true;
     for (int j = 0; j < n_mats; ++j) {
-      tiles_even = tiles_even && (n_out[j] / 128) % 2 == 0;
       call.w_map[j] = &wm[j]->map;
       call.n_out[j] = n_out[j];
       call.col_off[j] = col;
@@ -415,7 +411,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     call.x_lo_row = Ma;
     call.M = M;
     call.K = k_in;
-    call.splits = (bf16_out || act) ? 1 : gemm_tc_splits(gemm_tc_plan(M, tiles_even), tiles, k_in / 64, c->n_ctas);
+    call.splits = (bf16_out || act) ? 1 : gemm_tc_splits(gemm_tc_plan(M), tiles, k_in / 64, c->n_ctas);
     call.out = out;
     call.plane_stride = (size_t)M * ldc;
     call.ldc = ldc;
@@ -727,7 +723,7 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
       const int Mp = (row_counts[i] + 15) / 16 * 16;
       if (row_counts[i] > 1024 || c->xmaps.count(Mp)) continue;
       XMaps xm;
-      const int box = gemm_tc_plan(row_counts[i], false).slab_rows;
+      const int box = gemm_tc_plan(row_counts[i]).slab_rows;
       const bool ok = make_tensor_map_bf16(&xm.h, c->ws + c->lay.xs_h, 2L * Ma, c->cfg.d_model, box) == SJD_OK &&
                       make_tensor_map_bf16(&xm.attn, c->ws + c->lay.xs_attn, 2L * Ma, nq, box) == SJD_OK &&
                       make_tensor_map_bf16(&xm.act, c->ws + c->lay.xs_act, 2L * Ma, c->cfg.ffn_hidden, box) == SJD_OK;

@@ -6,16 +6,17 @@
 // job is to keep every SM's TMA queue full.  Larger M (batches of images with wide windows, up to
 // 1024 rows) is cut into token slabs of at most 128 rows; the CTAs of the slabs of one weight tile
 // are neighbours in the grid, so the tile comes from HBM once and from L2 for the other slabs.  With
-// several slabs the kernel is bound by the tensor pipe (both activation planes are multiplied).
-// Optionally (SJD_GEMM_WIDE_W_TILES = 2) a CTA of a multi-slab launch takes two adjacent weight tiles
-// against one activation tile (two accumulators, all 512 TMEM columns, one CTA per SM: 64 instead of
-// 96 operand bytes per MMA clock); measured 10-15 % slower than two independent CTAs per SM.
+// several slabs the kernel is bound by the tensor pipe (both activation planes are multiplied) and, in
+// this tiling, by shared-memory bandwidth: a 128 x 256 MMA tile moves 96 KB through shared memory per 512
+// tensor clocks.  (Measured and removed: two adjacent weight tiles per CTA against one activation tile,
+// 10-15 % slower than two independent CTAs per SM.)
 //   * W is the 128-row operand of tcgen05.mma (M = 128), the tokens are the N dimension.  The fp32
 //     activations arrive split into two bf16 planes, hi = bf16(x) and lo = bf16(x - hi); both planes
 //     are columns of the same MMA (N = 2 * Mp), and the epilogue adds the two halves: activations keep
 //     ~16 bits of mantissa at no cost in weight bytes.  (Multiplying the hi plane alone, i.e. plain
-//     bf16 activations, halves the tensor work of the many-row case but misses the 2e-2 logits
-//     tolerance at d_model 4096 already after two layers; it stays a compile-time option.)
+//     bf16 activations, would halve the tensor work of the many-row case but misses the 2e-2 logits
+//     tolerance at d_model 4096 already after two layers: 4.0e-2.  So both planes, always, and the
+//     useful tensor throughput of the many-row case cannot pass half the peak.)
 //   * One CTA per (128-row weight tile, K split); two CTAs are resident per SM.  A launch covers up to
 //     three weight matrices that share the activation operand (Q|K|V, gate|up), so their tiles form
 //     one grid.  With more than one K split every CTA writes an fp32 partial plane; the consumer
@@ -58,12 +59,6 @@ constexpr int kMaxStages = 8;
 #ifndef SJD_GEMM_CTAS_PER_SM
 #define SJD_GEMM_CTAS_PER_SM 2
 #endif
-#ifndef SJD_GEMM_WIDE_W_TILES
-#define SJD_GEMM_WIDE_W_TILES 1             // weight tiles per CTA in launches with several token slabs (1 or 2)
-#endif
-#ifndef SJD_GEMM_SPLIT_MAX_M
-#define SJD_GEMM_SPLIT_MAX_M 1024           // most rows for which both the hi and the lo plane are multiplied
-#endif
 constexpr int kSmemBudget = SJD_GEMM_SMEM_BUDGET;
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
@@ -72,10 +67,8 @@ struct GemmParams {
   size_t plane_stride;    // elements between planes
   int ldc;
   int M;                  // valid token rows
-  int Mp;                 // token rows of one slab, a multiple of 16 (MMA N = x_planes * Mp)
-  int n_slabs;            // token slabs; CTA blockIdx.x = (weight tile / w_tiles) * n_slabs + slab
-  int w_tiles;            // adjacent weight tiles per CTA (1 or 2), each with its own accumulator (= template WT)
-  int x_planes;           // 2: hi and lo planes of the activations, 1: hi only
+  int Mp;                 // token rows of one slab, a multiple of 16 (MMA N = 2 * Mp: hi and lo plane)
+  int n_slabs;            // token slabs; CTA blockIdx.x = weight tile * n_slabs + slab
   int x_lo_row;           // row of the lo plane inside the activation tensor map
   int k_blocks, splits;   // K / 64, K splits (gridDim.y)
   int tile_end[3];        // matrix j owns tiles [tile_end[j-1], tile_end[j])
@@ -205,9 +198,8 @@ __device__ __forceinline__ bool epilogue_all(bool pred) {
 }
 
 // ---------------------------------------------------------------------------------- kernel
-// WT: weight tiles per CTA, XP: activation planes multiplied (compile-time so that the common
-// shape, one tile and both planes, keeps fully unrolled issue loops)
-template <int WT, int XP, bool GU>
+// GU: the gate|up launch that applies SwiGLU in its epilogue
+template <bool GU>
 __global__ void __launch_bounds__(kThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant__ CUtensorMap w_map1,
                const __grid_constant__ CUtensorMap w_map2, const __grid_constant__ CUtensorMap x_map, const GemmParams p) {
@@ -216,6 +208,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap w_map0, const __grid_constant
   __shared__ uint32_t s_tmem_base;
   __shared__ float s_scale[TILE_N];   // per-row output scales of this CTA's token slab (epilogue)
 
+  constexpr int WT = 1;   // weight tiles (accumulators) per CTA
+  constexpr int XP = 2;   // activation planes multiplied: hi and lo
   pdl_trigger();   // the next kernel in the stream may be scheduled as soon as every CTA got here
   SJD_TL(TL_GEMM, 0, threadIdx.x == 0);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -493,26 +487,21 @@ int make_tensor_map_bf16(TensorMap *out, const void *base, long rows, long cols,
 
 bool gemm_tc_supported(int M, int N, int K) { return M >= 1 && M <= 1024 && N % TILE_N == 0 && K % TILE_K == 0; }
 
-// How M token rows are laid over the MMA N dimension (at most 256 columns per accumulator): slabs of
-// at most 128 rows with both activation planes (256 rows where only the hi plane is multiplied).
-// `tiles_even`: every weight matrix of the launch has an even number of 128-row tiles.
-GemmTcPlan gemm_tc_plan(int M, bool tiles_even) {
+// How M token rows are laid over the MMA N dimension (at most 256 columns per accumulator, two per token
+// row: hi and lo plane): slabs of at most 128 rows.
+GemmTcPlan gemm_tc_plan(int M) {
   GemmTcPlan pl;
-  pl.x_planes = M <= SJD_GEMM_SPLIT_MAX_M ? 2 : 1;
-  const int cap = 256 / pl.x_planes;
-  pl.n_slabs = (M + cap - 1) / cap;
+  pl.n_slabs = (M + 127) / 128;
   const int per = (M + pl.n_slabs - 1) / pl.n_slabs;
   pl.slab_rows = (per + 15) / 16 * 16;
-  pl.w_tiles = (SJD_GEMM_WIDE_W_TILES == 2 && pl.n_slabs >= 2 && tiles_even) ? 2 : 1;
   return pl;
 }
 
-// K splits for a launch of `tiles` weight tiles: a single wave of the resident CTAs (two per SM, one
-// when a CTA holds two accumulators), at least 16 k-blocks (256 KB of weights) per CTA so that
+// K splits for a launch of `tiles` weight tiles: a single wave of the resident CTAs (two per SM), at least 16 k-blocks (256 KB of weights) per CTA so that
 // set-up and drain stay small next to the streaming
 int gemm_tc_splits(const GemmTcPlan &pl, int tiles, int k_blocks, int n_sms) {
-  const int ctas = tiles / pl.w_tiles * pl.n_slabs;
-  int s = ((pl.w_tiles == 2 ? 1 : SJD_GEMM_CTAS_PER_SM) * n_sms) / (ctas > 0 ? ctas : 1);
+  const int ctas = tiles * pl.n_slabs;
+  int s = (SJD_GEMM_CTAS_PER_SM * n_sms) / (ctas > 0 ? ctas : 1);
   const int cap = k_blocks / SJD_GEMM_MIN_KB > 1 ? k_blocks / SJD_GEMM_MIN_KB : 1;
   s = s > cap ? cap : s;
   s = s > 16 ? 16 : s;
@@ -528,14 +517,11 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   if (R > TILE_N || (gu && (R > TILE_N / 2 || g.n_mats != 2 || g.n_out[0] != g.n_out[1] || g.splits != 1)))
     return SJD_ERR_BAD_ARG;
   int tiles = 0;
-  bool tiles_even = true;
   for (int j = 0; j < 3; ++j) {
     if (j < g.n_mats && !(gu && j == 1)) {
       if (g.M < 1 || g.M > 1024 || g.K % TILE_K != 0 || g.n_out[j] < 1) return SJD_ERR_UNSUPPORTED;
       if (R == TILE_N && g.n_out[j] % TILE_N != 0) return SJD_ERR_UNSUPPORTED;
-      const int t = (g.n_out[j] + R - 1) / R;
-      tiles += t;
-      tiles_even = tiles_even && t % 2 == 0;
+      tiles += (g.n_out[j] + R - 1) / R;
     }
     p.tile_end[j] = tiles;
     p.col_off[j] = j < g.n_mats ? g.col_off[j] : 0;
@@ -545,14 +531,10 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.out = g.out;
   p.plane_stride = g.plane_stride;
   p.ldc = g.ldc;
-  GemmTcPlan pl = gemm_tc_plan(g.M, tiles_even);
-  if (gu || R != TILE_N) pl.w_tiles = 1;
-  if (gu && pl.x_planes != 2) return SJD_ERR_UNSUPPORTED;
+  const GemmTcPlan pl = gemm_tc_plan(g.M);
   p.M = g.M;
   p.Mp = pl.slab_rows;
   p.n_slabs = pl.n_slabs;
-  p.w_tiles = pl.w_tiles;
-  p.x_planes = pl.x_planes;
   p.x_lo_row = g.x_lo_row;
   p.k_blocks = g.K / TILE_K;
   p.splits = g.splits;
@@ -566,11 +548,11 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   p.act_hi = g.act_hi;
   p.act_lo_off = g.act_lo_off;
   p.F = gu ? g.n_out[0] : 0;
-  const int stage_bytes = p.w_tiles * W_TILE_BYTES + p.x_planes * p.Mp * TILE_K * 2;
-  const int ctas = tiles / p.w_tiles * p.n_slabs;
+  const int stage_bytes = W_TILE_BYTES + 2 * p.Mp * TILE_K * 2;
+  const int ctas = tiles * p.n_slabs;
   // one CTA per SM or fewer: give each the deeper ring
   const int budget =
-      (p.w_tiles == 2 || (SJD_GEMM_DEEP_RING && g.n_sms > 0 && ctas * g.splits <= g.n_sms)) ? 2 * kSmemBudget : kSmemBudget;
+      (SJD_GEMM_DEEP_RING && g.n_sms > 0 && ctas * g.splits <= g.n_sms) ? 2 * kSmemBudget : kSmemBudget;
   int stages = budget / stage_bytes;
   stages = stages > kMaxStages ? kMaxStages : stages;
   if (stages < 2) return SJD_ERR_UNSUPPORTED;
@@ -587,24 +569,15 @@ int launch_gemm_tc(const GemmTcCall &g, cudaStream_t stream) {
   if (dev < 0 || dev >= 64) return SJD_ERR_UNSUPPORTED;
   if (!configured[dev]) {
     const int max_dyn = 2 * kSmemBudget + 2048;
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<2, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
-    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<1, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
+    SJD_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dyn));
     configured[dev] = true;
   }
   const dim3 grid(ctas, g.splits);
   if (gu)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 2, true>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
-  else if (p.w_tiles == 1 && p.x_planes == 2)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 2, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
-  else if (p.w_tiles == 2 && p.x_planes == 2)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 2, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
-  else if (p.w_tiles == 1)
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<1, 1, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<true>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   else
-    SJD_CUDA(launch_kernel(gemm_tc_kernel<2, 1, false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
+    SJD_CUDA(launch_kernel(gemm_tc_kernel<false>, grid, dim3(kThreads), smem, stream, w0, w1, w2, xm, p));
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -55,3 +55,32 @@ def test_two_ranks_reproduce_the_single_rank_result():
         assert p.exitcode == 0
     assert everything == [[1000 * s + t for t in range(3)] for s in range(5)]
     assert slowest == 11.0
+
+
+def test_bench_starts_one_rank_per_gpu_when_no_launcher_did(monkeypatch):
+    """`python bench.py --gpus N` without torchrun: bench starts the N ranks itself; every rank gets its
+    RANK / LOCAL_RANK / WORLD_SIZE and a rendezvous on 127.0.0.1 (checked with the process spawner and the
+    per-rank body replaced by recorders: no GPU involved)."""
+    import argparse
+    import importlib.util
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_under_test", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    seen = []
+
+    def fake_run(args, wl):
+        seen.append({k: os.environ[k] for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")})
+
+    def fake_spawn(fn, args=(), nprocs=1, join=True):
+        for i in range(nprocs):
+            fn(i, *args)
+
+    monkeypatch.setattr(bench, "run_library", fake_run)
+    monkeypatch.setattr(mp, "spawn", fake_spawn)
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT"):
+        monkeypatch.setenv(k, "unset")   # restored by monkeypatch afterwards
+    bench.launch_ranks(argparse.Namespace(gpus=3), None)
+    assert [s["RANK"] for s in seen] == ["0", "1", "2"] and [s["LOCAL_RANK"] for s in seen] == ["0", "1", "2"]
+    assert all(s["WORLD_SIZE"] == "3" and s["MASTER_ADDR"] == "127.0.0.1" for s in seen)
+    assert len({s["MASTER_PORT"] for s in seen}) == 1 and int(seen[0]["MASTER_PORT"]) > 0
