@@ -11,7 +11,7 @@ attention BATCH PREFIX [--window W --heads H --kv-heads KVH --head-dim D]: the w
 verify  the isolated verify-and-resample kernel (sjd_verify) on the synthetic verification workload;
         reports 2*B*W*V*2 bytes / time (current and previous logits read once each).
 
-The same commands are the ones the ncu captures under profiles/ were taken with.
+Each call is small enough (a few launches of one kernel, buffers of a few hundred MB) to be captured under ncu.
 """
 from __future__ import annotations
 
