@@ -35,10 +35,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # DRAM traffic of the dominant kernel (gemm_tc_kernel) from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum) of the four projection launches of one decoder layer inside a step: 409.58 MB read +
+# dram__bytes_write.sum) of the four projection launches of one decoder layer inside a step: 409.76 MB read +
 # written for 404.75 MB of weights.  Traffic grows in proportion to the weight bytes of a launch, so a step's
 # launches scale by that ratio.  Valid only for the kernel source the counters were taken with.
-GEMM_TRAFFIC = {"source_sha256_16": "a01bee506214a0f9", "dram_bytes_per_weight_byte": 409.58 / 404.75}
+GEMM_TRAFFIC = {"source_sha256_16": "7a7d0504b4d33207", "dram_bytes_per_weight_byte": 409.76 / 404.75}
 
 
 def gemm_traffic_per_launch(algorithmic_bytes_per_launch):
