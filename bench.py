@@ -501,6 +501,7 @@ def main():
     ap.add_argument("--table", action="store_true",
                     help="whole-image generation under the baseline schedules and SJD (rows A-D and no-refinement)")
     ap.add_argument("--n-generate", type=int, default=0, help="image tokens per image for --table (default: the workload's)")
+    ap.add_argument("--temperature", type=float, default=0.0, help="override the sampling temperature (default: the workload's, 1.0)")
     ap.add_argument("--guidance", type=float, default=0.0,
                     help="classifier-free guidance weight (the paper runs 3.0): two streams per image, 2 x batch x W rows")
     args = ap.parse_args()
@@ -510,6 +511,8 @@ def main():
         wl = wl.with_(prompt_len=args.prompt_len)
     if args.window:
         wl = wl.with_(window=args.window)
+    if args.temperature > 0:
+        wl = wl.with_(temperature=args.temperature)
     if args.impl == "reference":
         run_reference(args, wl)
     elif args.table:
