@@ -22,8 +22,8 @@
  *     stream).  Work is enqueued asynchronously; no call synchronises the
  *     device except sjd_init (table upload) and sjd_last_device_status.
  *   - Matrices are row-major [out_features][in_features] (y = x W^T).
- *   - All sequences of a batch share prompt length, n_generate and the
- *     sampling configuration; the Philox counter carries the sequence id.
+ *   - All sequences of a batch share n_generate and the sampling configuration (prompt lengths may
+ *     differ: sjd_prefill_ragged); the Philox counter carries the sequence id.
  *
  * Random numbers: Philox4x32-10 (Salmon et al., SC'11), key = 64-bit seed,
  * counter = (absolute position, step index, sequence id, stream tag).
@@ -195,6 +195,18 @@ int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weights *weights
  */
 int sjd_prefill(sjd_ctx *ctx, int batch, const int32_t *prompt, int prompt_len,
                 const sjd_sample_cfg *sample, void *cuda_stream);
+
+/*
+ * sjd_prefill for a ragged batch: sequence b uses the first prompt_lens[b] tokens of row b of `prompt`
+ * (device int32 [batch][row_stride]); prompt_lens is a HOST array of `batch` lengths in 1..row_stride.
+ * Every sequence keeps its own positions (its image starts right after its own prompt: nothing is padded),
+ * generates n_generate tokens and finishes on its own; under guidance the two streams of an image must have
+ * prompts of one length.  (Sec. 4.1, first sentence: "after pre-filling the tokens of text prompts";
+ * prompts of different lengths in one batch are this library's generalisation.)
+ * Errors: as sjd_prefill; CAPACITY is judged by the longest prompt.
+ */
+int sjd_prefill_ragged(sjd_ctx *ctx, int batch, const int32_t *prompt, const int32_t *prompt_lens, int row_stride,
+                       const sjd_sample_cfg *sample, void *cuda_stream);
 
 /*
  * One SJD iteration for every sequence of the batch (Sec. 4.1 Steps 1-4):

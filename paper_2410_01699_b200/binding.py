@@ -29,7 +29,8 @@ TORCH_DTYPES = {SJD_F32: torch.float32, SJD_BF16: torch.bfloat16}
 EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_get_window", "sjd_peek_logits",
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
            "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static",
-           "sjd_gemm_workspace_bytes", "sjd_gemm", "sjd_attention_workspace_bytes", "sjd_attention", "sjd_get_info"]
+           "sjd_gemm_workspace_bytes", "sjd_gemm", "sjd_attention_workspace_bytes", "sjd_attention", "sjd_get_info",
+           "sjd_prefill_ragged"]
 
 
 class SJDError(RuntimeError):
@@ -95,6 +96,9 @@ def lib():
                            C.c_size_t]
     L.sjd_prefill.restype = C.c_int
     L.sjd_prefill.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.POINTER(sjd_sample_cfg), C.c_void_p]
+    L.sjd_prefill_ragged.restype = C.c_int
+    L.sjd_prefill_ragged.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(C.c_int32), C.c_int,
+                                     C.POINTER(sjd_sample_cfg), C.c_void_p]
     L.sjd_step.restype = C.c_int
     L.sjd_step.argtypes = [C.c_void_p, C.POINTER(sjd_step_out), C.c_void_p]
     L.sjd_get_window.restype = C.c_int
@@ -287,6 +291,16 @@ class Context:
         self.batch, self.window = int(prompt.shape[0]), int(sample.window)
         _check(lib().sjd_prefill(self._ctx, self.batch, _ptr(prompt), int(prompt.shape[1]), C.byref(sample),
                                  _stream()), "sjd_prefill")
+
+    def prefill_ragged(self, prompt, prompt_lens, sample: sjd_sample_cfg):
+        """prompt: int32 cuda tensor [B][row_stride]; prompt_lens: B host integers (sequence b uses the first
+        prompt_lens[b] tokens of its row)."""
+        assert prompt.dtype == torch.int32 and prompt.is_cuda and prompt.is_contiguous()
+        self._prompt = prompt
+        self.batch, self.window = int(prompt.shape[0]), int(sample.window)
+        lens = (C.c_int32 * self.batch)(*[int(x) for x in prompt_lens])
+        _check(lib().sjd_prefill_ragged(self._ctx, self.batch, _ptr(prompt), lens, int(prompt.shape[1]), C.byref(sample),
+                                        _stream()), "sjd_prefill_ragged")
 
     def step(self, out: StepOut | None = None):
         _check(lib().sjd_step(self._ctx, C.byref(out.c) if out is not None else None, _stream()), "sjd_step")

@@ -176,7 +176,7 @@ struct SeqState {
   int32_t *in_tok;      // [B][W] model inputs of the next step
   int32_t *in_pos;      // [B][W] their absolute positions, -1 = inactive row
   int32_t max_seq;
-  int32_t prompt_len;
+  const int32_t *prompt_lens;   // [B] prompt length of every sequence (ragged batches)
   int32_t n_generate;
   int32_t init;
   int32_t grid_stride;

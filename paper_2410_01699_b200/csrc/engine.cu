@@ -48,6 +48,7 @@ struct Layout {
   size_t xs_h, xs_attn, xs_act, gemm_planes, ss_part;
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t ring, ring_stats, n_prev, w_prev;   // Sec. 4.2 (d): retained logits rows (max_ring > 0)
+  size_t prompt_lens;                        // [max_batch] prompt length of every sequence
   size_t total;
 };
 
@@ -132,6 +133,7 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.ring_stats = take(ring_rows * sizeof(RowStats));
   L.n_prev = take((size_t)c.max_batch * 4);
   L.w_prev = take((size_t)c.max_batch * 4);
+  L.prompt_lens = take((size_t)c.max_batch * 4);
   L.total = off;
   return L;
 }
@@ -183,10 +185,12 @@ struct Tracer {
   }
 };
 
-__global__ void prefill_setup_kernel(const int32_t *prompt, int P, SeqState st, uint32_t *step, int32_t *counters,
+// prompt: [B][ld] token ids, sequence b uses the first st.prompt_lens[b] of its row
+__global__ void prefill_setup_kernel(const int32_t *prompt, int ld, SeqState st, uint32_t *step, int32_t *counters,
                                      int B) {
   const int b = blockIdx.x;
-  for (int i = threadIdx.x; i < P; i += blockDim.x) st.committed[(size_t)b * st.max_seq + i] = prompt[(size_t)b * P + i];
+  const int P = st.prompt_lens[b];
+  for (int i = threadIdx.x; i < P; i += blockDim.x) st.committed[(size_t)b * st.max_seq + i] = prompt[(size_t)b * ld + i];
   if (threadIdx.x == 0) {
     st.n[b] = P;
     st.w_eff[b] = 0;
@@ -198,12 +202,14 @@ __global__ void prefill_setup_kernel(const int32_t *prompt, int P, SeqState st, 
   }
 }
 
-__global__ void prefill_inputs_kernel(const int32_t *prompt, int P, int c0, int rows, int32_t *in_tok, int32_t *in_pos) {
+__global__ void prefill_inputs_kernel(const int32_t *prompt, int ld, const int32_t *prompt_lens, int c0, int rows,
+                                      int32_t *in_tok, int32_t *in_pos) {
   const int b = blockIdx.x;
+  const int P = prompt_lens[b];
   for (int k = threadIdx.x; k < rows; k += blockDim.x) {
     const int pos = c0 + k;
     const bool act = pos < P - 1;
-    in_tok[b * rows + k] = act ? prompt[(size_t)b * P + pos] : 0;
+    in_tok[b * rows + k] = act ? prompt[(size_t)b * ld + pos] : 0;
     in_pos[b * rows + k] = act ? pos : -1;
   }
 }
@@ -234,7 +240,8 @@ struct sjd_ctx {
   std::vector<const void *> q_norm, k_norm;   // QK-norm gains per layer (null entries: the plain model)
   QkNorm qk_norm(int l) const { return QkNorm{q_norm[l], k_norm[l], cfg.rms_eps}; }
   sjd_sample_cfg sample;
-  int batch, prompt_len, window;
+  int batch, prompt_len, window;   // prompt_len: the longest prompt of the batch
+  std::vector<int32_t> prompt_lens;  // per sequence (host copy; the device copy is in the workspace)
   bool prefilled;
   uint32_t host_step;  // number of sjd_step calls since prefill == device step index
   cudaStream_t last_stream;
@@ -286,7 +293,7 @@ struct sjd_ctx {
     st.in_tok = at<int32_t>(lay.in_tok);
     st.in_pos = at<int32_t>(lay.in_pos);
     st.max_seq = cfg.max_seq;
-    st.prompt_len = prompt_len;
+    st.prompt_lens = at<int32_t>(lay.prompt_lens);
     st.n_generate = sample.n_generate;
     st.init = sample.init;
     st.grid_stride = sample.grid_stride;
@@ -696,19 +703,38 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
 
 extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int prompt_len, const sjd_sample_cfg *sample,
                            void *cuda_stream) {
-  if (!c || !prompt || !sample || batch < 1 || prompt_len < 1) return SJD_ERR_BAD_ARG;
+  if (batch < 1 || batch > (1 << 20)) return SJD_ERR_BAD_ARG;
+  const std::vector<int32_t> lens((size_t)batch, prompt_len);
+  return sjd_prefill_ragged(c, batch, prompt, lens.data(), prompt_len, sample, cuda_stream);
+}
+
+extern "C" int sjd_prefill_ragged(sjd_ctx *c, int batch, const int32_t *prompt, const int32_t *prompt_lens, int row_stride,
+                                  const sjd_sample_cfg *sample, void *cuda_stream) {
+  if (!c || !prompt || !prompt_lens || !sample || batch < 1 || row_stride < 1) return SJD_ERR_BAD_ARG;
+  int prompt_len = 0;   // the longest
+  for (int b = 0; b < batch; ++b) {
+    if (prompt_lens[b] < 1 || prompt_lens[b] > row_stride) return SJD_ERR_BAD_ARG;
+    prompt_len = prompt_lens[b] > prompt_len ? prompt_lens[b] : prompt_len;
+  }
   int rc = check_sample_cfg(sample, c->cfg.vocab);
   if (rc != SJD_OK) return rc;
   if (sample->n_generate < 0) return SJD_ERR_BAD_ARG;
   if (batch > c->cfg.max_batch || sample->window > c->cfg.max_window) return SJD_ERR_CAPACITY;
   if ((long)prompt_len + sample->n_generate > c->cfg.max_seq) return SJD_ERR_CAPACITY;
-  if (sample->guidance != 0.0f && batch % 2 != 0) return SJD_ERR_BAD_ARG;   // streams come in pairs
+  if (sample->guidance != 0.0f) {   // streams come in pairs that share every position
+    if (batch % 2 != 0) return SJD_ERR_BAD_ARG;
+    for (int b = 0; b < batch; b += 2)
+      if (prompt_lens[b] != prompt_lens[b + 1]) return SJD_ERR_BAD_ARG;
+  }
   if (sample->init == SJD_INIT_RESAMPLE_ABOVE && c->cfg.max_ring < sample->grid_stride + sample->window)
     return SJD_ERR_CAPACITY;   // a retained row must outlive the window that draws from it
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   c->sample = *sample;
   c->batch = batch;
   c->prompt_len = prompt_len;
+  c->prompt_lens.assign(prompt_lens, prompt_lens + batch);
+  SJD_CUDA(cudaMemcpyAsync(c->ws + c->lay.prompt_lens, c->prompt_lens.data(), (size_t)batch * sizeof(int32_t),
+                           cudaMemcpyHostToDevice, stream));
   c->window = sample->window;
   c->host_step = 0;
   c->last_stream = stream;
@@ -731,13 +757,13 @@ extern "C" int sjd_prefill(sjd_ctx *c, int batch, const int32_t *prompt, int pro
     }
   }
   const SeqState st = c->state();
-  prefill_setup_kernel<<<batch, 128, 0, stream>>>(prompt, prompt_len, st, c->at<uint32_t>(c->lay.step),
+  prefill_setup_kernel<<<batch, 128, 0, stream>>>(prompt, row_stride, st, c->at<uint32_t>(c->lay.step),
                                                   c->at<int32_t>(c->lay.counters), batch);
   SJD_CHECK_LAUNCH();
   // cache keys/values of c[0..P-1) in chunks of max_window rows per sequence
   const int rows = c->cfg.max_window;
   for (int c0 = 0; c0 < prompt_len - 1; c0 += rows) {
-    prefill_inputs_kernel<<<batch, 64, 0, stream>>>(prompt, prompt_len, c0, rows, st.in_tok, st.in_pos);
+    prefill_inputs_kernel<<<batch, 64, 0, stream>>>(prompt, row_stride, st.prompt_lens, c0, rows, st.in_tok, st.in_pos);
     SJD_CHECK_LAUNCH();
     rc = forward(c, rows, nullptr, stream);
     if (rc != SJD_OK) return rc;

@@ -1190,7 +1190,8 @@ __device__ void draw_fresh_slots(const VerifyParams &p, int b, uint32_t step, in
   __syncthreads();
   const int m = (a < w_eff) ? a + 1 : w_eff;
   const int base = p.st.n[sb], n2 = base + m;
-  const int w2 = max(0, min(W, p.st.prompt_len + p.st.n_generate - n2));
+  const int prompt_len = p.st.prompt_lens[sb];
+  const int w2 = max(0, min(W, prompt_len + p.st.n_generate - n2));
   int kept = (a < w_eff) ? min(w_eff - a - 1, w2) : 0;
   if (p.schedule == SJD_SCHEDULE_NO_REFINE) kept = 0;
   const float inv_t = 1.0f / p.temperature;
@@ -1204,7 +1205,7 @@ __device__ void draw_fresh_slots(const VerifyParams &p, int b, uint32_t step, in
     } else {   // (d): the position one grid row above; its most recent row is in this pass's buffer if it was
                // inside the window just verified, else in the ring (every image position passes through a window)
       const int src = t_pos - p.st.grid_stride;
-      if (src >= p.st.prompt_len) {
+      if (src >= prompt_len) {
         if (src >= base) k = src - base < w_eff ? src - base : -1;
         else if (p.ring) k = -2 - src % p.ring_len;
       }
@@ -1292,7 +1293,7 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
 
   int w2 = 0, kept = 0;
   if (p.e2e) {
-    const int total = p.st.prompt_len + p.st.n_generate;
+    const int total = p.st.prompt_lens[sb] + p.st.n_generate;
     w2 = max(0, min(W, total - n2));
     kept = (a < w_eff) ? min(w_eff - a - 1, w2) : 0;
     if (p.schedule == SJD_SCHEDULE_NO_REFINE) kept = 0;   // every slot of the new window is initialised afresh
@@ -1326,7 +1327,7 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
       const int stride = p.st.init == SJD_INIT_COPY_ABOVE ? p.st.grid_stride
                          : p.st.init == SJD_INIT_COPY_LEFT ? 1 : 0;
       const int src = t_pos - stride;
-      if (p.st.init != SJD_INIT_RANDOM && stride > 0 && src >= p.st.prompt_len) {
+      if (p.st.init != SJD_INIT_RANDOM && stride > 0 && src >= p.st.prompt_lens[sb]) {
         tok = src < n2 ? p.st.committed[(size_t)sb * p.st.max_seq + src] : nd[src - n2];
         kind = SJD_Q_ONEHOT;
         q = 1.0f;

@@ -121,6 +121,42 @@ def test_tiny_batch_of_three_and_ragged_window():
     assert all(s.st.n == wl.prompt_len + 61 for s in seqs)
 
 
+@pytest.mark.parametrize("name,lens", [("tiny", (16, 5, 11)), ("small-bf16", (24, 7, 1))])
+def test_ragged_prompts(name, lens):
+    """Prompts of different lengths in one batch (sjd_prefill_ragged): every sequence keeps its own positions
+    and finishes on its own; lock-step with one checker per sequence, each on its own prompt."""
+    wl = WORKLOADS[name]
+    n_generate, window = 40, wl.window
+    weights = make_weights(wl, gain_jitter=0.1)
+    batch, stride = len(lens), max(lens)
+    prompt = make_prompt(wl.with_(prompt_len=stride), batch)
+    cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=stride + n_generate + 8, max_window=window)
+    ctx = B.Context(cfg, B.weights_to_device(weights))
+    sample = B.make_sample_cfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window,
+                               init=INIT_COPY_ABOVE, grid_stride=wl.grid_stride, n_generate=n_generate)
+    scfg = SampleCfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window,
+                     init=INIT_COPY_ABOVE, grid_stride=wl.grid_stride, n_generate=n_generate, logits_dtype=wl.dtype)
+    ctx.prefill_ragged(torch.from_numpy(prompt).cuda(), lens, sample)
+    out = B.StepOut(batch, window)
+    ctx.get_window(out)
+    h = out.host()
+    seqs = [LockStepSequence(wl.with_(prompt_len=lens[b]), weights, prompt[b][:lens[b]], scfg, b, LOGIT_TOL[wl.dtype])
+            for b in range(batch)]
+    for b, s in enumerate(seqs):
+        s.check_window(h["draft"][b], h["q_kind"][b], h["q_draft"][b], h["total_committed"][b])
+    steps = 0
+    while any(s.st.n < lens[b] + n_generate for b, s in enumerate(seqs)):
+        ctx.step(out)
+        logits = ctx.peek_logits().to(torch.float64).cpu().numpy()
+        h = out.host()
+        for b, s in enumerate(seqs):
+            s.step(logits[b], {k: v[b] for k, v in h.items()})
+        steps += 1
+        assert steps <= n_generate
+    assert ctx.device_status() == B.SJD_OK
+    assert [s.st.n for s in seqs] == [l + n_generate for l in lens]
+
+
 def test_tiny_window_of_one_is_ordinary_sampling():
     wl = WORKLOADS["tiny"]
     ctx, seqs, steps, _ = run_lockstep(wl, window=1, n_generate=24)
