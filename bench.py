@@ -243,7 +243,8 @@ def run_library(args, wl):
 
     weights = make_weights(wl, device=dev)
     max_seq = wl.prompt_len + wl.n_generate + 8
-    ctx = B.Context(B.make_model_cfg(wl, batch * streams, max_seq, wl.window), weights, device=dev)
+    kv_pages = batch * streams * (-(-(wl.prompt_len + wl.n_generate) // 64)) if args.paged_kv else 0
+    ctx = B.Context(B.make_model_cfg(wl, batch * streams, max_seq, wl.window, kv_pages=kv_pages), weights, device=dev)
     sample = B.make_sample_cfg(wl.temperature, wl.top_k, wl.philox_seed, wl.window, B.SJD_INIT_RANDOM,
                                wl.grid_stride, wl.n_generate, seq_base=seq_base, guidance=args.guidance)
     prompt_host = torch.from_numpy(make_prompt(wl, batch * streams * world)[seq_base * streams:(seq_base + batch) * streams]
@@ -396,7 +397,7 @@ def run_library(args, wl):
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(wl, batch), guidance=args.guidance, rows_per_step=rows),
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(wl, batch), guidance=args.guidance, rows_per_step=rows, kv_cache="paged-64" if args.paged_kv else "contiguous"),
                 "clocks": clk, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
                 "cpu_baseline": cpu,
                 "timing": {"blocks": len(block_ms), "steps_per_block": args.steps,
@@ -502,6 +503,7 @@ def main():
                     help="whole-image generation under the baseline schedules and SJD (rows A-D and no-refinement)")
     ap.add_argument("--n-generate", type=int, default=0, help="image tokens per image for --table (default: the workload's)")
     ap.add_argument("--temperature", type=float, default=0.0, help="override the sampling temperature (default: the workload's, 1.0)")
+    ap.add_argument("--paged-kv", action="store_true", help="keep the KV cache in 64-position pages (same results)")
     ap.add_argument("--guidance", type=float, default=0.0,
                     help="classifier-free guidance weight (the paper runs 3.0): two streams per image, 2 x batch x W rows")
     args = ap.parse_args()

@@ -106,7 +106,13 @@ typedef struct {
   int32_t max_ring; /* logits rows retained per image for SJD_INIT_RESAMPLE_ABOVE: at least grid_stride +   */
                     /* window (each costs vocab elements of dtype in the workspace); 0 if that strategy is  */
                     /* not used                                                                            */
+  int32_t kv_pages; /* 0: every sequence owns max_seq cache rows.  > 0: paged cache (the paper has none; a    */
+                    /* serving-side layout): the batch shares a pool of kv_pages pages of SJD_KV_PAGE         */
+                    /* positions, and sjd_prefill gives each sequence the ceil((prompt_len + n_generate) /    */
+                    /* SJD_KV_PAGE) pages it needs (SJD_ERR_CAPACITY when the pool is too small); results are */
+                    /* identical to the contiguous layout                                                     */
 } sjd_model_cfg;
+#define SJD_KV_PAGE 64
 
 /* Device pointers, borrowed.  Per-layer entries are HOST arrays of n_layers device pointers. */
 typedef struct {

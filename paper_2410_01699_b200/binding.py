@@ -46,7 +46,8 @@ class sjd_model_cfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim", "ffn_hidden",
                                          "vocab")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32),
-                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_window", C.c_int32), ("max_ring", C.c_int32)]
+                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_window", C.c_int32), ("max_ring", C.c_int32),
+                ("kv_pages", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -155,10 +156,11 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_model_cfg(wl, max_batch: int, max_seq: int, max_window: int, max_ring: int = 0) -> sjd_model_cfg:
+def make_model_cfg(wl, max_batch: int, max_seq: int, max_window: int, max_ring: int = 0,
+                   kv_pages: int = 0) -> sjd_model_cfg:
     """wl: anything with the model fields of inputs.Workload."""
     return sjd_model_cfg(wl.n_layers, wl.d_model, wl.n_heads, wl.n_kv_heads, wl.head_dim, wl.ffn_hidden, wl.vocab,
-                         wl.rope_theta, wl.rms_eps, DTYPES[wl.dtype], max_batch, max_seq, max_window, max_ring)
+                         wl.rope_theta, wl.rms_eps, DTYPES[wl.dtype], max_batch, max_seq, max_window, max_ring, kv_pages)
 
 
 def make_sample_cfg(temperature=1.0, top_k=2000, seed=0, window=16, init=SJD_INIT_RANDOM, grid_stride=0,

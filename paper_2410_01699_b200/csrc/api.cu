@@ -221,8 +221,9 @@ extern "C" int sjd_attention(int batch, int window, int n_heads, int n_kv_heads,
   if (rc != SJD_OK) return rc;
   const int splits = attn_splits(n_heads, batch);
   const int M = batch * window;
-  rc = launch_attention_mma(kv_map, 0, q, in_pos, partial, out, HiLoOut{nullptr, 0}, status, M, window, n_heads, n_kv_heads,
-                            head_dim, splits, stream);
+  const KvLayout contiguous = {const_cast<void *>(kv_cache), n_kv_heads, max_seq, head_dim, nullptr, 0, 0, 1};
+  rc = launch_attention_mma(kv_map, 0, contiguous, q, in_pos, partial, out, HiLoOut{nullptr, 0}, status, M, window,
+                            n_heads, n_kv_heads, head_dim, splits, stream);
   if (rc != SJD_OK || splits == 1) return rc;
   return launch_attention_combine(partial, in_pos, out, M, n_heads, head_dim, splits, stream, HiLoOut{nullptr, 0});
 }

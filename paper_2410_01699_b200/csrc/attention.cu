@@ -57,10 +57,8 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
   const int k_begin = s * chunk;
   const int k_end = min(len, k_begin + chunk);
 
-  const T *kbase = reinterpret_cast<const T *>(kv.base) +
-                   ((size_t)(b * 2 + 0) * kv.n_kv_heads + kvh) * (size_t)kv.max_seq * hd;
-  const T *vbase = reinterpret_cast<const T *>(kv.base) +
-                   ((size_t)(b * 2 + 1) * kv.n_kv_heads + kvh) * (size_t)kv.max_seq * hd;
+  static_assert(KV_PAGE % TK == 0, "a key tile must lie inside one cache page");
+  const T *cache = reinterpret_cast<const T *>(kv.base);
   const float scale = rsqrtf((float)hd);
 
   float m_run[MAXQ], l_run[MAXQ], o[MAXQ][MAXD];
@@ -74,12 +72,14 @@ __global__ void __launch_bounds__(NWARPS * 32) attention_partial_kernel(
 
   for (int t0 = k_begin; t0 < k_end; t0 += TK) {
     const int nk = min(TK, k_end - t0);
+    const T *kbase = cache + kv_row_offset(kv, b, 0, kvh, t0);   // the tile's rows are contiguous
+    const T *vbase = cache + kv_row_offset(kv, b, 1, kvh, t0);
     for (int i = tid; i < TK * hd; i += blockDim.x) {
       const int r = i / hd, d = i % hd;
       float kx = 0.0f, vx = 0.0f;
       if (r < nk) {
-        kx = to_f<T>(kbase[(size_t)(t0 + r) * hd + d]);
-        vx = to_f<T>(vbase[(size_t)(t0 + r) * hd + d]);
+        kx = to_f<T>(kbase[(size_t)r * hd + d]);
+        vx = to_f<T>(vbase[(size_t)r * hd + d]);
       }
       Ks[r * (hd + 1) + d] = kx;
       Vs[r * hd + d] = vx;

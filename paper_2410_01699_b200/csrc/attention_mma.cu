@@ -91,6 +91,9 @@ struct AttnParams {
   int *status;
   int rows_per_seq, n_heads, n_kv_heads, splits;
   int plane0;            // first cache plane of this layer: planes are [b][k|v][kv_head]
+  // paged cache: planes are [page][layer][k|v][kv_head], one page (KT positions) per tile
+  const int32_t *page_table;   // [B][pages_per_seq]; null: contiguous
+  int pages_per_seq, layer, n_layers;
 };
 
 template <int HD, int KG>
@@ -139,13 +142,19 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
   auto issue = [&](int t) {   // thread 0: load tile t into its stage
     const int s = t % kStagesAttn;
     uint8_t *dst = smem + s * STAGE_BYTES;
-    const int key0 = k_begin + t * KT;
+    int key0 = k_begin + t * KT, pk = plane_k, pv = plane_v;
+    if (p.page_table != nullptr) {   // k_begin is a multiple of KT: tile t is exactly one page
+      const int page = __ldg(p.page_table + b * p.pages_per_seq + key0 / KT);
+      pk = ((page * p.n_layers + p.layer) * 2 + 0) * p.n_kv_heads + kvh;
+      pv = pk + p.n_kv_heads;
+      key0 = 0;
+    }
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&bar_full[s])), "r"(STAGE_BYTES)
                  : "memory");
 #pragma unroll
     for (int hf = 0; hf < HALVES; ++hf) {
-      tma_load_3d(dst + hf * (KT * 128), &kv_map, hf * 64, key0, plane_k, &bar_full[s]);
-      tma_load_3d(dst + TILE_BYTES + hf * (KT * 128), &kv_map, hf * 64, key0, plane_v, &bar_full[s]);
+      tma_load_3d(dst + hf * (KT * 128), &kv_map, hf * 64, key0, pk, &bar_full[s]);
+      tma_load_3d(dst + TILE_BYTES + hf * (KT * 128), &kv_map, hf * 64, key0, pv, &bar_full[s]);
     }
   };
   if (tid == 0)
@@ -404,7 +413,8 @@ bool attention_mma_supported(int head_dim, int rows_per_seq) { return (head_dim 
 
 // With splits > 1 the kernel leaves partial records and the caller merges them with the combine kernel of
 // attention.cu; with a single key range it writes `out` (and `hilo`) itself and no merge is needed.
-int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
+int launch_attention_mma(const TensorMap &kv_map, int plane0, KvLayout kv, const float *q, const int32_t *in_pos,
+                         float *partial,
                          float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads,
                          int head_dim, int splits, cudaStream_t stream) {
   if (!attention_mma_supported(head_dim, rows_per_seq) || M % rows_per_seq != 0) return SJD_ERR_UNSUPPORTED;
@@ -420,6 +430,11 @@ int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, co
   p.n_kv_heads = n_kv_heads;
   p.splits = splits;
   p.plane0 = plane0;
+  static_assert(KT == KV_PAGE, "one key tile per cache page");
+  p.page_table = kv.page_table;
+  p.pages_per_seq = kv.pages_per_seq;
+  p.layer = kv.layer;
+  p.n_layers = kv.n_layers;
   const int threads = 128;   // four warps: 16-row bands x key groups
   const int kg = rows_per_seq <= 16 ? 4 : rows_per_seq <= 32 ? 2 : 1;
   const dim3 grid(n_heads, M / rows_per_seq, splits);

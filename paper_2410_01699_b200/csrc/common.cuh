@@ -319,10 +319,24 @@ int launch_rmsnorm(int dtype, const float *x, const void *gain, float *h, int M,
                    HiLoOut hilo = HiLoOut{nullptr, 0});
 // Rotate q and k by their absolute position (pairs i, i + hd/2), store q as fp32 [M][H*hd],
 // append k and v to the cache row in_pos[m] of sequence m / rows_per_seq.  Rows with in_pos < 0 are skipped.
-struct KvLayout {        // cache of one layer: [B][2][KVh][max_seq][hd]
+// Cache of one layer.  Contiguous: base is this layer's [B][2][KVh][max_seq][hd].  Paged (page_table != null): base is
+// the pool [page][layer][2][KVh][KV_PAGE][hd] shared by all layers, and logical page i of sequence b (positions
+// i * KV_PAGE .. i * KV_PAGE + KV_PAGE - 1) lives in physical page page_table[b * pages_per_seq + i].
+constexpr int KV_PAGE = 64;
+struct KvLayout {
   void *base;
   int n_kv_heads, max_seq, head_dim;
+  const int32_t *page_table;
+  int pages_per_seq, layer, n_layers;
 };
+// element offset of the cache row (sequence b, which = 0 keys / 1 values, kv head kh, position pos)
+__device__ __forceinline__ size_t kv_row_offset(const KvLayout &kv, int b, int which, int kh, int pos) {
+  if (kv.page_table == nullptr)
+    return (((size_t)(b * 2 + which) * kv.n_kv_heads + kh) * kv.max_seq + pos) * kv.head_dim;
+  const int page = kv.page_table[b * kv.pages_per_seq + pos / KV_PAGE];
+  return (((((size_t)page * kv.n_layers + kv.layer) * 2 + which) * kv.n_kv_heads + kh) * KV_PAGE + pos % KV_PAGE) *
+         kv.head_dim;
+}
 // QK-norm variant: every head of q and of k is RMS-normalised over its head_dim entries (gains of `dtype`,
 // length head_dim) before the rotary step; null gains: the plain model.
 struct QkNorm {
@@ -346,7 +360,9 @@ int launch_attention_combine(const float *partial, const int32_t *in_pos, float 
 // tensor-core split-KV attention for bf16 caches (attention_mma.cu)
 int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_seq, int head_dim);
 bool attention_mma_supported(int head_dim, int rows_per_seq);
-int launch_attention_mma(const TensorMap &kv_map, int plane0, const float *q, const int32_t *in_pos, float *partial,
+// plane0: first plane of this layer in the contiguous map [planes][max_seq][hd]; with kv.page_table set the map is
+// the pool's [planes][KV_PAGE][hd] and the plane of a tile comes from the page table.
+int launch_attention_mma(const TensorMap &kv_map, int plane0, KvLayout kv, const float *q, const int32_t *in_pos, float *partial,
                          float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads,
                          int head_dim, int splits, cudaStream_t stream);
 

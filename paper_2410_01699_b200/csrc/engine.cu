@@ -49,6 +49,7 @@ struct Layout {
   size_t committed, n, w_eff, draft, q_kind, q_row, q_draft, in_tok, in_pos;
   size_t ring, ring_stats, n_prev, w_prev;   // Sec. 4.2 (d): retained logits rows (max_ring > 0)
   size_t prompt_lens;                        // [max_batch] prompt length of every sequence
+  size_t page_table;                         // [max_batch][pages_per_seq] (paged cache, kv_pages > 0)
   size_t total;
 };
 
@@ -59,7 +60,7 @@ bool cfg_valid(const sjd_model_cfg *c) {
     return false;
   if (c->head_dim % 2 != 0 || c->n_heads % c->n_kv_heads != 0) return false;
   if (!(c->rms_eps > 0.0f) || !(c->rope_theta > 0.0f)) return false;
-  if (c->max_ring < 0) return false;
+  if (c->max_ring < 0 || c->kv_pages < 0) return false;
   return true;
 }
 
@@ -74,7 +75,10 @@ Layout make_layout(const sjd_model_cfg &c) {
     off += align256(bytes);
     return o;
   };
-  L.kv = take((size_t)c.n_layers * c.max_batch * 2 * nk * c.max_seq * es);
+  // contiguous: max_seq rows for every sequence; paged: kv_pages pages shared by the batch plus one spare page
+  // that unassigned table entries point to
+  L.kv = c.kv_pages > 0 ? take((size_t)(c.kv_pages + 1) * c.n_layers * 2 * nk * KV_PAGE * es)
+                        : take((size_t)c.n_layers * c.max_batch * 2 * nk * c.max_seq * es);
   L.logits[0] = take(Mx * c.vocab * es);
   L.logits[1] = take(Mx * c.vocab * es);
   L.stats[0] = take(Mx * sizeof(RowStats));
@@ -134,6 +138,7 @@ Layout make_layout(const sjd_model_cfg &c) {
   L.n_prev = take((size_t)c.max_batch * 4);
   L.w_prev = take((size_t)c.max_batch * 4);
   L.prompt_lens = take((size_t)c.max_batch * 4);
+  L.page_table = take(c.kv_pages > 0 ? (size_t)c.max_batch * ((c.max_seq + KV_PAGE - 1) / KV_PAGE) * 4 : 0);
   L.total = off;
   return L;
 }
@@ -242,6 +247,7 @@ struct sjd_ctx {
   sjd_sample_cfg sample;
   int batch, prompt_len, window;   // prompt_len: the longest prompt of the batch
   std::vector<int32_t> prompt_lens;  // per sequence (host copy; the device copy is in the workspace)
+  std::vector<int32_t> page_table;   // paged cache: host copy of [max_batch][pages_per_seq]
   bool prefilled;
   uint32_t host_step;  // number of sjd_step calls since prefill == device step index
   cudaStream_t last_stream;
@@ -299,13 +305,24 @@ struct sjd_ctx {
     st.grid_stride = sample.grid_stride;
     return st;
   }
+  int pages_per_seq() const { return (cfg.max_seq + KV_PAGE - 1) / KV_PAGE; }
   KvLayout kv_layer(int l) const {
     KvLayout kv;
     const size_t per_layer = (size_t)cfg.max_batch * 2 * cfg.n_kv_heads * cfg.max_seq * cfg.head_dim * esize(cfg.dtype);
-    kv.base = ws + lay.kv + (size_t)l * per_layer;
     kv.n_kv_heads = cfg.n_kv_heads;
     kv.max_seq = cfg.max_seq;
     kv.head_dim = cfg.head_dim;
+    kv.layer = l;
+    kv.n_layers = cfg.n_layers;
+    if (cfg.kv_pages > 0) {   // one pool for all layers; the page table says where a sequence's rows are
+      kv.base = ws + lay.kv;
+      kv.page_table = reinterpret_cast<const int32_t *>(ws + lay.page_table);
+      kv.pages_per_seq = pages_per_seq();
+    } else {
+      kv.base = ws + lay.kv + (size_t)l * per_layer;
+      kv.page_table = nullptr;
+      kv.pages_per_seq = 0;
+    }
     return kv;
   }
 };
@@ -452,7 +469,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     const KvLayout kv = c->kv_layer(l);
     SJD_TR(TC_OTHER, launch_qkv_finish(dt, ps, rs, st.in_pos, rope, q, kv, M, rows_per_seq, g.n_heads, c->qk_norm(l), stream));
     if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
-      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, q, st.in_pos, partial, attn,
+      SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, kv, q, st.in_pos, partial, attn,
                                                 hl_attn, status, M, rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim,
                                                 att_splits, stream));
       if (att_splits > 1)
@@ -686,10 +703,14 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
     }
     // the cache as one 3-D tensor map for the tensor-core attention; unwritten rows must read as finite
     // numbers (a masked probability of 0 times NaN would poison the output), so the cache starts at zero
-    const long planes = (long)L * cfg->max_batch * 2 * cfg->n_kv_heads;
+    // (paged cache: the planes are the pool's [page][layer][k|v][kv_head], each KV_PAGE rows long)
+    const bool paged = cfg->kv_pages > 0;
+    const long planes = paged ? (long)(cfg->kv_pages + 1) * L * 2 * cfg->n_kv_heads
+                              : (long)L * cfg->max_batch * 2 * cfg->n_kv_heads;
+    const long plane_rows = paged ? KV_PAGE : cfg->max_seq;
     if (attention_mma_supported(cfg->head_dim, cfg->max_window) &&
-        make_kv_tensor_map(&c->kv_map, c->ws + lay.kv, planes, cfg->max_seq, cfg->head_dim) == SJD_OK &&
-        cudaMemset(c->ws + lay.kv, 0, (size_t)planes * cfg->max_seq * cfg->head_dim * 2) == cudaSuccess)
+        make_kv_tensor_map(&c->kv_map, c->ws + lay.kv, planes, plane_rows, cfg->head_dim) == SJD_OK &&
+        cudaMemset(c->ws + lay.kv, 0, (size_t)planes * plane_rows * cfg->head_dim * 2) == cudaSuccess)
       c->kv_map_valid = true;
     for (int l = 0; l < L; ++l) {
       const LayerMaps &lm = c->wmaps[l];
@@ -732,6 +753,21 @@ extern "C" int sjd_prefill_ragged(sjd_ctx *c, int batch, const int32_t *prompt, 
   c->sample = *sample;
   c->batch = batch;
   c->prompt_len = prompt_len;
+  if (c->cfg.kv_pages > 0) {
+    // every sequence gets the pages its own prompt and generated tokens need, in order, from page 0; entries
+    // past a sequence's last page point to the spare page
+    const int pps = c->pages_per_seq();
+    c->page_table.assign((size_t)c->cfg.max_batch * pps, c->cfg.kv_pages);
+    long next = 0;
+    for (int b = 0; b < batch; ++b) {
+      const int need = (prompt_lens[b] + sample->n_generate + KV_PAGE - 1) / KV_PAGE;
+      if (next + need > c->cfg.kv_pages) return SJD_ERR_CAPACITY;
+      for (int i = 0; i < need; ++i) c->page_table[(size_t)b * pps + i] = (int32_t)(next + i);
+      next += need;
+    }
+    SJD_CUDA(cudaMemcpyAsync(c->ws + c->lay.page_table, c->page_table.data(), c->page_table.size() * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, stream));
+  }
   c->prompt_lens.assign(prompt_lens, prompt_lens + batch);
   SJD_CUDA(cudaMemcpyAsync(c->ws + c->lay.prompt_lens, c->prompt_lens.data(), (size_t)batch * sizeof(int32_t),
                            cudaMemcpyHostToDevice, stream));

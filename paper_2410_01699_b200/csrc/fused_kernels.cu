@@ -103,8 +103,7 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   const int hd = kv.head_dim, half = hd >> 1, nkv = kv.n_kv_heads;
   const int nq = n_heads * hd, nk = nkv * hd;
   const size_t rbase = (size_t)m * ps.ld;
-  T *kbase = reinterpret_cast<T *>(kv.base) + (size_t)b * 2 * nkv * kv.max_seq * hd;
-  T *vbase = kbase + (size_t)nkv * kv.max_seq * hd;
+  T *cache = reinterpret_cast<T *>(kv.base);
   // the block's 64-thread groups walk over the head slots of the row (one pass when the grid has a
   // block for every four slots, several when many rows share fewer blocks per row)
   const int stride = gridDim.y * (blockDim.x >> 6);
@@ -141,14 +140,14 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
         q[(size_t)m * nq + slot * hd + j] = r1;
         q[(size_t)m * nq + slot * hd + j + half] = r2;
       } else {
-        T *dst = kbase + ((size_t)(slot - n_heads) * kv.max_seq + pos) * hd;
+        T *dst = cache + kv_row_offset(kv, b, 0, slot - n_heads, pos);
         dst[j] = from_f<T>(r1);
         dst[j + half] = from_f<T>(r2);
       }
     }
   } else {
     const int kh = slot - n_heads - nkv;
-    T *dst = vbase + ((size_t)kh * kv.max_seq + pos) * hd;
+    T *dst = cache + kv_row_offset(kv, b, 1, kh, pos);
     for (int j = lt; j < hd; j += 64)
       dst[j] = from_f<T>(sc * sum_planes(ps, rbase + nq + nk + kh * hd + j));
   }

@@ -138,8 +138,7 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t 
   const int nq = n_heads * hd, nk = nkv * hd;
   const float *row = qkv + (size_t)m * (nq + 2 * nk);
   const float2 *cs = rope + (size_t)pos * half;
-  T *kbase = reinterpret_cast<T *>(kv.base) + (size_t)b * 2 * nkv * kv.max_seq * hd;
-  T *vbase = kbase + (size_t)nkv * kv.max_seq * hd;
+  T *cache = reinterpret_cast<T *>(kv.base);
   // rotated pairs of q and k
   for (int i = threadIdx.x; i < (n_heads + nkv) * half; i += blockDim.x) {
     const int head = i / half, j = i % half;
@@ -161,14 +160,14 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, const int32_t 
     } else {
       const int kh = head - n_heads;
       const float x1 = g1 * row[nq + kh * hd + j], x2 = g2 * row[nq + kh * hd + j + half];
-      T *dst = kbase + ((size_t)kh * kv.max_seq + pos) * hd;
+      T *dst = cache + kv_row_offset(kv, b, 0, kh, pos);
       dst[j] = from_f<T>(x1 * c.x - x2 * c.y);
       dst[j + half] = from_f<T>(x2 * c.x + x1 * c.y);
     }
   }
   for (int i = threadIdx.x; i < nk; i += blockDim.x) {
     const int kh = i / hd, j = i % hd;
-    vbase[((size_t)kh * kv.max_seq + pos) * hd + j] = from_f<T>(row[nq + nk + i]);
+    cache[kv_row_offset(kv, b, 1, kh, pos) + j] = from_f<T>(row[nq + nk + i]);
   }
 }
 

@@ -28,7 +28,7 @@ def test_library_exports_every_declared_function():
 
 
 def test_struct_sizes_match_the_header_layout():
-    assert C.sizeof(B.sjd_model_cfg) == 14 * 4
+    assert C.sizeof(B.sjd_model_cfg) == 15 * 4
     assert C.sizeof(B.sjd_weights) == 14 * 8
     assert C.sizeof(B.sjd_sample_cfg) == 48
     assert B.sjd_sample_cfg.guidance.offset == 36 and B.sjd_sample_cfg.schedule.offset == 40
@@ -53,7 +53,13 @@ def test_workspace_size_query():
     kv = 32 * 2 * 32 * 128 * 2432 * 2
     logits = 2 * 32 * 65536 * 2
     assert kv + logits < nbytes < kv + logits + (256 << 20)
-    for field, bad in (("n_layers", 0), ("head_dim", 63), ("n_kv_heads", 5), ("max_window", 0), ("dtype", 7)):
+    # paged cache: the pool (plus its spare page) replaces max_batch x max_seq rows
+    paged = B.make_model_cfg(wl, max_batch=8, max_seq=2432, max_window=32, kv_pages=40)
+    pool = 41 * 32 * 2 * 32 * 64 * 128 * 2
+    rest = B.sjd_workspace_bytes(B.make_model_cfg(wl, 8, 2432, 32)) - 8 * kv
+    assert pool + rest <= B.sjd_workspace_bytes(paged) < pool + rest + (1 << 20)
+    for field, bad in (("n_layers", 0), ("head_dim", 63), ("n_kv_heads", 5), ("max_window", 0), ("dtype", 7),
+                       ("kv_pages", -1)):
         c = B.make_model_cfg(wl, 1, 2432, 32)
         setattr(c, field, bad)
         assert B.sjd_workspace_bytes(c) == 0, field

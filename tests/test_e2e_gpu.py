@@ -121,19 +121,33 @@ def test_tiny_batch_of_three_and_ragged_window():
     assert all(s.st.n == wl.prompt_len + 61 for s in seqs)
 
 
-@pytest.mark.parametrize("name,lens", [("tiny", (16, 5, 11)), ("small-bf16", (24, 7, 1))])
-def test_ragged_prompts(name, lens):
+@pytest.mark.parametrize("name,over,lens,kv_pages", [
+    ("tiny", {}, (16, 5, 11), 0), ("small-bf16", {}, (24, 7, 1), 0),
+    ("tiny", {}, (70, 5, 130), 6), ("small-bf16", {}, (100, 7, 64), 6),
+    ("small-bf16", dict(head_dim=128, n_heads=4, n_kv_heads=2), (90, 130), 6)])
+def test_ragged_prompts(name, over, lens, kv_pages):
     """Prompts of different lengths in one batch (sjd_prefill_ragged): every sequence keeps its own positions
-    and finishes on its own; lock-step with one checker per sequence, each on its own prompt."""
-    wl = WORKLOADS[name]
+    and finishes on its own; lock-step with one checker per sequence, each on its own prompt.  With kv_pages the
+    cache is paged: the sequences' rows sit in pool pages handed out at pre-fill (a sequence's pages are not
+    where a contiguous layout would put them, and its rows cross page boundaries), which the oracle knows
+    nothing about, so agreement shows the paging changes no result."""
+    wl = WORKLOADS[name].with_(**over)
     n_generate, window = 40, wl.window
     weights = make_weights(wl, gain_jitter=0.1)
     batch, stride = len(lens), max(lens)
     prompt = make_prompt(wl.with_(prompt_len=stride), batch)
-    cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=stride + n_generate + 8, max_window=window)
+    cfg = B.make_model_cfg(wl, max_batch=batch, max_seq=stride + n_generate + 8, max_window=window,
+                           kv_pages=kv_pages)
     ctx = B.Context(cfg, B.weights_to_device(weights))
     sample = B.make_sample_cfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window,
                                init=INIT_COPY_ABOVE, grid_stride=wl.grid_stride, n_generate=n_generate)
+    if kv_pages:   # one page short: refused before anything is enqueued
+        small = B.Context(B.make_model_cfg(wl, max_batch=batch, max_seq=stride + n_generate + 8, max_window=window,
+                                           kv_pages=kv_pages - 1), B.weights_to_device(weights))
+        with pytest.raises(B.SJDError) as e:
+            small.prefill_ragged(torch.from_numpy(prompt).cuda(), lens, sample)
+        assert e.value.status == B.SJD_ERR_CAPACITY
+        del small
     scfg = SampleCfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window,
                      init=INIT_COPY_ABOVE, grid_stride=wl.grid_stride, n_generate=n_generate, logits_dtype=wl.dtype)
     ctx.prefill_ragged(torch.from_numpy(prompt).cuda(), lens, sample)
