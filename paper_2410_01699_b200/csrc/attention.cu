@@ -164,6 +164,44 @@ __global__ void attention_combine_kernel(const float *__restrict__ partial, cons
   const float *src = partial + ((size_t)m * n_heads + h) * splits * (hd + 2);
   const size_t base = ((size_t)m * n_heads + h) * hd;
   float *dst = out + base;
+  constexpr int NS = 8;
+  if (splits <= NS && hd <= (int)blockDim.x) {
+    // Few key ranges (the usual case): every thread fetches the row's position, all record heads and its own
+    // entry of every record at once, so the kernel costs one memory round trip instead of three in a row.
+    // Same arithmetic, in the same order, as the general path below.
+    const int d = threadIdx.x;
+    const int pos = in_pos[m];
+    float mm[NS], ll[NS], vv[NS];
+#pragma unroll
+    for (int s = 0; s < NS; ++s) {
+      const bool on = s < splits;
+      mm[s] = on ? src[(size_t)s * (hd + 2)] : -INFINITY;
+      ll[s] = on ? src[(size_t)s * (hd + 2) + 1] : 0.0f;
+      vv[s] = on && d < hd ? src[(size_t)s * (hd + 2) + 2 + d] : 0.0f;
+    }
+    if (d >= hd) return;
+    float v = 0.0f;
+    if (pos >= 0) {
+      float gmax = -INFINITY;
+#pragma unroll
+      for (int s = 0; s < NS; ++s) gmax = fmaxf(gmax, mm[s]);
+      float denom = 0.0f, acc = 0.0f;
+#pragma unroll
+      for (int s = 0; s < NS; ++s)
+        if (s < splits && mm[s] > -INFINITY) denom += ll[s] * expf(mm[s] - gmax);
+#pragma unroll
+      for (int s = 0; s < NS; ++s)
+        if (s < splits) acc += vv[s] * (mm[s] > -INFINITY ? expf(mm[s] - gmax) : 0.0f);
+      v = denom > 0.0f ? acc / denom : 0.0f;
+    }
+    dst[d] = v;
+    if (hilo.base) {
+      const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+      hilo.base[base + d] = hi;
+      hilo.base[hilo.lo_offset + base + d] = __float2bfloat16_rn(v - __bfloat162float(hi));
+    }
+    return;
+  }
   if (in_pos[m] < 0) {
     for (int d = threadIdx.x; d < hd; d += blockDim.x) {
       dst[d] = 0.0f;

@@ -96,61 +96,69 @@ __global__ void qkv_finish_kernel(PlaneSet ps, RowScale rs, const int32_t *__res
   pdl_wait();
   SJD_TL(TL_QKV, 1, threadIdx.x == 0);
   const int m = blockIdx.x, lt = threadIdx.x & 63;
-  const int pos = in_pos[m];
-  const float sc = row_scale_warp(rs, m);   // before any thread leaves: the warp shares the loads
-  if (pos < 0) return;
   const int b = m / rows_per_seq;
   const int hd = kv.head_dim, half = hd >> 1, nkv = kv.n_kv_heads;
   const int nq = n_heads * hd, nk = nkv * hd;
   const size_t rbase = (size_t)m * ps.ld;
   T *cache = reinterpret_cast<T *>(kv.base);
+  // The loads of the projection planes depend on nothing, the row's position and RMS scale are loads of their
+  // own and the rotary entry depends on the position: the plane loads of a slot are issued first, so that the
+  // kernel waits for two memory round trips in a row and not three.
+  int pos = 0;
+  float sc = 0.0f;
+  bool first = true;
   // the block's 64-thread groups walk over the head slots of the row (one pass when the grid has a
   // block for every four slots, several when many rows share fewer blocks per row)
   const int stride = gridDim.y * (blockDim.x >> 6);
   for (int slot = blockIdx.y * (blockDim.x >> 6) + (threadIdx.x >> 6); slot < n_heads + 2 * nkv; slot += stride) {
-  if (slot < n_heads + nkv) {
+    const bool is_v = slot >= n_heads + nkv;
     const bool is_q = slot < n_heads;
-    const int col0 = is_q ? slot * hd : nq + (slot - n_heads) * hd;
-    // head_dim <= 128: a thread of the group owns at most one rotary pair (j, j + half) of the head
-    {
-      const int j = lt;
-      const bool has = j < half;
-      float x1 = 0.0f, x2 = 0.0f;
-      if (has) {
-        x1 = sc * sum_planes(ps, rbase + col0 + j);
-        x2 = sc * sum_planes(ps, rbase + col0 + j + half);
-      }
-      if (qkn.q_gain) {   // QK-norm: RMS over the head's entries, held by the 64 threads of this group
-        const int grp = threadIdx.x >> 6;
-        const float ws = warp_sum(x1 * x1 + x2 * x2);
-        if ((threadIdx.x & 31) == 0) s_ss[threadIdx.x >> 5] = ws;
-        asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory");
-        const float rinv = rsqrtf((s_ss[2 * grp] + s_ss[2 * grp + 1]) / (float)hd + qkn.eps);
-        asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory");   // the sums are reused by the group's next head
-        if (has) {
-          const T *gain = reinterpret_cast<const T *>(is_q ? qkn.q_gain : qkn.k_gain);
-          x1 *= rinv * to_f<T>(gain[j]);
-          x2 *= rinv * to_f<T>(gain[j + half]);
-        }
-      }
-      if (!has) continue;
-      const float2 c = rope[(size_t)pos * half + j];
-      const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
-      if (is_q) {
-        q[(size_t)m * nq + slot * hd + j] = r1;
-        q[(size_t)m * nq + slot * hd + j + half] = r2;
-      } else {
-        T *dst = cache + kv_row_offset(kv, b, 0, slot - n_heads, pos);
-        dst[j] = from_f<T>(r1);
-        dst[j + half] = from_f<T>(r2);
+    // head_dim <= 128: a thread of the group owns at most one rotary pair (j, j + half) of a q or k head,
+    // or the entries j and j + 64 of a v head
+    const int col0 = is_q ? slot * hd : is_v ? nq + nk + (slot - n_heads - nkv) * hd : nq + (slot - n_heads) * hd;
+    const int ja = lt, jb = is_v ? lt + 64 : lt + half;
+    const bool has_a = is_v ? ja < hd : ja < half, has_b = is_v ? jb < hd : ja < half;
+    float x1 = 0.0f, x2 = 0.0f;
+    if (has_a) x1 = sum_planes(ps, rbase + col0 + ja);
+    if (has_b) x2 = sum_planes(ps, rbase + col0 + jb);
+    if (first) {   // uniform over the block
+      pos = in_pos[m];
+      sc = row_scale_warp(rs, m);   // before any thread leaves: the warp shares the loads
+      first = false;
+      if (pos < 0) return;
+    }
+    x1 *= sc;
+    x2 *= sc;
+    if (is_v) {
+      T *dst = cache + kv_row_offset(kv, b, 1, slot - n_heads - nkv, pos);
+      if (has_a) dst[ja] = from_f<T>(x1);
+      if (has_b) dst[jb] = from_f<T>(x2);
+      continue;
+    }
+    if (qkn.q_gain) {   // QK-norm: RMS over the head's entries, held by the 64 threads of this group
+      const int grp = threadIdx.x >> 6;
+      const float ws = warp_sum(x1 * x1 + x2 * x2);
+      if ((threadIdx.x & 31) == 0) s_ss[threadIdx.x >> 5] = ws;
+      asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory");
+      const float rinv = rsqrtf((s_ss[2 * grp] + s_ss[2 * grp + 1]) / (float)hd + qkn.eps);
+      asm volatile("bar.sync %0, 64;" ::"r"(grp + 1) : "memory");   // the sums are reused by the group's next head
+      if (has_a) {
+        const T *gain = reinterpret_cast<const T *>(is_q ? qkn.q_gain : qkn.k_gain);
+        x1 *= rinv * to_f<T>(gain[ja]);
+        x2 *= rinv * to_f<T>(gain[jb]);
       }
     }
-  } else {
-    const int kh = slot - n_heads - nkv;
-    T *dst = cache + kv_row_offset(kv, b, 1, kh, pos);
-    for (int j = lt; j < hd; j += 64)
-      dst[j] = from_f<T>(sc * sum_planes(ps, rbase + nq + nk + kh * hd + j));
-  }
+    if (!has_a) continue;
+    const float2 c = rope[(size_t)pos * half + ja];
+    const float r1 = x1 * c.x - x2 * c.y, r2 = x2 * c.x + x1 * c.y;
+    if (is_q) {
+      q[(size_t)m * nq + slot * hd + ja] = r1;
+      q[(size_t)m * nq + slot * hd + jb] = r2;
+    } else {
+      T *dst = cache + kv_row_offset(kv, b, 0, slot - n_heads, pos);
+      dst[ja] = from_f<T>(r1);
+      dst[jb] = from_f<T>(r2);
+    }
   }
 }
 
