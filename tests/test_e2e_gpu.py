@@ -190,7 +190,8 @@ def test_tiny_top1_is_greedy_decoding():
     assert steps <= 48
 
 
-def run_lockstep_guided(wl, images, guidance, max_steps=None, init=INIT_RANDOM, window=None, n_generate=None, schedule=0):
+def run_lockstep_guided(wl, images, guidance, max_steps=None, init=INIT_RANDOM, window=None, n_generate=None, schedule=0,
+                        kv_pages=0):
     """Lock-step under classifier-free guidance: 2 * images sequences in the library (conditional and
     unconditional stream of each image, prompts of one length with different tokens), one checker per image."""
     window = window or wl.window
@@ -198,7 +199,7 @@ def run_lockstep_guided(wl, images, guidance, max_steps=None, init=INIT_RANDOM, 
     weights = make_weights(wl, gain_jitter=0.1)
     prompt = make_prompt(wl, 2 * images)       # rows 2i / 2i+1: conditional / unconditional prompt of image i
     cfg = B.make_model_cfg(wl, max_batch=2 * images, max_seq=wl.prompt_len + n_generate + 8, max_window=window,
-                           max_ring=wl.grid_stride + window if init == INIT_RESAMPLE_ABOVE else 0)
+                           max_ring=wl.grid_stride + window if init == INIT_RESAMPLE_ABOVE else 0, kv_pages=kv_pages)
     ctx = B.Context(cfg, B.weights_to_device(weights))
     sample = B.make_sample_cfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=window,
                                init=init, grid_stride=wl.grid_stride, n_generate=n_generate, guidance=guidance,
@@ -238,13 +239,17 @@ def test_tiny_guided_generation():
         assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
 
 
-@pytest.mark.parametrize("name,init,schedule", [("tiny", INIT_RESAMPLE_ABOVE, 0), ("small-bf16", INIT_RESAMPLE_ABOVE, 0),
-                                                ("small-bf16", INIT_RESAMPLE_LEFT, 2), ("tiny", INIT_RANDOM, 1)])
-def test_guided_generation_with_the_other_options(name, init, schedule):
+@pytest.mark.parametrize("name,init,schedule,kv_pages", [
+    ("tiny", INIT_RESAMPLE_ABOVE, 0, 0), ("small-bf16", INIT_RESAMPLE_ABOVE, 0, 0),
+    ("small-bf16", INIT_RESAMPLE_LEFT, 2, 0), ("tiny", INIT_RANDOM, 1, 0),
+    ("small-bf16", INIT_RESAMPLE_ABOVE, 0, 8), ("tiny", INIT_COPY_ABOVE, 0, 8)])
+def test_guided_generation_with_the_other_options(name, init, schedule, kv_pages):
     """Guidance together with the initialisations that draw from predicted distributions (the ring then
-    holds mixed rows, one per image position), with the no-refinement ablation and with the Jacobi schedule."""
+    holds mixed rows, one per image position), with the no-refinement ablation, with the Jacobi schedule and
+    with the paged cache (four streams of two pages each)."""
     wl = WORKLOADS[name]
-    seqs, steps = run_lockstep_guided(wl, images=2, guidance=3.0, n_generate=50, init=init, schedule=schedule)
+    seqs, steps = run_lockstep_guided(wl, images=2, guidance=3.0, n_generate=50, init=init, schedule=schedule,
+                                      kv_pages=kv_pages)
     for s in seqs:
         assert s.st.n == wl.prompt_len + 50
 
