@@ -317,6 +317,16 @@ def test_small_bf16_gqa_generation():
         assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
 
 
+def test_small_bf16_128_rows():
+    """8 images x W = 16 = 128 rows per pass: the largest single slab (256 MMA columns, two-stage ring) through
+    pre-fill and three steps."""
+    wl = WORKLOADS["small-bf16"]
+    ctx, seqs, steps, _ = run_lockstep(wl, batch=8, max_steps=3)
+    for s in seqs:
+        assert s.max_logit_err <= 2e-2
+        assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
+
+
 def test_small_bf16_many_rows():
     """20 images x W = 16 = 320 rows per pass: the token-slab form of the projections (three slabs of
     112 rows) through pre-fill and three steps."""

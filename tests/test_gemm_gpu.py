@@ -33,6 +33,8 @@ def _tolerance(x, w, k):
     (64, 2048, 1024),     # W = 64
     (128, 512, 256),      # widest supported window batch
     (32, 65536, 512),     # 512 tiles (vocabulary-sized N)
+    (112, 768, 1024),     # 112 rows in one slab: accumulators of 224 columns
+    (128, 22016, 4096),   # four images x W = 32 on the gate|up projection: 172 tiles on 148 SMs
     (129, 256, 512),      # first row count cut into token slabs: two of 80 rows (the second holds 49)
     (256, 1024, 1024),    # two full slabs of 128 rows
     (300, 384, 640),      # three ragged slabs of 112 rows (the last holds 76)
