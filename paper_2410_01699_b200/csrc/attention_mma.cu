@@ -94,26 +94,7 @@ struct AttnParams {
   // paged cache: planes are [page][layer][k|v][kv_head], one page (KT positions) per tile
   const int32_t *page_table;   // [B][pages_per_seq]; null: contiguous
   int pages_per_seq, layer, n_layers;
-  int cluster_merge;     // splits > 1 and the CTAs of one (head, sequence) form a thread-block cluster along z:
-                         // they merge their key ranges through distributed shared memory and write `out` themselves
 };
-
-// ---- thread-block cluster helpers (the key ranges of one head form a cluster; no multicast anywhere)
-__device__ __forceinline__ void cluster_arrive_wait() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// address of this CTA's shared-memory location `local` in the CTA of rank `rank` of the cluster
-__device__ __forceinline__ uint32_t cluster_map(uint32_t local, uint32_t rank) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
-  return remote;
-}
-__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
-}
 
 template <int HD, int KG>
 __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams p) {
@@ -310,8 +291,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
     // leave no copy in flight: wait (bounded) for the stages that were armed
     if (tid == 0)
       for (int t = 0; t < n_tiles && t < kStagesAttn; ++t) bar_wait(&bar_full[t % kStagesAttn], 0);
-    if (!p.cluster_merge) return;
-    __syncthreads();   // in a cluster every CTA still has to pass the barriers below (its output is void anyway)
+    return;
   }
 
   SJD_TL(TL_ATTN, 2, threadIdx.x == 0);
@@ -340,8 +320,7 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
       }
     }
     __syncthreads();
-    if (kg > 0 && !p.cluster_merge) return;
-    if (kg == 0) {
+    if (kg > 0) return;
 #pragma unroll
     for (int og = 1; og < KG; ++og) {
       const float *src = xch + ((size_t)((og - 1) * n_rw + rw) * 16) * REC;
@@ -362,55 +341,6 @@ __global__ void __launch_bounds__(128) attention_mma_kernel(const __grid_constan
         }
       }
     }
-  }
-  }
-  if (p.cluster_merge) {
-    // ---- several key ranges, one cluster: every CTA leaves its rows' records (max, sum, output) in its own
-    // shared memory; after a cluster barrier CTA s merges rows s, s + S, ... from all S CTAs in rank order
-    // (fixed order: deterministic), normalises and writes the output and its hi/lo planes; a second barrier
-    // keeps every CTA's shared memory alive until its peers have read it.
-    constexpr int REC = HD + 2;
-    constexpr int FIN_OFF = (3 * 16 * REC * 4 + 1023) / 1024 * 1024;   // behind the key-group exchange area
-    float *fin = reinterpret_cast<float *>(smem + FIN_OFF);
-    if (kg == 0) {
-#pragma unroll
-      for (int rr = 0; rr < 2; ++rr) {
-        float *row = fin + (size_t)(rw * 16 + g + rr * 8) * REC;
-        if (tq == 0) {
-          row[0] = m_run[rr];
-          row[1] = l_run[rr];
-        }
-#pragma unroll
-        for (int i = 0; i < HD / 8; ++i)
-          *reinterpret_cast<float2 *>(row + 2 + i * 8 + tq * 2) = make_float2(o[i][rr * 2], o[i][rr * 2 + 1]);
-      }
-    }
-    cluster_arrive_wait();
-    const int S = p.splits;
-    const uint32_t fin_local = smem_addr(fin);
-    for (int idx = tid; idx < ((W - split + S - 1) / S) * HD; idx += blockDim.x) {
-      const int r = split + (idx / HD) * S, col = idx % HD;
-      float mx = -INFINITY;
-      for (int j = 0; j < S; ++j) mx = fmaxf(mx, ld_cluster_f32(cluster_map(fin_local + (uint32_t)(r * REC) * 4u, (uint32_t)j)));
-      float l = 0.0f, acc = 0.0f;
-      for (int j = 0; j < S; ++j) {
-        const uint32_t rec = cluster_map(fin_local + (uint32_t)(r * REC) * 4u, (uint32_t)j);
-        const float m_j = ld_cluster_f32(rec);
-        const float a_j = m_j > -INFINITY ? exp2f(m_j - mx) : 0.0f;
-        l += ld_cluster_f32(rec + 4u) * a_j;
-        acc += ld_cluster_f32(rec + 8u + (uint32_t)col * 4u) * a_j;
-      }
-      const float v = l > 0.0f ? acc / l : 0.0f;   // inactive rows: zeros
-      const size_t at = ((size_t)(m0 + r) * p.n_heads + h) * HD + col;
-      p.out[at] = v;
-      if (p.hilo.base) {
-        const __nv_bfloat16 vh = __float2bfloat16_rn(v);
-        p.hilo.base[at] = vh;
-        p.hilo.base[p.hilo.lo_offset + at] = __float2bfloat16_rn(v - __bfloat162float(vh));
-      }
-    }
-    cluster_arrive_wait();
-    return;
   }
   if (p.splits == 1) {
     // ---- a single key range: normalise and write the output rows (and their hi/lo planes) directly
@@ -481,12 +411,12 @@ int make_kv_tensor_map(TensorMap *out, const void *base, long planes, long max_s
 
 bool attention_mma_supported(int head_dim, int rows_per_seq) { return (head_dim == 64 || head_dim == 128) && rows_per_seq <= 64; }
 
-// With a single key range, or with 2..8 ranges and cluster_merge (their CTAs then form a thread-block cluster and
-// merge through distributed shared memory), the kernel writes `out` (and `hilo`) itself; else it leaves
-// partial records and the caller merges them with the combine kernel of attention.cu.
+// With splits > 1 the kernel leaves partial records and the caller merges them with the combine kernel of
+// attention.cu; with a single key range it writes `out` (and `hilo`) itself and no merge is needed.
 int launch_attention_mma(const TensorMap &kv_map, int plane0, KvLayout kv, const float *q, const int32_t *in_pos,
-                         float *partial, float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads,
-                         int n_kv_heads, int head_dim, int splits, cudaStream_t stream, bool cluster_merge) {
+                         float *partial,
+                         float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads,
+                         int head_dim, int splits, cudaStream_t stream) {
   if (!attention_mma_supported(head_dim, rows_per_seq) || M % rows_per_seq != 0) return SJD_ERR_UNSUPPORTED;
   AttnParams p;
   p.q = q;
@@ -505,7 +435,6 @@ int launch_attention_mma(const TensorMap &kv_map, int plane0, KvLayout kv, const
   p.pages_per_seq = kv.pages_per_seq;
   p.layer = kv.layer;
   p.n_layers = kv.n_layers;
-  p.cluster_merge = (cluster_merge && splits > 1 && splits <= 8) ? 1 : 0;
   const int threads = 128;   // four warps: 16-row bands x key groups
   const int kg = rows_per_seq <= 16 ? 4 : rows_per_seq <= 32 ? 2 : 1;
   const dim3 grid(n_heads, M / rows_per_seq, splits);
@@ -513,10 +442,7 @@ int launch_attention_mma(const TensorMap &kv_map, int plane0, KvLayout kv, const
   const size_t smem = (size_t)kStagesAttn * 2 * KT * head_dim * 2 + 1024;
   auto launch = [&](auto kernel) -> int {
     SJD_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    if (p.cluster_merge)
-      SJD_CUDA(launch_kernel_cluster(kernel, grid, dim3(threads), smem, stream, dim3(1, 1, splits), km, p));
-    else
-      SJD_CUDA(launch_kernel(kernel, grid, dim3(threads), smem, stream, km, p));
+    SJD_CUDA(launch_kernel(kernel, grid, dim3(threads), smem, stream, km, p));
     SJD_CHECK_LAUNCH();
     return SJD_OK;
   };

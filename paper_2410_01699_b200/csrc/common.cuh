@@ -56,27 +56,6 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   cfg.numAttrs = g_pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
-// the same with a thread-block cluster of `cluster` CTAs (grid dimensions must be multiples of it)
-template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kernel_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                                         dim3 cluster, Args &&...args) {
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = cluster.x;
-  attr[0].val.clusterDim.y = cluster.y;
-  attr[0].val.clusterDim.z = cluster.z;
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = g_pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -385,6 +364,6 @@ bool attention_mma_supported(int head_dim, int rows_per_seq);
 // the pool's [planes][KV_PAGE][hd] and the plane of a tile comes from the page table.
 int launch_attention_mma(const TensorMap &kv_map, int plane0, KvLayout kv, const float *q, const int32_t *in_pos, float *partial,
                          float *out, HiLoOut hilo, int *status, int M, int rows_per_seq, int n_heads, int n_kv_heads,
-                         int head_dim, int splits, cudaStream_t stream, bool cluster_merge = false);
+                         int head_dim, int splits, cudaStream_t stream);
 
 }  // namespace sjd

@@ -277,7 +277,6 @@ struct sjd_ctx {
   bool gu_fused = false; // gate|up projection with SwiGLU in its epilogue (every layer has the maps for it)
   int gu_rows = 0;       // feature rows of the gate (and of the up) matrix per CTA of that launch
   int head_rows = 0;     // weight rows per CTA of the logits projection (0: 128)
-  int attn_cluster = 0;  // > 1: the key ranges of a head form a thread-block cluster of at most this many CTAs
   WMap wmap_head_r;      // lm_head in boxes of head_rows rows
   int n_ctas = 0;
   std::vector<LayerMaps> wmaps;
@@ -401,11 +400,7 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
   float *planes = c->at<float>(c->lay.gemm_planes);
   int *status = c->at<int>(c->lay.status);
   const float2 *rope = c->at<float2>(c->lay.rope);
-  int att_splits = attention_splits(g.n_heads, c->batch);
-  // key ranges of a head as one thread-block cluster that merges through distributed shared memory (no merge
-  // launch): at most attn_cluster ranges then
-  const bool att_cluster = c->attn_cluster > 1 && att_splits > 1;
-  if (att_cluster && att_splits > c->attn_cluster) att_splits = c->attn_cluster;
+  const int att_splits = attention_splits(g.n_heads, c->batch);
   const int Ma = c->rows_alloc();
   const HiLoOut hl_h{c->at<__nv_bfloat16>(c->lay.xs_h), (size_t)Ma * d};
   const HiLoOut hl_attn{c->at<__nv_bfloat16>(c->lay.xs_attn), (size_t)Ma * nq};
@@ -476,8 +471,8 @@ int forward_tc(sjd_ctx *c, const XMaps &xm, int rows_per_seq, void *logits_out, 
     if (c->kv_map_valid && attention_mma_supported(g.head_dim, rows_per_seq)) {
       SJD_TR(TC_ATTENTION, launch_attention_mma(c->kv_map, l * g.max_batch * 2 * g.n_kv_heads, kv, q, st.in_pos, partial, attn,
                                                 hl_attn, status, M, rows_per_seq, g.n_heads, g.n_kv_heads, g.head_dim,
-                                                att_splits, stream, att_cluster));
-      if (att_splits > 1 && !att_cluster)
+                                                att_splits, stream));
+      if (att_splits > 1)
         SJD_TR(TC_ATTENTION,
                launch_attention_combine(partial, st.in_pos, attn, M, g.n_heads, g.head_dim, att_splits, stream, hl_attn));
     } else {
@@ -698,10 +693,6 @@ extern "C" int sjd_init(sjd_ctx **out, const sjd_model_cfg *cfg, const sjd_weigh
     }
     // logits projection: optional tile height below 128 rows (SJD_HEAD_ROWS; measured on the 7B shapes: 112
     // rows = two full waves of CTAs is 4 % slower than 128 rows in 1.7 waves, so the default stays 128)
-    if (const char *e = getenv("SJD_ATTN_CLUSTER")) {   // tuning: 2, 4 or 8
-      const int v = atoi(e);
-      if (v == 2 || v == 4 || v == 8) c->attn_cluster = v;
-    }
     if (const char *e = getenv("SJD_HEAD_ROWS")) {
       const int r = atoi(e);
       if (r >= 8 && r < 128 && c->wmap_head.valid &&
