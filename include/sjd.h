@@ -235,6 +235,14 @@ int sjd_step(sjd_ctx *ctx, const sjd_step_out *out, void *cuda_stream);
  * n_committed, committed and flags of `out` are not written. */
 int sjd_get_window(sjd_ctx *ctx, const sjd_step_out *out, void *cuda_stream);
 
+/* The output of Algorithm 1: the tokens fixed so far.  tokens: device int32 [images][row_stride], image i
+ * receives its prompt followed by the tokens it has accepted (under guidance: the conditional stream, which
+ * holds the same accepted tokens as the unconditional one); entries past its count are not written.
+ * counts: device int32 [images], prompt length + accepted tokens of each image (may be null).
+ * images = the batch of the pre-fill (half of it under guidance).  Asynchronous on the stream.
+ * Errors: STATE (no prefill), BAD_ARG, CAPACITY (row_stride below a sequence's prompt + n_generate). */
+int sjd_get_tokens(sjd_ctx *ctx, int32_t *tokens, int row_stride, int32_t *counts, void *cuda_stream);
+
 /* Copy the stored logits of the last step, [batch][window][vocab] in cfg.dtype,
  * to dst (device or host); for parity checks.  Errors: STATE, CAPACITY (bytes too small). */
 int sjd_peek_logits(sjd_ctx *ctx, void *dst, size_t bytes, void *cuda_stream);

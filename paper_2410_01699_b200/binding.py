@@ -30,7 +30,7 @@ EXPORTS = ["sjd_workspace_bytes", "sjd_init", "sjd_prefill", "sjd_step", "sjd_ge
            "sjd_verify_workspace_bytes", "sjd_verify", "sjd_last_device_status", "sjd_last_cuda_error",
            "sjd_destroy", "sjd_strerror", "sjd_launch_count", "sjd_trace", "sjd_trace_read", "sjd_verify_static",
            "sjd_gemm_workspace_bytes", "sjd_gemm", "sjd_attention_workspace_bytes", "sjd_attention", "sjd_get_info",
-           "sjd_prefill_ragged"]
+           "sjd_prefill_ragged", "sjd_get_tokens"]
 
 
 class SJDError(RuntimeError):
@@ -102,6 +102,8 @@ def lib():
                                      C.POINTER(sjd_sample_cfg), C.c_void_p]
     L.sjd_step.restype = C.c_int
     L.sjd_step.argtypes = [C.c_void_p, C.POINTER(sjd_step_out), C.c_void_p]
+    L.sjd_get_tokens.restype = C.c_int
+    L.sjd_get_tokens.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
     L.sjd_get_window.restype = C.c_int
     L.sjd_get_window.argtypes = [C.c_void_p, C.POINTER(sjd_step_out), C.c_void_p]
     L.sjd_peek_logits.restype = C.c_int
@@ -285,12 +287,14 @@ class Context:
         self._ctx = C.c_void_p()
         _check(lib().sjd_init(C.byref(self._ctx), C.byref(cfg), C.byref(w), _ptr(self.workspace), nbytes), "sjd_init")
         self.batch = self.window = 0
+        self._guided = False
 
     def prefill(self, prompt, sample: sjd_sample_cfg):
         """prompt: int32 cuda tensor [B][P]."""
         assert prompt.dtype == torch.int32 and prompt.is_cuda and prompt.is_contiguous()
         self._prompt = prompt
         self.batch, self.window = int(prompt.shape[0]), int(sample.window)
+        self._guided = float(sample.guidance) != 0.0
         _check(lib().sjd_prefill(self._ctx, self.batch, _ptr(prompt), int(prompt.shape[1]), C.byref(sample),
                                  _stream()), "sjd_prefill")
 
@@ -300,6 +304,7 @@ class Context:
         assert prompt.dtype == torch.int32 and prompt.is_cuda and prompt.is_contiguous()
         self._prompt = prompt
         self.batch, self.window = int(prompt.shape[0]), int(sample.window)
+        self._guided = float(sample.guidance) != 0.0
         lens = (C.c_int32 * self.batch)(*[int(x) for x in prompt_lens])
         _check(lib().sjd_prefill_ragged(self._ctx, self.batch, _ptr(prompt), lens, int(prompt.shape[1]), C.byref(sample),
                                         _stream()), "sjd_prefill_ragged")
@@ -309,6 +314,16 @@ class Context:
 
     def get_window(self, out: StepOut):
         _check(lib().sjd_get_window(self._ctx, C.byref(out.c), _stream()), "sjd_get_window")
+
+    def get_tokens(self, row_stride: int | None = None):
+        """(tokens int32 [images][row_stride], counts int32 [images]) on the device: every image's prompt and the
+        tokens fixed so far; see sjd_get_tokens."""
+        images = self.batch // 2 if self._guided else self.batch
+        row_stride = int(row_stride or self.cfg.max_seq)
+        tokens = torch.zeros(images, row_stride, dtype=torch.int32, device=self.device)
+        counts = torch.zeros(images, dtype=torch.int32, device=self.device)
+        _check(lib().sjd_get_tokens(self._ctx, _ptr(tokens), row_stride, _ptr(counts), _stream()), "sjd_get_tokens")
+        return tokens, counts
 
     def peek_logits(self):
         t = torch.empty(self.batch, self.window, self.cfg.vocab, dtype=TORCH_DTYPES[self.cfg.dtype], device=self.device)

@@ -231,6 +231,15 @@ __global__ void get_window_kernel(SeqState st, sjd_step_out o, int W, int stream
   if (threadIdx.x == 0 && o.total_committed) o.total_committed[b] = st.n[sb];
 }
 
+// one block per image: the fixed tokens of its (first) stream
+__global__ void get_tokens_kernel(SeqState st, int32_t *tokens, int row_stride, int32_t *counts, int streams) {
+  const int b = blockIdx.x, sb = b * streams;
+  const int n = st.n[sb];
+  for (int i = threadIdx.x; i < n && i < row_stride; i += blockDim.x)
+    tokens[(size_t)b * row_stride + i] = st.committed[(size_t)sb * st.max_seq + i];
+  if (threadIdx.x == 0 && counts) counts[b] = n;
+}
+
 }  // namespace
 }  // namespace sjd
 
@@ -891,6 +900,16 @@ extern "C" int sjd_get_window(sjd_ctx *c, const sjd_step_out *out, void *cuda_st
   if (!c->prefilled) return SJD_ERR_STATE;
   const int streams = c->sample.guidance != 0.0f ? 2 : 1;
   get_window_kernel<<<c->batch / streams, 64, 0, (cudaStream_t)cuda_stream>>>(c->state(), *out, c->window, streams);
+  SJD_CHECK_LAUNCH();
+  return SJD_OK;
+}
+
+extern "C" int sjd_get_tokens(sjd_ctx *c, int32_t *tokens, int row_stride, int32_t *counts, void *cuda_stream) {
+  if (!c || !tokens || row_stride < 1) return SJD_ERR_BAD_ARG;
+  if (!c->prefilled) return SJD_ERR_STATE;
+  if ((long)row_stride < (long)c->prompt_len + c->sample.n_generate) return SJD_ERR_CAPACITY;
+  const int streams = c->sample.guidance != 0.0f ? 2 : 1;
+  get_tokens_kernel<<<c->batch / streams, 256, 0, (cudaStream_t)cuda_stream>>>(c->state(), tokens, row_stride, counts, streams);
   SJD_CHECK_LAUNCH();
   return SJD_OK;
 }

@@ -57,7 +57,37 @@ def run_lockstep(wl, batch=1, max_steps=None, init=INIT_RANDOM, check_logits_eve
         if max_steps and steps >= max_steps:
             break
     assert ctx.device_status() == B.SJD_OK
+    # the sequences as the library hands them out (sjd_get_tokens): prompt + every token fixed so far
+    tokens, counts = ctx.get_tokens()
+    tokens, counts = tokens.cpu().numpy(), counts.cpu().numpy()
+    for b, s in enumerate(seqs):
+        assert int(counts[b]) == s.st.n
+        assert [int(t) for t in tokens[b][:s.st.n]] == s.st.committed
     return ctx, seqs, steps, out
+
+
+@pytest.mark.parametrize("name,batch,guidance", [("tiny", 3, 0.0), ("small-bf16", 2, 0.0), ("small-bf16", 4, 3.0)])
+def test_generate_reproduces_the_lockstep_run(name, batch, guidance):
+    """generate() (iterations enqueued without the host looking at them, DONE flags read every few
+    iterations, sjd_get_tokens at the end) yields exactly the sequences of the run that was checked against
+    the oracle step by step: the kernels are deterministic, so a second context must repeat them."""
+    from paper_2410_01699_b200.generate import generate
+    wl = WORKLOADS[name]
+    n_generate = 45
+    if guidance:
+        checked, _ = run_lockstep_guided(wl, images=batch // 2, guidance=guidance, n_generate=n_generate)
+    else:
+        _, checked, _, _ = run_lockstep(wl, batch=batch, n_generate=n_generate)
+    weights = make_weights(wl, gain_jitter=0.1)
+    ctx = B.Context(B.make_model_cfg(wl, batch, wl.prompt_len + n_generate + 8, wl.window), B.weights_to_device(weights))
+    sample = B.make_sample_cfg(temperature=wl.temperature, top_k=wl.top_k, seed=wl.philox_seed, window=wl.window,
+                               init=INIT_RANDOM, grid_stride=wl.grid_stride, n_generate=n_generate, guidance=guidance)
+    tokens, counts, steps = generate(ctx, torch.from_numpy(make_prompt(wl, batch)).cuda(), sample, check_every=5)
+    tokens, counts = tokens.cpu().numpy(), counts.cpu().numpy()
+    assert steps <= n_generate and len(checked) == len(counts)
+    for i, s in enumerate(checked):
+        assert int(counts[i]) == wl.prompt_len + n_generate
+        assert [int(t) for t in tokens[i][:counts[i]]] == s.st.committed
 
 
 def test_tiny_fp32_full_generation():
