@@ -90,6 +90,36 @@ def test_generate_reproduces_the_lockstep_run(name, batch, guidance):
         assert [int(t) for t in tokens[i][:counts[i]]] == s.st.committed
 
 
+@pytest.mark.parametrize("name,init,kv_pages", [("tiny", INIT_RESAMPLE_ABOVE, 0), ("small-bf16", INIT_RESAMPLE_ABOVE, 6),
+                                                ("small-bf16", INIT_COPY_LEFT, 0)])
+def test_second_prefill_starts_clean(name, init, kv_pages):
+    """A context that has generated one batch and is pre-filled again (other prompts, other lengths of batch)
+    yields what a fresh context yields: no window state, retained row, cache row or page of the first run
+    leaks into the second."""
+    from paper_2410_01699_b200.generate import generate
+    wl = WORKLOADS[name]
+    n_generate = 40
+    weights = B.weights_to_device(make_weights(wl, gain_jitter=0.1))
+    ring = wl.grid_stride + wl.window if init == INIT_RESAMPLE_ABOVE else 0
+
+    def ctx():
+        return B.Context(B.make_model_cfg(wl, 3, wl.prompt_len + n_generate + 8, wl.window, max_ring=ring,
+                                          kv_pages=kv_pages), weights)
+
+    def sample(seed):
+        return B.make_sample_cfg(temperature=wl.temperature, top_k=wl.top_k, seed=seed, window=wl.window, init=init,
+                                 grid_stride=wl.grid_stride, n_generate=n_generate)
+
+    prompts = torch.from_numpy(make_prompt(wl, 5)).cuda()
+    used = ctx()
+    generate(used, prompts[:3].contiguous(), sample(11))
+    again, counts_a, _ = generate(used, prompts[3:].contiguous(), sample(12))
+    fresh, counts_f, _ = generate(ctx(), prompts[3:].contiguous(), sample(12))
+    assert torch.equal(counts_a, counts_f)
+    n = int(counts_f[0])
+    assert torch.equal(again[:, :n], fresh[:, :n])
+
+
 def test_tiny_fp32_full_generation():
     """The tiny fp32 configuration end to end: 256 tokens, W = 16, top-k 64, random initialisation."""
     wl = WORKLOADS["tiny"]
