@@ -23,7 +23,8 @@
 // (about a dozen block barriers per row).  Rows with NaN/+inf, without a finite entry, with the
 // K-th largest entry more than 4095 codes below the maximum (e.g. a positive maximum and a negative
 // threshold) or next to +-0 use the general route above; both routes produce the same threshold and
-// the same weights.
+// the same weights.  Longer bf16 rows (the 184320-entry head) take the same route streamed: a full block
+// passes the row through its registers in segments of 65536 entries, once per phase (long_statistics).
 #include <float.h>
 
 #include <type_traits>
@@ -594,9 +595,8 @@ __device__ uint32_t rr_load_max(RegRow &row, const uint4 *g, const uint4 *g2, fl
 // `z_hist` (optional): the softmax denominator from the histogram alone -- all entries of a bin share one
 // value, so Z = sum over the kept bins of count * 2^((value - max) * scale) -- for rows whose chunk
 // sums nobody needs (the previous-iteration row when its statistics are not cached).
-__device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, Scratch &sc, uint32_t &tau_key,
-                          float scale, double *z_hist) {
-  using E = Elt<__nv_bfloat16>;
+// histogram pass of rr_select over the vectors held in `row` (those with local index below NV)
+__device__ __forceinline__ void rr_hist_add(const RegRow &row, int NV, uint32_t kmax, Scratch &sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int j0 = warp * 256 + lane;
   const uint32_t kmax2 = kmax | (kmax << 16);
@@ -614,7 +614,13 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
       }
     }
   }
-  __syncthreads();
+}
+
+// walk of rr_select over the finished histogram (every warp for itself)
+__device__ __forceinline__ bool rr_walk(uint32_t kmax, uint32_t K, Scratch &sc, uint32_t &tau_key, float scale,
+                                        double *z_hist) {
+  using E = Elt<__nv_bfloat16>;
+  const int lane = threadIdx.x & 31;
   // The walk: 32 adjacent bins per step (conflict-free).  A step that does not reach the K-th entry costs one
   // load and one warp-wide integer sum; only the step that does is scanned.  For z_hist every lane
   // accumulates the mass of its own bins and the warp adds the lanes up once, at the end.
@@ -652,13 +658,21 @@ __device__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, 
   return false;
 }
 
+__device__ __forceinline__ bool rr_select(const RegRow &row, int NV, uint32_t kmax, uint32_t K, Scratch &sc,
+                                          uint32_t &tau_key, float scale, double *z_hist) {
+  rr_hist_add(row, NV, kmax, sc);
+  __syncthreads();
+  return rr_walk(kmax, K, sc, tau_key, scale, z_hist);
+}
+
 // chunk sums of a weight functor evaluated on registers -> sc.chunk_sum.  One barrier.
 // Every lane holds eight slot sums; the warp adds them up transposed (each exchange halves the number of
 // slots a lane still carries: 4 + 2 + 1 + 1 + 1 shuffles instead of 8 x 5), in a fixed order.
+// `chunk0`: chunk index of this block's first vector (rows streamed in segments), NC then counts the whole row's chunks.
 template <typename F>
-__device__ __forceinline__ void rr_chunk_sums(const F &wf, int NV, Scratch &sc) {
+__device__ __forceinline__ void rr_chunk_sums(const F &wf, int NV, Scratch &sc, int chunk0 = 0, int n_chunks = -1) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int NC = (NV + 31) >> 5;
+  const int NC = n_chunks >= 0 ? n_chunks : (NV + 31) >> 5;
   float s[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -686,7 +700,7 @@ __device__ __forceinline__ void rr_chunk_sums(const F &wf, int NV, Scratch &sc) 
   e += __shfl_xor_sync(0xffffffffu, e, 2);
   e += __shfl_xor_sync(0xffffffffu, e, 1);
   const int slot = (lane >> 2) & 7;   // bit 4 -> slot bit 2, bit 3 -> bit 1, bit 2 -> bit 0
-  if ((lane & 3) == 0 && warp * 8 + slot < NC) sc.chunk_sum[warp * 8 + slot] = e;
+  if ((lane & 3) == 0 && chunk0 + warp * 8 + slot < NC) sc.chunk_sum[chunk0 + warp * 8 + slot] = e;
   __syncthreads();
 }
 
@@ -716,10 +730,13 @@ __device__ __forceinline__ WarpPrefix rr_prefix(int NC, const Scratch &sc) {
 
 // Inverse CDF (token order) over weights held in registers: every warp finds the chunk, the warp that
 // owns it finds the entry (same rules as sample_icdf) and publishes it.  One barrier.
+// wf(c, w): this lane's eight weights of chunk c, asked of the warp that owns the chunk (chunk c of a row
+// streamed in segments of 8 * blockDim vectors belongs to warp (c mod 8 * warps) / 8).
 template <typename F>
 __device__ void rr_icdf(const F &wf, int NV, const WarpPrefix &wp, float u, Scratch &sc, int &tok, float &tok_w) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NC = (NV + 31) >> 5;
+  const int seg_chunks = (int)(blockDim.x >> 5) * 8;
   const double target = (double)u * wp.total;
   const int lo = min(NC, lane * wp.per), hi = min(NC, lo + wp.per);
   // inside this lane's group: first chunk with positive mass whose interval holds the target; last positive chunk
@@ -761,9 +778,9 @@ __device__ void rr_icdf(const F &wf, int NV, const WarpPrefix &wp, float u, Scra
       sc.tok = 0;
       sc.tok_w = 0.0f;
     }
-  } else if (warp == (c >> 3)) {
+  } else if (warp == ((c % seg_chunks) >> 3)) {
     float w[8];
-    wf(c & 7, w);
+    wf(c, w);
     float sum = 0.0f;
 #pragma unroll
     for (int t = 0; t < 8; ++t) sum += w[t];
@@ -881,6 +898,106 @@ __device__ bool rr_statistics(RegRow &row, const __nv_bfloat16 *g, const __nv_bf
   return true;
 }
 
+// ------------------------------------------------------------------------------------ rows longer than the registers
+// bf16 rows of more than 8 * blockDim vectors (V = 184320: 23040 vectors against 8192) take the same phases with
+// the row streamed through the registers one segment of 8 * blockDim vectors at a time; every phase reads the
+// row again (it was written by the preceding kernel and sits in L2): maximum, histogram, masked weights and
+// chunk sums.  The chunk numbering is the one of a row held at once (chunk = 32 consecutive vectors), so the
+// prefix and the search over sc.chunk_sum are shared; the search re-reads the one chunk it ends in.
+__device__ __forceinline__ void seg_load(RegRow &row, const uint4 *g, const uint4 *g2, float gw, int NV, int seg) {
+  const int j0 = seg * 8 * (int)blockDim.x + (int)(threadIdx.x >> 5) * 256 + (int)(threadIdx.x & 31);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int j = j0 + i * 32;
+    row.v[i] = j < NV ? rr_load_vec(g, g2, gw, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+  }
+}
+// vector j of the row with the entries below the threshold replaced by -inf (what rr_mask_below leaves in a RegRow)
+__device__ __forceinline__ uint4 load_masked_vec(const uint4 *g, const uint4 *g2, float gw, int NV, int j, float tau_f) {
+  if (j >= NV) return make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+  const uint4 v = rr_load_vec(g, g2, gw, j);
+  const __nv_bfloat16 t1 = __float2bfloat16_rn(tau_f);
+  const __nv_bfloat162 t2 = __halves2bfloat162(t1, t1);
+  uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t m = __hge2_mask(as_bf2(w[k]), t2);
+    w[k] = (w[k] & m) | (0xFF80FF80u & ~m);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// rr_statistics for a streamed row.  Barriers: 1 (maximum) + 1 (histogram) + one per segment (chunk sums).
+__device__ bool long_statistics(const __nv_bfloat16 *g, const __nv_bfloat16 *g2, float gw, int V, int d, int d_slot, int top_k,
+                                float inv_t, Scratch &sc, RowFast &out, bool want_chunks) {
+  using E = Elt<__nv_bfloat16>;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
+  const int NV = V >> 3, NC = (NV + 31) >> 5;
+  const int seg_v = 8 * nt, n_seg = (NV + seg_v - 1) / seg_v;
+  const uint4 *gv = reinterpret_cast<const uint4 *>(g), *gv2 = reinterpret_cast<const uint4 *>(g2);
+  const bool need_select = top_k < V;
+  RegRow row;
+  // ---- maximum (and the entry at the draft token)
+  if (need_select)
+    for (int i = tid; i < 1024; i += nt) reinterpret_cast<uint4 *>(sc.hist12)[i] = make_uint4(0u, 0u, 0u, 0u);
+  __nv_bfloat162 m2 = as_bf2(0xFF80FF80u);
+  for (int seg = 0; seg < n_seg; ++seg) {
+    seg_load(row, gv, gv2, gw, NV, seg);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) m2 = __hmax2_nan(m2, as_bf2(word_of(row.v[i], w)));
+    }
+  }
+  if (tid == 0 && d >= 0) {
+    uint32_t bits = (uint32_t)__ldg(reinterpret_cast<const unsigned short *>(g) + d);
+    if (g2) {
+      const float c = E::val(bits), u = E::val((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(g2) + d));
+      bits = E::bits(fmaf(gw, c - u, u));
+    }
+    sc.d_bits[d_slot] = bits;
+  }
+  const __nv_bfloat16 m1 = __hmax_nan(__low2bfloat16(m2), __high2bfloat16(m2));
+  const uint32_t mbits = (uint32_t)__bfloat16_as_ushort(m1);
+  uint32_t kmax = (mbits & 0x7FFFu) > 0x7F80u ? 0xFFFFu : E::key(mbits);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) sc.redu[warp] = kmax;
+  __syncthreads();
+  kmax = 0;
+  for (int w = 0; w < nw; ++w) kmax = max(kmax, sc.redu[w]);
+  if (kmax >= 0xFF80u || kmax <= 0x007Fu) return false;
+  // ---- threshold
+  uint32_t tau_key = 0;
+  const float scale = inv_t * 1.4426950408889634f;
+  const bool from_hist = need_select && !want_chunks;
+  out.z_hist = -1.0;
+  if (need_select) {
+    for (int seg = 0; seg < n_seg; ++seg) {
+      seg_load(row, gv, gv2, gw, NV, seg);
+      rr_hist_add(row, NV - seg * seg_v, kmax, sc);
+    }
+    __syncthreads();
+    if (!rr_walk(kmax, (uint32_t)top_k, sc, tau_key, scale, from_hist ? &out.z_hist : nullptr)) return false;
+  }
+  out.st.tau_key = tau_key;
+  out.st.xmax = E::val(E::unkey(kmax));
+  out.st.flags = 0;
+  out.tau_f = need_select ? E::val(E::unkey(tau_key)) : -INFINITY;
+  const float xmax = out.st.xmax, tau_f = out.tau_f;
+  if (from_hist) {
+    __syncthreads();   // sc.d_bits is read below; the walk above read the histogram the next row clears
+  } else {
+    for (int seg = 0; seg < n_seg; ++seg) {
+      seg_load(row, gv, gv2, gw, NV, seg);
+      if (need_select) rr_mask_below(row, tau_f);
+      rr_chunk_sums([&](int i, float *w) { rr_p_weights(row.v[i], xmax, scale, w); }, NV, sc, seg * nw * 8, NC);
+    }
+  }
+  const float dv = E::val(sc.d_bits[d_slot]);
+  out.d_weight = (d >= 0 && dv >= tau_f) ? exp2_neg((dv - xmax) * scale) : 0.0f;
+  return true;
+}
+
 // The logits rows of window slot k of image b: this iteration's (p) and the one the draft was drawn from
 // (q, row qr of the other buffer); under guidance the unconditional stream's rows beside them (else null).
 template <typename T>
@@ -908,25 +1025,23 @@ __device__ __forceinline__ RowRefs<T> row_refs(const VerifyParams &p, int b, int
   return rr;
 }
 
-__device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowRefs<__nv_bfloat16> &rows, int kind, int d,
+template <bool STREAM_OK>
+__device__ void rr_residual(const VerifyParams &p, const RegRow *row_in, const RowRefs<__nv_bfloat16> &rows, int kind, int d,
                             const RowStats &ps, const RowStats &qs, float u_res, Scratch &sc, int &tok, uint32_t &flags);
 
-template <typename T>
-__device__ bool fast_row(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
-                         const RowRefs<T> &rows, float inv_t, float u_acc, float u_res, float u_draft, RowOut &ro) {
-  return false;
-}
 
 constexpr int kResampleDeferred = -2;   // RowOut.resample_tok of a rejected row whose Eq. 2 draw is still to be made
 
-template <>
-__device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
-                                        const RowRefs<__nv_bfloat16> &rows, float inv_t, float u_acc, float u_res,
-                                        float u_draft, RowOut &ro) {
+// STREAM_OK: the instantiation for full blocks, which also takes rows too long for the registers
+template <bool STREAM_OK>
+__device__ bool fast_row_bf16(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
+                              const RowRefs<__nv_bfloat16> &rows, float inv_t, float u_acc, float u_res,
+                              float u_draft, RowOut &ro) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x;
   const int V = p.V, NV = V >> 3, NC = (NV + 31) >> 5;
-  if (NV > 8 * (int)blockDim.x) return false;
+  const bool streamed = STREAM_OK && NV > 8 * (int)blockDim.x;   // too long for the registers: see long_statistics
+  if (NV > 8 * (int)blockDim.x && (!STREAM_OK || NC > kMaxChunks)) return false;
   const bool d_ok = d >= 0 && d < V;
   const int dd = d_ok ? d : -1;
   const float scale = inv_t * 1.4426950408889634f;
@@ -952,7 +1067,9 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
       q_d = d_ok ? (E::key(bits) >= qs.tau_key ? exp2_neg((E::val(bits) - qs.xmax) * scale) : 0.0f) / qs.z : 1.0f;
     } else {
       RowFast qfast;
-      if (!rr_statistics(row, rows.q, rows.q2, p.guidance, V, dd, 0, p.top_k, inv_t, sc, qfast, false)) return false;
+      if (!(streamed ? long_statistics(rows.q, rows.q2, p.guidance, V, dd, 0, p.top_k, inv_t, sc, qfast, false)
+                     : rr_statistics(row, rows.q, rows.q2, p.guidance, V, dd, 0, p.top_k, inv_t, sc, qfast, false)))
+        return false;
       qs = qfast.st;
       qs.z = (float)(qfast.z_hist >= 0.0 ? qfast.z_hist : rr_prefix(NC, sc).total);
       if (tid == 0) p.stats[cur ^ 1][r] = qs;
@@ -967,7 +1084,9 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   SJD_TL(TL_VERIFY, 10, tid == 0);
   // ---- this iteration's distribution (entries below the threshold are -inf in `row` from here on)
   RowFast pfast;
-  if (!rr_statistics(row, rows.p, rows.p2, p.guidance, V, dd, 1, p.top_k, inv_t, sc, pfast, true)) return false;
+  if (!(streamed ? long_statistics(rows.p, rows.p2, p.guidance, V, dd, 1, p.top_k, inv_t, sc, pfast, true)
+                 : rr_statistics(row, rows.p, rows.p2, p.guidance, V, dd, 1, p.top_k, inv_t, sc, pfast, true)))
+    return false;
   const WarpPrefix wpp = rr_prefix(NC, sc);
   RowStats ps = pfast.st;
   ps.z = (float)wpp.total;
@@ -989,7 +1108,15 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   auto p_w = [&](int i, float *w) { rr_p_weights(reg_slot(row, i), xmax_p, scale, w); };
   int redraft_tok;
   float redraft_w;
-  rr_icdf(p_w, NV, wpp, u_draft, sc, redraft_tok, redraft_w);
+  if (streamed) {
+    const uint4 *pg = reinterpret_cast<const uint4 *>(rows.p), *pg2 = reinterpret_cast<const uint4 *>(rows.p2);
+    const float tau_f = pfast.tau_f;
+    rr_icdf([&](int c, float *w) {
+      rr_p_weights(load_masked_vec(pg, pg2, p.guidance, NV, c * 32 + (tid & 31), tau_f), xmax_p, scale, w);
+    }, NV, wpp, u_draft, sc, redraft_tok, redraft_w);
+  } else {
+    rr_icdf([&](int c, float *w) { p_w(c & 7, w); }, NV, wpp, u_draft, sc, redraft_tok, redraft_w);
+  }
   const float redraft_p = redraft_w / ps.z;
   SJD_TL(TL_VERIFY, 12, tid == 0);
 
@@ -1000,7 +1127,7 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   int resample_tok = accept ? -1 : kResampleDeferred;
   if (!accept && !p.defer_residual && p.schedule != SJD_SCHEDULE_JACOBI) {
     __syncthreads();
-    rr_residual(p, row, rows, kind, d, ps, qs, u_res, sc, resample_tok, flags);
+    rr_residual<STREAM_OK>(p, streamed ? nullptr : &row, rows, kind, d, ps, qs, u_res, sc, resample_tok, flags);
   }
   ro.p_draft = p_d; ro.q_draft = q_d; ro.thr = thr; ro.accept = accept ? 1 : 0;
   ro.redraft_tok = redraft_tok; ro.redraft_p = redraft_p; ro.resample_tok = resample_tok;
@@ -1015,10 +1142,23 @@ __device__ bool fast_row<__nv_bfloat16>(const VerifyParams &p, Scratch &sc, int 
   return true;
 }
 
+template <typename T, bool STREAM_OK>
+__device__ __forceinline__ bool fast_row(const VerifyParams &p, Scratch &sc, int r, int b, int kind, int d, int qr, int cur,
+                                         const RowRefs<T> &rows, float inv_t, float u_acc, float u_res, float u_draft,
+                                         RowOut &ro) {
+  if constexpr (std::is_same<T, __nv_bfloat16>::value)
+    return fast_row_bf16<STREAM_OK>(p, sc, r, b, kind, d, qr, cur, rows, inv_t, u_acc, u_res, u_draft, ro);
+  else
+    return false;
+}
+
 // Eq. 2 on a p row held in registers (entries below its threshold may already have been replaced by
 // -inf): residual weights max(0, p - q), their chunk sums and the inverse-CDF draw; the q row is read
 // from global memory (L2) vector by vector as it is needed.  Block-wide; returns the token and flags.
-__device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowRefs<__nv_bfloat16> &rows, int kind, int d,
+// row_in == null: the p row is too long for the registers and is streamed from global memory as well (only in
+// the instantiation for full blocks, STREAM_OK: smaller blocks never meet such a row).
+template <bool STREAM_OK>
+__device__ void rr_residual(const VerifyParams &p, const RegRow *row_in, const RowRefs<__nv_bfloat16> &rows, int kind, int d,
                             const RowStats &ps, const RowStats &qs, float u_res, Scratch &sc, int &tok, uint32_t &flags) {
   using E = Elt<__nv_bfloat16>;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1032,9 +1172,7 @@ __device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowR
   // c = -max * scale - log2(Z); entries below the threshold contribute nothing
   const float cp = -ps.xmax * scale - log2f(ps.z), cq = -qs.xmax * scale - log2f(qs.z);
   const float q_uniform = 1.0f / (float)V;
-  auto r_w = [&](int i, float *w) {   // max(0, p - q) of the eight entries of slot i
-    const int j = j0 + i * 32;
-    const uint4 pv = reg_slot(row, i);
+  auto r_vec = [&](const uint4 &pv, int j, float *w) {   // max(0, p - q) of the eight entries of vector j
     uint4 qv = make_uint4(0, 0, 0, 0);
     if (kind == SJD_Q_ROW && j < NV) qv = rr_load_vec(qg, qg2, p.guidance, j);
 #pragma unroll
@@ -1057,28 +1195,61 @@ __device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowR
       }
     }
   };
+  auto p_vec = [&](const uint4 &pv, float *w) {   // the p row's own weights (empty residual: sample from p)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t px = word_of(pv, k);
+      const float lo = __uint_as_float(px << 16), hi = __uint_as_float(px & 0xFFFF0000u);
+      w[2 * k] = lo >= tau_p ? exp2_neg((lo - ps.xmax) * scale) : 0.0f;
+      w[2 * k + 1] = hi >= tau_p ? exp2_neg((hi - ps.xmax) * scale) : 0.0f;
+    }
+  };
   float wsel;
+  if (STREAM_OK && row_in == nullptr) {
+    // ---- a row streamed in segments (see long_statistics): chunk sums segment by segment, the search re-reads
+    // the vectors of the chunk it ends in
+    const uint4 *pg = reinterpret_cast<const uint4 *>(rows.p), *pg2 = reinterpret_cast<const uint4 *>(rows.p2);
+    const int nw = blockDim.x >> 5, seg_v = 8 * (int)blockDim.x, n_seg = (NV + seg_v - 1) / seg_v;
+    const uint4 filler = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+    RegRow seg_row;
+    for (int seg = 0; seg < n_seg; ++seg) {
+      seg_load(seg_row, pg, pg2, p.guidance, NV, seg);
+      rr_chunk_sums([&](int i, float *w) { r_vec(seg_row.v[i], seg * seg_v + j0 + i * 32, w); }, NV, sc, seg * nw * 8, NC);
+    }
+    WarpPrefix wr = rr_prefix(NC, sc);
+    if (wr.total > 0.0) {
+      rr_icdf([&](int c, float *w) {
+        const int j = c * 32 + lane;
+        r_vec(j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : filler, j, w);
+      }, NV, wr, u_res, sc, tok, wsel);
+    } else {
+      flags |= SJD_FLAG_RESIDUAL_EMPTY;
+      __syncthreads();
+      for (int seg = 0; seg < n_seg; ++seg) {
+        seg_load(seg_row, pg, pg2, p.guidance, NV, seg);
+        rr_chunk_sums([&](int i, float *w) { p_vec(seg_row.v[i], w); }, NV, sc, seg * nw * 8, NC);
+      }
+      wr = rr_prefix(NC, sc);
+      rr_icdf([&](int c, float *w) {
+        const int j = c * 32 + lane;
+        p_vec(j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : filler, w);
+      }, NV, wr, u_res, sc, tok, wsel);
+    }
+    return;
+  }
+  const RegRow &row = *row_in;
+  auto r_w = [&](int i, float *w) { r_vec(reg_slot(row, i), j0 + i * 32, w); };
   rr_chunk_sums(r_w, NV, sc);
   WarpPrefix wr = rr_prefix(NC, sc);
   if (wr.total > 0.0) {
-    rr_icdf(r_w, NV, wr, u_res, sc, tok, wsel);
+    rr_icdf([&](int c, float *w) { r_w(c & 7, w); }, NV, wr, u_res, sc, tok, wsel);
   } else {
     flags |= SJD_FLAG_RESIDUAL_EMPTY;
-    const float c0 = ps.xmax;
-    auto p_w = [&](int i, float *w) {
-      const uint4 pv = reg_slot(row, i);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const uint32_t px = word_of(pv, k);
-        const float lo = __uint_as_float(px << 16), hi = __uint_as_float(px & 0xFFFF0000u);
-        w[2 * k] = lo >= tau_p ? exp2_neg((lo - c0) * scale) : 0.0f;
-        w[2 * k + 1] = hi >= tau_p ? exp2_neg((hi - c0) * scale) : 0.0f;
-      }
-    };
+    auto p_w = [&](int i, float *w) { p_vec(reg_slot(row, i), w); };
     __syncthreads();
     rr_chunk_sums(p_w, NV, sc);
     wr = rr_prefix(NC, sc);
-    rr_icdf(p_w, NV, wr, u_res, sc, tok, wsel);
+    rr_icdf([&](int c, float *w) { p_w(c & 7, w); }, NV, wr, u_res, sc, tok, wsel);
   }
 }
 
@@ -1086,11 +1257,8 @@ __device__ void rr_residual(const VerifyParams &p, const RegRow &row, const RowR
 // grids of more than one wave): run by every thread of the sequence's last block before the window slide.
 // The row's statistics and those of its draft's law were published by the block that verified it; the p
 // row is read again into registers (it is still in L2).
-template <typename T>
-__device__ void deferred_residual(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {}
-
-template <>
-__device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {
+template <bool STREAM_OK>
+__device__ void deferred_residual_bf16(const VerifyParams &p, int b, uint32_t step, int cur, Scratch &sc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int W = p.W, NV = p.V >> 3;
   const int w_eff = p.w_eff ? p.w_eff[p.paired ? 2 * b : b] : W;
@@ -1128,16 +1296,20 @@ __device__ void deferred_residual<__nv_bfloat16>(const VerifyParams &p, int b, u
   RowStats qs;
   qs.tau_key = 0; qs.xmax = 0.0f; qs.z = 1.0f; qs.flags = 0;
   if (kind == SJD_Q_ROW) qs = load_stats(rows.qstats);
-  RegRow row;
-  const int j0 = warp * 256 + lane;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int j = j0 + i * 32;
-    row.v[i] = j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-  }
   uint32_t flags = 0;
   int tok;
-  rr_residual(p, row, rows, kind, d, ps, qs, u_res, sc, tok, flags);
+  if (STREAM_OK && NV > 8 * (int)blockDim.x) {   // a row streamed in segments
+    rr_residual<STREAM_OK>(p, nullptr, rows, kind, d, ps, qs, u_res, sc, tok, flags);
+  } else {
+    RegRow row;
+    const int j0 = warp * 256 + lane;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int j = j0 + i * 32;
+      row.v[i] = j < NV ? rr_load_vec(pg, pg2, p.guidance, j) : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+    }
+    rr_residual<STREAM_OK>(p, &row, rows, kind, d, ps, qs, u_res, sc, tok, flags);
+  }
   if (tid == 0) {
     ro[a].resample_tok = tok;
     ro[a].flags = __ldcg(&ro[a].flags) | flags;
@@ -1383,7 +1555,8 @@ __device__ void finalize_sequence(const VerifyParams &p, int b, uint32_t step, S
 }
 
 // ------------------------------------------------------------------------------------ kernel
-template <typename T, int MAXT>
+// STREAM: the instantiation launched for bf16 rows too long for the registers of a block (see long_statistics)
+template <typename T, int MAXT, bool STREAM = false>
 __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1) verify_rows_kernel(const VerifyParams p) {
   using E = Elt<T>;
   extern __shared__ uint4 dyn_smem[];
@@ -1424,7 +1597,7 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
 
     RowOut fast_out;
     const bool fast_done = p.fast && (((uintptr_t)rows.q | (uintptr_t)rows.p) & 15u) == 0 &&
-                           fast_row<T>(p, sc, r, b, kind, d, qr, cur, rows, inv_t, u_acc, u_res, u_draft, fast_out);
+                           fast_row<T, STREAM>(p, sc, r, b, kind, d, qr, cur, rows, inv_t, u_acc, u_res, u_draft, fast_out);
     if (fast_done) {
       if (tid == 0) p.row_out[r] = fast_out;
     } else {
@@ -1525,7 +1698,9 @@ __global__ void __launch_bounds__(MAXT, MAXT <= 256 ? SJD_VERIFY_MIN_BLOCKS : 1)
   if (!sc.is_last) return;
   __threadfence();
   SJD_TL(TL_VERIFY, 14, tid == 0);
-  if (p.fast && p.defer_residual) deferred_residual<T>(p, b, step, cur, sc);
+  if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    if (p.fast && p.defer_residual) deferred_residual_bf16<STREAM>(p, b, step, cur, sc);
+  }
   if (p.e2e && (p.st.init == SJD_INIT_RESAMPLE_LEFT || p.st.init == SJD_INIT_RESAMPLE_ABOVE))
     draw_fresh_slots<T>(p, b, step, cur, sc);
   finalize_sequence(p, b, step, sc);
@@ -1600,10 +1775,12 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
   int threads = nv_max <= 1024 ? 128 : nv_max <= 4096 ? 256 : nv_max <= 16384 ? 512 : 1024;
   // rows a block can hold in registers, eight vectors per thread
   p.fast = 0;
-  if (std::is_same<T, __nv_bfloat16>::value && p.staged && p.V % VEC == 0 && p.V / VEC <= 8 * kMaxThreads &&
+  // (longer rows, up to kMaxChunks chunks, stream through the registers of a full block in segments)
+  const bool in_registers = p.V / VEC <= 8 * kMaxThreads;
+  if (std::is_same<T, __nv_bfloat16>::value && (p.staged || !in_registers) && p.V % VEC == 0 &&
       ((uintptr_t)p.logits[0] & 15u) == 0 && ((uintptr_t)p.logits[1] & 15u) == 0) {
     p.fast = 1;
-    threads = (p.V / VEC + 255) / 256 * 32;
+    threads = in_registers ? (p.V / VEC + 255) / 256 * 32 : kMaxThreads;
     threads = threads < 64 ? 64 : threads;
     // no staging buffer: the rows live in registers; the odd row that needs the general route (a NaN, a
     // threshold out of the histogram's reach) re-reads global memory instead, and more blocks fit an SM
@@ -1627,6 +1804,7 @@ static int launch_verify_t(const VerifyParams &p_in, cudaStream_t stream) {
     return SJD_OK;
   };
   if (threads <= 256) return launch(verify_rows_kernel<T, 256>);
+  if (p.fast && !in_registers) return launch(verify_rows_kernel<T, kMaxThreads, true>);
   return launch(verify_rows_kernel<T, kMaxThreads>);
 }
 

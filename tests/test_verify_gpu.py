@@ -97,7 +97,10 @@ def test_verify_ratio_corner_cases():
     ("f32", 1000, 7, 1000),      # top_k == V: no filtering
     ("bf16", 4099, 5, 1),        # top-1
     ("bf16", 65536, 4, 2000),    # 128 KB rows (the 7B head)
-    ("bf16", 184320, 2, 2048),   # rows larger than shared memory
+    ("bf16", 184320, 2, 2048),   # rows longer than a block's registers: streamed in three segments (the 8B head)
+    ("bf16", 100000, 5, 2000),   # two segments, the second partial (12500 vectors against 8192)
+    ("bf16", 184320, 3, 184320), # streamed rows, top_k == V: no threshold
+    ("bf16", 262000, 2, 4000),   # the longest row the chunk table covers: four segments
     ("f32", 50000, 3, 500),      # fp32 rows beyond the staging buffer
 ])
 def test_verify_shapes(dtype, vocab, window, top_k):
@@ -109,6 +112,20 @@ def test_verify_mixed_laws():
     """Slots whose draft came from a uniform initialisation (q = 1/V) or a copy (point mass)."""
     case = make_verify_case(6, window=16, vocab=4096, top_k=300, seed=11, mixed_kinds=True)
     _check_case(case)
+
+
+def test_verify_mixed_laws_on_streamed_rows():
+    """The same on rows too long for the registers (drift 3: most drafts are rejected, so Eq. 2 runs on streamed
+    rows against uniform, copied and predicted drafts)."""
+    case = make_verify_case(3, window=6, vocab=100000, top_k=2000, seed=12, mixed_kinds=True, drift=3.0)
+    _check_case(case, max_flag_frac=0.06)
+
+
+def test_verify_streamed_rows_in_a_grid_of_several_waves():
+    """160 streamed rows on 148 SMs: the rejected rows leave Eq. 2 to their sequence's last block, which streams
+    the two rows again."""
+    case = make_verify_case(10, window=16, vocab=70000, top_k=2000, seed=13, drift=2.0)
+    _check_case(case, max_flag_frac=0.06)
 
 
 def test_verify_temperature_and_ties():
