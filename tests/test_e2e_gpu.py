@@ -377,6 +377,22 @@ def test_small_bf16_gqa_generation():
         assert s.stats.flagged <= max(3, 0.03 * s.stats.decisions), s.stats
 
 
+@pytest.mark.parametrize("guidance,init", [(0.0, INIT_RESAMPLE_ABOVE), (3.0, INIT_RESAMPLE_LEFT), (3.0, INIT_RANDOM)])
+def test_small_bf16_vocabulary_longer_than_the_registers(guidance, init):
+    """A 70016-entry vocabulary on the small bf16 model: every logits row is verified on the streamed form of
+    the register route (two segments), with cached statistics of the previous rows, with the rows of the two
+    guidance streams mixed as they are loaded, and with retained rows as the drafts' laws."""
+    wl = WORKLOADS["small-bf16"].with_(vocab=70016, top_k=2000)
+    if guidance:
+        seqs, steps = run_lockstep_guided(wl, images=1, guidance=guidance, n_generate=40, init=init)
+    else:
+        _, seqs, steps, _ = run_lockstep(wl, batch=2, init=init, n_generate=40)
+    for s in seqs:
+        assert s.st.n == wl.prompt_len + 40
+        assert s.max_logit_err <= 2e-2
+        assert s.stats.flagged <= max(3, 0.04 * s.stats.decisions), s.stats
+
+
 def test_small_bf16_128_rows():
     """8 images x W = 16 = 128 rows per pass: the largest single slab (256 MMA columns, two-stage ring) through
     pre-fill and three steps."""
